@@ -1,0 +1,315 @@
+/*
+ * FFD oracle: a plain, slow, fp64 CPU statement of the sparse decode-attention path of
+ * "Faster Than Flash" (FFD): 2-bit mid-rise key quantizer (App. A.1), approximate scores from the
+ * 2-bit keys, pseudo-max over sink + local blocks (Sec. 3.2, Alg. 1 "Pseudo-max estimation"),
+ * top-delta block selection (Eq. 1, Alg. 1 "Top-delta selection"), exact softmax attention over the
+ * kept blocks (Alg. 1 "Fine-grained refinement"), and dense softmax attention.
+ *
+ * THIS IS TEST INFRASTRUCTURE.  It exists to define correctness for the CUDA library and to be timed as
+ * a reported CPU baseline.  It shares no code with the CUDA path and the product never calls it.
+ *
+ * Style: every step is the definition written out, token by token and channel by channel, in double
+ * precision on the exact values of the bf16 / fp16 inputs.  No blocking, no fusion, no reordering.  The
+ * only parallelism is an OpenMP loop over independent (sequence, query head) pairs.
+ *
+ * Readings of the paper that this file fixes (each is a reading, not something the paper prints; the
+ * ones marked "parity unpinned" have no independent pin):
+ *   - bit width 2, codebook {-1.5,-0.5,+0.5,+1.5}, scale = absmax/1.5            (App. A.1, printed)
+ *   - one scale per (64-token block, KV head, channel), absmax over the block's valid rows;
+ *     stored as fp16 = RNE(fp32(absmax)/1.5f), saturated at 65504             (parity unpinned)
+ *   - nearest level written as comparisons: |x| >= s -> outer level, x = 0 -> +0.5; this equals the
+ *     arg-min of App. A.1 everywhere except exact ties
+ *   - approximate scores and the pseudo-max carry 1/sqrt(d); delta is a natural-log logit gap (Eq. 1-2)
+ *   - the pseudo-max uses the quantized scores (Alg. 1), so the kept set is never empty
+ *   - sink set = first n_sink blocks, local set = last n_local blocks (incl. the partial tail)
+ *                                                                              (parity unpinned)
+ *   - selection is per query head; whole 64-token blocks are kept or skipped  (parity unpinned)
+ *   - the partial tail block is quantized over its valid rows; rows past seq_len never contribute
+ *                                                                              (parity unpinned)
+ *   - refinement uses the full 16-bit K (the two-term form of Sec. 3.3 equals q.k when the residual
+ *     is exact), softmax over the kept tokens only
+ *
+ * Layouts (all host pointers, row-major, innermost last):
+ *   q        bf16 bits  [B, Hq, D]
+ *   k_cache  bf16 bits  [num_pages, Hkv, BLK, D]      v_cache the same
+ *   codes    u8 0..3    [num_pages, Hkv, BLK, D]      level = code - 1.5
+ *   scales   fp16 bits  [num_pages, Hkv, D]
+ *   block_table int32   [B, max_blocks]  logical block -> physical page; NULL = b*max_blocks + blk
+ *   seq_lens int32      [B]
+ *   query head h belongs to KV head h / (Hq/Hkv).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+static int g_threads = 1;
+
+void ffd_oracle_set_threads(int n) { g_threads = n < 1 ? 1 : n; }
+int ffd_oracle_get_threads(void) { return g_threads; }
+int ffd_oracle_max_threads(void) {
+#ifdef _OPENMP
+    return omp_get_num_procs();
+#else
+    return 1;
+#endif
+}
+
+/* ---- number formats -------------------------------------------------------------------------- */
+
+/* bf16 is the top half of an IEEE binary32. */
+static double bf16_value(uint16_t bits) {
+    uint32_t u = (uint32_t)bits << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* IEEE binary16: 1 sign, 5 exponent (bias 15), 10 fraction bits. */
+static double fp16_value(uint16_t bits) {
+    int sign = (bits >> 15) & 1;
+    int expo = (bits >> 10) & 0x1f;
+    int frac = bits & 0x3ff;
+    double v;
+    if (expo == 0) v = ldexp((double)frac, -24);                 /* subnormal: frac * 2^-24 */
+    else if (expo == 31) v = frac ? NAN : INFINITY;
+    else v = ldexp(1.0 + (double)frac / 1024.0, expo - 15);
+    return sign ? -v : v;
+}
+
+/* Round a finite non-negative binary32 to binary16, ties to even, by the definition: pick the fp16
+ * quantum for the value's binade, round the ratio to the nearest even integer. */
+static uint16_t fp16_round_nonneg(float f) {
+    double v = (double)f;
+    if (v == 0.0) return 0;
+    int e;
+    (void)frexp(v, &e);            /* v = m * 2^e, m in [0.5,1)  ->  floor(log2 v) = e-1 */
+    int binade = e - 1;
+    if (binade < -14) binade = -14; /* subnormal range shares the quantum 2^-24 */
+    double quantum = ldexp(1.0, binade - 10);
+    double n = rint(v / quantum);   /* default rounding mode: to nearest, ties to even */
+    double r = n * quantum;
+    if (r >= 65536.0) return 0x7c00; /* overflow to +inf (unreachable after saturation) */
+    if (r == 0.0) return 0;
+    (void)frexp(r, &e);
+    binade = e - 1;
+    if (binade < -14) return (uint16_t)ldexp(r, 24);             /* subnormal */
+    double frac = r / ldexp(1.0, binade) - 1.0;                  /* in [0,1) */
+    return (uint16_t)(((binade + 15) << 10) | (int)(frac * 1024.0));
+}
+
+/* exported so tests can pin the two conversions against a library's */
+double ffd_oracle_fp16_value(uint16_t bits) { return fp16_value(bits); }
+double ffd_oracle_bf16_value(uint16_t bits) { return bf16_value(bits); }
+uint16_t ffd_oracle_fp16_round(float f) { return fp16_round_nonneg(f); }
+
+static int64_t page_of(const int32_t* block_table, int b, int blk, int max_blocks) {
+    return block_table ? (int64_t)block_table[(int64_t)b * max_blocks + blk]
+                       : (int64_t)b * max_blocks + blk;
+}
+
+static int valid_rows(int seq_len, int blk, int BLK) {
+    int rows = seq_len - blk * BLK;
+    return rows > BLK ? BLK : rows;
+}
+
+/* ---- App. A.1: the quantizer ----------------------------------------------------------------- */
+
+/* One (page, KV head) tile.  For every channel c: a = max over valid rows of |K[r,c]|;
+ * s = fp16(fp32(a)/1.5f) saturated at 65504; code by comparisons against s. */
+static void quantize_tile(const uint16_t* k_tile, int rows, int BLK, int D, uint8_t* codes, uint16_t* scales) {
+    for (int c = 0; c < D; ++c) {
+        float a = 0.0f;
+        for (int r = 0; r < rows; ++r) {
+            float x = (float)fabs(bf16_value(k_tile[(int64_t)r * D + c]));
+            if (x > a) a = x;
+        }
+        float s32 = a / 1.5f;                     /* IEEE binary32 division, round to nearest */
+        if (s32 > 65504.0f) s32 = 65504.0f;
+        uint16_t sbits = fp16_round_nonneg(s32);
+        scales[c] = sbits;
+        double s = fp16_value(sbits);
+        for (int r = 0; r < BLK; ++r) {
+            uint8_t code = 0;                     /* padding rows: don't-care, written as 0 */
+            if (r < rows) {
+                double x = bf16_value(k_tile[(int64_t)r * D + c]);
+                int neg = x < 0.0;                /* -0.0 is not negative */
+                int big = fabs(x) >= s;
+                code = neg ? (big ? 0 : 1) : (big ? 3 : 2);
+            }
+            codes[(int64_t)r * D + c] = code;
+        }
+    }
+}
+
+/* Quantize every logical block of every sequence that holds at least one valid token. */
+int ffd_oracle_quantize(const uint16_t* k_cache, uint8_t* codes, uint16_t* scales, const int32_t* block_table,
+                        const int32_t* seq_lens, int B, int Hkv, int D, int BLK, int max_blocks, int num_pages) {
+    for (int b = 0; b < B; ++b) {
+        int nb = (seq_lens[b] + BLK - 1) / BLK;
+        if (nb > max_blocks) return 2;
+        for (int blk = 0; blk < nb; ++blk) {
+            int64_t page = page_of(block_table, b, blk, max_blocks);
+            if (page < 0 || page >= num_pages) return 3;
+            int rows = valid_rows(seq_lens[b], blk, BLK);
+            for (int g = 0; g < Hkv; ++g) {
+                int64_t tile = page * Hkv + g;
+                quantize_tile(k_cache + tile * BLK * D, rows, BLK, D, codes + tile * BLK * D, scales + tile * D);
+            }
+        }
+    }
+    return 0;
+}
+
+/* ---- Alg. 1 for one (sequence, query head) ---------------------------------------------------- */
+
+typedef struct {
+    const uint16_t *q, *k_cache, *v_cache, *scales;
+    const uint8_t* codes;
+    const int32_t *block_table, *seq_lens;
+    int B, Hq, Hkv, D, BLK, max_blocks, num_pages, n_sink, n_local;
+    double sm_scale, delta;
+    const uint8_t* forced_mask; /* nullable [B,Hq,max_blocks]: use these decisions instead of top-delta */
+    double *out, *lse, *block_max, *mtilde;
+    uint8_t* kept;
+} decode_args;
+
+static void softmax_attention_over_mask(const decode_args* a, int b, int h, const uint8_t* keep, double* out,
+                                        double* lse) {
+    int D = a->D, BLK = a->BLK, g = h / (a->Hq / a->Hkv);
+    int N = a->seq_lens[b], nb = (N + BLK - 1) / BLK;
+    const uint16_t* qv = a->q + ((int64_t)b * a->Hq + h) * D;
+    /* pass 1: the exact logits of kept tokens and their maximum */
+    double* s = (double*)malloc(sizeof(double) * (size_t)(nb > 0 ? nb : 1) * BLK);
+    double M = -INFINITY;
+    for (int blk = 0; blk < nb; ++blk) {
+        if (!keep[blk]) continue;
+        int64_t tile = page_of(a->block_table, b, blk, a->max_blocks) * a->Hkv + g;
+        int rows = valid_rows(N, blk, BLK);
+        for (int r = 0; r < rows; ++r) {
+            double dot = 0.0;
+            for (int c = 0; c < D; ++c) dot += bf16_value(qv[c]) * bf16_value(a->k_cache[(tile * BLK + r) * D + c]);
+            s[blk * BLK + r] = a->sm_scale * dot;
+            if (s[blk * BLK + r] > M) M = s[blk * BLK + r];
+        }
+    }
+    /* pass 2: softmax weights and the weighted sum of V */
+    double L = 0.0;
+    for (int c = 0; c < D; ++c) out[c] = 0.0;
+    for (int blk = 0; blk < nb; ++blk) {
+        if (!keep[blk]) continue;
+        int64_t tile = page_of(a->block_table, b, blk, a->max_blocks) * a->Hkv + g;
+        int rows = valid_rows(N, blk, BLK);
+        for (int r = 0; r < rows; ++r) {
+            double p = exp(s[blk * BLK + r] - M);
+            L += p;
+            for (int c = 0; c < D; ++c) out[c] += p * bf16_value(a->v_cache[(tile * BLK + r) * D + c]);
+        }
+    }
+    if (L > 0.0) {
+        for (int c = 0; c < D; ++c) out[c] /= L;
+        *lse = M + log(L);
+    } else {
+        *lse = -INFINITY; /* empty sequence: zeros */
+    }
+    free(s);
+}
+
+static void decode_one(const decode_args* a, int b, int h) {
+    int D = a->D, BLK = a->BLK, g = h / (a->Hq / a->Hkv);
+    int N = a->seq_lens[b], nb = (N + BLK - 1) / BLK;
+    const uint16_t* qv = a->q + ((int64_t)b * a->Hq + h) * D;
+    int64_t row = ((int64_t)b * a->Hq + h);
+    double* bm = a->block_max + row * a->max_blocks;
+    uint8_t* keep = a->kept + row * a->max_blocks;
+
+    /* approximate scores from the dequantized 2-bit keys; per-block maximum */
+    for (int blk = 0; blk < nb; ++blk) {
+        int64_t tile = page_of(a->block_table, b, blk, a->max_blocks) * a->Hkv + g;
+        int rows = valid_rows(N, blk, BLK);
+        double best = -INFINITY;
+        for (int r = 0; r < rows; ++r) {
+            double dot = 0.0;
+            for (int c = 0; c < D; ++c) {
+                double khat = ((double)a->codes[(tile * BLK + r) * D + c] - 1.5) * fp16_value(a->scales[tile * D + c]);
+                dot += bf16_value(qv[c]) * khat;
+            }
+            double s_approx = a->sm_scale * dot;
+            if (s_approx > best) best = s_approx;
+        }
+        bm[blk] = best;
+    }
+    /* pseudo-max over the sink and local blocks */
+    double mt = -INFINITY;
+    for (int blk = 0; blk < nb; ++blk)
+        if (blk < a->n_sink || blk >= nb - a->n_local)
+            if (bm[blk] > mt) mt = bm[blk];
+    a->mtilde[row] = mt;
+    /* top-delta test */
+    for (int blk = 0; blk < nb; ++blk) {
+        if (a->forced_mask) keep[blk] = a->forced_mask[row * a->max_blocks + blk];
+        else keep[blk] = isinf(a->delta) ? 1 : (bm[blk] >= mt - a->delta);
+    }
+    /* exact attention over the kept blocks */
+    softmax_attention_over_mask(a, b, h, keep, a->out + row * D, a->lse + row);
+}
+
+static int check_geometry(const decode_args* a) {
+    if (a->Hq % a->Hkv) return 1;
+    for (int b = 0; b < a->B; ++b) {
+        int nb = (a->seq_lens[b] + a->BLK - 1) / a->BLK;
+        if (a->seq_lens[b] < 0 || nb > a->max_blocks) return 2;
+        for (int blk = 0; blk < nb; ++blk) {
+            int64_t page = page_of(a->block_table, b, blk, a->max_blocks);
+            if (page < 0 || page >= a->num_pages) return 3;
+        }
+    }
+    return 0;
+}
+
+/* Sparse decode step.  Rows of kept / block_max beyond a sequence's block count are left untouched.
+ * units: nullable list of n_units (b, h) pairs to compute; NULL = all B*Hq pairs. */
+int ffd_oracle_decode(const uint16_t* q, const uint16_t* k_cache, const uint16_t* v_cache, const uint8_t* codes,
+                      const uint16_t* scales, const int32_t* block_table, const int32_t* seq_lens, int B, int Hq,
+                      int Hkv, int D, int BLK, int max_blocks, int num_pages, int n_sink, int n_local,
+                      double sm_scale, double delta, const uint8_t* forced_mask, const int32_t* units, int n_units,
+                      double* out, double* lse, uint8_t* kept, double* block_max, double* mtilde) {
+    decode_args a = {q, k_cache, v_cache, scales, codes, block_table, seq_lens, B, Hq, Hkv, D, BLK, max_blocks,
+                     num_pages, n_sink, n_local, sm_scale, delta, forced_mask, out, lse, block_max, mtilde, kept};
+    int rc = check_geometry(&a);
+    if (rc) return rc;
+    if (isnan(delta) || delta < 0.0) return 4;
+    int total = units ? n_units : B * Hq;
+#pragma omp parallel for schedule(dynamic, 1) num_threads(g_threads)
+    for (int u = 0; u < total; ++u) {
+        int b = units ? units[2 * u] : u / Hq;
+        int h = units ? units[2 * u + 1] : u % Hq;
+        decode_one(&a, b, h);
+    }
+    return 0;
+}
+
+/* Dense softmax attention over every valid token: softmax(q K^T / sqrt(d)) V. */
+int ffd_oracle_dense(const uint16_t* q, const uint16_t* k_cache, const uint16_t* v_cache, const int32_t* block_table,
+                     const int32_t* seq_lens, int B, int Hq, int Hkv, int D, int BLK, int max_blocks, int num_pages,
+                     double sm_scale, const int32_t* units, int n_units, double* out, double* lse) {
+    decode_args a = {q, k_cache, v_cache, NULL, NULL, block_table, seq_lens, B, Hq, Hkv, D, BLK, max_blocks,
+                     num_pages, 0, 0, sm_scale, INFINITY, NULL, out, lse, NULL, NULL, NULL};
+    int rc = check_geometry(&a);
+    if (rc) return rc;
+    int total = units ? n_units : B * Hq;
+#pragma omp parallel for schedule(dynamic, 1) num_threads(g_threads)
+    for (int u = 0; u < total; ++u) {
+        int b = units ? units[2 * u] : u / Hq;
+        int h = units ? units[2 * u + 1] : u % Hq;
+        uint8_t* all = (uint8_t*)malloc((size_t)(max_blocks > 0 ? max_blocks : 1));
+        memset(all, 1, (size_t)(max_blocks > 0 ? max_blocks : 1));
+        int64_t row = (int64_t)b * Hq + h;
+        softmax_attention_over_mask(&a, b, h, all, out + row * D, lse + row);
+        free(all);
+    }
+    return 0;
+}

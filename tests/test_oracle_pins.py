@@ -1,0 +1,474 @@
+"""Pins for the CPU oracle: it is checked against what the paper and the mathematics fix, never against itself.
+
+Each test names the passage it pins.  None of them needs a GPU.
+"""
+import json
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_00097_b200.workloads import make_workload, repage
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+CODEBOOK = np.array([-1.5, -0.5, 0.5, 1.5])   # App. A.1, printed
+INF = float("inf")
+
+
+def bf16_bits(x):
+    """float array -> bf16 bit patterns (values must already be bf16-representable or are rounded by torch)."""
+    t = torch.as_tensor(np.asarray(x, dtype=np.float32)).to(torch.bfloat16)
+    return t.view(torch.int16).numpy().view(np.uint16)
+
+
+def bits_to_f64(bits):
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+# ---------------------------------------------------------------------------------------------------------
+# number formats: pinned to numpy's IEEE conversions
+# ---------------------------------------------------------------------------------------------------------
+
+def test_fp16_decode_matches_numpy_exhaustively(oracle):
+    bits = np.arange(65536, dtype=np.uint16)
+    want = bits.view(np.float16).astype(np.float64)
+    got = np.array([oracle.fp16_value(int(b)) for b in bits])
+    both_nan = np.isnan(want) & np.isnan(got)
+    assert np.all((want == got) | both_nan)
+    assert math.copysign(1.0, oracle.fp16_value(0x8000)) == -1.0
+
+
+def test_fp16_rounding_matches_numpy(oracle):
+    rng = np.random.default_rng(5)
+    xs = np.concatenate([
+        np.abs(rng.standard_normal(20000)).astype(np.float32) * np.float32(3.0),
+        (10.0 ** rng.uniform(-9, 4.8, 20000)).astype(np.float32),
+        np.arange(0, 2048, dtype=np.float32) * np.float32(2.0 ** -25),          # subnormal ties
+        np.array([0.0, 65504.0, 65503.9, 2.0 ** -24, 2.0 ** -25, 1.0 + 2.0 ** -11, 1.0 + 3 * 2.0 ** -11],
+                 dtype=np.float32),
+    ])
+    xs = xs[xs <= 65504.0]
+    want = xs.astype(np.float16).view(np.uint16)
+    got = np.array([oracle.fp16_round(float(x)) for x in xs], dtype=np.uint16)
+    assert np.array_equal(want, got)
+
+
+def test_bf16_decode_matches_numpy(oracle):
+    bits = np.arange(0, 65536, 7, dtype=np.uint16)
+    want = bits_to_f64(bits)
+    got = np.array([oracle.bf16_value(int(b)) for b in bits])
+    ok = (want == got) | (np.isnan(want) & np.isnan(got))
+    assert np.all(ok)
+
+
+# ---------------------------------------------------------------------------------------------------------
+# App. A.1: quantizer
+# ---------------------------------------------------------------------------------------------------------
+
+def _one_column(values_bits):
+    """A cache of one page, one head, BLK = len(values), D = 1 holding the given bf16 column."""
+    n = len(values_bits)
+    return values_bits.reshape(1, 1, n, 1).copy(), np.array([n], dtype=np.int32)
+
+
+@pytest.mark.parametrize("absmax", [1.5, 2.71875, 0.01226806640625, 1000.0, 3.0e-5])
+def test_codes_equal_argmin_over_all_bf16_values(oracle, absmax):
+    """App. A.1: x_q = argmin_c |x/s - c| with s = max|x|/1.5, checked on every bf16 value below the maximum."""
+    allbits = np.arange(65536, dtype=np.uint16)
+    vals = bits_to_f64(allbits)
+    keep = np.isfinite(vals) & (np.abs(vals) <= absmax)
+    column = np.concatenate([allbits[keep], bf16_bits([absmax])])
+    k, seq = _one_column(column)
+    codes, scales = oracle.quantize(k, None, seq, 1)
+    x = bits_to_f64(column)
+    # printed scale rule, evaluated by numpy in the stated precisions
+    want_scale = (np.float32(absmax) / np.float32(1.5)).astype(np.float16)
+    assert scales[0, 0, 0] == want_scale.view(np.uint16)
+    s = float(want_scale)
+    dist = np.abs(x[:, None] / s - CODEBOOK[None, :])
+    order = np.sort(dist, axis=1)
+    clear = (order[:, 1] - order[:, 0]) > 1e-9
+    got = codes[0, 0, :, 0]
+    assert np.array_equal(got[clear], np.argmin(dist, axis=1)[clear])
+    # where fp64 cannot separate the two nearest levels (tiny |x|, or x next to a decision point) evaluate the
+    # arg-min in exact rational arithmetic; only exact ties are left out
+    fs = Fraction(s)
+    levels = [Fraction(-3, 2), Fraction(-1, 2), Fraction(1, 2), Fraction(3, 2)]
+    exact_ties = 0
+    for i in np.where(~clear)[0]:
+        d = [abs(Fraction(float(x[i])) / fs - c) for c in levels]
+        best = min(d)
+        winners = [j for j in range(4) if d[j] == best]
+        if len(winners) > 1:
+            exact_ties += 1
+            continue
+        assert got[i] == winners[0], (x[i], got[i], winners)
+    assert exact_ties <= 6                                       # x in {+-0, +-s} (and nothing else)
+    # the stated tie rule: |x| = s goes to the outer level, +-0 to +0.5
+    ties = {s: 3, -s: 0, 0.0: 2}
+    for v, c in ties.items():
+        idx = np.where(x == v)[0]                               # +-s is present only when s is a bf16 value
+        assert len(idx) > 0 or v != 0.0
+        assert np.all(got[idx] == c), (v, got[idx])
+    negzero = np.where(column == 0x8000)[0]
+    assert np.all(got[negzero] == 2)
+
+
+def test_quantizer_roundtrip_bound_and_extremes(oracle):
+    """Mid-rise grid: every reconstruction is a non-zero level times s; |x - x_hat| <= s/2 up to the fp16
+    rounding of s (bound s*(0.5 + 1.5*2^-10)); the absmax element maps to +-1.5 s."""
+    w = make_workload("C1", N=1024, tail=13)
+    codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
+    K = bits_to_f64(w.bits("k_cache"))
+    S = scales.view(np.float16).astype(np.float64)[:, :, None, :]
+    nb = w.num_blocks(0)
+    for blk in range(nb):
+        rows = min(64, int(w.seq_lens[0]) - 64 * blk)
+        k = K[blk, :, :rows]
+        c = codes[blk, :, :rows]
+        s = S[blk]
+        a = np.abs(k).max(axis=1, keepdims=True)
+        assert np.array_equal(scales[blk].view(np.float16),
+                              (a[:, 0].astype(np.float32) / np.float32(1.5)).astype(np.float16))
+        khat = (c.astype(np.float64) - 1.5) * s
+        assert np.all(np.abs(khat) >= 0.5 * s - 1e-12)          # zero-free grid
+        assert np.all(np.abs(k - khat) <= s * (0.5 + 1.5 * 2.0 ** -10) + 1e-12)
+        at_max = np.abs(k) == a
+        assert np.all(np.abs(khat[at_max]) == np.broadcast_to(1.5 * s, k.shape)[at_max])
+        assert np.all(np.sign(khat[k != 0]) == np.sign(k[k != 0]))
+
+
+def test_padding_rows_do_not_move_the_scale(oracle):
+    w = make_workload("C1", N=512, tail=40)
+    codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
+    k2 = w.bits("k_cache").copy()
+    last = w.num_blocks(0) - 1
+    rows = int(w.seq_lens[0]) - 64 * last
+    assert np.all(bits_to_f64(k2[last, :, rows:]) > 9000)       # the generator's poison is there
+    k2[last, :, rows:] = bf16_bits([-3.0e4])[0]
+    codes2, scales2 = oracle.quantize(k2, w.block_table, w.seq_lens, w.max_blocks)
+    assert np.array_equal(scales, scales2)
+    assert np.array_equal(codes[:, :, :rows], codes2[:, :, :rows])
+    assert scales.view(np.float16).astype(np.float64).max() < 10.0
+
+
+# ---------------------------------------------------------------------------------------------------------
+# hand-worked example (tests/golden/worked_example.json)
+# ---------------------------------------------------------------------------------------------------------
+
+@pytest.fixture(scope="module")
+def golden():
+    with open(os.path.join(HERE, "golden", "worked_example.json")) as f:
+        return json.load(f)
+
+
+def _run_golden(oracle, g, case, delta, V=None):
+    K = np.array(case["K"], dtype=np.float32)                    # [nb, BLK, D]
+    nb, BLK, D = K.shape
+    k = bf16_bits(K).reshape(nb, 1, BLK, D)
+    v = bf16_bits(np.full((nb, 1, BLK, D), 100.0) if V is None else V).reshape(nb, 1, BLK, D)
+    q = bf16_bits(np.array(case["q"], dtype=np.float32)).reshape(1, 1, D)
+    seq = np.array([nb * BLK], dtype=np.int32)
+    codes, scales = oracle.quantize(k, None, seq, nb)
+    r = oracle.decode(q, k, v, codes, scales, None, seq, nb, delta, n_sink=g["n_sink"], n_local=g["n_local"],
+                      sm_scale=g["sm_scale"])
+    return codes, scales, r
+
+
+def test_golden_case_a_codes_scores_masks(oracle, golden):
+    case = golden["case_A"]
+    codes, scales, r = _run_golden(oracle, golden, case, 3.0)
+    assert np.array_equal(codes[:, 0], np.array(case["codes"], dtype=np.uint8))
+    assert np.all(scales == case["scale_fp16_bits"])
+    assert np.array_equal(r.block_max[0, 0], np.array(case["block_max"]))
+    assert r.mtilde[0, 0] == case["mtilde"]
+    for d, want in case["kept"].items():
+        _, _, rr = _run_golden(oracle, golden, case, float(d))
+        assert list(rr.kept[0, 0]) == want, d
+
+
+def test_golden_case_a_output_is_softmax_over_kept_tokens(oracle, golden):
+    case = golden["case_A"]
+    nb, BLK, D = np.array(case["K"]).shape
+    V = np.full((nb, BLK, D), 100.0, dtype=np.float32)
+    for j, (blk, row) in enumerate(case["V_onehot_tokens"]):
+        V[blk, row] = 0.0
+        V[blk, row, j] = 1.0
+    _, _, r = _run_golden(oracle, golden, case, case["delta_for_output"], V=V)
+    w = np.exp(np.array(case["exponents"]))
+    assert np.allclose(r.out[0, 0], w / w.sum(), rtol=0, atol=1e-15)
+    assert abs(r.lse[0, 0] - (case["lse_offset"] + math.log(w.sum()))) < 1e-14
+
+
+def test_golden_case_b_delta_is_a_natural_log_gap_on_scaled_scores(oracle, golden):
+    """Eq. 1-2 and the printed constants: a token exactly delta = 5 below the peak carries e^-5 of the peak's
+    weight, printed as about 0.67 % and about 1/148."""
+    case = golden["case_B"]
+    for d, want in case["kept"].items():
+        _, _, rr = _run_golden(oracle, golden, case, float(d))
+        assert list(rr.kept[0, 0]) == want, d
+        assert np.array_equal(rr.block_max[0, 0], np.array(case["block_max"]))
+    nb, BLK, D = np.array(case["K"]).shape
+    V = np.zeros((nb, BLK, D), dtype=np.float32)
+    V[tuple(case["peak_token"])][0] = 1.0
+    V[tuple(case["threshold_token"])][1] = 1.0
+    _, _, r = _run_golden(oracle, golden, case, 5.0, V=V)
+    ratio = r.out[0, 0, 1] / r.out[0, 0, 0]
+    assert abs(ratio * 100 - case["printed_ratio_percent"]) < 0.005
+    assert round(1.0 / ratio) == case["printed_ratio_inverse"]
+    assert abs(1.0 / math.exp(-7.0) - 1096) < 1.0                # the second printed constant
+
+
+# ---------------------------------------------------------------------------------------------------------
+# dense attention and delta = +inf against a library routine
+# ---------------------------------------------------------------------------------------------------------
+
+def _torch_dense(w):
+    """softmax(q K^T / sqrt(d)) V by torch's scaled_dot_product_attention in fp64 (GQA by repetition)."""
+    outs = []
+    for b in range(w.B):
+        N = int(w.seq_lens[b])
+        pages = [w.page(b, blk) for blk in range(w.num_blocks(b))]
+        K = w.k_cache[pages].double().permute(1, 0, 2, 3).reshape(w.Hkv, -1, 128)[:, :N]
+        V = w.v_cache[pages].double().permute(1, 0, 2, 3).reshape(w.Hkv, -1, 128)[:, :N]
+        K = K.repeat_interleave(w.G, dim=0)
+        V = V.repeat_interleave(w.G, dim=0)
+        q = w.q[b].double().unsqueeze(1)
+        outs.append(torch.nn.functional.scaled_dot_product_attention(q, K, V).squeeze(1))
+    return torch.stack(outs).numpy()
+
+
+@pytest.mark.parametrize("name,kw", [("C1", dict(N=1500)), ("C5", dict(B=3, lens=(300, 900)))])
+def test_dense_and_delta_inf_equal_library_softmax_attention(oracle, name, kw):
+    w = make_workload(name, **kw)
+    want = _torch_dense(w)
+    out, lse = oracle.dense(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), w.block_table, w.seq_lens,
+                            w.max_blocks)
+    assert np.abs(out - want).max() < 1e-12
+    codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
+    r = oracle.decode(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), codes, scales, w.block_table, w.seq_lens,
+                      w.max_blocks, INF)
+    assert np.abs(r.out - want).max() < 1e-12
+    assert np.abs(r.lse - lse).max() < 1e-12
+    for b in range(w.B):
+        assert np.all(r.kept[b, :, : w.num_blocks(b)] == 1)
+        assert np.all(r.kept[b, :, w.num_blocks(b):] == 0)
+
+
+# ---------------------------------------------------------------------------------------------------------
+# Alg. 1 re-derived by brute force on small inputs (numpy matrices, written from the algorithm box)
+# ---------------------------------------------------------------------------------------------------------
+
+def _brute_force(w, codes, scales, delta, n_sink, n_local):
+    B, Hq, G = w.B, w.Hq, w.G
+    out = np.zeros((B, Hq, 128))
+    kept = np.zeros((B, Hq, w.max_blocks), dtype=np.uint8)
+    mt = np.zeros((B, Hq))
+    Kc = bits_to_f64(w.bits("k_cache"))
+    Vc = bits_to_f64(w.bits("v_cache"))
+    Q = bits_to_f64(w.bits("q"))
+    S = scales.view(np.float16).astype(np.float64)
+    for b in range(B):
+        N = int(w.seq_lens[b])
+        nb = w.num_blocks(b)
+        pages = [w.page(b, i) for i in range(nb)]
+        for h in range(Hq):
+            g = h // G
+            Khat = np.concatenate([CODEBOOK[codes[p, g]] * S[p, g][None, :] for p in pages])[:N]
+            approx = Khat @ Q[b, h] / math.sqrt(128)
+            token_block = np.arange(N) // 64
+            bm = np.array([approx[token_block == i].max() for i in range(nb)])
+            S_set = [i for i in range(nb) if i < n_sink or i >= nb - n_local]
+            m = max(bm[i] for i in S_set)
+            sel = bm >= m - delta
+            kept[b, h, :nb] = sel
+            mt[b, h] = m
+            Kx = np.concatenate([Kc[p, g] for p in pages])[:N]
+            Vx = np.concatenate([Vc[p, g] for p in pages])[:N]
+            tok = sel[token_block]
+            logits = Kx[tok] @ Q[b, h] / math.sqrt(128)
+            p_ = np.exp(logits - logits.max())
+            out[b, h] = (p_ / p_.sum()) @ Vx[tok]
+    return out, kept, mt
+
+
+@pytest.mark.parametrize("delta", [0.0, 2.0, 6.0])
+def test_decode_equals_brute_force_on_small_inputs(oracle, delta):
+    w = make_workload("C5", B=3, lens=(700, 2600), variant=2)      # ragged tails, paged, GQA 4
+    codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
+    r = oracle.decode(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), codes, scales, w.block_table, w.seq_lens,
+                      w.max_blocks, delta, n_sink=1, n_local=4)
+    out, kept, mt = _brute_force(w, codes, scales, delta, 1, 4)
+    assert np.abs(r.mtilde - mt).max() < 1e-11
+    assert np.array_equal(r.kept, kept)
+    assert np.abs(r.out - out).max() < 1e-11
+
+
+# ---------------------------------------------------------------------------------------------------------
+# properties of the selection rule and of the output
+# ---------------------------------------------------------------------------------------------------------
+
+@pytest.fixture(scope="module")
+def small(oracle):
+    w = make_workload("C2", N=6000)
+    codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
+    return w, codes, scales
+
+
+def _decode(oracle, w, codes, scales, delta, **kw):
+    return oracle.decode(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), codes, scales, w.block_table,
+                         w.seq_lens, w.max_blocks, delta, **kw)
+
+
+def test_planted_needles_are_kept_and_most_blocks_are_skipped(oracle, small):
+    w, codes, scales = small
+    r = _decode(oracle, w, codes, scales, 6.0)
+    nb = w.num_blocks(0)
+    for (b, g), blocks in w.needles.items():
+        assert len(blocks) >= 2
+        for h in range(g * w.G, (g + 1) * w.G):
+            for blk in blocks:
+                assert r.kept[b, h, blk] == 1
+    assert r.kept[:, :, :nb].mean() < 0.1
+
+
+def test_mask_monotone_in_delta_nonempty_and_superset_of_global_max_rule(oracle, small):
+    """Sec. 5.2: the pseudo-max never exceeds the global approximate max, so the kept set contains the one
+    the global-max rule would keep; the block that attains the pseudo-max always passes (delta >= 0)."""
+    w, codes, scales = small
+    nb = w.num_blocks(0)
+    prev = None
+    for delta in [0.0, 1.0, 4.0, 6.0, 8.0, 30.0, INF]:
+        r = _decode(oracle, w, codes, scales, delta)
+        k = r.kept[0, :, :nb].astype(bool)
+        assert np.all(k.sum(-1) >= 1)
+        gmax = r.block_max[0, :, :nb].max(-1)
+        assert np.all(r.mtilde[0] <= gmax + 1e-15)
+        if np.isfinite(delta):
+            would = r.block_max[0, :, :nb] >= (gmax[:, None] - delta)
+            assert np.all(k | ~would)
+        if prev is not None:
+            assert np.all(k | ~prev)
+        prev = k
+    assert np.all(prev)
+    # no-sink variant: the pseudo-max underestimates and the rule falls back to keeping (almost) everything
+    w2 = make_workload("C2", N=6000, sink=False)
+    c2, s2 = oracle.quantize(w2.bits("k_cache"), None, w2.seq_lens, w2.max_blocks)
+    r2 = _decode(oracle, w2, c2, s2, 6.0)
+    assert r2.kept[0, :, :nb].mean() > 0.9
+
+
+def test_delta_zero_keeps_the_pseudo_max_block(oracle, small):
+    w, codes, scales = small
+    nb = w.num_blocks(0)
+    r = _decode(oracle, w, codes, scales, 0.0)
+    in_S = np.array([i < 1 or i >= nb - 16 for i in range(nb)])
+    for h in range(w.Hq):
+        bm = r.block_max[0, h, :nb]
+        arg = int(np.argmax(np.where(in_S, bm, -np.inf)))
+        assert r.kept[0, h, arg] == 1
+        assert bm[arg] == r.mtilde[0, h]
+
+
+def test_constant_values_give_constant_output_and_output_stays_in_range(oracle, small):
+    w, codes, scales = small
+    v2 = w.bits("v_cache").copy()
+    v2[...] = bf16_bits([0.75])[0]
+    r = oracle.decode(w.bits("q"), w.bits("k_cache"), v2, codes, scales, None, w.seq_lens, w.max_blocks, 6.0)
+    assert np.abs(r.out - 0.75).max() < 1e-12
+    r = _decode(oracle, w, codes, scales, 6.0)
+    V = bits_to_f64(w.bits("v_cache"))
+    nb = w.num_blocks(0)
+    for h in range(0, w.Hq, 5):
+        g = h // w.G
+        blocks = np.where(r.kept[0, h, :nb])[0]
+        rows = np.concatenate([V[blk, g, : min(64, 6000 - 64 * blk)] for blk in blocks])
+        assert np.all(r.out[0, h] <= rows.max(0) + 1e-12) and np.all(r.out[0, h] >= rows.min(0) - 1e-12)
+
+
+def test_sparse_lse_below_dense_lse_and_close_output(oracle, small):
+    w, codes, scales = small
+    r = _decode(oracle, w, codes, scales, 6.0)
+    out, lse = oracle.dense(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), None, w.seq_lens, w.max_blocks)
+    assert np.all(r.lse <= lse + 1e-12)
+    cos = (r.out * out).sum(-1) / np.linalg.norm(r.out, axis=-1) / np.linalg.norm(out, axis=-1)
+    assert cos.min() > 0.999                                      # Sec. 5.1 recall metric on needle data
+
+
+def test_single_kept_block_closed_form(oracle, small):
+    w, codes, scales = small
+    forced = np.zeros((1, w.Hq, w.max_blocks), dtype=np.uint8)
+    blk = 17
+    forced[:, :, blk] = 1
+    r = _decode(oracle, w, codes, scales, 6.0, forced_mask=forced)
+    K = w.k_cache[blk].double()
+    V = w.v_cache[blk].double()
+    for h in range(w.Hq):
+        g = h // w.G
+        logits = (K[g] @ w.q[0, h].double()) / math.sqrt(128)
+        want = torch.softmax(logits, 0) @ V[g]
+        assert np.abs(r.out[0, h] - want.numpy()).max() < 1e-12
+        assert abs(r.lse[0, h] - float(torch.logsumexp(logits, 0))) < 1e-12
+
+
+def test_permuting_middle_blocks_permutes_mask_and_keeps_output(oracle):
+    w = make_workload("C1", N=4096)
+    nb = w.num_blocks(0)
+    codes, scales = oracle.quantize(w.bits("k_cache"), None, w.seq_lens, w.max_blocks)
+    r = _decode(oracle, w, codes, scales, 6.0)
+    perm = np.arange(nb)
+    rng = np.random.default_rng(3)
+    mid = np.arange(1, nb - 16)
+    perm[mid] = rng.permutation(mid)
+    w2 = make_workload("C1", N=4096)
+    w2.k_cache = w.k_cache[perm].clone()
+    w2.v_cache = w.v_cache[perm].clone()
+    c2, s2 = oracle.quantize(w2.bits("k_cache"), None, w2.seq_lens, w2.max_blocks)
+    r2 = _decode(oracle, w2, c2, s2, 6.0)
+    assert np.array_equal(r2.kept[0, :, :nb], r.kept[0, :, :nb][:, perm])
+    assert np.abs(r2.out - r.out).max() < 1e-12
+
+
+def test_paged_equals_contiguous_and_poison_is_never_read(oracle):
+    w = make_workload("C1", N=3000)
+    wp = repage(w)
+    c, s = oracle.quantize(w.bits("k_cache"), None, w.seq_lens, w.max_blocks)
+    cp, sp = oracle.quantize(wp.bits("k_cache"), wp.block_table, wp.seq_lens, wp.max_blocks)
+    r = _decode(oracle, w, c, s, 6.0)
+    rp = _decode(oracle, wp, cp, sp, 6.0)
+    assert np.array_equal(r.kept, rp.kept)
+    assert np.array_equal(r.out, rp.out)
+    assert np.abs(r.out).max() < 10.0
+
+
+def test_scan_error_concentrates_as_the_theorem_says(oracle):
+    """App. B theorem, used as a soft check: with sigma = s/2 per channel (half a quantization step) and
+    alpha = |q|/sqrt(d), the frequency of |s_hat - s| >= lambda stays under 2 exp(-lambda^2 / (2 sigma^2 alpha^2))."""
+    w = make_workload("C2", N=4096, sink=False)
+    codes, scales = oracle.quantize(w.bits("k_cache"), None, w.seq_lens, w.max_blocks)
+    K = bits_to_f64(w.bits("k_cache"))[:, 0].reshape(-1, 128)
+    S = scales.view(np.float16).astype(np.float64)[:, 0]
+    Khat = (CODEBOOK[codes[:, 0]] * S[:, None, :]).reshape(-1, 128)
+    q = bits_to_f64(w.bits("q"))[0, 0]
+    err = (Khat - K) @ q / math.sqrt(128)
+    sigma = S.max() / 2
+    alpha = np.linalg.norm(q) / math.sqrt(128)
+    for lam in [1.0, 2.0, 3.0]:
+        bound = 2 * math.exp(-lam ** 2 / (2 * sigma ** 2 * alpha ** 2))
+        assert (np.abs(err) >= lam).mean() <= bound
+    assert abs(err.mean()) < 0.2
+
+
+def test_empty_sequence_and_argument_errors(oracle):
+    w = make_workload("C1", N=256)
+    codes, scales = oracle.quantize(w.bits("k_cache"), None, w.seq_lens, w.max_blocks)
+    seq0 = np.array([0], dtype=np.int32)
+    r = oracle.decode(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), codes, scales, None, seq0, w.max_blocks, 6.0)
+    assert np.all(r.out == 0) and np.all(np.isneginf(r.lse))
+    with pytest.raises(ValueError):
+        _decode(oracle, w, codes, scales, -1.0)
+    with pytest.raises(ValueError):
+        _decode(oracle, w, codes, scales, float("nan"))
