@@ -1,0 +1,142 @@
+/*
+ * ffd.h - C ABI of the B200 (sm_100a) FFD sparse decode-attention library.
+ *
+ * The library implements one decode step of "Faster Flash Decoding" (FFD) for one attention layer:
+ * keys are kept twice, as 16-bit K and as a 2-bit mid-rise "thumbnail" with per-channel scales; a step
+ * scans the thumbnails of every 64-token block, skips blocks whose best approximate score lies more than
+ * delta below a pseudo-max taken from the sink and local blocks, and runs exact softmax attention over the
+ * kept blocks only.
+ *
+ * Conventions for every entry point
+ *   - All data pointers are DEVICE pointers, 16-byte aligned, owned by the caller; `cfg` and output
+ *     size pointers are HOST pointers.  The library allocates no device memory and keeps no state.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only enqueue work;
+ *     nothing synchronizes except ffd_read_device_status.
+ *   - Host-detectable problems return a non-zero ffd_status and launch nothing.
+ *   - Layouts (row-major, innermost last), D = head_dim = 128, BLK = block_tokens = 64:
+ *       q        bf16  [batch, num_q_heads, D]
+ *       k_cache  bf16  [num_pages, num_kv_heads, BLK, D]     (v_cache the same)
+ *       k_quant  u8    [num_pages, num_kv_heads, 2048]       packed 2-bit codes, physical order below
+ *       k_scales fp16  [num_pages, num_kv_heads, D]          one scale per (page, KV head, channel)
+ *       block_table int32 [batch, max_blocks_per_seq]        logical block -> physical page;
+ *                                                            NULL = page b*max_blocks_per_seq + blk
+ *       seq_lens int32 [batch]                               tokens in each sequence (0 allowed)
+ *     Token t of sequence b lives in logical block t/64, row t%64.  Query head h uses KV head
+ *     h / (num_q_heads / num_kv_heads).
+ *   - Physical order of k_quant: a (page, head) tile is 4 groups of 16 tokens, 512 bytes each.  Inside a
+ *     group, 32 lanes own 16 bytes each: lane = 4*r + j holds 32-bit words W0..W3 for tokens r (W0, W2)
+ *     and r+8 (W1, W3) of the group.  Bits [2i+1:2i] of the low / high half of W0 (W1) hold the codes of
+ *     channels 32j+4i and 32j+4i+1; those of W2 (W3) hold channels 32j+4i+2 and 32j+4i+3 (i = 0..7).
+ *     A code c in 0..3 stands for level c - 1.5.  ffd_unpack_codes returns the canonical form.
+ */
+#ifndef FFD_H_
+#define FFD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    FFD_OK = 0,
+    FFD_ERR_NULL = 1,          /* a required pointer is NULL */
+    FFD_ERR_SHAPE = 2,         /* batch / heads / block counts out of range */
+    FFD_ERR_UNSUPPORTED = 3,   /* head_dim != 128, block_tokens != 64, quant_bits != 2, group size not 1..4 ... */
+    FFD_ERR_ALIGN = 4,         /* a device pointer is not 16-byte aligned */
+    FFD_ERR_WORKSPACE = 5,     /* workspace smaller than ffd_workspace_bytes reports */
+    FFD_ERR_DELTA = 6,         /* delta is NaN or negative */
+    FFD_ERR_CUDA = 7,          /* a CUDA runtime call failed (launch error, wrong device ...) */
+    FFD_ERR_DEVICE_STATUS = 8  /* a kernel recorded a problem in the workspace status word */
+} ffd_status;
+
+/* bits of the device status word (ffd_read_device_status) */
+#define FFD_DEV_BAD_PAGE 1u     /* a block_table entry was outside [0, num_pages); that block was skipped */
+#define FFD_DEV_BAD_SEQ_LEN 2u  /* a seq_len was negative or above max_blocks_per_seq*64; clamped */
+
+typedef struct {
+    int32_t num_q_heads;
+    int32_t num_kv_heads;
+    int32_t head_dim;        /* 128 */
+    int32_t block_tokens;    /* 64 */
+    int32_t quant_bits;      /* 2 */
+    int32_t n_sink_blocks;   /* size of the sink set S_global in blocks (>= 0) */
+    int32_t n_local_blocks;  /* size of the local set S_local in blocks, counted from the last block (>= 0);
+                                n_sink_blocks + n_local_blocks must be >= 1 */
+    float sm_scale;          /* 0 => 1/sqrt(head_dim) */
+    int32_t out_dtype;       /* 0: bf16 output, 1: fp32 output */
+} ffd_config;
+
+const char* ffd_status_string(ffd_status status);
+
+/* Bytes of device workspace ffd_decode / ffd_decode_dense need for this geometry (host call, no CUDA). */
+ffd_status ffd_workspace_bytes(const ffd_config* cfg, int32_t batch, int32_t max_blocks_per_seq, size_t* bytes);
+
+/* Zeroes the status word at the head of a freshly allocated workspace.  Call once before the first decode
+ * with that workspace (the status word is sticky across calls until ffd_read_device_status clears it). */
+ffd_status ffd_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Cache append: quantize keys to 2-bit thumbnails (App. A.1, "Symmetric Mid-rise Uniform Quantization").
+ * For every sequence b, every logical block that holds a token in [first_token[b], seq_lens[b]) is
+ * (re)quantized over its valid rows r < min(64, seq_lens[b] - 64*blk): per channel
+ *   s = fp16_rne(min(fp32(max_r |K[r,c]|) / 1.5f, 65504)),  code = x<0 ? (|x|>=s ? 0 : 1) : (|x|>=s ? 3 : 2)
+ * (the nearest level of {-1.5,-0.5,+0.5,+1.5}*s; ties go outward, +-0 to +0.5).  Codes of rows past the
+ * sequence end are unspecified.  first_token NULL means 0 (quantize everything).
+ * Writes k_quant and k_scales of the touched (page, head) tiles only.  Blocks whose block_table entry is
+ * outside [0, num_pages) are skipped; a seq_len outside [0, max_blocks_per_seq*64] is clamped.
+ */
+ffd_status ffd_quantize_keys(const ffd_config* cfg, const void* k_cache, void* k_quant, void* k_scales,
+                             const int32_t* block_table, const int32_t* seq_lens, const int32_t* first_token,
+                             int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages, void* stream);
+
+/*
+ * One sparse decode step (Alg. 1; Sec. 3.2 Eq. 1 and the pseudo-max equation; Sec. 3.3 kernel steps).
+ * Per query head h of sequence b, with sm = sm_scale and khat = (code - 1.5) * scale:
+ *   approx[t]  = sm * sum_c q[c] * khat[t,c]                      every valid token t
+ *   bm[blk]    = max of approx over the block's valid tokens
+ *   m_tilde    = max of bm over blocks blk < n_sink_blocks or blk >= nb - n_local_blocks
+ *   keep[blk]  = bm[blk] >= m_tilde - delta                        (delta = +inf keeps every block)
+ *   out        = softmax over tokens of kept blocks of (sm * q . K[t]) applied to V;  lse = log-sum-exp
+ * K and V of a block are read if any query head of the KV group keeps it; a head gives zero weight to
+ * blocks it did not keep.  seq_len 0 gives out = 0 and lse = -inf.
+ *   out       [batch, num_q_heads, D], bf16 or fp32 per cfg->out_dtype; bf16 is the rounding of the fp32 result
+ *   lse       nullable fp32 [batch, num_q_heads]
+ *   kept_mask nullable u8 [batch, num_q_heads, max_blocks_per_seq]: 0/1 for blk < nb, others untouched
+ *   block_max nullable fp32 [batch, num_q_heads, max_blocks_per_seq]: bm (same validity)
+ * delta must be >= 0 or +inf.  Arithmetic: approximate scores are fp32-accurate (tensor-core products of
+ * exact operands, fp32 accumulation); exact scores bf16 x bf16 -> fp32; P.V with P split in two bf16 pieces.
+ * Device-detected problems (bad page index, seq_len beyond max_blocks_per_seq*64) skip / clamp the
+ * offending work and set bits in the workspace status word; nothing traps.
+ */
+ffd_status ffd_decode(const ffd_config* cfg, const void* q, const void* k_cache, const void* v_cache,
+                      const void* k_quant, const void* k_scales, const int32_t* block_table,
+                      const int32_t* seq_lens, int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages,
+                      float delta, void* out, float* lse, uint8_t* kept_mask, float* block_max, void* workspace,
+                      size_t workspace_bytes, void* stream);
+
+/*
+ * Dense decode attention over every valid token (the exact baseline the paper compares against in
+ * Sec. 4.2): out = softmax(sm * q K^T) V, split over the sequence and merged.  Same layouts as ffd_decode.
+ */
+ffd_status ffd_decode_dense(const ffd_config* cfg, const void* q, const void* k_cache, const void* v_cache,
+                            const int32_t* block_table, const int32_t* seq_lens, int32_t batch,
+                            int32_t max_blocks_per_seq, int32_t num_pages, void* out, float* lse, void* workspace,
+                            size_t workspace_bytes, void* stream);
+
+/*
+ * Canonical view of the packed thumbnails (App. A.1 codebook index): codes u8 [num_pages, num_kv_heads, 64, 128]
+ * with values 0..3, level = code - 1.5.  Used to compare codes bit for bit with another implementation.
+ */
+ffd_status ffd_unpack_codes(const ffd_config* cfg, const void* k_quant, uint8_t* codes, int32_t num_pages,
+                            void* stream);
+
+/* Waits for `stream`, copies the workspace status word to *status_bits (HOST) and clears it on the device.
+ * Returns FFD_ERR_DEVICE_STATUS if any bit was set. */
+ffd_status ffd_read_device_status(void* workspace, void* stream, uint32_t* status_bits);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FFD_H_ */

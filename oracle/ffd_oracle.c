@@ -10,7 +10,8 @@
  *
  * Style: every step is the definition written out, token by token and channel by channel, in double
  * precision on the exact values of the bf16 / fp16 inputs.  No blocking, no fusion, no reordering.  The
- * only parallelism is an OpenMP loop over independent (sequence, query head) pairs.
+ * only parallelism is an OpenMP loop over independent units: (sequence, query head) pairs in the decode
+ * functions, blocks in the quantizer.
  *
  * Readings of the paper that this file fixes (each is a reading, not something the paper prints; the
  * ones marked "parity unpinned" have no independent pin):
@@ -150,10 +151,17 @@ int ffd_oracle_quantize(const uint16_t* k_cache, uint8_t* codes, uint16_t* scale
                         const int32_t* seq_lens, int B, int Hkv, int D, int BLK, int max_blocks, int num_pages) {
     for (int b = 0; b < B; ++b) {
         int nb = (seq_lens[b] + BLK - 1) / BLK;
-        if (nb > max_blocks) return 2;
+        if (seq_lens[b] < 0 || nb > max_blocks) return 2;
         for (int blk = 0; blk < nb; ++blk) {
             int64_t page = page_of(block_table, b, blk, max_blocks);
             if (page < 0 || page >= num_pages) return 3;
+        }
+    }
+    for (int b = 0; b < B; ++b) {
+        int nb = (seq_lens[b] + BLK - 1) / BLK;
+#pragma omp parallel for schedule(static) num_threads(g_threads)
+        for (int blk = 0; blk < nb; ++blk) {
+            int64_t page = page_of(block_table, b, blk, max_blocks);
             int rows = valid_rows(seq_lens[b], blk, BLK);
             for (int g = 0; g < Hkv; ++g) {
                 int64_t tile = page * Hkv + g;

@@ -1,0 +1,473 @@
+// Kernels and C-ABI host layer of the FFD sparse decode-attention library (sm_100a).
+#include <cuda_runtime.h>
+#include <math.h>
+#include <string.h>
+
+#include "../../include/ffd.h"
+#include "ffd_kernels.cuh"
+
+namespace ffd {
+
+// ---- quantize (App. A.1) ----------------------------------------------------------------------------------
+// One CTA of 128 threads per (logical block, KV head, sequence).  The K tile goes through shared memory
+// once: thread c owns channel c for the absmax / scale, then thread (mt, lane) assembles its 16 bytes of the
+// packed layout.
+struct QuantParams {
+    const __nv_bfloat16* k_cache;
+    uint8_t* k_quant;
+    __half* k_scales;
+    const int32_t* block_table;
+    const int32_t* seq_lens;
+    const int32_t* first_token;
+    int Hkv, max_blocks, num_pages;
+};
+
+__device__ __forceinline__ uint32_t quant_code(float x, float s) {
+    const bool neg = x < 0.f;
+    const bool big = fabsf(x) >= s;
+    return neg ? (big ? 0u : 1u) : (big ? 3u : 2u);
+}
+
+__global__ void __launch_bounds__(128) quantize_kernel(QuantParams p) {
+    const int blk = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+    int n = p.seq_lens[b];
+    const int cap = p.max_blocks * kBlk;
+    n = n < 0 ? 0 : (n > cap ? cap : n);
+    const int nb = (n + kBlk - 1) / kBlk;
+    const int first = p.first_token ? max(p.first_token[b], 0) / kBlk : 0;
+    if (blk >= nb || blk < first) return;
+    const int page = p.block_table ? p.block_table[(size_t)b * p.max_blocks + blk] : b * p.max_blocks + blk;
+    if (page < 0 || page >= p.num_pages) return;
+    const int rows = min(kBlk, n - blk * kBlk);
+    const size_t tile = (size_t)page * p.Hkv + g;
+
+    __shared__ __align__(16) __nv_bfloat16 sk[kBlk * kD];
+    __shared__ float ss[kD];
+    const uint4* src = reinterpret_cast<const uint4*>(p.k_cache + tile * kBlk * kD);
+    uint4* dst = reinterpret_cast<uint4*>(sk);
+    const int tid = threadIdx.x;
+#pragma unroll
+    for (int x = 0; x < 8; ++x) dst[tid + 128 * x] = ldg_stream(src + tid + 128 * x);
+    __syncthreads();
+    {
+        float a = 0.f;
+        for (int r = 0; r < rows; ++r) a = fmaxf(a, fabsf(__bfloat162float(sk[r * kD + tid])));
+        float s32 = __fdiv_rn(a, 1.5f);
+        s32 = fminf(s32, 65504.f);
+        const __half s = __float2half_rn(s32);
+        p.k_scales[tile * kD + tid] = s;
+        ss[tid] = __half2float(s);
+    }
+    __syncthreads();
+    const int mt = tid >> 5, lane = tid & 31, r = lane >> 2, j = lane & 3;
+    uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int c = 32 * j + 4 * i + u;
+            const float s = ss[c];
+            const uint32_t lo_row = quant_code(__bfloat162float(sk[(16 * mt + r) * kD + c]), s);
+            const uint32_t hi_row = quant_code(__bfloat162float(sk[(16 * mt + r + 8) * kD + c]), s);
+            const int shift = 2 * i + 16 * (u & 1);
+            w[(u >> 1) * 2 + 0] |= lo_row << shift;   // W0 / W2: token r
+            w[(u >> 1) * 2 + 1] |= hi_row << shift;   // W1 / W3: token r + 8
+        }
+    }
+    uint4* out = reinterpret_cast<uint4*>(p.k_quant + tile * kCodeBytes);
+    out[mt * 32 + lane] = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// canonical codes [pages, Hkv, 64, 128] from the packed layout
+__global__ void __launch_bounds__(128) unpack_kernel(const uint8_t* k_quant, uint8_t* codes, size_t tiles) {
+    const size_t tile = blockIdx.x;
+    if (tile >= tiles) return;
+    const int tid = threadIdx.x;
+    const int mt = tid >> 5, lane = tid & 31, r = lane >> 2, j = lane & 3;
+    const uint4 v = reinterpret_cast<const uint4*>(k_quant + tile * kCodeBytes)[mt * 32 + lane];
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint8_t* dst = codes + tile * kBlk * kD;
+    for (int i = 0; i < 8; ++i)
+        for (int u = 0; u < 4; ++u) {
+            const int c = 32 * j + 4 * i + u;
+            const int shift = 2 * i + 16 * (u & 1);
+            dst[(16 * mt + r) * kD + c] = (w[(u >> 1) * 2 + 0] >> shift) & 3u;
+            dst[(16 * mt + r + 8) * kD + c] = (w[(u >> 1) * 2 + 1] >> shift) & 3u;
+        }
+}
+
+// ---- pseudo-max (Sec. 3.2; Alg. 1 "Pseudo-max estimation") ------------------------------------------------
+// One CTA per (KV head, sequence): its warps scan the sink and local blocks and reduce the block maxima.
+__global__ void __launch_bounds__(kWarps * 32) pseudomax_kernel(DecodeParams p) {
+    const int g = blockIdx.x, b = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n = clamped_seq_len(p, b);
+    const int nb = (n + kBlk - 1) / kBlk;
+    const int ns = min(p.n_sink, nb);
+    const int local_begin = max(nb - p.n_local, ns);
+    const int count = ns + (nb - local_begin);
+    __shared__ float smax[kWarps][kMaxG];
+    ScanQuery sq;
+    scan_setup(sq, p.q + ((size_t)b * p.Hq + (size_t)g * p.G) * kD, p.G, lane);
+    float best = -INFINITY;
+    for (int s = warp; s < count; s += kWarps) {
+        const int blk = s < ns ? s : local_begin + (s - ns);
+        const int page = page_of(p, b, blk);
+        if (page < 0) continue;
+        const size_t tile = (size_t)page * p.Hkv + g;
+        const int rows = min(kBlk, n - blk * kBlk);
+        const float bm = scan_block(reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes),
+                                    reinterpret_cast<const uint4*>(p.k_scales + tile * kD), sq, lane, rows,
+                                    p.sm_scale);
+        best = fmaxf(best, bm);
+    }
+    if (lane < kMaxG) smax[warp][lane] = best;
+    __syncthreads();
+    if (threadIdx.x < p.G) {
+        float m = -INFINITY;
+        for (int w = 0; w < kWarps; ++w) m = fmaxf(m, smax[w][threadIdx.x]);
+        p.mtilde[(size_t)b * p.Hq + g * p.G + threadIdx.x] = m;
+    }
+}
+
+// ---- fused scan -> select -> attend over one split of one (sequence, KV head) ---------------------------
+template <bool SPARSE>
+__global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(DecodeParams p) {
+    const int split = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r = lane >> 2, j = lane & 3;
+    const int n = clamped_seq_len(p, b);
+    const int nb = (n + kBlk - 1) / kBlk;
+    const int blk_begin = split * p.blocks_per_split;
+    const int blk_end = min(nb, blk_begin + p.blocks_per_split);
+
+    __shared__ int next_blk;
+    __shared__ float sm_m[kWarps][kMaxG], sm_l[kWarps][kMaxG];
+    __shared__ __align__(16) float sm_acc[kWarps][kMaxG][kD];
+    if (threadIdx.x == 0) next_blk = blk_begin;
+    __syncthreads();
+
+    const __nv_bfloat16* q_group = p.q + ((size_t)b * p.Hq + (size_t)g * p.G) * kD;
+    const size_t head0 = (size_t)b * p.Hq + (size_t)g * p.G;
+    AttendState st;
+    attend_setup(st, q_group, p.G, lane);
+    ScanQuery sq;
+    float thr = -INFINITY;
+    if (SPARSE) {
+        scan_setup(sq, q_group, p.G, lane);
+        if (j < p.G) thr = p.mtilde[head0 + j] - p.delta;   // delta = +inf -> -inf: everything passes
+    }
+    const unsigned group_mask = (1u << p.G) - 1u;
+    const float logit_scale_log2 = p.sm_scale * kLog2e;
+
+    for (;;) {
+        int blk = 0;
+        if (lane == 0) blk = atomicAdd(&next_blk, 1);
+        blk = __shfl_sync(kFull, blk, 0);
+        if (blk >= blk_end) break;
+        const int page = page_of(p, b, blk);
+        if (page < 0) continue;
+        const size_t tile = (size_t)page * p.Hkv + g;
+        const int rows = min(kBlk, n - blk * kBlk);
+        unsigned keep4 = group_mask;
+        if (SPARSE) {
+            const float bm = scan_block(reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes),
+                                        reinterpret_cast<const uint4*>(p.k_scales + tile * kD), sq, lane, rows,
+                                        p.sm_scale);
+            const bool keep = (j < p.G) && (bm >= thr);
+            keep4 = __ballot_sync(kFull, keep) & 0xFu;
+            if (r == 0 && j < p.G) {
+                const size_t o = (head0 + j) * p.max_blocks + blk;
+                if (p.kept_mask) p.kept_mask[o] = keep ? 1 : 0;
+                if (p.block_max) p.block_max[o] = bm;
+            }
+        }
+        if (keep4)
+            attend_block(st, reinterpret_cast<const uint4*>(p.k_cache + tile * kBlk * kD),
+                         reinterpret_cast<const uint4*>(p.v_cache + tile * kBlk * kD), lane, rows, keep4,
+                         logit_scale_log2);
+    }
+
+    // fold the warp's state: row sums over the 4 lanes of a row, bf16 remainder rows onto the main rows
+    float l = st.l;
+    l += __shfl_xor_sync(kFull, l, 1);
+    l += __shfl_xor_sync(kFull, l, 2);
+#pragma unroll
+    for (int nt = 0; nt < 16; ++nt) {
+        st.acc[nt][0] += __shfl_xor_sync(kFull, st.acc[nt][0], 16);
+        st.acc[nt][1] += __shfl_xor_sync(kFull, st.acc[nt][1], 16);
+    }
+    if (r < kMaxG) {
+        if (j == 0) { sm_m[warp][r] = st.m; sm_l[warp][r] = l; }
+#pragma unroll
+        for (int nt = 0; nt < 16; ++nt) {
+            sm_acc[warp][r][attend_channel(nt, 2 * j)] = st.acc[nt][0];
+            sm_acc[warp][r][attend_channel(nt, 2 * j + 1)] = st.acc[nt][1];
+        }
+    }
+    __syncthreads();
+    // merge the warps; thread t owns head t/64 and channels 2*(t%64), +1
+    const int h = threadIdx.x >> 6, c = (threadIdx.x & 63) * 2;
+    if (h < p.G) {
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) M = fmaxf(M, sm_m[w][h]);
+        float L = 0.f, a0 = 0.f, a1 = 0.f;
+        if (M != -INFINITY) {
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) {
+                const float f = exp2f(sm_m[w][h] - M);
+                L += f * sm_l[w][h];
+                a0 += f * sm_acc[w][h][c];
+                a1 += f * sm_acc[w][h][c + 1];
+            }
+        }
+        const size_t slot = (head0 + h) * p.splits + split;
+        if (c == 0) { p.part_ml[2 * slot] = M; p.part_ml[2 * slot + 1] = L; }
+        *reinterpret_cast<float2*>(p.part_acc + slot * kD + c) = make_float2(a0, a1);
+    }
+}
+
+// ---- split combine (FlashDecoding-style log-sum-exp merge) -------------------------------------------------
+__global__ void __launch_bounds__(kD) combine_kernel(DecodeParams p) {
+    const size_t head = (size_t)blockIdx.y * p.Hq + blockIdx.x;
+    const int c = threadIdx.x;
+    const float* ml = p.part_ml + head * p.splits * 2;
+    float M = -INFINITY;
+    for (int s = 0; s < p.splits; ++s)
+        if (ml[2 * s + 1] > 0.f) M = fmaxf(M, ml[2 * s]);
+    float L = 0.f, a = 0.f;
+    if (M != -INFINITY) {
+        for (int s = 0; s < p.splits; ++s) {
+            const float ls = ml[2 * s + 1];
+            if (!(ls > 0.f)) continue;
+            const float f = exp2f(ml[2 * s] - M);
+            L += f * ls;
+            a += f * p.part_acc[(head * p.splits + s) * kD + c];
+        }
+    }
+    const float o = L > 0.f ? a / L : 0.f;
+    if (p.out_fp32) reinterpret_cast<float*>(p.out)[head * kD + c] = o;
+    else reinterpret_cast<__nv_bfloat16*>(p.out)[head * kD + c] = __float2bfloat16_rn(o);
+    if (p.lse && c == 0) p.lse[head] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
+}
+
+__global__ void clear_status_kernel(uint32_t* status) { *status = 0u; }
+
+// ---- host side --------------------------------------------------------------------------------------------
+
+struct Plan {
+    int blocks_per_split, splits;
+    size_t off_mtilde, off_ml, off_acc, total;
+};
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Split geometry is a pure function of (batch, KV heads, max blocks) so that ffd_workspace_bytes and the
+// launch agree.  Aim for at least two CTAs per SM before making splits longer than 8 blocks.
+static Plan make_plan(const ffd_config* cfg, int batch, int max_blocks) {
+    Plan pl;
+    int bps = 32;
+    const long units = (long)batch * cfg->num_kv_heads;
+    while (bps > 8 && units * ((max_blocks + bps - 1) / bps) < 2 * 148) bps /= 2;
+    pl.blocks_per_split = bps;
+    pl.splits = max_blocks > 0 ? (max_blocks + bps - 1) / bps : 1;
+    const size_t heads = (size_t)batch * cfg->num_q_heads;
+    pl.off_mtilde = 256;
+    pl.off_ml = align_up(pl.off_mtilde + heads * sizeof(float), 256);
+    pl.off_acc = align_up(pl.off_ml + heads * pl.splits * 2 * sizeof(float), 256);
+    pl.total = align_up(pl.off_acc + heads * pl.splits * kD * sizeof(float), 256);
+    return pl;
+}
+
+static ffd_status check_config(const ffd_config* cfg) {
+    if (!cfg) return FFD_ERR_NULL;
+    if (cfg->head_dim != kD || cfg->block_tokens != kBlk || cfg->quant_bits != 2) return FFD_ERR_UNSUPPORTED;
+    if (cfg->num_q_heads <= 0 || cfg->num_kv_heads <= 0 || cfg->num_q_heads % cfg->num_kv_heads) return FFD_ERR_SHAPE;
+    if (cfg->num_q_heads / cfg->num_kv_heads > kMaxG) return FFD_ERR_UNSUPPORTED;
+    if (cfg->n_sink_blocks < 0 || cfg->n_local_blocks < 0 || cfg->n_sink_blocks + cfg->n_local_blocks < 1)
+        return FFD_ERR_SHAPE;
+    if (cfg->out_dtype != 0 && cfg->out_dtype != 1) return FFD_ERR_UNSUPPORTED;
+    if (!(cfg->sm_scale >= 0.f) || isinf(cfg->sm_scale)) return FFD_ERR_SHAPE;
+    return FFD_OK;
+}
+
+static bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+static ffd_status check_geometry(int batch, int max_blocks, int num_pages) {
+    if (batch <= 0 || batch > 65535 || max_blocks <= 0 || num_pages <= 0) return FFD_ERR_SHAPE;
+    if ((long)max_blocks * kBlk > 0x7fffffffL) return FFD_ERR_SHAPE;
+    return FFD_OK;
+}
+
+static ffd_status launch_status() { return cudaGetLastError() == cudaSuccess ? FFD_OK : FFD_ERR_CUDA; }
+
+static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, const void* k_cache,
+                             const void* v_cache, const void* k_quant, const void* k_scales,
+                             const int32_t* block_table, const int32_t* seq_lens, int batch, int max_blocks,
+                             int num_pages, float delta, void* out, float* lse, uint8_t* kept_mask,
+                             float* block_max, void* workspace, size_t workspace_bytes, void* stream) {
+    ffd_status st = check_config(cfg);
+    if (st) return st;
+    if (!q || !k_cache || !v_cache || !seq_lens || !out || !workspace) return FFD_ERR_NULL;
+    if (sparse && (!k_quant || !k_scales)) return FFD_ERR_NULL;
+    st = check_geometry(batch, max_blocks, num_pages);
+    if (st) return st;
+    if (cfg->num_kv_heads > 65535) return FFD_ERR_SHAPE;
+    if (sparse && (isnan(delta) || delta < 0.f)) return FFD_ERR_DELTA;
+    const void* ptrs[] = {q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, out, lse, block_max, workspace};
+    for (const void* ptr : ptrs)
+        if (ptr && misaligned(ptr)) return FFD_ERR_ALIGN;
+    const Plan pl = make_plan(cfg, batch, max_blocks);
+    if (workspace_bytes < pl.total) return FFD_ERR_WORKSPACE;
+
+    DecodeParams p;
+    memset(&p, 0, sizeof p);
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.k_cache = static_cast<const __nv_bfloat16*>(k_cache);
+    p.v_cache = static_cast<const __nv_bfloat16*>(v_cache);
+    p.k_quant = static_cast<const uint8_t*>(k_quant);
+    p.k_scales = static_cast<const __half*>(k_scales);
+    p.block_table = block_table;
+    p.seq_lens = seq_lens;
+    p.batch = batch;
+    p.Hq = cfg->num_q_heads;
+    p.Hkv = cfg->num_kv_heads;
+    p.G = p.Hq / p.Hkv;
+    p.max_blocks = max_blocks;
+    p.num_pages = num_pages;
+    p.n_sink = cfg->n_sink_blocks;
+    p.n_local = cfg->n_local_blocks;
+    p.blocks_per_split = pl.blocks_per_split;
+    p.splits = pl.splits;
+    p.sm_scale = cfg->sm_scale > 0.f ? cfg->sm_scale : 1.0f / sqrtf((float)kD);
+    p.delta = delta;
+    char* ws = static_cast<char*>(workspace);
+    p.status = reinterpret_cast<uint32_t*>(ws);
+    p.mtilde = reinterpret_cast<float*>(ws + pl.off_mtilde);
+    p.part_ml = reinterpret_cast<float*>(ws + pl.off_ml);
+    p.part_acc = reinterpret_cast<float*>(ws + pl.off_acc);
+    p.kept_mask = kept_mask;
+    p.block_max = block_max;
+    p.out = out;
+    p.lse = lse;
+    p.out_fp32 = cfg->out_dtype;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const dim3 grid(p.splits, p.Hkv, batch);
+    if (sparse) {
+        pseudomax_kernel<<<dim3(p.Hkv, batch), kWarps * 32, 0, s>>>(p);
+        decode_kernel<true><<<grid, kWarps * 32, 0, s>>>(p);
+    } else {
+        decode_kernel<false><<<grid, kWarps * 32, 0, s>>>(p);
+    }
+    combine_kernel<<<dim3(p.Hq, batch), kD, 0, s>>>(p);
+    return launch_status();
+}
+
+}  // namespace ffd
+
+using namespace ffd;
+
+extern "C" {
+
+const char* ffd_status_string(ffd_status status) {
+    switch (status) {
+        case FFD_OK: return "ok";
+        case FFD_ERR_NULL: return "required pointer is NULL";
+        case FFD_ERR_SHAPE: return "shape or count out of range";
+        case FFD_ERR_UNSUPPORTED: return "unsupported configuration (needs head_dim 128, block 64, 2 bits, group <= 4)";
+        case FFD_ERR_ALIGN: return "device pointer not 16-byte aligned";
+        case FFD_ERR_WORKSPACE: return "workspace too small";
+        case FFD_ERR_DELTA: return "delta must be >= 0 or +inf";
+        case FFD_ERR_CUDA: return "CUDA runtime error";
+        case FFD_ERR_DEVICE_STATUS: return "a kernel recorded a problem in the status word";
+    }
+    return "unknown status";
+}
+
+ffd_status ffd_workspace_bytes(const ffd_config* cfg, int32_t batch, int32_t max_blocks_per_seq, size_t* bytes) {
+    ffd_status st = check_config(cfg);
+    if (st) return st;
+    if (!bytes) return FFD_ERR_NULL;
+    st = check_geometry(batch, max_blocks_per_seq, 1);
+    if (st) return st;
+    *bytes = make_plan(cfg, batch, max_blocks_per_seq).total;
+    return FFD_OK;
+}
+
+ffd_status ffd_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+    if (!workspace) return FFD_ERR_NULL;
+    if (workspace_bytes < 256) return FFD_ERR_WORKSPACE;
+    if (misaligned(workspace)) return FFD_ERR_ALIGN;
+    clear_status_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<uint32_t*>(workspace));
+    return launch_status();
+}
+
+ffd_status ffd_quantize_keys(const ffd_config* cfg, const void* k_cache, void* k_quant, void* k_scales,
+                             const int32_t* block_table, const int32_t* seq_lens, const int32_t* first_token,
+                             int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages, void* stream) {
+    ffd_status st = check_config(cfg);
+    if (st) return st;
+    if (!k_cache || !k_quant || !k_scales || !seq_lens) return FFD_ERR_NULL;
+    st = check_geometry(batch, max_blocks_per_seq, num_pages);
+    if (st) return st;
+    if (cfg->num_kv_heads > 65535) return FFD_ERR_SHAPE;
+    const void* ptrs[] = {k_cache, k_quant, k_scales, block_table, seq_lens, first_token};
+    for (const void* ptr : ptrs)
+        if (ptr && misaligned(ptr)) return FFD_ERR_ALIGN;
+    QuantParams p{static_cast<const __nv_bfloat16*>(k_cache), static_cast<uint8_t*>(k_quant),
+                  static_cast<__half*>(k_scales), block_table, seq_lens, first_token,
+                  cfg->num_kv_heads, max_blocks_per_seq, num_pages};
+    quantize_kernel<<<dim3(max_blocks_per_seq, cfg->num_kv_heads, batch), 128, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    return launch_status();
+}
+
+ffd_status ffd_decode(const ffd_config* cfg, const void* q, const void* k_cache, const void* v_cache,
+                      const void* k_quant, const void* k_scales, const int32_t* block_table,
+                      const int32_t* seq_lens, int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages,
+                      float delta, void* out, float* lse, uint8_t* kept_mask, float* block_max, void* workspace,
+                      size_t workspace_bytes, void* stream) {
+    return run_decode(true, cfg, q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, batch,
+                      max_blocks_per_seq, num_pages, delta, out, lse, kept_mask, block_max, workspace,
+                      workspace_bytes, stream);
+}
+
+ffd_status ffd_decode_dense(const ffd_config* cfg, const void* q, const void* k_cache, const void* v_cache,
+                            const int32_t* block_table, const int32_t* seq_lens, int32_t batch,
+                            int32_t max_blocks_per_seq, int32_t num_pages, void* out, float* lse, void* workspace,
+                            size_t workspace_bytes, void* stream) {
+    return run_decode(false, cfg, q, k_cache, v_cache, nullptr, nullptr, block_table, seq_lens, batch,
+                      max_blocks_per_seq, num_pages, INFINITY, out, lse, nullptr, nullptr, workspace,
+                      workspace_bytes, stream);
+}
+
+ffd_status ffd_unpack_codes(const ffd_config* cfg, const void* k_quant, uint8_t* codes, int32_t num_pages,
+                            void* stream) {
+    ffd_status st = check_config(cfg);
+    if (st) return st;
+    if (!k_quant || !codes) return FFD_ERR_NULL;
+    if (num_pages <= 0) return FFD_ERR_SHAPE;
+    if (misaligned(k_quant) || misaligned(codes)) return FFD_ERR_ALIGN;
+    const size_t tiles = (size_t)num_pages * cfg->num_kv_heads;
+    if (tiles > 0x7fffffffu) return FFD_ERR_SHAPE;
+    unpack_kernel<<<(unsigned)tiles, 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint8_t*>(k_quant), codes, tiles);
+    return launch_status();
+}
+
+ffd_status ffd_read_device_status(void* workspace, void* stream, uint32_t* status_bits) {
+    if (!workspace || !status_bits) return FFD_ERR_NULL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(status_bits, workspace, sizeof(uint32_t), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return FFD_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return FFD_ERR_CUDA;
+    if (*status_bits) {
+        clear_status_kernel<<<1, 1, 0, s>>>(static_cast<uint32_t*>(workspace));
+        if (cudaGetLastError() != cudaSuccess) return FFD_ERR_CUDA;
+        return FFD_ERR_DEVICE_STATUS;
+    }
+    return FFD_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,326 @@
+// Device code of the FFD sparse decode-attention path for sm_100a.
+//
+// Work unit: one (sequence b, KV head g) pair owns the G <= 4 query heads of its GQA group; its cache is a
+// list of 64-token blocks, each a contiguous 16 KB K tile, 16 KB V tile, 2 KB of packed 2-bit codes and
+// 256 B of fp16 scales.  One warp processes one block at a time:
+//   scan   : 2-bit codes -> fp16 subnormal integers (one AND per register), per-block B operand
+//            q*scale split in two fp16 pieces, 40 mma.sync.m16n8k16 (tokens x (head,piece) x channels)
+//   select : block max per head vs (m_tilde - delta)                                   (Eq. 1, Alg. 1)
+//   attend : S^T = Q K^T and O = P V with mma.sync bf16, online softmax in registers   (Alg. 1 refinement)
+// A CTA merges its warps' partial (m, l, acc) in shared memory; a combine kernel merges the splits.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+
+namespace ffd {
+
+constexpr int kD = 128;            // head_dim
+constexpr int kBlk = 64;           // tokens per block
+constexpr int kTileBytes = kBlk * kD * 2;
+constexpr int kCodeBytes = kBlk * kD / 4;
+constexpr int kWarps = 8;          // warps per decode CTA
+constexpr int kMaxG = 4;           // query heads per KV head handled by one warp
+constexpr unsigned kFull = 0xffffffffu;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+constexpr uint32_t kDevBadPage = 1u;
+constexpr uint32_t kDevBadSeqLen = 2u;
+
+struct DecodeParams {
+    const __nv_bfloat16* q;
+    const __nv_bfloat16* k_cache;
+    const __nv_bfloat16* v_cache;
+    const uint8_t* k_quant;
+    const __half* k_scales;
+    const int32_t* block_table;
+    const int32_t* seq_lens;
+    int batch, Hq, Hkv, G, max_blocks, num_pages;
+    int n_sink, n_local;
+    int blocks_per_split, splits;
+    float sm_scale;          // logit scale
+    float delta;             // +inf allowed
+    uint32_t* status;        // workspace status word
+    float* mtilde;           // [B, Hq]   (workspace)
+    float* part_ml;          // [B, Hq, S, 2]   m (log2 domain), l
+    float* part_acc;         // [B, Hq, S, 128]
+    uint8_t* kept_mask;      // nullable [B, Hq, max_blocks]
+    float* block_max;        // nullable [B, Hq, max_blocks]
+    void* out;               // [B, Hq, 128] bf16 or fp32
+    float* lse;              // nullable [B, Hq]
+    int out_fp32;
+};
+
+// ---- small helpers --------------------------------------------------------------------------------------
+
+__device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                        uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// rows 8..15 of A are zero and rows 8..15 of the result are never used
+__device__ __forceinline__ void mma_bf16_top(float& c0, float& c1, uint32_t a0, uint32_t a2, uint32_t b0,
+                                             uint32_t b1) {
+    float z0 = 0.f, z1 = 0.f;
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+        : "+f"(c0), "+f"(c1), "+f"(z0), "+f"(z1)
+        : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
+
+// physical page of logical block `blk`; returns -1 (and flags) when the table entry is out of range
+__device__ __forceinline__ int page_of(const DecodeParams& p, int b, int blk) {
+    int page = p.block_table ? p.block_table[(size_t)b * p.max_blocks + blk] : b * p.max_blocks + blk;
+    if (page < 0 || page >= p.num_pages) {
+        atomicOr(p.status, kDevBadPage);
+        return -1;
+    }
+    return page;
+}
+
+__device__ __forceinline__ int clamped_seq_len(const DecodeParams& p, int b) {
+    int n = p.seq_lens[b];
+    int cap = p.max_blocks * kBlk;
+    if (n < 0 || n > cap) {
+        atomicOr(p.status, kDevBadSeqLen);
+        n = n < 0 ? 0 : cap;
+    }
+    return n;
+}
+
+// ---- scan: approximate scores of one block from its 2-bit codes -----------------------------------------
+//
+// MMA shape: M = 16 tokens, N = 8 = 4 heads x {hi, lo} piece of q*scale, K = 16 channels.
+// Lane = 4*r + j.  As a B-fragment owner the lane serves column n = lane/4 = 2*head + piece and the 32
+// channels 32j..32j+31; k-step i (0..7) uses channels 32j+4i..32j+4i+3.
+//
+// A operand: the two code bits of a channel stay where they are in the packed word; masking them out leaves
+// the fp16 subnormal code * 4^e * 2^-24 with e = i (i < 5) or i - 5 (after a shift by 10 bits).  The factor
+// 4^e is undone by pre-scaling q with 4^(2-e); the level offset -1.5 is applied afterwards from
+// sum_c q*scale, which one extra MMA per k-step with A = 4^e * 2^-24 provides.
+//
+// B operand: v = (q * 4^(2-e)) * scale has at most 8 + 11 significant bits; hi = fp16(v) and
+// lo = fma(q, scale, -hi) represent it exactly (barring underflow), so the products are exact and only the
+// fp32 accumulation rounds.
+
+struct ScanQuery {
+    uint32_t qh[16];  // half2: q of head (lane/8), channels 32j+4i+{0,1} (qh[2i]) and +{2,3} (qh[2i+1]), pre-scaled
+    int piece;        // (lane/4) & 1
+};
+
+__device__ __forceinline__ float scan_pos_scale(int i) {
+    const int e = i < 5 ? i : i - 5;
+    return e == 0 ? 16.f : e == 1 ? 4.f : e == 2 ? 1.f : e == 3 ? 0.25f : 0.0625f;
+}
+
+__device__ __forceinline__ void scan_setup(ScanQuery& sq, const __nv_bfloat16* q_group /* [G][128] */, int G,
+                                           int lane) {
+    const int n = lane >> 2, j = lane & 3;
+    const int head = n >> 1;
+    sq.piece = n & 1;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        float v[4] = {0.f, 0.f, 0.f, 0.f};
+        if (head < G) {
+            const __nv_bfloat16* src = q_group + head * kD + 32 * j + 4 * i;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) v[u] = __bfloat162float(src[u]) * scan_pos_scale(i);
+        }
+        __half2 a = __floats2half2_rn(v[0], v[1]);
+        __half2 c = __floats2half2_rn(v[2], v[3]);
+        sq.qh[2 * i] = *reinterpret_cast<uint32_t*>(&a);
+        sq.qh[2 * i + 1] = *reinterpret_cast<uint32_t*>(&c);
+    }
+}
+
+// Returns, in every lane, the block maximum of the approximate logits (sm_scale applied) of head lane%4
+// over the first `rows` tokens of the block.
+__device__ __forceinline__ float scan_block(const uint4* __restrict__ codes_tile, const uint4* __restrict__ scales_tile,
+                                            const ScanQuery& sq, int lane, int rows, float sm_scale) {
+    const int j = lane & 3, r = lane >> 2;
+    uint4 w[4];
+#pragma unroll
+    for (int mt = 0; mt < 4; ++mt) w[mt] = ldg_stream(codes_tile + mt * 32 + lane);
+    uint32_t sc[16];
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        uint4 s = __ldg(scales_tile + 4 * j + x);
+        sc[4 * x] = s.x; sc[4 * x + 1] = s.y; sc[4 * x + 2] = s.z; sc[4 * x + 3] = s.w;
+    }
+    uint32_t bfrag[16];
+#pragma unroll
+    for (int x = 0; x < 16; ++x) {
+        __half2 qv = *reinterpret_cast<const __half2*>(&sq.qh[x]);
+        __half2 sv = *reinterpret_cast<const __half2*>(&sc[x]);
+        __half2 hi = __hmul2(qv, sv);
+        __half2 lo = __hfma2(qv, sv, __hneg2(hi));
+        __half2 pick = sq.piece ? lo : hi;
+        bfrag[x] = *reinterpret_cast<uint32_t*>(&pick);
+    }
+    float acc[4][4];
+    float off[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+        for (int x = 0; x < 4; ++x) acc[mt][x] = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int e = i < 5 ? i : i - 5;
+        const uint32_t mask = 0x00030003u << (2 * e);
+        const uint32_t one = 0x00010001u << (2 * e);
+#pragma unroll
+        for (int mt = 0; mt < 4; ++mt) {
+            uint32_t x0 = w[mt].x, x1 = w[mt].y, x2 = w[mt].z, x3 = w[mt].w;
+            if (i >= 5) { x0 >>= 10; x1 >>= 10; x2 >>= 10; x3 >>= 10; }
+            mma_f16(acc[mt], x0 & mask, x1 & mask, x2 & mask, x3 & mask, bfrag[2 * i], bfrag[2 * i + 1]);
+        }
+        mma_f16(off, one, one, one, one, bfrag[2 * i], bfrag[2 * i + 1]);
+    }
+    float best = -INFINITY;
+#pragma unroll
+    for (int mt = 0; mt < 4; ++mt) {
+        float t0 = acc[mt][0] + acc[mt][1];
+        float t1 = acc[mt][2] + acc[mt][3];
+        if (16 * mt + r < rows) best = fmaxf(best, t0);
+        if (16 * mt + r + 8 < rows) best = fmaxf(best, t1);
+    }
+    best = fmaxf(best, __shfl_xor_sync(kFull, best, 4));
+    best = fmaxf(best, __shfl_xor_sync(kFull, best, 8));
+    best = fmaxf(best, __shfl_xor_sync(kFull, best, 16));
+    // sum_c (code - 1.5) q s = 2^20 * (acc - 1.5 * off)
+    return (best - 1.5f * (off[0] + off[1])) * (1048576.0f * sm_scale);
+}
+
+// ---- attend: exact attention of one block, online softmax state in registers ------------------------------
+//
+// S^T = Q K^T : M = 16 rows (row r < 4: head r, row r + 4: the same head again, rows 8..15 zero), N = 8 tokens,
+//               K = 16 channels.  A lane (n = lane/4, j) reads 16 contiguous bytes of token n's key per load.
+// O = P V     : M = same rows (r < 4 carries the bf16 rounding of P, r + 4 the remainder), N = 8 channels,
+//               K = 16 tokens.  V rows are paired in registers with byte permutes.
+// Channel order inside the contractions is a fixed permutation chosen so that every global load is a full
+// 16-byte vector and every 32-byte sector fetched is fully used.
+
+struct AttendState {
+    uint32_t qa[16];   // A fragments of Q: qa[2s] (k = 2j..2j+1), qa[2s+1] (k = 2j+8..2j+9) of k-step s
+    float m;           // running max of row r%4 in the log2 domain (-inf when nothing seen)
+    float l;           // this lane's share of the running sum
+    float acc[16][2];  // O fragments: n-tile nt, columns 2j, 2j+1
+};
+
+__device__ __forceinline__ void attend_setup(AttendState& st, const __nv_bfloat16* q_group, int G, int lane) {
+    const int r = lane >> 2, j = lane & 3;
+    const int head = r & 3;
+#pragma unroll
+    for (int l4 = 0; l4 < 4; ++l4) {
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (head < G) v = *reinterpret_cast<const uint4*>(q_group + head * kD + 32 * l4 + 8 * j);
+        st.qa[4 * l4 + 0] = v.x; st.qa[4 * l4 + 1] = v.y; st.qa[4 * l4 + 2] = v.z; st.qa[4 * l4 + 3] = v.w;
+    }
+    st.m = -INFINITY;
+    st.l = 0.f;
+#pragma unroll
+    for (int nt = 0; nt < 16; ++nt) st.acc[nt][0] = st.acc[nt][1] = 0.f;
+}
+
+// keep4: bit h set when head h attends to this block.  rows: valid tokens in the block (1..64).
+__device__ __forceinline__ void attend_block(AttendState& st, const uint4* __restrict__ k_tile,
+                                             const uint4* __restrict__ v_tile, int lane, int rows, unsigned keep4,
+                                             float logit_scale_log2) {
+    const int r = lane >> 2, j = lane & 3;
+    const bool mine = (keep4 >> (r & 3)) & 1u;
+    float s[8][2];
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+        s[nt][0] = s[nt][1] = 0.f;
+        const uint4* src = k_tile + (8 * nt + r) * 16 + j;
+        uint4 kv[4];
+#pragma unroll
+        for (int l4 = 0; l4 < 4; ++l4) kv[l4] = ldg_stream(src + 4 * l4);
+#pragma unroll
+        for (int l4 = 0; l4 < 4; ++l4) {
+            mma_bf16_top(s[nt][0], s[nt][1], st.qa[4 * l4 + 0], st.qa[4 * l4 + 1], kv[l4].x, kv[l4].y);
+            mma_bf16_top(s[nt][0], s[nt][1], st.qa[4 * l4 + 2], st.qa[4 * l4 + 3], kv[l4].z, kv[l4].w);
+        }
+    }
+    // online softmax (log2 domain)
+    float mx = -INFINITY;
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+            const int tok = 8 * nt + 2 * j + x;
+            float t = s[nt][x] * logit_scale_log2;
+            t = (mine && tok < rows) ? t : -INFINITY;
+            s[nt][x] = t;
+            mx = fmaxf(mx, t);
+        }
+    mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 2));
+    const float m_new = fmaxf(st.m, mx);
+    const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+    const float alpha = exp2f(st.m - m_use);
+    st.m = m_new;
+    float psum = 0.f;
+    uint32_t pa[8];  // A fragments of P: pa[2kt] (tokens 16kt+2j..), pa[2kt+1] (tokens 16kt+8+2j..)
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+        float p0 = exp2f(s[nt][0] - m_use), p1 = exp2f(s[nt][1] - m_use);
+        psum += p0 + p1;
+        float h0 = bf16_round(p0), h1 = bf16_round(p1);
+        pa[nt] = (r < 4) ? pack_bf16(h0, h1) : pack_bf16(p0 - h0, p1 - h1);
+    }
+    st.l = st.l * alpha + psum;
+#pragma unroll
+    for (int nt = 0; nt < 16; ++nt) { st.acc[nt][0] *= alpha; st.acc[nt][1] *= alpha; }
+    // O += P V
+#pragma unroll
+    for (int kt = 0; kt < 4; ++kt) {
+        const int t0 = 16 * kt + 2 * j;
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+            uint4 v[4];
+#pragma unroll
+            for (int tt = 0; tt < 4; ++tt) {
+                const int tok = t0 + (tt & 1) + ((tt >> 1) << 3);
+                v[tt] = ldg_stream(v_tile + tok * 16 + hf * 8 + r);
+                if (tok >= rows) v[tt] = make_uint4(0u, 0u, 0u, 0u);   // never multiply 0 by stale memory
+            }
+            const uint32_t* x0 = reinterpret_cast<const uint32_t*>(&v[0]);
+            const uint32_t* x1 = reinterpret_cast<const uint32_t*>(&v[1]);
+            const uint32_t* x2 = reinterpret_cast<const uint32_t*>(&v[2]);
+            const uint32_t* x3 = reinterpret_cast<const uint32_t*>(&v[3]);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t b0e = __byte_perm(x0[c], x1[c], 0x5410), b1e = __byte_perm(x2[c], x3[c], 0x5410);
+                uint32_t b0o = __byte_perm(x0[c], x1[c], 0x7632), b1o = __byte_perm(x2[c], x3[c], 0x7632);
+                const int nt = 8 * hf + 2 * c;
+                mma_bf16_top(st.acc[nt][0], st.acc[nt][1], pa[2 * kt], pa[2 * kt + 1], b0e, b1e);
+                mma_bf16_top(st.acc[nt + 1][0], st.acc[nt + 1][1], pa[2 * kt], pa[2 * kt + 1], b0o, b1o);
+            }
+        }
+    }
+}
+
+// output channel of O fragment (n-tile nt, column n)
+__device__ __forceinline__ int attend_channel(int nt, int n) { return 64 * (nt >> 3) + 8 * n + (nt & 7); }
+
+}  // namespace ffd

@@ -1,0 +1,196 @@
+"""Thin ctypes binding over the C ABI declared in ``include/ffd.h``.
+
+Argument marshalling only: every step of the path runs in the CUDA library.  PyTorch supplies device memory
+and streams.  The library is loaded from ``libffd_b200.so`` next to this file; if it is missing the import of
+any entry point raises (there is no CPU fallback).
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+from dataclasses import dataclass
+
+import torch
+
+from .build import LIB_PATH
+
+FFD_OK = 0
+STATUS_NAMES = {0: "FFD_OK", 1: "FFD_ERR_NULL", 2: "FFD_ERR_SHAPE", 3: "FFD_ERR_UNSUPPORTED", 4: "FFD_ERR_ALIGN",
+                5: "FFD_ERR_WORKSPACE", 6: "FFD_ERR_DELTA", 7: "FFD_ERR_CUDA", 8: "FFD_ERR_DEVICE_STATUS"}
+DEV_BAD_PAGE = 1
+DEV_BAD_SEQ_LEN = 2
+
+EXPORTS = ["ffd_status_string", "ffd_workspace_bytes", "ffd_workspace_init", "ffd_quantize_keys", "ffd_decode",
+           "ffd_decode_dense", "ffd_unpack_codes", "ffd_read_device_status"]
+
+
+class FfdError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)} ({status_string(status)})")
+
+
+class ffd_config(ctypes.Structure):
+    _fields_ = [("num_q_heads", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+                ("block_tokens", ctypes.c_int32), ("quant_bits", ctypes.c_int32), ("n_sink_blocks", ctypes.c_int32),
+                ("n_local_blocks", ctypes.c_int32), ("sm_scale", ctypes.c_float), ("out_dtype", ctypes.c_int32)]
+
+
+@dataclass
+class Config:
+    num_q_heads: int
+    num_kv_heads: int
+    head_dim: int = 128
+    block_tokens: int = 64
+    quant_bits: int = 2
+    n_sink_blocks: int = 1
+    n_local_blocks: int = 16
+    sm_scale: float = 0.0          # 0 -> 1/sqrt(head_dim)
+    out_dtype: int = 1             # 0 bf16, 1 fp32
+
+    def c(self) -> ffd_config:
+        return ffd_config(self.num_q_heads, self.num_kv_heads, self.head_dim, self.block_tokens, self.quant_bits,
+                          self.n_sink_blocks, self.n_local_blocks, self.sm_scale, self.out_dtype)
+
+
+_lib = None
+_vp = ctypes.c_void_p
+
+
+def load_library() -> ctypes.CDLL:
+    """Load the CUDA library; fails loudly when it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_00097_b200.build` "
+                              "(there is no fallback path)")
+        lib = ctypes.CDLL(LIB_PATH)
+        cfgp = ctypes.POINTER(ffd_config)
+        i32 = ctypes.c_int32
+        lib.ffd_status_string.restype = ctypes.c_char_p
+        lib.ffd_status_string.argtypes = [ctypes.c_int]
+        lib.ffd_workspace_bytes.argtypes = [cfgp, i32, i32, ctypes.POINTER(ctypes.c_size_t)]
+        lib.ffd_workspace_init.argtypes = [_vp, ctypes.c_size_t, _vp]
+        lib.ffd_quantize_keys.argtypes = [cfgp, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, _vp]
+        lib.ffd_decode.argtypes = [cfgp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, ctypes.c_float, _vp, _vp,
+                                   _vp, _vp, _vp, ctypes.c_size_t, _vp]
+        lib.ffd_decode_dense.argtypes = [cfgp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, _vp, _vp, _vp,
+                                         ctypes.c_size_t, _vp]
+        lib.ffd_unpack_codes.argtypes = [cfgp, _vp, _vp, i32, _vp]
+        lib.ffd_read_device_status.argtypes = [_vp, _vp, ctypes.POINTER(ctypes.c_uint32)]
+        for name in EXPORTS:
+            if name != "ffd_status_string":
+                getattr(lib, name).restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return load_library().ffd_status_string(int(status)).decode()
+
+
+def _p(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(status: int, where: str):
+    if status != FFD_OK:
+        raise FfdError(status, where)
+
+
+def ffd_workspace_bytes(cfg: Config, batch: int, max_blocks_per_seq: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(load_library().ffd_workspace_bytes(ctypes.byref(cfg.c()), batch, max_blocks_per_seq, ctypes.byref(n)),
+           "ffd_workspace_bytes")
+    return int(n.value)
+
+
+def new_workspace(cfg: Config, batch: int, max_blocks_per_seq: int, device="cuda", stream=None) -> torch.Tensor:
+    """Allocate (with torch) and initialise a workspace for this geometry."""
+    ws = torch.empty(ffd_workspace_bytes(cfg, batch, max_blocks_per_seq), dtype=torch.uint8, device=device)
+    _check(load_library().ffd_workspace_init(_p(ws), ws.numel(), _stream(stream)), "ffd_workspace_init")
+    return ws
+
+
+def ffd_quantize_keys(cfg: Config, k_cache, k_quant, k_scales, block_table, seq_lens, first_token=None, *,
+                      max_blocks_per_seq: int, stream=None):
+    num_pages = k_cache.shape[0]
+    _check(load_library().ffd_quantize_keys(ctypes.byref(cfg.c()), _p(k_cache), _p(k_quant), _p(k_scales),
+                                            _p(block_table), _p(seq_lens), _p(first_token), seq_lens.numel(),
+                                            max_blocks_per_seq, num_pages, _stream(stream)), "ffd_quantize_keys")
+
+
+def ffd_decode(cfg: Config, q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, delta: float, out, *,
+               max_blocks_per_seq: int, workspace, lse=None, kept_mask=None, block_max=None, stream=None):
+    _check(load_library().ffd_decode(ctypes.byref(cfg.c()), _p(q), _p(k_cache), _p(v_cache), _p(k_quant),
+                                     _p(k_scales), _p(block_table), _p(seq_lens), q.shape[0], max_blocks_per_seq,
+                                     k_cache.shape[0], ctypes.c_float(delta), _p(out), _p(lse), _p(kept_mask),
+                                     _p(block_max), _p(workspace), workspace.numel(), _stream(stream)), "ffd_decode")
+
+
+def ffd_decode_dense(cfg: Config, q, k_cache, v_cache, block_table, seq_lens, out, *, max_blocks_per_seq: int,
+                     workspace, lse=None, stream=None):
+    _check(load_library().ffd_decode_dense(ctypes.byref(cfg.c()), _p(q), _p(k_cache), _p(v_cache), _p(block_table),
+                                           _p(seq_lens), q.shape[0], max_blocks_per_seq, k_cache.shape[0], _p(out),
+                                           _p(lse), _p(workspace), workspace.numel(), _stream(stream)),
+           "ffd_decode_dense")
+
+
+def ffd_unpack_codes(cfg: Config, k_quant, codes, stream=None):
+    _check(load_library().ffd_unpack_codes(ctypes.byref(cfg.c()), _p(k_quant), _p(codes), k_quant.shape[0],
+                                           _stream(stream)), "ffd_unpack_codes")
+
+
+def ffd_read_device_status(workspace, stream=None) -> int:
+    """Synchronises the stream; returns the status bits (0 = clean) and clears them on the device."""
+    bits = ctypes.c_uint32(0)
+    st = load_library().ffd_read_device_status(_p(workspace), _stream(stream), ctypes.byref(bits))
+    if st not in (FFD_OK, 8):
+        raise FfdError(st, "ffd_read_device_status")
+    return int(bits.value)
+
+
+class DeviceCache:
+    """Device-resident copy of a synthetic workload plus the buffers one decode step needs (test / bench helper:
+    it only allocates with torch and forwards to the entry points above)."""
+
+    def __init__(self, w, cfg: Config | None = None, device="cuda"):
+        self.w = w
+        self.cfg = cfg or Config(w.Hq, w.Hkv)
+        self.device = device
+        self.q = w.q.to(device)
+        self.k_cache = w.k_cache.to(device)
+        self.v_cache = w.v_cache.to(device)
+        self.seq_lens = torch.from_numpy(w.seq_lens).to(device)
+        self.block_table = None if w.block_table is None else torch.from_numpy(w.block_table).to(device)
+        P, Hkv = w.num_pages, w.Hkv
+        self.k_quant = torch.zeros(P, Hkv, 2048, dtype=torch.uint8, device=device)
+        self.k_scales = torch.zeros(P, Hkv, 128, dtype=torch.float16, device=device)
+        self.workspace = new_workspace(self.cfg, w.B, w.max_blocks, device)
+        odt = torch.float32 if self.cfg.out_dtype == 1 else torch.bfloat16
+        self.out = torch.zeros(w.B, w.Hq, 128, dtype=odt, device=device)
+        self.lse = torch.zeros(w.B, w.Hq, dtype=torch.float32, device=device)
+
+    def quantize(self, first_token=None):
+        ffd_quantize_keys(self.cfg, self.k_cache, self.k_quant, self.k_scales, self.block_table, self.seq_lens,
+                          first_token, max_blocks_per_seq=self.w.max_blocks)
+
+    def decode(self, delta, kept_mask=None, block_max=None):
+        ffd_decode(self.cfg, self.q, self.k_cache, self.v_cache, self.k_quant, self.k_scales, self.block_table,
+                   self.seq_lens, delta, self.out, max_blocks_per_seq=self.w.max_blocks, workspace=self.workspace,
+                   lse=self.lse, kept_mask=kept_mask, block_max=block_max)
+
+    def dense(self):
+        ffd_decode_dense(self.cfg, self.q, self.k_cache, self.v_cache, self.block_table, self.seq_lens, self.out,
+                         max_blocks_per_seq=self.w.max_blocks, workspace=self.workspace, lse=self.lse)
+
+    def canonical_codes(self):
+        codes = torch.zeros(self.w.num_pages, self.w.Hkv, 64, 128, dtype=torch.uint8, device=self.device)
+        ffd_unpack_codes(self.cfg, self.k_quant, codes)
+        return codes

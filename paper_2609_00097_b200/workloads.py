@@ -71,7 +71,7 @@ class Workload:
         return (int(self.seq_lens[b]) + BLOCK_TOKENS - 1) // BLOCK_TOKENS
 
     def bits(self, name: str) -> np.ndarray:
-        """bf16 tensor -> uint16 bit patterns (what the oracle takes)."""
+        """bf16 tensor -> uint16 bit patterns (for host-side consumers that take raw bits)."""
         return getattr(self, name).view(torch.int16).numpy().view(np.uint16)
 
 

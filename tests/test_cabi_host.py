@@ -1,0 +1,97 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports what include/ffd.h declares, and
+rejects bad arguments before touching CUDA."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2609_00097_b200 import build, ffd
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build_library()
+    return ffd.load_library()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "ffd.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ffd_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(lib):
+    names = declared_functions()
+    assert len(names) >= 8
+    for name in names:
+        assert hasattr(lib, name), name
+    assert sorted(n for n in names if not n.startswith("ffd_decode_static")) == sorted(
+        n for n in ffd.EXPORTS if n in names)
+
+
+def test_status_strings(lib):
+    for code in range(9):
+        assert len(ffd.status_string(code)) > 1
+
+
+def test_workspace_bytes_grows_with_geometry():
+    cfg = ffd.Config(32, 8)
+    a = ffd.ffd_workspace_bytes(cfg, 1, 512)
+    b = ffd.ffd_workspace_bytes(cfg, 4, 2048)
+    assert 0 < a < b
+    assert a % 256 == 0
+
+
+@pytest.mark.parametrize("field,value,status", [
+    ("head_dim", 64, 3), ("block_tokens", 32, 3), ("quant_bits", 4, 3), ("num_kv_heads", 5, 2),
+    ("num_q_heads", 64, 3), ("n_local_blocks", -1, 2), ("out_dtype", 7, 3), ("sm_scale", -1.0, 2),
+])
+def test_bad_config_is_rejected(field, value, status):
+    cfg = ffd.Config(32, 8)
+    setattr(cfg, field, value)
+    with pytest.raises(ffd.FfdError) as e:
+        ffd.ffd_workspace_bytes(cfg, 1, 16)
+    assert e.value.status == status
+
+
+def test_null_and_range_arguments_are_rejected_before_any_launch(lib):
+    cfg = ffd.Config(32, 8).c()
+    vp = ctypes.c_void_p
+    fake = vp(0x1000)            # aligned, never dereferenced: validation fails first
+    odd = vp(0x1008)
+    # NULL q
+    assert lib.ffd_decode(ctypes.byref(cfg), None, fake, fake, fake, fake, None, fake, 1, 16, 16,
+                          ctypes.c_float(6.0), fake, None, None, None, fake, 1 << 30, None) == 1
+    # negative / NaN delta
+    for d in (-1.0, float("nan")):
+        assert lib.ffd_decode(ctypes.byref(cfg), fake, fake, fake, fake, fake, None, fake, 1, 16, 16,
+                              ctypes.c_float(d), fake, None, None, None, fake, 1 << 30, None) == 6
+    # misaligned pointer
+    assert lib.ffd_decode(ctypes.byref(cfg), odd, fake, fake, fake, fake, None, fake, 1, 16, 16,
+                          ctypes.c_float(6.0), fake, None, None, None, fake, 1 << 30, None) == 4
+    # workspace too small
+    assert lib.ffd_decode(ctypes.byref(cfg), fake, fake, fake, fake, fake, None, fake, 1, 16, 16,
+                          ctypes.c_float(6.0), fake, None, None, None, fake, 16, None) == 5
+    # batch 0
+    assert lib.ffd_decode_dense(ctypes.byref(cfg), fake, fake, fake, None, fake, 0, 16, 16, fake, None, fake,
+                                1 << 30, None) == 2
+    assert lib.ffd_quantize_keys(ctypes.byref(cfg), None, fake, fake, None, fake, None, 1, 16, 16, None) == 1
+    assert lib.ffd_unpack_codes(ctypes.byref(cfg), fake, fake, 0, None) == 2
+    assert lib.ffd_read_device_status(None, None, None) == 1
+
+
+def test_oracle_and_cuda_paths_share_no_code():
+    """The oracle imports nothing from the CUDA package and the package imports nothing from the oracle."""
+    pkg = os.path.join(ROOT, "paper_2609_00097_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in text.lower(), f
+    for f in os.listdir(os.path.join(ROOT, "oracle")):
+        if f.endswith((".py", ".c")):
+            text = open(os.path.join(ROOT, "oracle", f)).read()
+            assert "paper_2609_00097_b200" not in text and "ffd.h" not in text, f
