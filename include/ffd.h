@@ -136,6 +136,14 @@ ffd_status ffd_unpack_codes(const ffd_config* cfg, const void* k_quant, uint8_t*
  * Returns FFD_ERR_DEVICE_STATUS if any bit was set. */
 ffd_status ffd_read_device_status(void* workspace, void* stream, uint32_t* status_bits);
 
+/*
+ * Measurement hook (process-wide, not thread-safe; the only state the library keeps): while both events are
+ * non-NULL, ffd_decode and ffd_decode_dense record `start` right before and `stop` right after their fused
+ * scan-select-attend kernel on the call's stream, so a benchmark can time that kernel alone.  Both are
+ * cudaEvent_t passed as void*; pass NULL, NULL to switch the hook off.  No counterpart in the paper.
+ */
+ffd_status ffd_profile_events(void* start_event, void* stop_event);
+
 #ifdef __cplusplus
 }
 #endif

@@ -111,7 +111,9 @@ class DecodeResult:
 def _units(units):
     if units is None:
         return None, 0
-    u = np.ascontiguousarray(np.asarray(units, dtype=np.int32).reshape(-1, 2))
+    # duplicates would make two threads write the same output row: keep each (b, h) once
+    u = np.unique(np.asarray(units, dtype=np.int32).reshape(-1, 2), axis=0)
+    u = np.ascontiguousarray(u)
     return u, len(u)
 
 

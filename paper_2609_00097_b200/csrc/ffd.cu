@@ -116,9 +116,10 @@ __global__ void __launch_bounds__(kWarps * 32) pseudomax_kernel(DecodeParams p) 
         if (page < 0) continue;
         const size_t tile = (size_t)page * p.Hkv + g;
         const int rows = min(kBlk, n - blk * kBlk);
-        const float bm = scan_block(reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes),
-                                    reinterpret_cast<const uint4*>(p.k_scales + tile * kD), sq, lane, rows,
-                                    p.sm_scale);
+        float band;
+        const float bm = scan_block<true>(reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes),
+                                          reinterpret_cast<const uint4*>(p.k_scales + tile * kD), sq, lane, rows,
+                                          p.sm_scale, band);
         best = fmaxf(best, bm);
     }
     if (lane < kMaxG) smax[warp][lane] = best;
@@ -171,9 +172,13 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(DecodeParams p) 
         const int rows = min(kBlk, n - blk * kBlk);
         unsigned keep4 = group_mask;
         if (SPARSE) {
-            const float bm = scan_block(reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes),
-                                        reinterpret_cast<const uint4*>(p.k_scales + tile * kD), sq, lane, rows,
-                                        p.sm_scale);
+            const uint4* codes_tile = reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes);
+            const uint4* scales_tile = reinterpret_cast<const uint4*>(p.k_scales + tile * kD);
+            float band;
+            float bm = scan_block<false>(codes_tile, scales_tile, sq, lane, rows, p.sm_scale, band);
+            // too close to call with the fast accumulation: redo the block with the arithmetic m_tilde used
+            if (__any_sync(kFull, (j < p.G) && fabsf(bm - thr) <= band))
+                bm = scan_block<true>(codes_tile, scales_tile, sq, lane, rows, p.sm_scale, band);
             const bool keep = (j < p.G) && (bm >= thr);
             keep4 = __ballot_sync(kFull, keep) & 0xFu;
             if (r == 0 && j < p.G) {
@@ -300,6 +305,8 @@ static ffd_status check_geometry(int batch, int max_blocks, int num_pages) {
     return FFD_OK;
 }
 
+static cudaEvent_t g_prof_start = nullptr, g_prof_stop = nullptr;
+
 static ffd_status launch_status() { return cudaGetLastError() == cudaSuccess ? FFD_OK : FFD_ERR_CUDA; }
 
 static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, const void* k_cache,
@@ -355,12 +362,16 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const dim3 grid(p.splits, p.Hkv, batch);
+    const bool prof = g_prof_start && g_prof_stop;
     if (sparse) {
         pseudomax_kernel<<<dim3(p.Hkv, batch), kWarps * 32, 0, s>>>(p);
+        if (prof) cudaEventRecord(g_prof_start, s);
         decode_kernel<true><<<grid, kWarps * 32, 0, s>>>(p);
     } else {
+        if (prof) cudaEventRecord(g_prof_start, s);
         decode_kernel<false><<<grid, kWarps * 32, 0, s>>>(p);
     }
+    if (prof) cudaEventRecord(g_prof_stop, s);
     combine_kernel<<<dim3(p.Hq, batch), kD, 0, s>>>(p);
     return launch_status();
 }
@@ -454,6 +465,13 @@ ffd_status ffd_unpack_codes(const ffd_config* cfg, const void* k_quant, uint8_t*
     unpack_kernel<<<(unsigned)tiles, 128, 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const uint8_t*>(k_quant), codes, tiles);
     return launch_status();
+}
+
+ffd_status ffd_profile_events(void* start_event, void* stop_event) {
+    if ((start_event == nullptr) != (stop_event == nullptr)) return FFD_ERR_NULL;
+    g_prof_start = static_cast<cudaEvent_t>(start_event);
+    g_prof_stop = static_cast<cudaEvent_t>(stop_event);
+    return FFD_OK;
 }
 
 ffd_status ffd_read_device_status(void* workspace, void* stream, uint32_t* status_bits) {

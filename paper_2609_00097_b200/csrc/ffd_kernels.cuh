@@ -25,6 +25,9 @@ constexpr unsigned kFull = 0xffffffffu;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
+// bound on the relative error of the chained tensor-core accumulation in the fast scan (measured ~2.3e-6)
+constexpr float kScanBandRel = 1.2e-5f;
+
 constexpr uint32_t kDevBadPage = 1u;
 constexpr uint32_t kDevBadSeqLen = 2u;
 
@@ -154,8 +157,16 @@ __device__ __forceinline__ void scan_setup(ScanQuery& sq, const __nv_bfloat16* q
 
 // Returns, in every lane, the block maximum of the approximate logits (sm_scale applied) of head lane%4
 // over the first `rows` tokens of the block.
+//
+// PRECISE = false chains the 8 k-steps through the tensor-core accumulator.  That accumulation truncates every
+// addend when it aligns it, which costs up to a few 1e-5 of a logit at |logit| ~ 40; `band` returns a bound on
+// that error.  PRECISE = true starts every k-step from a zero accumulator (alignment then happens at the size of
+// single products) and adds the eight partial sums with round-to-nearest fp32 adds; it is used for the
+// pseudo-max and for blocks whose fast result lands within `band` of the threshold, so that both decisions rest
+// on the same, deterministic, ~1e-5-accurate arithmetic.
+template <bool PRECISE>
 __device__ __forceinline__ float scan_block(const uint4* __restrict__ codes_tile, const uint4* __restrict__ scales_tile,
-                                            const ScanQuery& sq, int lane, int rows, float sm_scale) {
+                                            const ScanQuery& sq, int lane, int rows, float sm_scale, float& band) {
     const int j = lane & 3, r = lane >> 2;
     uint4 w[4];
 #pragma unroll
@@ -191,9 +202,23 @@ __device__ __forceinline__ float scan_block(const uint4* __restrict__ codes_tile
         for (int mt = 0; mt < 4; ++mt) {
             uint32_t x0 = w[mt].x, x1 = w[mt].y, x2 = w[mt].z, x3 = w[mt].w;
             if (i >= 5) { x0 >>= 10; x1 >>= 10; x2 >>= 10; x3 >>= 10; }
-            mma_f16(acc[mt], x0 & mask, x1 & mask, x2 & mask, x3 & mask, bfrag[2 * i], bfrag[2 * i + 1]);
+            if (PRECISE) {
+                float part[4] = {0.f, 0.f, 0.f, 0.f};
+                mma_f16(part, x0 & mask, x1 & mask, x2 & mask, x3 & mask, bfrag[2 * i], bfrag[2 * i + 1]);
+#pragma unroll
+                for (int x = 0; x < 4; ++x) acc[mt][x] += part[x];
+            } else {
+                mma_f16(acc[mt], x0 & mask, x1 & mask, x2 & mask, x3 & mask, bfrag[2 * i], bfrag[2 * i + 1]);
+            }
         }
-        mma_f16(off, one, one, one, one, bfrag[2 * i], bfrag[2 * i + 1]);
+        if (PRECISE) {
+            float part[4] = {0.f, 0.f, 0.f, 0.f};
+            mma_f16(part, one, one, one, one, bfrag[2 * i], bfrag[2 * i + 1]);
+            off[0] += part[0];
+            off[1] += part[1];
+        } else {
+            mma_f16(off, one, one, one, one, bfrag[2 * i], bfrag[2 * i + 1]);
+        }
     }
     float best = -INFINITY;
 #pragma unroll
@@ -207,7 +232,10 @@ __device__ __forceinline__ float scan_block(const uint4* __restrict__ codes_tile
     best = fmaxf(best, __shfl_xor_sync(kFull, best, 8));
     best = fmaxf(best, __shfl_xor_sync(kFull, best, 16));
     // sum_c (code - 1.5) q s = 2^20 * (acc - 1.5 * off)
-    return (best - 1.5f * (off[0] + off[1])) * (1048576.0f * sm_scale);
+    const float o = 1.5f * (off[0] + off[1]);
+    const float unit = 1048576.0f * sm_scale;
+    band = kScanBandRel * (fabsf(best) + fabsf(o)) * unit;
+    return (best - o) * unit;
 }
 
 // ---- attend: exact attention of one block, online softmax state in registers ------------------------------

@@ -22,7 +22,7 @@ DEV_BAD_PAGE = 1
 DEV_BAD_SEQ_LEN = 2
 
 EXPORTS = ["ffd_status_string", "ffd_workspace_bytes", "ffd_workspace_init", "ffd_quantize_keys", "ffd_decode",
-           "ffd_decode_dense", "ffd_unpack_codes", "ffd_read_device_status"]
+           "ffd_decode_dense", "ffd_unpack_codes", "ffd_read_device_status", "ffd_profile_events"]
 
 
 class FfdError(RuntimeError):
@@ -79,6 +79,7 @@ def load_library() -> ctypes.CDLL:
                                          ctypes.c_size_t, _vp]
         lib.ffd_unpack_codes.argtypes = [cfgp, _vp, _vp, i32, _vp]
         lib.ffd_read_device_status.argtypes = [_vp, _vp, ctypes.POINTER(ctypes.c_uint32)]
+        lib.ffd_profile_events.argtypes = [_vp, _vp]
         for name in EXPORTS:
             if name != "ffd_status_string":
                 getattr(lib, name).restype = ctypes.c_int
@@ -154,6 +155,14 @@ def ffd_read_device_status(workspace, stream=None) -> int:
     if st not in (FFD_OK, 8):
         raise FfdError(st, "ffd_read_device_status")
     return int(bits.value)
+
+
+def ffd_profile_events(start: "torch.cuda.Event | None", stop: "torch.cuda.Event | None"):
+    """Time the fused kernel alone: events must have been created with enable_timing=True and recorded once
+    (torch creates the CUDA event lazily on first record)."""
+    a = None if start is None else ctypes.c_void_p(start.cuda_event)
+    b = None if stop is None else ctypes.c_void_p(stop.cuda_event)
+    _check(load_library().ffd_profile_events(a, b), "ffd_profile_events")
 
 
 class DeviceCache:

@@ -70,7 +70,8 @@ def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None):
     for b, h in rows:
         nb = w.num_blocks(b)
         assert np.all(kept[b, h, nb:] == 255), "mask written past the sequence's blocks"
-        assert np.abs(bm[b, h, :nb] - r.block_max[b, h, :nb]).max() < 5e-5
+        # debug output: fast-scan values carry the tensor-core accumulation error (~2e-6 of the accumulator size)
+        assert np.all(np.abs(bm[b, h, :nb] - r.block_max[b, h, :nb]) < 1e-4 + 6e-6 * np.abs(r.block_max[b, h, :nb]))
         diff = kept[b, h, :nb] != r.kept[b, h, :nb]
         if diff.any():
             differs = True
@@ -111,6 +112,8 @@ SMALL = [
     ("C4", dict(N=16384), None),                            # no sink needle, recency band, m_tilde < max
     ("C5", dict(B=4, lens=(1000, 5000)), None),             # paged, per-sequence lengths, partial tails
     ("C2", dict(N=6000, sink=False), None),                 # no-sink variant: everything kept
+    ("C3", dict(N=8192, B=8), None),                        # enough units for long splits: several blocks per warp
+    ("C5", dict(B=16, lens=(2000, 4200)), None),
 ]
 
 
@@ -225,7 +228,7 @@ def test_full_size_configs_on_sampled_heads(ffd, oracle, name, kw, n_units):
     rng = np.random.default_rng(11)
     units = sorted({(int(rng.integers(w.B)), int(rng.integers(w.Hq))) for _ in range(4 * n_units)})[:n_units]
     if w.flat_heads:   # make sure both head kinds are sampled
-        units = units[: n_units - 2] + [(0, w.flat_heads[0] * w.G), (w.B - 1, 0)]
+        units = sorted(set(units[: n_units - 2] + [(0, w.flat_heads[0] * w.G), (w.B - 1, 0)]))
     # oracle quantizer on the sampled KV heads only would need a sub-cache; the GPU codes were verified bit-exact
     # on the small configs, and here the oracle runs its own quantizer over the whole cache
     codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
