@@ -54,6 +54,7 @@ typedef enum {
 /* bits of the device status word (ffd_read_device_status) */
 #define FFD_DEV_BAD_PAGE 1u     /* a block_table entry was outside [0, num_pages); that block was skipped */
 #define FFD_DEV_BAD_SEQ_LEN 2u  /* a seq_len was negative or above max_blocks_per_seq*64; clamped */
+#define FFD_DEV_TIMEOUT 4u      /* a bounded wait for an asynchronous copy ran out; that split's result is incomplete */
 
 typedef struct {
     int32_t num_q_heads;

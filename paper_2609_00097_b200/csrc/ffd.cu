@@ -5,6 +5,7 @@
 
 #include "../../include/ffd.h"
 #include "ffd_kernels.cuh"
+#include "ffd_fused.cuh"
 
 namespace ffd {
 
@@ -96,9 +97,11 @@ __global__ void __launch_bounds__(128) unpack_kernel(const uint8_t* k_quant, uin
         }
 }
 
+constexpr int kPmWarps = 8;
+
 // ---- pseudo-max (Sec. 3.2; Alg. 1 "Pseudo-max estimation") ------------------------------------------------
 // One CTA per (KV head, sequence): its warps scan the sink and local blocks and reduce the block maxima.
-__global__ void __launch_bounds__(kWarps * 32) pseudomax_kernel(DecodeParams p) {
+__global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p) {
     const int g = blockIdx.x, b = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n = clamped_seq_len(p, b);
@@ -106,34 +109,47 @@ __global__ void __launch_bounds__(kWarps * 32) pseudomax_kernel(DecodeParams p) 
     const int ns = min(p.n_sink, nb);
     const int local_begin = max(nb - p.n_local, ns);
     const int count = ns + (nb - local_begin);
-    __shared__ float smax[kWarps][kMaxG];
+    __shared__ float smax[kPmWarps][kMaxG];
     ScanQuery sq;
     scan_setup(sq, p.q + ((size_t)b * p.Hq + (size_t)g * p.G) * kD, p.G, lane);
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *p.item_counter = 0u;
+    if (warp == 0) {   // the scan warps of the fused kernel reload these per work item
+        uint4* dst = reinterpret_cast<uint4*>(p.qfrag) + ((size_t)(b * p.Hkv + g) * 32 + lane) * 4;
+#pragma unroll
+        for (int x = 0; x < 4; ++x) dst[x] = make_uint4(sq.qh[4 * x], sq.qh[4 * x + 1], sq.qh[4 * x + 2], sq.qh[4 * x + 3]);
+    }
     float best = -INFINITY;
-    for (int s = warp; s < count; s += kWarps) {
+    for (int s = warp; s < count; s += kPmWarps) {
         const int blk = s < ns ? s : local_begin + (s - ns);
         const int page = page_of(p, b, blk);
         if (page < 0) continue;
         const size_t tile = (size_t)page * p.Hkv + g;
         const int rows = min(kBlk, n - blk * kBlk);
         float band;
-        const float bm = scan_block<true>(reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes),
-                                          reinterpret_cast<const uint4*>(p.k_scales + tile * kD), sq, lane, rows,
-                                          p.sm_scale, band);
-        best = fmaxf(best, bm);
+        ScanRegs sr;
+        scan_load(sr, reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes),
+                  reinterpret_cast<const uint4*>(p.k_scales + tile * kD), lane);
+        best = fmaxf(best, scan_compute<true>(sr, sq, lane, rows, p.sm_scale, band));
     }
     if (lane < kMaxG) smax[warp][lane] = best;
     __syncthreads();
     if (threadIdx.x < p.G) {
         float m = -INFINITY;
-        for (int w = 0; w < kWarps; ++w) m = fmaxf(m, smax[w][threadIdx.x]);
+        for (int w = 0; w < kPmWarps; ++w) m = fmaxf(m, smax[w][threadIdx.x]);
         p.mtilde[(size_t)b * p.Hq + g * p.G + threadIdx.x] = m;
     }
 }
 
 // ---- fused scan -> select -> attend over one split of one (sequence, KV head) ---------------------------
+struct BlockRef {
+    int blk;        // logical block, -1 = none
+    int rows;       // valid tokens
+    size_t tile;    // (page, KV head) tile index
+};
+
 template <bool SPARSE>
 __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(DecodeParams p) {
+    extern __shared__ __align__(1024) unsigned char smem[];
     const int split = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int r = lane >> 2, j = lane & 3;
@@ -144,8 +160,16 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(DecodeParams p) 
 
     __shared__ int next_blk;
     __shared__ float sm_m[kWarps][kMaxG], sm_l[kWarps][kMaxG];
-    __shared__ __align__(16) float sm_acc[kWarps][kMaxG][kD];
+    const uint32_t kslot = smem_u32(smem) + warp * 2 * kSlotBytes;
+    const uint32_t vslot = kslot + kSlotBytes;
+    const uint32_t kbar = smem_u32(smem) + kWarps * 2 * kSlotBytes + warp * 16;
+    const uint32_t vbar = kbar + 8;
     if (threadIdx.x == 0) next_blk = blk_begin;
+    if (lane == 0) {
+        mbar_init(kbar, 32);
+        mbar_init(vbar, 32);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
     __syncthreads();
 
     const __nv_bfloat16* q_group = p.q + ((size_t)b * p.Hq + (size_t)g * p.G) * kD;
@@ -160,38 +184,81 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(DecodeParams p) 
     }
     const unsigned group_mask = (1u << p.G) - 1u;
     const float logit_scale_log2 = p.sm_scale * kLog2e;
+    const uint4* kbase = reinterpret_cast<const uint4*>(p.k_cache);
+    const uint4* vbase = reinterpret_cast<const uint4*>(p.v_cache);
+    constexpr size_t kTileVec = kTileBytes / 16;
 
-    for (;;) {
-        int blk = 0;
-        if (lane == 0) blk = atomicAdd(&next_blk, 1);
-        blk = __shfl_sync(kFull, blk, 0);
-        if (blk >= blk_end) break;
-        const int page = page_of(p, b, blk);
-        if (page < 0) continue;
-        const size_t tile = (size_t)page * p.Hkv + g;
-        const int rows = min(kBlk, n - blk * kBlk);
+    // next block of this split for this warp (skipping blocks whose page index is bad)
+    auto fetch = [&]() {
+        BlockRef ref{-1, 0, 0};
+        for (;;) {
+            int blk = 0;
+            if (lane == 0) blk = atomicAdd(&next_blk, 1);
+            blk = __shfl_sync(kFull, blk, 0);
+            if (blk >= blk_end) return ref;
+            const int page = page_of(p, b, blk);
+            if (page < 0) continue;
+            ref.blk = blk;
+            ref.rows = min(kBlk, n - blk * kBlk);
+            ref.tile = (size_t)page * p.Hkv + g;
+            return ref;
+        }
+    };
+    auto load_codes = [&](ScanRegs& sr, const BlockRef& ref) {
+        scan_load(sr, reinterpret_cast<const uint4*>(p.k_quant + ref.tile * kCodeBytes),
+                  reinterpret_cast<const uint4*>(p.k_scales + ref.tile * kD), lane);
+    };
+
+    BlockRef cur = fetch();
+    ScanRegs cur_regs;
+    if (SPARSE && cur.blk >= 0) load_codes(cur_regs, cur);
+    BlockRef pending{-1, 0, 0};     // kept block whose K/V copies are in flight
+    unsigned pending_keep = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+
+    while (cur.blk >= 0 && ok) {
+        // prefetch the next block's codes into registers before working on this one
+        const BlockRef nxt = fetch();
+        ScanRegs nxt_regs;
+        if (SPARSE && nxt.blk >= 0) load_codes(nxt_regs, nxt);
+
         unsigned keep4 = group_mask;
         if (SPARSE) {
-            const uint4* codes_tile = reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes);
-            const uint4* scales_tile = reinterpret_cast<const uint4*>(p.k_scales + tile * kD);
             float band;
-            float bm = scan_block<false>(codes_tile, scales_tile, sq, lane, rows, p.sm_scale, band);
+            float bm = scan_compute<false>(cur_regs, sq, lane, cur.rows, p.sm_scale, band);
             // too close to call with the fast accumulation: redo the block with the arithmetic m_tilde used
             if (__any_sync(kFull, (j < p.G) && fabsf(bm - thr) <= band))
-                bm = scan_block<true>(codes_tile, scales_tile, sq, lane, rows, p.sm_scale, band);
+                bm = scan_compute<true>(cur_regs, sq, lane, cur.rows, p.sm_scale, band);
             const bool keep = (j < p.G) && (bm >= thr);
             keep4 = __ballot_sync(kFull, keep) & 0xFu;
             if (r == 0 && j < p.G) {
-                const size_t o = (head0 + j) * p.max_blocks + blk;
+                const size_t o = (head0 + j) * p.max_blocks + cur.blk;
                 if (p.kept_mask) p.kept_mask[o] = keep ? 1 : 0;
                 if (p.block_max) p.block_max[o] = bm;
             }
         }
-        if (keep4)
-            attend_block(st, reinterpret_cast<const uint4*>(p.k_cache + tile * kBlk * kD),
-                         reinterpret_cast<const uint4*>(p.v_cache + tile * kBlk * kD), lane, rows, keep4,
-                         logit_scale_log2);
+        if (keep4) {
+            const uint4* ksrc = kbase + cur.tile * kTileVec;
+            const uint4* vsrc = vbase + cur.tile * kTileVec;
+            if (pending.blk >= 0) {
+                ok = attend_block(st, kslot, vslot, kbar, vbar, phase, ksrc, vsrc, lane, pending.rows, pending_keep,
+                                  logit_scale_log2);
+            } else {
+                tile_copy_async(kslot, ksrc, lane, kbar);
+                tile_copy_async(vslot, vsrc, lane, vbar);
+            }
+            pending = cur;
+            pending_keep = keep4;
+        }
+        cur = nxt;
+        if (SPARSE) cur_regs = nxt_regs;
     }
+    if (ok && pending.blk >= 0)
+        ok = attend_block(st, kslot, vslot, kbar, vbar, phase, nullptr, nullptr, lane, pending.rows, pending_keep,
+                          logit_scale_log2);
+    cp_async_drain();
+    if (!ok && lane == 0) atomicOr(p.status, kDevTimeout);
 
     // fold the warp's state: row sums over the 4 lanes of a row, bf16 remainder rows onto the main rows
     float l = st.l;
@@ -202,18 +269,20 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(DecodeParams p) 
         st.acc[nt][0] += __shfl_xor_sync(kFull, st.acc[nt][0], 16);
         st.acc[nt][1] += __shfl_xor_sync(kFull, st.acc[nt][1], 16);
     }
+    // the warp's own K slot is free now: it holds the warp's [4][128] accumulators for the merge
+    float* my_acc = reinterpret_cast<float*>(smem + (size_t)warp * 2 * kSlotBytes);
     if (r < kMaxG) {
         if (j == 0) { sm_m[warp][r] = st.m; sm_l[warp][r] = l; }
 #pragma unroll
         for (int nt = 0; nt < 16; ++nt) {
-            sm_acc[warp][r][attend_channel(nt, 2 * j)] = st.acc[nt][0];
-            sm_acc[warp][r][attend_channel(nt, 2 * j + 1)] = st.acc[nt][1];
+            my_acc[r * kD + attend_channel(nt, 2 * j)] = st.acc[nt][0];
+            my_acc[r * kD + attend_channel(nt, 2 * j + 1)] = st.acc[nt][1];
         }
     }
     __syncthreads();
-    // merge the warps; thread t owns head t/64 and channels 2*(t%64), +1
-    const int h = threadIdx.x >> 6, c = (threadIdx.x & 63) * 2;
-    if (h < p.G) {
+    // merge the warps; each work item is one head and a pair of channels
+    for (int item = threadIdx.x; item < p.G * (kD / 2); item += kWarps * 32) {
+        const int h = item / (kD / 2), c = (item % (kD / 2)) * 2;
         float M = -INFINITY;
 #pragma unroll
         for (int w = 0; w < kWarps; ++w) M = fmaxf(M, sm_m[w][h]);
@@ -222,9 +291,10 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(DecodeParams p) 
 #pragma unroll
             for (int w = 0; w < kWarps; ++w) {
                 const float f = exp2f(sm_m[w][h] - M);
+                const float* wacc = reinterpret_cast<const float*>(smem + (size_t)w * 2 * kSlotBytes) + h * kD + c;
                 L += f * sm_l[w][h];
-                a0 += f * sm_acc[w][h][c];
-                a1 += f * sm_acc[w][h][c + 1];
+                a0 += f * wacc[0];
+                a1 += f * wacc[1];
             }
         }
         const size_t slot = (head0 + h) * p.splits + split;
@@ -262,8 +332,9 @@ __global__ void clear_status_kernel(uint32_t* status) { *status = 0u; }
 // ---- host side --------------------------------------------------------------------------------------------
 
 struct Plan {
-    int blocks_per_split, splits;
-    size_t off_mtilde, off_ml, off_acc, total;
+    int blocks_per_split, splits;     // dense path
+    int total_items;                  // fused path
+    size_t off_mtilde, off_qfrag, off_ml, off_acc, off_fml, off_facc, total;
 };
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -278,10 +349,15 @@ static Plan make_plan(const ffd_config* cfg, int batch, int max_blocks) {
     pl.blocks_per_split = bps;
     pl.splits = max_blocks > 0 ? (max_blocks + bps - 1) / bps : 1;
     const size_t heads = (size_t)batch * cfg->num_q_heads;
+    pl.total_items = ((max_blocks + kItemBlocks - 1) / kItemBlocks) * batch * cfg->num_kv_heads;
+    const size_t fslots = (size_t)pl.total_items * kNA * kMaxG;
     pl.off_mtilde = 256;
-    pl.off_ml = align_up(pl.off_mtilde + heads * sizeof(float), 256);
+    pl.off_qfrag = align_up(pl.off_mtilde + heads * sizeof(float), 256);
+    pl.off_ml = align_up(pl.off_qfrag + (size_t)batch * cfg->num_kv_heads * 32 * 16 * sizeof(uint32_t), 256);
     pl.off_acc = align_up(pl.off_ml + heads * pl.splits * 2 * sizeof(float), 256);
-    pl.total = align_up(pl.off_acc + heads * pl.splits * kD * sizeof(float), 256);
+    pl.off_fml = align_up(pl.off_acc + heads * pl.splits * kD * sizeof(float), 256);
+    pl.off_facc = align_up(pl.off_fml + fslots * 2 * sizeof(float), 256);
+    pl.total = align_up(pl.off_facc + fslots * kD * sizeof(float), 256);
     return pl;
 }
 
@@ -320,7 +396,8 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
     if (sparse && (!k_quant || !k_scales)) return FFD_ERR_NULL;
     st = check_geometry(batch, max_blocks, num_pages);
     if (st) return st;
-    if (cfg->num_kv_heads > 65535) return FFD_ERR_SHAPE;
+    if (cfg->num_kv_heads > 65535 || cfg->num_q_heads > 65535) return FFD_ERR_SHAPE;
+    if ((double)num_pages * cfg->num_kv_heads >= 4294967296.0) return FFD_ERR_SHAPE;
     if (sparse && (isnan(delta) || delta < 0.f)) return FFD_ERR_DELTA;
     const void* ptrs[] = {q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, out, lse, block_max, workspace};
     for (const void* ptr : ptrs)
@@ -354,6 +431,11 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
     p.mtilde = reinterpret_cast<float*>(ws + pl.off_mtilde);
     p.part_ml = reinterpret_cast<float*>(ws + pl.off_ml);
     p.part_acc = reinterpret_cast<float*>(ws + pl.off_acc);
+    p.qfrag = reinterpret_cast<uint32_t*>(ws + pl.off_qfrag);
+    p.fpart_ml = reinterpret_cast<float*>(ws + pl.off_fml);
+    p.fpart_acc = reinterpret_cast<float*>(ws + pl.off_facc);
+    p.total_items = pl.total_items;
+    p.item_counter = reinterpret_cast<uint32_t*>(ws + 64);
     p.kept_mask = kept_mask;
     p.block_max = block_max;
     p.out = out;
@@ -364,15 +446,24 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
     const dim3 grid(p.splits, p.Hkv, batch);
     const bool prof = g_prof_start && g_prof_stop;
     if (sparse) {
-        pseudomax_kernel<<<dim3(p.Hkv, batch), kWarps * 32, 0, s>>>(p);
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            cudaFuncSetAttribute(fused_sparse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem) != cudaSuccess)
+            return FFD_ERR_CUDA;
+        pseudomax_kernel<<<dim3(p.Hkv, batch), kPmWarps * 32, 0, s>>>(p);
         if (prof) cudaEventRecord(g_prof_start, s);
-        decode_kernel<true><<<grid, kWarps * 32, 0, s>>>(p);
+        fused_sparse_kernel<<<min(p.total_items, sms), kFusedThreads, kFusedSmem, s>>>(p);
+        if (prof) cudaEventRecord(g_prof_stop, s);
+        fused_combine_kernel<<<dim3(p.Hq, batch), kD, 0, s>>>(p);
     } else {
+        if (cudaFuncSetAttribute(decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem) != cudaSuccess)
+            return FFD_ERR_CUDA;
         if (prof) cudaEventRecord(g_prof_start, s);
-        decode_kernel<false><<<grid, kWarps * 32, 0, s>>>(p);
+        decode_kernel<false><<<grid, kWarps * 32, kDecodeSmem, s>>>(p);
+        if (prof) cudaEventRecord(g_prof_stop, s);
+        combine_kernel<<<dim3(p.Hq, batch), kD, 0, s>>>(p);
     }
-    if (prof) cudaEventRecord(g_prof_stop, s);
-    combine_kernel<<<dim3(p.Hq, batch), kD, 0, s>>>(p);
     return launch_status();
 }
 

@@ -7,6 +7,10 @@
 //            q*scale split in two fp16 pieces, 40 mma.sync.m16n8k16 (tokens x (head,piece) x channels)
 //   select : block max per head vs (m_tilde - delta)                                   (Eq. 1, Alg. 1)
 //   attend : S^T = Q K^T and O = P V with mma.sync bf16, online softmax in registers   (Alg. 1 refinement)
+// Only kept blocks move their K and V: each warp owns one 16 KB K slot and one 16 KB V slot in shared memory,
+// filled by 16-byte cp.async copies into an XOR-swizzled layout and tracked by one mbarrier per slot.  The warp
+// scans one block ahead, so the next kept block's K (V) copy is issued as soon as the current block's Q K^T
+// (P V) has released the slot and overlaps the rest of the work.
 // A CTA merges its warps' partial (m, l, acc) in shared memory; a combine kernel merges the splits.
 #pragma once
 #include <cuda_bf16.h>
@@ -19,7 +23,10 @@ constexpr int kD = 128;            // head_dim
 constexpr int kBlk = 64;           // tokens per block
 constexpr int kTileBytes = kBlk * kD * 2;
 constexpr int kCodeBytes = kBlk * kD / 4;
-constexpr int kWarps = 8;          // warps per decode CTA
+constexpr int kWarps = 7;          // warps per decode CTA: 7 x (16 KB K slot + 16 KB V slot) of shared memory
+constexpr int kSlotBytes = kTileBytes;
+constexpr int kDecodeSmem = kWarps * 2 * kSlotBytes + 128;   // + mbarriers
+constexpr long long kSpinCycles = 2000000000LL;   // bounded mbarrier wait (~1 s of SM clocks); then report and stop
 constexpr int kMaxG = 4;           // query heads per KV head handled by one warp
 constexpr unsigned kFull = 0xffffffffu;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -30,6 +37,7 @@ constexpr float kScanBandRel = 1.2e-5f;
 
 constexpr uint32_t kDevBadPage = 1u;
 constexpr uint32_t kDevBadSeqLen = 2u;
+constexpr uint32_t kDevTimeout = 4u;
 
 struct DecodeParams {
     const __nv_bfloat16* q;
@@ -46,8 +54,13 @@ struct DecodeParams {
     float delta;             // +inf allowed
     uint32_t* status;        // workspace status word
     float* mtilde;           // [B, Hq]   (workspace)
-    float* part_ml;          // [B, Hq, S, 2]   m (log2 domain), l
-    float* part_acc;         // [B, Hq, S, 128]
+    float* part_ml;          // dense path: [B, Hq, S, 2]   m (log2 domain), l
+    float* part_acc;         // dense path: [B, Hq, S, 128]
+    uint32_t* qfrag;         // [B, Hkv, 32 lanes, 16] pre-scaled fp16 query fragments of the scan (workspace)
+    float* fpart_ml;         // fused path: [items, attend warps, 4 heads, 2]
+    float* fpart_acc;        // fused path: [items, attend warps, 4 heads, 128]
+    int total_items;         // fused path: work items = ceil(max_blocks / 32) * B * Hkv
+    uint32_t* item_counter;  // fused path: next work item to hand out (workspace; zeroed by the pseudo-max kernel)
     uint8_t* kept_mask;      // nullable [B, Hq, max_blocks]
     float* block_max;        // nullable [B, Hq, max_blocks]
     void* out;               // [B, Hq, 128] bf16 or fp32
@@ -81,6 +94,62 @@ __device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                  : "l"(p));
     return v;
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src) : "memory");
+}
+
+// the mbarrier receives one arrival from this thread once all its earlier cp.async copies have landed
+__device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void cp_async_drain() { asm volatile("cp.async.wait_all;\n" ::: "memory"); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
+}
+
+// Bounded wait for the phase with the given parity; false when the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    long long t0 = 0;
+    for (;;) {
+        uint32_t ok;
+        asm volatile(
+            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+        const long long now = clock64();
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > kSpinCycles) return false;
+    }
+}
+
+// Shared-memory tile layout: token T's 256-byte row keeps its place, its sixteen 16-byte chunks are XOR-ed with
+// swz(T) (bits 0..2 only).  With this every quarter-warp of the K and V fragment reads below, and of the copy
+// that fills the slot, touches eight different 16-byte bank groups.
+__device__ __forceinline__ uint32_t swz(uint32_t token) { return (((token >> 1) & 3u) << 1) ^ ((token & 1u) << 2); }
+
+// Copy one 16 KB (64 tokens x 256 B) tile into a slot: 32 coalesced 512-byte warp copies.
+__device__ __forceinline__ void tile_copy_async(uint32_t slot, const uint4* __restrict__ src, int lane, uint32_t bar) {
+    const uint32_t half = lane >> 4, c = lane & 15;
+#pragma unroll
+    for (int it = 0; it < 32; ++it) {
+        const uint32_t token = 2 * it + half;
+        cp_async16(slot + token * 256 + ((c ^ swz(token)) << 4), src + it * 32 + lane);
+    }
+    cp_async_arrive(bar);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -164,18 +233,28 @@ __device__ __forceinline__ void scan_setup(ScanQuery& sq, const __nv_bfloat16* q
 // single products) and adds the eight partial sums with round-to-nearest fp32 adds; it is used for the
 // pseudo-max and for blocks whose fast result lands within `band` of the threshold, so that both decisions rest
 // on the same, deterministic, ~1e-5-accurate arithmetic.
-template <bool PRECISE>
-__device__ __forceinline__ float scan_block(const uint4* __restrict__ codes_tile, const uint4* __restrict__ scales_tile,
-                                            const ScanQuery& sq, int lane, int rows, float sm_scale, float& band) {
-    const int j = lane & 3, r = lane >> 2;
-    uint4 w[4];
+struct ScanRegs {
+    uint4 w[4];   // packed codes of the four 16-token groups
+    uint4 s[4];   // this lane's 32 scales
+};
+
+__device__ __forceinline__ void scan_load(ScanRegs& sr, const uint4* __restrict__ codes_tile,
+                                          const uint4* __restrict__ scales_tile, int lane) {
 #pragma unroll
-    for (int mt = 0; mt < 4; ++mt) w[mt] = ldg_stream(codes_tile + mt * 32 + lane);
+    for (int mt = 0; mt < 4; ++mt) sr.w[mt] = ldg_stream(codes_tile + mt * 32 + lane);
+#pragma unroll
+    for (int x = 0; x < 4; ++x) sr.s[x] = __ldg(scales_tile + 4 * (lane & 3) + x);
+}
+
+template <bool PRECISE>
+__device__ __forceinline__ float scan_compute(const ScanRegs& sr, const ScanQuery& sq, int lane, int rows,
+                                              float sm_scale, float& band) {
+    const int r = lane >> 2;
+    const uint4* w = sr.w;
     uint32_t sc[16];
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
-        uint4 s = __ldg(scales_tile + 4 * j + x);
-        sc[4 * x] = s.x; sc[4 * x + 1] = s.y; sc[4 * x + 2] = s.z; sc[4 * x + 3] = s.w;
+        sc[4 * x] = sr.s[x].x; sc[4 * x + 1] = sr.s[x].y; sc[4 * x + 2] = sr.s[x].z; sc[4 * x + 3] = sr.s[x].w;
     }
     uint32_t bfrag[16];
 #pragma unroll
@@ -241,11 +320,11 @@ __device__ __forceinline__ float scan_block(const uint4* __restrict__ codes_tile
 // ---- attend: exact attention of one block, online softmax state in registers ------------------------------
 //
 // S^T = Q K^T : M = 16 rows (row r < 4: head r, row r + 4: the same head again, rows 8..15 zero), N = 8 tokens,
-//               K = 16 channels.  A lane (n = lane/4, j) reads 16 contiguous bytes of token n's key per load.
+//               K = 16 channels.  A lane (n = lane/4, j) reads 16 contiguous bytes of token n's key per read.
 // O = P V     : M = same rows (r < 4 carries the bf16 rounding of P, r + 4 the remainder), N = 8 channels,
 //               K = 16 tokens.  V rows are paired in registers with byte permutes.
-// Channel order inside the contractions is a fixed permutation chosen so that every global load is a full
-// 16-byte vector and every 32-byte sector fetched is fully used.
+// Channel order inside the contractions is a fixed permutation chosen so that every shared-memory read is a
+// full 16-byte vector of one token row.
 
 struct AttendState {
     uint32_t qa[16];   // A fragments of Q: qa[2s] (k = 2j..2j+1), qa[2s+1] (k = 2j+8..2j+9) of k-step s
@@ -270,25 +349,32 @@ __device__ __forceinline__ void attend_setup(AttendState& st, const __nv_bfloat1
 }
 
 // keep4: bit h set when head h attends to this block.  rows: valid tokens in the block (1..64).
-__device__ __forceinline__ void attend_block(AttendState& st, const uint4* __restrict__ k_tile,
-                                             const uint4* __restrict__ v_tile, int lane, int rows, unsigned keep4,
-                                             float logit_scale_log2) {
+// The block's K and V tiles are (being) copied into kslot / vslot; kbar / vbar complete when they have landed.
+// next_k / next_v: global tiles of the next kept block (nullptr = none); their copies are issued as soon as
+// this block has finished reading the respective slot.  Returns false if a wait ran out.
+__device__ __forceinline__ bool attend_block(AttendState& st, uint32_t kslot, uint32_t vslot, uint32_t kbar,
+                                             uint32_t vbar, uint32_t& phase, const uint4* next_k, const uint4* next_v,
+                                             int lane, int rows, unsigned keep4, float logit_scale_log2) {
     const int r = lane >> 2, j = lane & 3;
     const bool mine = (keep4 >> (r & 3)) & 1u;
+    if (!mbar_wait(kbar, phase & 1u)) return false;
     float s[8][2];
+    {
+        const uint32_t swz_k = swz(r);   // token 8*nt + r: the swizzle depends on r only
 #pragma unroll
-    for (int nt = 0; nt < 8; ++nt) {
-        s[nt][0] = s[nt][1] = 0.f;
-        const uint4* src = k_tile + (8 * nt + r) * 16 + j;
-        uint4 kv[4];
+        for (int nt = 0; nt < 8; ++nt) {
+            s[nt][0] = s[nt][1] = 0.f;
+            const uint32_t row = kslot + (8 * nt + r) * 256;
 #pragma unroll
-        for (int l4 = 0; l4 < 4; ++l4) kv[l4] = ldg_stream(src + 4 * l4);
-#pragma unroll
-        for (int l4 = 0; l4 < 4; ++l4) {
-            mma_bf16_top(s[nt][0], s[nt][1], st.qa[4 * l4 + 0], st.qa[4 * l4 + 1], kv[l4].x, kv[l4].y);
-            mma_bf16_top(s[nt][0], s[nt][1], st.qa[4 * l4 + 2], st.qa[4 * l4 + 3], kv[l4].z, kv[l4].w);
+            for (int l4 = 0; l4 < 4; ++l4) {
+                const uint4 kv = lds128(row + (((4 * l4 + j) ^ swz_k) << 4));
+                mma_bf16_top(s[nt][0], s[nt][1], st.qa[4 * l4 + 0], st.qa[4 * l4 + 1], kv.x, kv.y);
+                mma_bf16_top(s[nt][0], s[nt][1], st.qa[4 * l4 + 2], st.qa[4 * l4 + 3], kv.z, kv.w);
+            }
         }
     }
+    __syncwarp();   // every lane is done reading the K slot
+    if (next_k) tile_copy_async(kslot, next_k, lane, kbar);
     // online softmax (log2 domain)
     float mx = -INFINITY;
 #pragma unroll
@@ -320,6 +406,7 @@ __device__ __forceinline__ void attend_block(AttendState& st, const uint4* __res
 #pragma unroll
     for (int nt = 0; nt < 16; ++nt) { st.acc[nt][0] *= alpha; st.acc[nt][1] *= alpha; }
     // O += P V
+    if (!mbar_wait(vbar, phase & 1u)) return false;
 #pragma unroll
     for (int kt = 0; kt < 4; ++kt) {
         const int t0 = 16 * kt + 2 * j;
@@ -329,7 +416,8 @@ __device__ __forceinline__ void attend_block(AttendState& st, const uint4* __res
 #pragma unroll
             for (int tt = 0; tt < 4; ++tt) {
                 const int tok = t0 + (tt & 1) + ((tt >> 1) << 3);
-                v[tt] = ldg_stream(v_tile + tok * 16 + hf * 8 + r);
+                const uint32_t swz_v = (uint32_t)(j << 1) ^ ((uint32_t)(tt & 1) << 2);   // = swz(tok)
+                v[tt] = lds128(vslot + tok * 256 + (((8 * hf + r) ^ swz_v) << 4));
                 if (tok >= rows) v[tt] = make_uint4(0u, 0u, 0u, 0u);   // never multiply 0 by stale memory
             }
             const uint32_t* x0 = reinterpret_cast<const uint32_t*>(&v[0]);
@@ -346,6 +434,10 @@ __device__ __forceinline__ void attend_block(AttendState& st, const uint4* __res
             }
         }
     }
+    __syncwarp();   // every lane is done reading the V slot
+    if (next_v) tile_copy_async(vslot, next_v, lane, vbar);
+    phase ^= 1u;
+    return true;
 }
 
 // output channel of O fragment (n-tile nt, column n)
