@@ -30,53 +30,55 @@ __device__ __forceinline__ uint32_t quant_code(float x, float s) {
 }
 
 __global__ void __launch_bounds__(128) quantize_kernel(QuantParams p) {
-    const int blk = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+    const int g = blockIdx.y, b = blockIdx.z;
     int n = p.seq_lens[b];
     const int cap = p.max_blocks * kBlk;
     n = n < 0 ? 0 : (n > cap ? cap : n);
     const int nb = (n + kBlk - 1) / kBlk;
     const int first = p.first_token ? max(p.first_token[b], 0) / kBlk : 0;
-    if (blk >= nb || blk < first) return;
-    const int page = p.block_table ? p.block_table[(size_t)b * p.max_blocks + blk] : b * p.max_blocks + blk;
-    if (page < 0 || page >= p.num_pages) return;
-    const int rows = min(kBlk, n - blk * kBlk);
-    const size_t tile = (size_t)page * p.Hkv + g;
-
     __shared__ __align__(16) __nv_bfloat16 sk[kBlk * kD];
     __shared__ float ss[kD];
-    const uint4* src = reinterpret_cast<const uint4*>(p.k_cache + tile * kBlk * kD);
-    uint4* dst = reinterpret_cast<uint4*>(sk);
     const int tid = threadIdx.x;
+    // the grid's x extent is bounded; every CTA walks its share of the blocks that need (re)quantizing
+    for (int blk = first + blockIdx.x; blk < nb; blk += gridDim.x) {
+        const int page = p.block_table ? p.block_table[(size_t)b * p.max_blocks + blk] : b * p.max_blocks + blk;
+        if (page < 0 || page >= p.num_pages) continue;
+        const int rows = min(kBlk, n - blk * kBlk);
+        const size_t tile = (size_t)page * p.Hkv + g;
+        const uint4* src = reinterpret_cast<const uint4*>(p.k_cache + tile * kBlk * kD);
+        uint4* dst = reinterpret_cast<uint4*>(sk);
+        __syncthreads();   // the previous block's tile is no longer needed
 #pragma unroll
-    for (int x = 0; x < 8; ++x) dst[tid + 128 * x] = ldg_stream(src + tid + 128 * x);
-    __syncthreads();
-    {
-        float a = 0.f;
-        for (int r = 0; r < rows; ++r) a = fmaxf(a, fabsf(__bfloat162float(sk[r * kD + tid])));
-        float s32 = __fdiv_rn(a, 1.5f);
-        s32 = fminf(s32, 65504.f);
-        const __half s = __float2half_rn(s32);
-        p.k_scales[tile * kD + tid] = s;
-        ss[tid] = __half2float(s);
-    }
-    __syncthreads();
-    const int mt = tid >> 5, lane = tid & 31, r = lane >> 2, j = lane & 3;
-    uint32_t w[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int c = 32 * j + 4 * i + u;
-            const float s = ss[c];
-            const uint32_t lo_row = quant_code(__bfloat162float(sk[(16 * mt + r) * kD + c]), s);
-            const uint32_t hi_row = quant_code(__bfloat162float(sk[(16 * mt + r + 8) * kD + c]), s);
-            const int shift = 2 * i + 16 * (u & 1);
-            w[(u >> 1) * 2 + 0] |= lo_row << shift;   // W0 / W2: token r
-            w[(u >> 1) * 2 + 1] |= hi_row << shift;   // W1 / W3: token r + 8
+        for (int x = 0; x < 8; ++x) dst[tid + 128 * x] = ldg_stream(src + tid + 128 * x);
+        __syncthreads();
+        {
+            float a = 0.f;
+            for (int r = 0; r < rows; ++r) a = fmaxf(a, fabsf(__bfloat162float(sk[r * kD + tid])));
+            float s32 = __fdiv_rn(a, 1.5f);
+            s32 = fminf(s32, 65504.f);
+            const __half s = __float2half_rn(s32);
+            p.k_scales[tile * kD + tid] = s;
+            ss[tid] = __half2float(s);
         }
+        __syncthreads();
+        const int mt = tid >> 5, lane = tid & 31, r = lane >> 2, j = lane & 3;
+        uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int c = 32 * j + 4 * i + u;
+                const float s = ss[c];
+                const uint32_t lo_row = quant_code(__bfloat162float(sk[(16 * mt + r) * kD + c]), s);
+                const uint32_t hi_row = quant_code(__bfloat162float(sk[(16 * mt + r + 8) * kD + c]), s);
+                const int shift = 2 * i + 16 * (u & 1);
+                w[(u >> 1) * 2 + 0] |= lo_row << shift;   // W0 / W2: token r
+                w[(u >> 1) * 2 + 1] |= hi_row << shift;   // W1 / W3: token r + 8
+            }
+        }
+        uint4* out = reinterpret_cast<uint4*>(p.k_quant + tile * kCodeBytes);
+        out[mt * 32 + lane] = make_uint4(w[0], w[1], w[2], w[3]);
     }
-    uint4* out = reinterpret_cast<uint4*>(p.k_quant + tile * kCodeBytes);
-    out[mt * 32 + lane] = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
 // canonical codes [pages, Hkv, 64, 128] from the packed layout
@@ -113,10 +115,12 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
     ScanQuery sq;
     scan_setup(sq, p.q + ((size_t)b * p.Hq + (size_t)g * p.G) * kD, p.G, lane);
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *p.item_counter = 0u;
-    if (warp == 0) {   // the scan warps of the fused kernel reload these per work item
-        uint4* dst = reinterpret_cast<uint4*>(p.qfrag) + ((size_t)(b * p.Hkv + g) * 32 + lane) * 4;
+    unsigned char* rec = p.qrec + (size_t)(b * p.Hkv + g) * kQrecBytes;
+    if (warp == 0) {   // query record of this (sequence, KV head): the fused kernel stages it per work item
+        uint4* dst = reinterpret_cast<uint4*>(rec);
 #pragma unroll
-        for (int x = 0; x < 4; ++x) dst[x] = make_uint4(sq.qh[4 * x], sq.qh[4 * x + 1], sq.qh[4 * x + 2], sq.qh[4 * x + 3]);
+        for (int x = 0; x < 4; ++x)
+            dst[x * 32 + lane] = make_uint4(sq.qh[4 * x], sq.qh[4 * x + 1], sq.qh[4 * x + 2], sq.qh[4 * x + 3]);
     }
     float best = -INFINITY;
     for (int s = warp; s < count; s += kPmWarps) {
@@ -133,10 +137,16 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
     }
     if (lane < kMaxG) smax[warp][lane] = best;
     __syncthreads();
-    if (threadIdx.x < p.G) {
-        float m = -INFINITY;
-        for (int w = 0; w < kPmWarps; ++w) m = fmaxf(m, smax[w][threadIdx.x]);
-        p.mtilde[(size_t)b * p.Hq + g * p.G + threadIdx.x] = m;
+    if (threadIdx.x < 8) {
+        // thresholds m_tilde - delta for the scan (delta = +inf gives -inf: every block passes); unused heads: +inf
+        float thr = INFINITY;
+        if (threadIdx.x < p.G) {
+            float m = -INFINITY;
+            for (int w = 0; w < kPmWarps; ++w) m = fmaxf(m, smax[w][threadIdx.x]);
+            p.mtilde[(size_t)b * p.Hq + g * p.G + threadIdx.x] = m;
+            thr = m - p.delta;
+        }
+        reinterpret_cast<float*>(rec + 2048)[threadIdx.x] = thr;
     }
 }
 
@@ -303,30 +313,6 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(DecodeParams p) 
     }
 }
 
-// ---- split combine (FlashDecoding-style log-sum-exp merge) -------------------------------------------------
-__global__ void __launch_bounds__(kD) combine_kernel(DecodeParams p) {
-    const size_t head = (size_t)blockIdx.y * p.Hq + blockIdx.x;
-    const int c = threadIdx.x;
-    const float* ml = p.part_ml + head * p.splits * 2;
-    float M = -INFINITY;
-    for (int s = 0; s < p.splits; ++s)
-        if (ml[2 * s + 1] > 0.f) M = fmaxf(M, ml[2 * s]);
-    float L = 0.f, a = 0.f;
-    if (M != -INFINITY) {
-        for (int s = 0; s < p.splits; ++s) {
-            const float ls = ml[2 * s + 1];
-            if (!(ls > 0.f)) continue;
-            const float f = exp2f(ml[2 * s] - M);
-            L += f * ls;
-            a += f * p.part_acc[(head * p.splits + s) * kD + c];
-        }
-    }
-    const float o = L > 0.f ? a / L : 0.f;
-    if (p.out_fp32) reinterpret_cast<float*>(p.out)[head * kD + c] = o;
-    else reinterpret_cast<__nv_bfloat16*>(p.out)[head * kD + c] = __float2bfloat16_rn(o);
-    if (p.lse && c == 0) p.lse[head] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
-}
-
 __global__ void clear_status_kernel(uint32_t* status) { *status = 0u; }
 
 // ---- host side --------------------------------------------------------------------------------------------
@@ -334,7 +320,7 @@ __global__ void clear_status_kernel(uint32_t* status) { *status = 0u; }
 struct Plan {
     int blocks_per_split, splits;     // dense path
     int total_items;                  // fused path
-    size_t off_mtilde, off_qfrag, off_ml, off_acc, off_fml, off_facc, total;
+    size_t off_mtilde, off_qrec, off_ml, off_acc, off_fml, off_facc, total;
 };
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -352,8 +338,8 @@ static Plan make_plan(const ffd_config* cfg, int batch, int max_blocks) {
     pl.total_items = ((max_blocks + kItemBlocks - 1) / kItemBlocks) * batch * cfg->num_kv_heads;
     const size_t fslots = (size_t)pl.total_items * kNA * kMaxG;
     pl.off_mtilde = 256;
-    pl.off_qfrag = align_up(pl.off_mtilde + heads * sizeof(float), 256);
-    pl.off_ml = align_up(pl.off_qfrag + (size_t)batch * cfg->num_kv_heads * 32 * 16 * sizeof(uint32_t), 256);
+    pl.off_qrec = align_up(pl.off_mtilde + heads * sizeof(float), 256);
+    pl.off_ml = align_up(pl.off_qrec + (size_t)batch * cfg->num_kv_heads * kQrecBytes, 256);
     pl.off_acc = align_up(pl.off_ml + heads * pl.splits * 2 * sizeof(float), 256);
     pl.off_fml = align_up(pl.off_acc + heads * pl.splits * kD * sizeof(float), 256);
     pl.off_facc = align_up(pl.off_fml + fslots * 2 * sizeof(float), 256);
@@ -431,7 +417,7 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
     p.mtilde = reinterpret_cast<float*>(ws + pl.off_mtilde);
     p.part_ml = reinterpret_cast<float*>(ws + pl.off_ml);
     p.part_acc = reinterpret_cast<float*>(ws + pl.off_acc);
-    p.qfrag = reinterpret_cast<uint32_t*>(ws + pl.off_qfrag);
+    p.qrec = reinterpret_cast<unsigned char*>(ws + pl.off_qrec);
     p.fpart_ml = reinterpret_cast<float*>(ws + pl.off_fml);
     p.fpart_acc = reinterpret_cast<float*>(ws + pl.off_facc);
     p.total_items = pl.total_items;
@@ -455,14 +441,14 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
         if (prof) cudaEventRecord(g_prof_start, s);
         fused_sparse_kernel<<<min(p.total_items, sms), kFusedThreads, kFusedSmem, s>>>(p);
         if (prof) cudaEventRecord(g_prof_stop, s);
-        fused_combine_kernel<<<dim3(p.Hq, batch), kD, 0, s>>>(p);
+        combine_kernel<true><<<dim3(p.Hq, batch), kCombineThreads, 0, s>>>(p);
     } else {
         if (cudaFuncSetAttribute(decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem) != cudaSuccess)
             return FFD_ERR_CUDA;
         if (prof) cudaEventRecord(g_prof_start, s);
         decode_kernel<false><<<grid, kWarps * 32, kDecodeSmem, s>>>(p);
         if (prof) cudaEventRecord(g_prof_stop, s);
-        combine_kernel<<<dim3(p.Hq, batch), kD, 0, s>>>(p);
+        combine_kernel<false><<<dim3(p.Hq, batch), kCombineThreads, 0, s>>>(p);
     }
     return launch_status();
 }
@@ -521,7 +507,8 @@ ffd_status ffd_quantize_keys(const ffd_config* cfg, const void* k_cache, void* k
     QuantParams p{static_cast<const __nv_bfloat16*>(k_cache), static_cast<uint8_t*>(k_quant),
                   static_cast<__half*>(k_scales), block_table, seq_lens, first_token,
                   cfg->num_kv_heads, max_blocks_per_seq, num_pages};
-    quantize_kernel<<<dim3(max_blocks_per_seq, cfg->num_kv_heads, batch), 128, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    quantize_kernel<<<dim3(max_blocks_per_seq < 64 ? max_blocks_per_seq : 64, cfg->num_kv_heads, batch), 128, 0,
+                      static_cast<cudaStream_t>(stream)>>>(p);
     return launch_status();
 }
 

@@ -1,28 +1,36 @@
 // The fused sparse kernel: scan -> top-delta select -> exact attention over kept blocks, in one persistent launch.
 //
-// One CTA per SM, 12 warps in two roles that run concurrently:
-//   8 scan warps    stream the 2-bit codes and scales of every block through a private 3-stage cp.async ring
+// One CTA per SM, 16 warps in two roles that run concurrently (register budgets set with setmaxnreg):
+//   12 scan warps   stream the 2-bit codes and scales of every block through a private 3-stage cp.async ring
 //                   (3 blocks = 6.9 KB in flight per warp), compute the block maxima of the approximate scores
 //                   on the tensor cores and publish the keep decisions of one work item in a batch descriptor;
 //   4 attend warps  take the kept blocks of a published batch, stage their K and V tiles (16 KB each) through
 //                   private swizzled slots with cp.async + mbarrier and run the exact online-softmax attention.
-// A work item is 32 consecutive blocks of one (sequence, KV head).  Items are handed out dynamically: lane 0 of scan
-// warp 0 draws item numbers from a global counter two items ahead and shares them with the other scan warps
-// through a small ring and one named barrier per item; attend warps learn the item from the batch descriptor.
-// Scan warps run up to two items ahead of the attend warps (two batch descriptors, full/empty mbarriers).
+// A work item is 24 consecutive blocks of one (sequence, KV head).  Items are handed out dynamically: lane 0 of scan
+// warp 0 draws item numbers from a global counter three items ahead (the atomic's latency is never waited for),
+// publishes them in a small ring two items ahead and starts the copy of the item's query record (pre-scaled fp16
+// query fragments + thresholds, written by the pseudo-max kernel) into shared memory; one named barrier per item
+// keeps the scan warps in step.  Attend warps learn the item from the batch descriptor.  Scan warps run up to two
+// batches ahead of the attend warps (two descriptors, full/empty mbarriers).
 // Every mbarrier wait is bounded; on expiry the warp records kDevTimeout and the CTA winds down.
 #pragma once
 #include "ffd_kernels.cuh"
 
 namespace ffd {
 
-constexpr int kNS = 8;                 // scan warps
-constexpr int kNA = 4;                 // attend warps
+constexpr int kNS = 12;                // scan warps (three warpgroups)
+constexpr int kNA = 4;                 // attend warps (one warpgroup)
 constexpr int kFusedThreads = (kNS + kNA) * 32;
-constexpr int kItemBlocks = 32;        // blocks per work item
+constexpr int kScanRegs = 112;         // 12*32*112 + 4*32*176 = 65536 registers
+constexpr int kAttendRegs = (65536 - kNS * 32 * kScanRegs) / (kNA * 32);
+static_assert(kAttendRegs % 8 == 0 && kScanRegs % 8 == 0, "setmaxnreg takes multiples of 8");
+constexpr int kItemBlocks = 24;        // blocks per work item: two per scan warp
 constexpr int kRing = 3;               // code-ring stages per scan warp
 constexpr int kStageBytes = kCodeBytes + kD * 2;   // 2048 B codes + 256 B scales
 constexpr int kNB = 2;                 // batch descriptors in flight
+constexpr int kIdRing = 8;             // item numbers known ahead
+constexpr int kQrecRing = 4;           // query records staged ahead
+constexpr int kQrecBytes = 2048 + 32;  // [4][32 lanes] uint4 of fp16 query fragments, then 4 thresholds (+ pad)
 
 struct BatchDesc {
     int item;                          // work item of this batch; < 0: no more work
@@ -34,11 +42,15 @@ struct BatchDesc {
 
 constexpr int kOffSlots = 0;
 constexpr int kOffRing = kOffSlots + kNA * 2 * kSlotBytes;
-constexpr int kOffDesc = kOffRing + kNS * kRing * kStageBytes;
+constexpr int kOffQrec = kOffRing + kNS * kRing * kStageBytes;
+constexpr int kOffDesc = kOffQrec + kQrecRing * kQrecBytes;
 constexpr int kOffBars = kOffDesc + kNB * (int)sizeof(BatchDesc);
-constexpr int kOffIds = kOffBars + (2 * kNB + 2 * kNA) * 8;      // ring of 4 item numbers + abort flag
-constexpr int kFusedSmem = kOffIds + 8 * 4;
-static_assert(kOffBars % 8 == 0 && kOffRing % 16 == 0 && kOffDesc % 16 == 0, "alignment");
+constexpr int kNumBars = 2 * kNB + 2 * kNA + kQrecRing;          // full, empty, K/V slots, query records
+constexpr int kOffIds = kOffBars + kNumBars * 8;                 // ring of item numbers + abort flag
+constexpr int kFusedSmem = kOffIds + (kIdRing + 4) * 4;
+static_assert(kOffBars % 8 == 0 && kOffRing % 16 == 0 && kOffDesc % 16 == 0 && kOffQrec % 16 == 0, "alignment");
+static_assert(sizeof(BatchDesc) % 16 == 0, "descriptor size");
+static_assert(kFusedSmem <= 227 * 1024, "shared memory budget");
 
 struct Item {
     int b, g, blk0, nblk, n;           // nblk <= 0: nothing to do
@@ -46,8 +58,10 @@ struct Item {
 
 __device__ __forceinline__ Item decode_item(const DecodeParams& p, int item) {
     Item it;
+    // items are numbered from the END of the sequences backwards: the local window, whose blocks are the most
+    // likely to be kept (and therefore the most expensive), is handed out first
     const int units = p.batch * p.Hkv;
-    const int bg = item % units, split = item / units;
+    const int bg = item % units, split = p.total_items / units - 1 - item / units;
     it.b = bg / p.Hkv;
     it.g = bg % p.Hkv;
     it.n = clamped_seq_len(p, it.b);
@@ -74,33 +88,25 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
 
 __device__ __forceinline__ void scan_warps_barrier() { asm volatile("bar.sync 1, %0;\n" ::"n"(kNS * 32) : "memory"); }
 
-// Draw the next non-empty work item from the global counter (one thread); p.total_items when none is left.
-__device__ __forceinline__ int draw_item(const DecodeParams& p) {
-    for (;;) {
-        const int item = (int)atomicAdd(p.item_counter, 1u);
-        if (item >= p.total_items) return p.total_items;
-        if (decode_item(p, item).nblk > 0) return item;
-    }
-}
-
-// Position of a scan warp in its stream of blocks: batch after batch, local blocks w, w+8, w+16, w+24.
+// Position of a scan warp in its stream of blocks: item after item (in the order the item numbers were drawn),
+// local blocks w and w + 12.
 struct ScanCursor {
-    int bi;        // batch the cursor is in
-    Item it;       // nblk = 0 before the first batch
+    int seq;       // index of the drawn item the cursor is in
+    Item it;       // nblk = 0 before the first item
     int lb;
     bool end;      // ran into the end of the work
 };
 
-// Advance to this warp's next block.  Returns false when that block lies beyond the batches whose item numbers
-// are known (bi <= horizon) or beyond the end of the work; the cursor then stays where it can resume.
+// Advance to this warp's next block.  Returns false when that block lies beyond the items whose numbers are known
+// (seq <= horizon) or beyond the end of the work; the cursor then stays where it can resume.
 __device__ __forceinline__ bool cursor_next(ScanCursor& c, const DecodeParams& p, const volatile int* ids, int horizon,
                                             int w) {
     if (c.end) return false;
     int lb = c.lb + kNS;
     while (lb >= c.it.nblk) {
-        if (c.bi + 1 > horizon) { c.lb = lb - kNS; return false; }   // resume here later (lb is re-derived)
-        const int item = ids[(c.bi + 1) & 3];
-        ++c.bi;
+        if (c.seq + 1 > horizon) { c.lb = lb - kNS; return false; }
+        const int item = ids[(c.seq + 1) & (kIdRing - 1)];
+        ++c.seq;
         if (item >= p.total_items) { c.end = true; c.it.nblk = 0; return false; }
         c.it = decode_item(p, item);
         lb = w;
@@ -117,8 +123,10 @@ __device__ __forceinline__ void ring_issue(const DecodeParams& p, const ScanCurs
         const uint4* codes = reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes);
 #pragma unroll
         for (int x = 0; x < 4; ++x) cp_async16(stage + (x * 32 + lane) * 16, codes + x * 32 + lane);
+        // scales: 16-byte chunk 4j + x lands at position 4x + j, so the four chunks read together are adjacent
         if (lane < 16)
-            cp_async16(stage + kCodeBytes + lane * 16, reinterpret_cast<const uint4*>(p.k_scales + tile * kD) + lane);
+            cp_async16(stage + kCodeBytes + ((lane & 3) * 4 + (lane >> 2)) * 16,
+                       reinterpret_cast<const uint4*>(p.k_scales + tile * kD) + lane);
     }
     asm volatile("cp.async.commit_group;\n" ::: "memory");
 }
@@ -129,59 +137,118 @@ __device__ __forceinline__ void ring_wait(int younger) {
     else asm volatile("cp.async.wait_group 0;\n" ::: "memory");
 }
 
+// Warp 0 only: if `item` has work, copy its query record into the next slot of the record ring and report
+// completion on that slot's mbarrier.  Records are numbered like batches (items with work, in drawing order), so
+// every scan warp waits for every phase of every slot barrier and a parity wait can never see a stale phase.
+__device__ __forceinline__ void qrec_issue(const DecodeParams& p, int item, uint32_t qrecs, uint32_t qbars,
+                                           int& records, int lane) {
+    if (item >= p.total_items || decode_item(p, item).nblk <= 0) return;
+    const int slot = records & (kQrecRing - 1);
+    const int bg = item % (p.batch * p.Hkv);
+    const uint4* src = reinterpret_cast<const uint4*>(p.qrec + (size_t)bg * kQrecBytes);
+    for (int c = lane; c < kQrecBytes / 16; c += 32) cp_async16(qrecs + slot * kQrecBytes + c * 16, src + c);
+    cp_async_arrive(qbars + slot * 8);
+    ++records;
+}
+
+// The precise variant of the scan for one block, with the arithmetic m_tilde was computed in.  Kept out of line so
+// that its registers do not weigh on the fast path; it re-reads the block's codes and scales from global memory.
+__device__ __noinline__ float scan_block_precise(const uint4* codes_tile, const uint4* scales_tile, uint32_t qrec,
+                                                 int lane, int rows, float sm_scale) {
+    ScanRegs sr;
+    scan_load(sr, codes_tile, scales_tile, lane);
+    ScanQuery sq;
+    sq.piece = (lane >> 2) & 1;
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        const uint4 v = lds128(qrec + (x * 32 + lane) * 16);
+        sq.qh[4 * x] = v.x; sq.qh[4 * x + 1] = v.y; sq.qh[4 * x + 2] = v.z; sq.qh[4 * x + 3] = v.w;
+    }
+    float band;
+    return scan_compute<true>(sr, sq, lane, rows, sm_scale, band);
+}
+
 __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* smem, int w, int lane) {
     const int r = lane >> 2, j = lane & 3;
     const uint32_t ring = smem_u32(smem) + kOffRing + w * kRing * kStageBytes;
+    const uint32_t qrecs = smem_u32(smem) + kOffQrec;
     const uint32_t bars = smem_u32(smem) + kOffBars;
+    const uint32_t qbars = bars + (2 * kNB + 2 * kNA) * 8;
     BatchDesc* descs = reinterpret_cast<BatchDesc*>(smem + kOffDesc);
     volatile int* ids = reinterpret_cast<volatile int*>(smem + kOffIds);
-    volatile int* abort_flag = ids + 4;
+    volatile int* abort_flag = ids + kIdRing;
 
-    if (w == 0 && lane == 0) {
-        ids[0] = draw_item(p);
-        ids[1] = ids[0] < p.total_items ? draw_item(p) : p.total_items;
+    // warp 0 draws the first item numbers: two are published now, the third is held until the first iteration
+    int pend = p.total_items;
+    int records = 0;                // query records staged so far (warp 0)
+    if (w == 0) {
+        int id0 = 0, id1 = 0;
+        if (lane == 0) {
+            id0 = (int)atomicAdd(p.item_counter, 1u);
+            id1 = (int)atomicAdd(p.item_counter, 1u);
+            pend = (int)atomicAdd(p.item_counter, 1u);
+            ids[0] = min(id0, p.total_items);
+            ids[1] = min(id1, p.total_items);
+        }
+        id0 = min(__shfl_sync(kFull, id0, 0), p.total_items);
+        id1 = min(__shfl_sync(kFull, id1, 0), p.total_items);
+        qrec_issue(p, id0, qrecs, qbars, records, lane);
+        qrec_issue(p, id1, qrecs, qbars, records, lane);
     }
     ScanCursor ic;
-    ic.bi = -1;
+    ic.seq = -1;
     ic.it.nblk = 0;
     ic.lb = w - kNS;
     ic.end = false;
     int issued = 0, consumed = 0;   // this warp's blocks whose copies were started / whose data was taken
-    ScanQuery sq;
-    sq.piece = r & 1;
+    int bi = 0;                     // batches published so far
 
-    for (int bi = 0;; ++bi) {
-        const int slot = bi & 1, use = bi >> 1;
-        // the attend warps must have released this descriptor (two batches ago)
-        if (use > 0 && !mbar_wait(bars + (kNB + slot) * 8, (use - 1) & 1)) *abort_flag = 1;
-        if (w == 0 && lane == 0) {
-            const int prev = ids[(bi + 1) & 3];
-            ids[(bi + 2) & 3] = prev < p.total_items ? draw_item(p) : p.total_items;
+#pragma unroll 1
+    for (int seq = 0;; ++seq) {
+        if (w == 0) {   // publish the item number of seq + 2, draw the one of seq + 3, stage the record of seq + 2
+            int id2 = 0;
+            if (lane == 0) {
+                id2 = min(pend, p.total_items);
+                ids[(seq + 2) & (kIdRing - 1)] = id2;
+                pend = id2 < p.total_items ? (int)atomicAdd(p.item_counter, 1u) : p.total_items;
+            }
+            id2 = __shfl_sync(kFull, id2, 0);
+            qrec_issue(p, id2, qrecs, qbars, records, lane);
         }
         __syncwarp();
-        scan_warps_barrier();          // item numbers of batches bi, bi+1, bi+2 are visible to all scan warps
-        const int horizon = bi + 2;
-        const int item = ids[bi & 3];
-        BatchDesc& d = descs[slot];
+        scan_warps_barrier();          // item numbers of seq, seq + 1, seq + 2 are visible to all scan warps
+        const int horizon = seq + 2;
+        const int item = ids[seq & (kIdRing - 1)];
         if (item >= p.total_items || *abort_flag) {   // no more work: tell the attend warps
+            const int slot = bi & 1, use = bi >> 1;
+            if (use > 0 && !mbar_wait(bars + (kNB + slot) * 8, (use - 1) & 1)) *abort_flag = 1;
             if (lane == 0) {
-                if (w == 0) d.item = -1;
+                if (w == 0) descs[slot].item = -1;
                 mbar_arrive(bars + slot * 8);
             }
             break;
         }
         const Item it = decode_item(p, item);
-        const size_t head0 = (size_t)it.b * p.Hq + (size_t)it.g * p.G;
-        {   // pre-scaled fp16 query fragments written by the pseudo-max kernel
-            const uint4* qf = reinterpret_cast<const uint4*>(p.qfrag) + ((size_t)(it.b * p.Hkv + it.g) * 32 + lane) * 4;
-#pragma unroll
-            for (int x = 0; x < 4; ++x) {
-                const uint4 v = __ldg(qf + x);
-                sq.qh[4 * x] = v.x; sq.qh[4 * x + 1] = v.y; sq.qh[4 * x + 2] = v.z; sq.qh[4 * x + 3] = v.w;
-            }
+        // The prefetch cursor never trails the item being processed: everything of this warp before `seq` has been
+        // consumed, hence issued.  (It would otherwise fall behind during runs of empty items and read slots of the
+        // item-number ring that have been reused.)
+        if (ic.seq < seq) {
+            ic.seq = seq;
+            ic.it = it;
+            ic.lb = w - kNS;
         }
-        const float thr = (j < p.G) ? p.mtilde[head0 + j] - p.delta : -INFINITY;   // delta = +inf: all pass
+        if (it.nblk <= 0) continue;    // nothing in this item (sequence shorter than the longest): no batch
+        const int slot = bi & 1, use = bi >> 1;
+        // the attend warps must have released this descriptor (two batches ago); the query record must have landed
+        if (use > 0 && !mbar_wait(bars + (kNB + slot) * 8, (use - 1) & 1)) *abort_flag = 1;
+        if (!mbar_wait(qbars + (bi & (kQrecRing - 1)) * 8, (bi / kQrecRing) & 1)) *abort_flag = 1;
+        BatchDesc& d = descs[slot];
+        const uint32_t qrec = qrecs + (bi & (kQrecRing - 1)) * kQrecBytes;
+        const size_t head0 = (size_t)it.b * p.Hq + (size_t)it.g * p.G;
+        float thr;
+        asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(thr) : "r"(qrec + 2048 + j * 4));
         if (w == 0 && lane == 0) d.item = item;
+#pragma unroll 1
         for (int lb = w; lb < it.nblk; lb += kNS) {
             // keep the ring full: blocks consumed .. consumed + kRing - 1 of this warp's stream
             while (issued < consumed + kRing && cursor_next(ic, p, ids, horizon, w)) {
@@ -191,11 +258,15 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
             const uint32_t stage = ring + (consumed % kRing) * kStageBytes;
             ring_wait(issued - consumed - 1);
             __syncwarp();
-            ScanRegs sr;
+            // codes into registers; B operand straight from the staged scales and the item's query record
+            uint4 wv[4];
 #pragma unroll
-            for (int mt = 0; mt < 4; ++mt) sr.w[mt] = lds128(stage + (mt * 32 + lane) * 16);
+            for (int mt = 0; mt < 4; ++mt) wv[mt] = lds128(stage + (mt * 32 + lane) * 16);
+            uint32_t bfrag[16];
 #pragma unroll
-            for (int x = 0; x < 4; ++x) sr.s[x] = lds128(stage + kCodeBytes + (4 * j + x) * 16);
+            for (int x = 0; x < 4; ++x)
+                scan_bfrag4(bfrag + 4 * x, lds128(qrec + (x * 32 + lane) * 16),
+                            lds128(stage + kCodeBytes + (4 * x + j) * 16), r & 1);
             __syncwarp();   // the stage is free again
             ++consumed;
             if (issued < consumed + kRing && cursor_next(ic, p, ids, horizon, w)) {
@@ -209,10 +280,14 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
             unsigned keep4 = 0;
             if (page >= 0) {
                 float band;
-                float bm = scan_compute<false>(sr, sq, lane, rows, p.sm_scale, band);
-                // too close to call with the fast accumulation: redo with the arithmetic m_tilde was computed in
-                if (__any_sync(kFull, (j < p.G) && fabsf(bm - thr) <= band))
-                    bm = scan_compute<true>(sr, sq, lane, rows, p.sm_scale, band);
+                float bm = scan_mma<false>(wv, bfrag, lane, rows, p.sm_scale, band);
+                // too close to call (rare): a separate, non-inlined routine re-reads the block and redoes it precisely
+                if (__any_sync(kFull, (j < p.G) && fabsf(bm - thr) <= band)) {
+                    const size_t tile = (size_t)page * p.Hkv + it.g;
+                    bm = scan_block_precise(reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes),
+                                            reinterpret_cast<const uint4*>(p.k_scales + tile * kD), qrec, lane, rows,
+                                            p.sm_scale);
+                }
                 const bool keep = (j < p.G) && (bm >= thr);
                 keep4 = __ballot_sync(kFull, keep) & 0xFu;
                 if (r == 0 && j < p.G) {
@@ -229,6 +304,7 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(bars + slot * 8);   // this warp's share of the batch is published
+        ++bi;
     }
     cp_async_drain();
     if (*abort_flag && w == 0 && lane == 0) atomicOr(p.status, kDevTimeout);
@@ -351,79 +427,129 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodePa
             mbar_init(bars + s * 8, kNS);             // full: one arrival per scan warp
             mbar_init(bars + (kNB + s) * 8, kNA);     // empty: one arrival per attend warp
         }
-        for (int a = 0; a < 2 * kNA; ++a) mbar_init(bars + (2 * kNB + a) * 8, 32);
-        reinterpret_cast<volatile int*>(smem + kOffIds)[4] = 0;   // abort flag
+        for (int a = 0; a < 2 * kNA + kQrecRing; ++a) mbar_init(bars + (2 * kNB + a) * 8, 32);
+        reinterpret_cast<volatile int*>(smem + kOffIds)[kIdRing] = 0;   // abort flag
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     __syncthreads();
-    if (warp < kNS) scan_role(p, smem, warp, lane);
-    else attend_role(p, smem, warp - kNS, lane);
+    if (warp < kNS) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kScanRegs));
+        scan_role(p, smem, warp, lane);
+    } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kAttendRegs));
+        attend_role(p, smem, warp - kNS, lane);
+    }
 }
 
-// ---- combine for the fused kernel's partials ---------------------------------------------------------------
-// One CTA of 128 threads per (query head, sequence); partial e = (split, attend warp).
-__global__ void __launch_bounds__(kD) fused_combine_kernel(DecodeParams p) {
-    const int h = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
+// ---- split combine (FlashDecoding-style log-sum-exp merge) -------------------------------------------------
+// One CTA of 512 threads per (query head, sequence).  FUSED: partial e = (work item, attend warp) of the fused
+// kernel; otherwise partial e = split of the dense kernel.  Thread (el, cg) = (tid / 32, tid % 32) sums the
+// partials e = el, el + 16, ... for channels 4cg .. 4cg+3 with eight independent loads in flight; the sixteen
+// partial sums meet in shared memory.  Summation order is fixed, so results are reproducible.
+constexpr int kCombineThreads = 512;
+constexpr int kCombineChunk = 1024;
+
+template <bool FUSED>
+__device__ __forceinline__ size_t combine_slot(const DecodeParams& p, size_t head, int bg, int hl, int e) {
+    if (FUSED) {   // item number of split e / kNA (see decode_item), then the attend warp
+        const int units = p.batch * p.Hkv;
+        const int item = (p.total_items / units - 1 - e / kNA) * units + bg;
+        return ((size_t)item * kNA + (e % kNA)) * kMaxG + hl;
+    }
+    return head * p.splits + e;
+}
+
+template <bool FUSED>
+__global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p) {
+    const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+    const int el = tid >> 5, cg = tid & 31;
     const size_t head = (size_t)b * p.Hq + h;
-    const int g = h / p.G, hl = h % p.G;
+    const int g = h / p.G, hl = h % p.G, bg = b * p.Hkv + g;
     const int n = min(max(p.seq_lens[b], 0), p.max_blocks * kBlk);
-    const int nsplit = ((n + kBlk - 1) / kBlk + kItemBlocks - 1) / kItemBlocks;
-    const int units = p.batch * p.Hkv, bg = b * p.Hkv + g;
-    const int entries = nsplit * kNA;
-    __shared__ float wgt[kD];
-    __shared__ float red[kD / 32];
-    float M = -INFINITY, L = 0.f, acc = 0.f;
-    // pass 1: global max over all partials
-    for (int e = c; e < entries; e += kD) {
-        const size_t slot = (((size_t)(e / kNA) * units + bg) * kNA + (e % kNA)) * kMaxG + hl;
-        const float2 ml = *reinterpret_cast<const float2*>(p.fpart_ml + slot * 2);
-        if (ml.y > 0.f) M = fmaxf(M, ml.x);
+    const int nb = (n + kBlk - 1) / kBlk;
+    const int entries = FUSED ? ((nb + kItemBlocks - 1) / kItemBlocks) * kNA
+                              : min((nb + p.blocks_per_split - 1) / p.blocks_per_split, p.splits);
+    const float* ml = FUSED ? p.fpart_ml : p.part_ml;
+    const float* pacc = FUSED ? p.fpart_acc : p.part_acc;
+    __shared__ float s_w[kCombineChunk];
+    __shared__ float s_red[kCombineThreads / 32];
+    __shared__ float4 s_part[kCombineThreads / 32][32];
+
+    // global max over the non-empty partials
+    float M = -INFINITY;
+    for (int e = tid; e < entries; e += kCombineThreads) {
+        const float2 v = *reinterpret_cast<const float2*>(ml + combine_slot<FUSED>(p, head, bg, hl, e) * 2);
+        if (v.y > 0.f) M = fmaxf(M, v.x);
     }
 #pragma unroll
     for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(kFull, M, o));
-    if ((c & 31) == 0) red[c >> 5] = M;
+    if (cg == 0) s_red[el] = M;
     __syncthreads();
-    M = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
-    // pass 2: weights in chunks of 128 partials, then the weighted sum of their accumulators
-    for (int base = 0; base < entries && M != -INFINITY; base += kD) {
+    M = s_red[0];
+#pragma unroll
+    for (int x = 1; x < kCombineThreads / 32; ++x) M = fmaxf(M, s_red[x]);
+
+    float L = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int base = 0; base < entries && M != -INFINITY; base += kCombineChunk) {
+        const int cnt = min(kCombineChunk, entries - base);
         __syncthreads();
-        const int e = base + c;
-        float wv = 0.f;
-        if (e < entries) {
-            const size_t slot = (((size_t)(e / kNA) * units + bg) * kNA + (e % kNA)) * kMaxG + hl;
-            const float2 ml = *reinterpret_cast<const float2*>(p.fpart_ml + slot * 2);
-            if (ml.y > 0.f) {
-                wv = exp2f(ml.x - M);
-                L += wv * ml.y;
+        for (int x = tid; x < cnt; x += kCombineThreads) {
+            const float2 v = *reinterpret_cast<const float2*>(ml + combine_slot<FUSED>(p, head, bg, hl, base + x) * 2);
+            float wv = 0.f;
+            if (v.y > 0.f) {
+                wv = exp2f(v.x - M);
+                L += wv * v.y;
             }
+            s_w[x] = wv;
         }
-        wgt[c] = wv;
         __syncthreads();
-        const int cnt = min(kD, entries - base);
-        for (int x0 = 0; x0 < cnt; x0 += 8) {   // eight independent (predicated) loads in flight per thread
-            float v[8];
+        for (int x0 = el; x0 < cnt; x0 += 16 * 8) {
+            float4 v[8];
+            float wv[8];
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-                const int x = x0 + u;
-                const int e2 = base + x;
-                const size_t slot = (((size_t)(e2 / kNA) * units + bg) * kNA + (e2 % kNA)) * kMaxG + hl;
-                v[u] = (x < cnt && wgt[x] != 0.f) ? p.fpart_acc[slot * kD + c] : 0.f;
+                const int x = x0 + 16 * u;
+                wv[u] = x < cnt ? s_w[x] : 0.f;
+                v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (wv[u] != 0.f)
+                    v[u] = *reinterpret_cast<const float4*>(pacc + combine_slot<FUSED>(p, head, bg, hl, base + x) * kD +
+                                                            4 * cg);
             }
 #pragma unroll
-            for (int u = 0; u < 8; ++u) acc += (x0 + u < cnt ? wgt[x0 + u] : 0.f) * v[u];
+            for (int u = 0; u < 8; ++u) {
+                acc.x += wv[u] * v[u].x; acc.y += wv[u] * v[u].y; acc.z += wv[u] * v[u].z; acc.w += wv[u] * v[u].w;
+            }
         }
     }
-    // total L: every thread holds the share of the partials it weighted
 #pragma unroll
     for (int o = 16; o; o >>= 1) L += __shfl_xor_sync(kFull, L, o);
     __syncthreads();
-    if ((c & 31) == 0) red[c >> 5] = L;
+    if (cg == 0) s_red[el] = L;
+    s_part[el][cg] = acc;
     __syncthreads();
-    L = red[0] + red[1] + red[2] + red[3];
-    const float o = L > 0.f ? acc / L : 0.f;
-    if (p.out_fp32) reinterpret_cast<float*>(p.out)[head * kD + c] = o;
-    else reinterpret_cast<__nv_bfloat16*>(p.out)[head * kD + c] = __float2bfloat16_rn(o);
-    if (p.lse && c == 0) p.lse[head] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
+    if (tid < 32) {
+        L = 0.f;
+        float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int x = 0; x < kCombineThreads / 32; ++x) {
+            L += s_red[x];
+            const float4 v = s_part[x][tid];
+            t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
+        }
+        const float inv = L > 0.f ? 1.f / L : 0.f;
+        const float4 o = make_float4(t.x * inv, t.y * inv, t.z * inv, t.w * inv);
+        if (p.out_fp32) {
+            reinterpret_cast<float4*>(p.out)[head * (kD / 4) + tid] = o;
+        } else {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(o.x, o.y), hi = __floats2bfloat162_rn(o.z, o.w);
+            uint2 pk;
+            pk.x = *reinterpret_cast<uint32_t*>(&lo);
+            pk.y = *reinterpret_cast<uint32_t*>(&hi);
+            reinterpret_cast<uint2*>(p.out)[head * (kD / 4) + tid] = pk;
+        }
+        if (p.lse && tid == 0) p.lse[head] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
+    }
 }
 
 }  // namespace ffd

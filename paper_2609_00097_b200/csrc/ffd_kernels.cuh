@@ -26,6 +26,7 @@ constexpr int kCodeBytes = kBlk * kD / 4;
 constexpr int kWarps = 7;          // warps per decode CTA: 7 x (16 KB K slot + 16 KB V slot) of shared memory
 constexpr int kSlotBytes = kTileBytes;
 constexpr int kDecodeSmem = kWarps * 2 * kSlotBytes + 128;   // + mbarriers
+constexpr uint32_t kSuspendHintNs = 200000u;       // upper bound of one hardware-suspended try_wait
 constexpr long long kSpinCycles = 2000000000LL;   // bounded mbarrier wait (~1 s of SM clocks); then report and stop
 constexpr int kMaxG = 4;           // query heads per KV head handled by one warp
 constexpr unsigned kFull = 0xffffffffu;
@@ -56,7 +57,7 @@ struct DecodeParams {
     float* mtilde;           // [B, Hq]   (workspace)
     float* part_ml;          // dense path: [B, Hq, S, 2]   m (log2 domain), l
     float* part_acc;         // dense path: [B, Hq, S, 128]
-    uint32_t* qfrag;         // [B, Hkv, 32 lanes, 16] pre-scaled fp16 query fragments of the scan (workspace)
+    unsigned char* qrec;     // [B, Hkv] query records of the scan: fp16 fragments + thresholds (workspace)
     float* fpart_ml;         // fused path: [items, attend warps, 4 heads, 2]
     float* fpart_acc;        // fused path: [items, attend warps, 4 heads, 128]
     int total_items;         // fused path: work items = ceil(max_blocks / 32) * B * Hkv
@@ -119,15 +120,17 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
 }
 
-// Bounded wait for the phase with the given parity; false when the limit ran out.
+// Bounded wait for the phase with the given parity; false when the limit ran out.  The suspend-time hint lets the
+// hardware park the warp until the phase completes instead of polling: a waiting warp must not eat the issue
+// slots of the warps it is waiting for.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     long long t0 = 0;
     for (;;) {
         uint32_t ok;
         asm volatile(
-            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}\n"
             : "=r"(ok)
-            : "r"(bar), "r"(parity)
+            : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
             : "memory");
         if (ok) return true;
         const long long now = clock64();
@@ -246,26 +249,40 @@ __device__ __forceinline__ void scan_load(ScanRegs& sr, const uint4* __restrict_
     for (int x = 0; x < 4; ++x) sr.s[x] = __ldg(scales_tile + 4 * (lane & 3) + x);
 }
 
+// B operand of four k-step halves: hi / lo piece of (pre-scaled q) * scale for this lane's column
+__device__ __forceinline__ void scan_bfrag4(uint32_t* bfrag, const uint4& qv, const uint4& sv, int piece) {
+    const uint32_t q[4] = {qv.x, qv.y, qv.z, qv.w};
+    const uint32_t sc[4] = {sv.x, sv.y, sv.z, sv.w};
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        const __half2 a = *reinterpret_cast<const __half2*>(&q[x]);
+        const __half2 b = *reinterpret_cast<const __half2*>(&sc[x]);
+        const __half2 hi = __hmul2(a, b);
+        const __half2 lo = __hfma2(a, b, __hneg2(hi));
+        const __half2 pick = piece ? lo : hi;
+        bfrag[x] = *reinterpret_cast<const uint32_t*>(&pick);
+    }
+}
+
+template <bool PRECISE>
+__device__ __forceinline__ float scan_mma(const uint4 (&w)[4], const uint32_t (&bfrag)[16], int lane, int rows,
+                                          float sm_scale, float& band);
+
 template <bool PRECISE>
 __device__ __forceinline__ float scan_compute(const ScanRegs& sr, const ScanQuery& sq, int lane, int rows,
                                               float sm_scale, float& band) {
-    const int r = lane >> 2;
-    const uint4* w = sr.w;
-    uint32_t sc[16];
-#pragma unroll
-    for (int x = 0; x < 4; ++x) {
-        sc[4 * x] = sr.s[x].x; sc[4 * x + 1] = sr.s[x].y; sc[4 * x + 2] = sr.s[x].z; sc[4 * x + 3] = sr.s[x].w;
-    }
     uint32_t bfrag[16];
 #pragma unroll
-    for (int x = 0; x < 16; ++x) {
-        __half2 qv = *reinterpret_cast<const __half2*>(&sq.qh[x]);
-        __half2 sv = *reinterpret_cast<const __half2*>(&sc[x]);
-        __half2 hi = __hmul2(qv, sv);
-        __half2 lo = __hfma2(qv, sv, __hneg2(hi));
-        __half2 pick = sq.piece ? lo : hi;
-        bfrag[x] = *reinterpret_cast<uint32_t*>(&pick);
-    }
+    for (int x = 0; x < 4; ++x)
+        scan_bfrag4(bfrag + 4 * x, make_uint4(sq.qh[4 * x], sq.qh[4 * x + 1], sq.qh[4 * x + 2], sq.qh[4 * x + 3]),
+                    sr.s[x], sq.piece);
+    return scan_mma<PRECISE>(sr.w, bfrag, lane, rows, sm_scale, band);
+}
+
+template <bool PRECISE>
+__device__ __forceinline__ float scan_mma(const uint4 (&w)[4], const uint32_t (&bfrag)[16], int lane, int rows,
+                                          float sm_scale, float& band) {
+    const int r = lane >> 2;
     float acc[4][4];
     float off[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
