@@ -7,12 +7,13 @@
 //   4 attend warps  take the kept blocks of a published batch, stage their K and V tiles (16 KB each) through
 //                   private swizzled slots with cp.async + mbarrier and run the exact online-softmax attention.
 // A work item is 24 consecutive blocks of one (sequence, KV head).  Items are handed out dynamically: lane 0 of scan
-// warp 0 draws item numbers from a global counter three items ahead (the atomic's latency is never waited for),
-// publishes them in a small ring two items ahead and starts the copy of the item's query record (pre-scaled fp16
-// query fragments + thresholds, written by the pseudo-max kernel) into shared memory; one named barrier per item
-// keeps the scan warps in step.  Attend warps learn the item from the batch descriptor.  Scan warps run up to two
-// batches ahead of the attend warps (two descriptors, full/empty mbarriers).
-// Every mbarrier wait is bounded; on expiry the warp records kDevTimeout and the CTA winds down.
+// warp 0 draws item numbers from a global counter (the atomic for the next draw is always in flight, so its latency
+// is not waited for), skips items without blocks, decodes the item once and publishes it two items ahead in a tagged
+// ring in shared memory; it also starts the copy of the item's query record (pre-scaled fp16 query fragments +
+// thresholds, written by the pseudo-max kernel).  Readers check the tag; nobody divides or reloads sequence
+// lengths on the per-block path.  Scan warps run up to two batches ahead of the attend warps (two descriptors,
+// full/empty mbarriers), which also keeps all scan warps within one batch of each other.
+// Every wait is bounded; on expiry the warp records kDevTimeout and the CTA winds down.
 #pragma once
 #include "ffd_kernels.cuh"
 
@@ -28,13 +29,23 @@ constexpr int kItemBlocks = 24;        // blocks per work item: two per scan war
 constexpr int kRing = 3;               // code-ring stages per scan warp
 constexpr int kStageBytes = kCodeBytes + kD * 2;   // 2048 B codes + 256 B scales
 constexpr int kNB = 2;                 // batch descriptors in flight
-constexpr int kIdRing = 8;             // item numbers known ahead
+constexpr int kItemRing = 8;           // decoded items published ahead
 constexpr int kQrecRing = 4;           // query records staged ahead
 constexpr int kQrecBytes = 2048 + 32;  // [4][32 lanes] uint4 of fp16 query fragments, then 4 thresholds (+ pad)
 
+struct Item {
+    int item;                          // work item number; < 0: no more work
+    int b, g, blk0, nblk, n;           // sequence, KV head, first block, blocks (1..24), tokens of the sequence
+};
+
+struct ItemSlot {                      // entry `seq` of the published-item ring is valid when tag == seq
+    volatile int tag;
+    volatile int item, b, g, blk0, nblk, n;
+    int pad;
+};
+
 struct BatchDesc {
-    int item;                          // work item of this batch; < 0: no more work
-    int pad[3];
+    int item, b, g, nblk;              // work item of this batch; item < 0: no more work
     uint32_t tile[kItemBlocks];        // (page, KV head) tile of each block of the item
     uint8_t keep4[kItemBlocks];        // bit h: query head h of the group keeps the block; 0 = skipped
     uint8_t rows[kItemBlocks];         // valid tokens
@@ -46,22 +57,21 @@ constexpr int kOffQrec = kOffRing + kNS * kRing * kStageBytes;
 constexpr int kOffDesc = kOffQrec + kQrecRing * kQrecBytes;
 constexpr int kOffBars = kOffDesc + kNB * (int)sizeof(BatchDesc);
 constexpr int kNumBars = 2 * kNB + 2 * kNA + kQrecRing;          // full, empty, K/V slots, query records
-constexpr int kOffIds = kOffBars + kNumBars * 8;                 // ring of item numbers + abort flag
-constexpr int kFusedSmem = kOffIds + (kIdRing + 4) * 4;
+constexpr int kOffItems = kOffBars + kNumBars * 8;               // ring of decoded items
+constexpr int kOffStageTile = kOffItems + kItemRing * (int)sizeof(ItemSlot);   // tile index of each ring stage
+constexpr int kOffAbort = kOffStageTile + kNS * 4 * 4;
+constexpr int kFusedSmem = kOffAbort + 16;
 static_assert(kOffBars % 8 == 0 && kOffRing % 16 == 0 && kOffDesc % 16 == 0 && kOffQrec % 16 == 0, "alignment");
-static_assert(sizeof(BatchDesc) % 16 == 0, "descriptor size");
+static_assert(sizeof(BatchDesc) % 16 == 0 && sizeof(ItemSlot) == 32, "descriptor sizes");
 static_assert(kFusedSmem <= 227 * 1024, "shared memory budget");
 
-struct Item {
-    int b, g, blk0, nblk, n;           // nblk <= 0: nothing to do
-};
-
+// Items are numbered from the END of the sequences backwards: the local window, whose blocks are the most likely
+// to be kept (and therefore the most expensive), is handed out first.
 __device__ __forceinline__ Item decode_item(const DecodeParams& p, int item) {
     Item it;
-    // items are numbered from the END of the sequences backwards: the local window, whose blocks are the most
-    // likely to be kept (and therefore the most expensive), is handed out first
     const int units = p.batch * p.Hkv;
     const int bg = item % units, split = p.total_items / units - 1 - item / units;
+    it.item = item;
     it.b = bg / p.Hkv;
     it.g = bg % p.Hkv;
     it.n = clamped_seq_len(p, it.b);
@@ -84,50 +94,89 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
+// ---- published items ---------------------------------------------------------------------------------------
+
+__device__ __forceinline__ bool item_ready(const ItemSlot* ring, int seq) { return ring[seq & (kItemRing - 1)].tag == seq; }
+
+__device__ __forceinline__ Item item_read(const ItemSlot* ring, int seq) {
+    const ItemSlot& e = ring[seq & (kItemRing - 1)];
+    __threadfence_block();
+    Item it;
+    it.item = e.item; it.b = e.b; it.g = e.g; it.blk0 = e.blk0; it.nblk = e.nblk; it.n = e.n;
+    return it;
+}
+
+// bounded wait for entry `seq` (it is normally there long before it is needed)
+__device__ __forceinline__ bool item_wait(const ItemSlot* ring, int seq) {
+    if (item_ready(ring, seq)) return true;
+    const long long t0 = clock64();
+    while (!item_ready(ring, seq)) {
+        __nanosleep(64);
+        if (clock64() - t0 > kSpinCycles) return false;
+    }
+    return true;
+}
+
+// Lane 0 of scan warp 0: draw the next item that has blocks and publish it as entry `seq`.
+// `pend` holds the result of an atomicAdd issued earlier; `done` is set once the counter ran past the last item.
+__device__ __forceinline__ Item item_publish(const DecodeParams& p, ItemSlot* ring, int seq, int& pend, bool& done) {
+    Item it;
+    it.item = -1; it.b = it.g = it.blk0 = it.nblk = it.n = 0;
+    while (!done) {
+        const int cand = pend;
+        if (cand >= p.total_items) { done = true; break; }
+        pend = (int)atomicAdd(p.item_counter, 1u);   // keep the next draw in flight
+        const Item c = decode_item(p, cand);
+        if (c.nblk > 0) { it = c; break; }
+    }
+    ItemSlot& e = ring[seq & (kItemRing - 1)];
+    e.item = it.item; e.b = it.b; e.g = it.g; e.blk0 = it.blk0; e.nblk = it.nblk; e.n = it.n;
+    __threadfence_block();
+    e.tag = seq;
+    return it;
+}
+
 // ---- scan role ---------------------------------------------------------------------------------------------
 
-__device__ __forceinline__ void scan_warps_barrier() { asm volatile("bar.sync 1, %0;\n" ::"n"(kNS * 32) : "memory"); }
-
-// Position of a scan warp in its stream of blocks: item after item (in the order the item numbers were drawn),
-// local blocks w and w + 12.
+// Position of a scan warp in its stream of blocks: published item after published item, local blocks w and w + 12.
 struct ScanCursor {
-    int seq;       // index of the drawn item the cursor is in
-    Item it;       // nblk = 0 before the first item
+    int seq;       // published item the cursor is in (-1 before the first)
+    Item it;
     int lb;
     bool end;      // ran into the end of the work
 };
 
-// Advance to this warp's next block.  Returns false when that block lies beyond the items whose numbers are known
-// (seq <= horizon) or beyond the end of the work; the cursor then stays where it can resume.
-__device__ __forceinline__ bool cursor_next(ScanCursor& c, const DecodeParams& p, const volatile int* ids, int horizon,
-                                            int w) {
+// Advance to this warp's next block; false when the item it lies in has not been published yet (the cursor then
+// stays where it can resume) or when there is no more work.
+__device__ __forceinline__ bool cursor_next(ScanCursor& c, const ItemSlot* items, int w) {
     if (c.end) return false;
     int lb = c.lb + kNS;
     while (lb >= c.it.nblk) {
-        if (c.seq + 1 > horizon) { c.lb = lb - kNS; return false; }
-        const int item = ids[(c.seq + 1) & (kIdRing - 1)];
+        if (!item_ready(items, c.seq + 1)) { c.lb = lb - kNS; return false; }
+        c.it = item_read(items, c.seq + 1);
         ++c.seq;
-        if (item >= p.total_items) { c.end = true; c.it.nblk = 0; return false; }
-        c.it = decode_item(p, item);
+        if (c.it.item < 0) { c.end = true; c.it.nblk = 0; return false; }
         lb = w;
     }
     c.lb = lb;
     return true;
 }
 
-// start the copy of one block's codes + scales into a ring stage (one commit group)
-__device__ __forceinline__ void ring_issue(const DecodeParams& p, const ScanCursor& c, uint32_t stage, int lane) {
+// start the copy of one block's codes + scales into a ring stage (one commit group); remembers the block's tile
+__device__ __forceinline__ void ring_issue(const DecodeParams& p, const ScanCursor& c, uint32_t stage,
+                                           volatile int* stage_tile, int lane) {
     const int page = page_of(p, c.it.b, c.it.blk0 + c.lb);
-    if (page >= 0) {
-        const size_t tile = (size_t)page * p.Hkv + c.it.g;
-        const uint4* codes = reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes);
+    const int tile = page >= 0 ? page * p.Hkv + c.it.g : -1;
+    if (tile >= 0) {
+        const uint4* codes = reinterpret_cast<const uint4*>(p.k_quant + (size_t)tile * kCodeBytes);
 #pragma unroll
         for (int x = 0; x < 4; ++x) cp_async16(stage + (x * 32 + lane) * 16, codes + x * 32 + lane);
         // scales: 16-byte chunk 4j + x lands at position 4x + j, so the four chunks read together are adjacent
         if (lane < 16)
             cp_async16(stage + kCodeBytes + ((lane & 3) * 4 + (lane >> 2)) * 16,
-                       reinterpret_cast<const uint4*>(p.k_scales + tile * kD) + lane);
+                       reinterpret_cast<const uint4*>(p.k_scales + (size_t)tile * kD) + lane);
     }
+    if (lane == 0) *stage_tile = tile;
     asm volatile("cp.async.commit_group;\n" ::: "memory");
 }
 
@@ -137,18 +186,15 @@ __device__ __forceinline__ void ring_wait(int younger) {
     else asm volatile("cp.async.wait_group 0;\n" ::: "memory");
 }
 
-// Warp 0 only: if `item` has work, copy its query record into the next slot of the record ring and report
-// completion on that slot's mbarrier.  Records are numbered like batches (items with work, in drawing order), so
-// every scan warp waits for every phase of every slot barrier and a parity wait can never see a stale phase.
-__device__ __forceinline__ void qrec_issue(const DecodeParams& p, int item, uint32_t qrecs, uint32_t qbars,
-                                           int& records, int lane) {
-    if (item >= p.total_items || decode_item(p, item).nblk <= 0) return;
-    const int slot = records & (kQrecRing - 1);
-    const int bg = item % (p.batch * p.Hkv);
+// Warp 0 only: copy the query record of published item `seq` into slot seq % 4 of the record ring and report
+// completion on that slot's mbarrier.  Every scan warp waits for every record, in order, so a parity wait can
+// never see a stale phase.
+__device__ __forceinline__ void qrec_issue(const DecodeParams& p, int seq, int bg, uint32_t qrecs, uint32_t qbars,
+                                           int lane) {
+    const int slot = seq & (kQrecRing - 1);
     const uint4* src = reinterpret_cast<const uint4*>(p.qrec + (size_t)bg * kQrecBytes);
     for (int c = lane; c < kQrecBytes / 16; c += 32) cp_async16(qrecs + slot * kQrecBytes + c * 16, src + c);
     cp_async_arrive(qbars + slot * 8);
-    ++records;
 }
 
 // The precise variant of the scan for one block, with the arithmetic m_tilde was computed in.  Kept out of line so
@@ -175,25 +221,25 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
     const uint32_t bars = smem_u32(smem) + kOffBars;
     const uint32_t qbars = bars + (2 * kNB + 2 * kNA) * 8;
     BatchDesc* descs = reinterpret_cast<BatchDesc*>(smem + kOffDesc);
-    volatile int* ids = reinterpret_cast<volatile int*>(smem + kOffIds);
-    volatile int* abort_flag = ids + kIdRing;
+    ItemSlot* items = reinterpret_cast<ItemSlot*>(smem + kOffItems);
+    volatile int* stage_tile = reinterpret_cast<volatile int*>(smem + kOffStageTile) + w * 4;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffAbort);
+    const int units = p.batch * p.Hkv;
 
-    // warp 0 draws the first item numbers: two are published now, the third is held until the first iteration
+    // warp 0 publishes items 0 and 1 (and stages their records) before anybody starts
     int pend = p.total_items;
-    int records = 0;                // query records staged so far (warp 0)
+    bool done = false;
     if (w == 0) {
-        int id0 = 0, id1 = 0;
+        int item0 = -1, item1 = -1;
         if (lane == 0) {
-            id0 = (int)atomicAdd(p.item_counter, 1u);
-            id1 = (int)atomicAdd(p.item_counter, 1u);
             pend = (int)atomicAdd(p.item_counter, 1u);
-            ids[0] = min(id0, p.total_items);
-            ids[1] = min(id1, p.total_items);
+            item0 = item_publish(p, items, 0, pend, done).item;
+            item1 = item_publish(p, items, 1, pend, done).item;
         }
-        id0 = min(__shfl_sync(kFull, id0, 0), p.total_items);
-        id1 = min(__shfl_sync(kFull, id1, 0), p.total_items);
-        qrec_issue(p, id0, qrecs, qbars, records, lane);
-        qrec_issue(p, id1, qrecs, qbars, records, lane);
+        item0 = __shfl_sync(kFull, item0, 0);
+        item1 = __shfl_sync(kFull, item1, 0);
+        if (item0 >= 0) qrec_issue(p, 0, item0 % units, qrecs, qbars, lane);
+        if (item1 >= 0) qrec_issue(p, 1, item1 % units, qrecs, qbars, lane);
     }
     ScanCursor ic;
     ic.seq = -1;
@@ -201,61 +247,44 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
     ic.lb = w - kNS;
     ic.end = false;
     int issued = 0, consumed = 0;   // this warp's blocks whose copies were started / whose data was taken
-    int bi = 0;                     // batches published so far
 
 #pragma unroll 1
-    for (int seq = 0;; ++seq) {
-        if (w == 0) {   // publish the item number of seq + 2, draw the one of seq + 3, stage the record of seq + 2
-            int id2 = 0;
-            if (lane == 0) {
-                id2 = min(pend, p.total_items);
-                ids[(seq + 2) & (kIdRing - 1)] = id2;
-                pend = id2 < p.total_items ? (int)atomicAdd(p.item_counter, 1u) : p.total_items;
-            }
-            id2 = __shfl_sync(kFull, id2, 0);
-            qrec_issue(p, id2, qrecs, qbars, records, lane);
+    for (int seq = 0;; ++seq) {     // published item seq = batch seq
+        if (w == 0) {               // publish item seq + 2 and stage its record
+            int item2 = -1;
+            if (lane == 0) item2 = item_publish(p, items, seq + 2, pend, done).item;
+            item2 = __shfl_sync(kFull, item2, 0);
+            if (item2 >= 0) qrec_issue(p, seq + 2, item2 % units, qrecs, qbars, lane);
         }
-        __syncwarp();
-        scan_warps_barrier();          // item numbers of seq, seq + 1, seq + 2 are visible to all scan warps
-        const int horizon = seq + 2;
-        const int item = ids[seq & (kIdRing - 1)];
-        if (item >= p.total_items || *abort_flag) {   // no more work: tell the attend warps
-            const int slot = bi & 1, use = bi >> 1;
-            if (use > 0 && !mbar_wait(bars + (kNB + slot) * 8, (use - 1) & 1)) *abort_flag = 1;
+        if (!item_wait(items, seq)) *abort_flag = 1;
+        const Item it = item_read(items, seq);
+        const int slot = seq & 1, use = seq >> 1;
+        // the attend warps must have released this descriptor (two batches ago)
+        if (use > 0 && !mbar_wait(bars + (kNB + slot) * 8, (use - 1) & 1)) *abort_flag = 1;
+        BatchDesc& d = descs[slot];
+        if (it.item < 0 || *abort_flag) {   // no more work: tell the attend warps
             if (lane == 0) {
-                if (w == 0) descs[slot].item = -1;
+                if (w == 0) d.item = -1;
                 mbar_arrive(bars + slot * 8);
             }
             break;
         }
-        const Item it = decode_item(p, item);
-        // The prefetch cursor never trails the item being processed: everything of this warp before `seq` has been
-        // consumed, hence issued.  (It would otherwise fall behind during runs of empty items and read slots of the
-        // item-number ring that have been reused.)
-        if (ic.seq < seq) {
-            ic.seq = seq;
-            ic.it = it;
-            ic.lb = w - kNS;
-        }
-        if (it.nblk <= 0) continue;    // nothing in this item (sequence shorter than the longest): no batch
-        const int slot = bi & 1, use = bi >> 1;
-        // the attend warps must have released this descriptor (two batches ago); the query record must have landed
-        if (use > 0 && !mbar_wait(bars + (kNB + slot) * 8, (use - 1) & 1)) *abort_flag = 1;
-        if (!mbar_wait(qbars + (bi & (kQrecRing - 1)) * 8, (bi / kQrecRing) & 1)) *abort_flag = 1;
-        BatchDesc& d = descs[slot];
-        const uint32_t qrec = qrecs + (bi & (kQrecRing - 1)) * kQrecBytes;
+        // the item's query record must have landed
+        if (!mbar_wait(qbars + (seq & (kQrecRing - 1)) * 8, (seq / kQrecRing) & 1)) *abort_flag = 1;
+        const uint32_t qrec = qrecs + (seq & (kQrecRing - 1)) * kQrecBytes;
         const size_t head0 = (size_t)it.b * p.Hq + (size_t)it.g * p.G;
         float thr;
         asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(thr) : "r"(qrec + 2048 + j * 4));
-        if (w == 0 && lane == 0) d.item = item;
+        if (w == 0 && lane == 0) { d.item = it.item; d.b = it.b; d.g = it.g; d.nblk = it.nblk; }
 #pragma unroll 1
         for (int lb = w; lb < it.nblk; lb += kNS) {
             // keep the ring full: blocks consumed .. consumed + kRing - 1 of this warp's stream
-            while (issued < consumed + kRing && cursor_next(ic, p, ids, horizon, w)) {
-                ring_issue(p, ic, ring + (issued % kRing) * kStageBytes, lane);
+            while (issued < consumed + kRing && cursor_next(ic, items, w)) {
+                ring_issue(p, ic, ring + (issued % kRing) * kStageBytes, stage_tile + issued % kRing, lane);
                 ++issued;
             }
-            const uint32_t stage = ring + (consumed % kRing) * kStageBytes;
+            const int st = consumed % kRing;
+            const uint32_t stage = ring + st * kStageBytes;
             ring_wait(issued - consumed - 1);
             __syncwarp();
             // codes into registers; B operand straight from the staged scales and the item's query record
@@ -267,27 +296,25 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
             for (int x = 0; x < 4; ++x)
                 scan_bfrag4(bfrag + 4 * x, lds128(qrec + (x * 32 + lane) * 16),
                             lds128(stage + kCodeBytes + (4 * x + j) * 16), r & 1);
+            const int tile = stage_tile[st];
             __syncwarp();   // the stage is free again
             ++consumed;
-            if (issued < consumed + kRing && cursor_next(ic, p, ids, horizon, w)) {
-                ring_issue(p, ic, ring + (issued % kRing) * kStageBytes, lane);
+            if (issued < consumed + kRing && cursor_next(ic, items, w)) {
+                ring_issue(p, ic, ring + (issued % kRing) * kStageBytes, stage_tile + issued % kRing, lane);
                 ++issued;
             }
 
             const int blk = it.blk0 + lb;
-            const int page = page_of(p, it.b, blk);
             const int rows = min(kBlk, it.n - blk * kBlk);
             unsigned keep4 = 0;
-            if (page >= 0) {
+            if (tile >= 0) {
                 float band;
                 float bm = scan_mma<false>(wv, bfrag, lane, rows, p.sm_scale, band);
                 // too close to call (rare): a separate, non-inlined routine re-reads the block and redoes it precisely
-                if (__any_sync(kFull, (j < p.G) && fabsf(bm - thr) <= band)) {
-                    const size_t tile = (size_t)page * p.Hkv + it.g;
-                    bm = scan_block_precise(reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes),
-                                            reinterpret_cast<const uint4*>(p.k_scales + tile * kD), qrec, lane, rows,
-                                            p.sm_scale);
-                }
+                if (__any_sync(kFull, (j < p.G) && fabsf(bm - thr) <= band))
+                    bm = scan_block_precise(reinterpret_cast<const uint4*>(p.k_quant + (size_t)tile * kCodeBytes),
+                                            reinterpret_cast<const uint4*>(p.k_scales + (size_t)tile * kD), qrec, lane,
+                                            rows, p.sm_scale);
                 const bool keep = (j < p.G) && (bm >= thr);
                 keep4 = __ballot_sync(kFull, keep) & 0xFu;
                 if (r == 0 && j < p.G) {
@@ -297,14 +324,13 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
                 }
             }
             if (lane == 0) {
-                d.tile[lb] = page >= 0 ? (uint32_t)((size_t)page * p.Hkv + it.g) : 0u;
+                d.tile[lb] = tile >= 0 ? (uint32_t)tile : 0u;
                 d.keep4[lb] = (uint8_t)keep4;
                 d.rows[lb] = (uint8_t)rows;
             }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(bars + slot * 8);   // this warp's share of the batch is published
-        ++bi;
     }
     cp_async_drain();
     if (*abort_flag && w == 0 && lane == 0) atomicOr(p.status, kDevTimeout);
@@ -344,7 +370,8 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
         const BatchDesc& d = descs[slot];
         const int item = d.item;
         if (item < 0) break;
-        const Item it = decode_item(p, item);
+        Item it;
+        it.item = item; it.b = d.b; it.g = d.g; it.nblk = d.nblk;
         unsigned mine = my_entries(d, it.nblk, a, lane);
         const bool any = mine != 0;
         if (any) attend_setup(st, p.q + ((size_t)it.b * p.Hq + (size_t)it.g * p.G) * kD, p.G, lane);
@@ -368,7 +395,7 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
                 if (mbar_test(bars + (bi2 & 1) * 8, (bi2 >> 1) & 1)) {
                     const BatchDesc& d2 = descs[bi2 & 1];
                     if (d2.item >= 0) {
-                        const unsigned mine2 = my_entries(d2, decode_item(p, d2.item).nblk, a, lane);
+                        const unsigned mine2 = my_entries(d2, d2.nblk, a, lane);
                         if (mine2) {
                             const int nlb = __ffs(mine2) - 1;
                             next_k = kbase + (size_t)d2.tile[nlb] * kTileVec;
@@ -428,7 +455,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodePa
             mbar_init(bars + (kNB + s) * 8, kNA);     // empty: one arrival per attend warp
         }
         for (int a = 0; a < 2 * kNA + kQrecRing; ++a) mbar_init(bars + (2 * kNB + a) * 8, 32);
-        reinterpret_cast<volatile int*>(smem + kOffIds)[kIdRing] = 0;   // abort flag
+        for (int s = 0; s < kItemRing; ++s) reinterpret_cast<ItemSlot*>(smem + kOffItems)[s].tag = -1;
+        *reinterpret_cast<volatile int*>(smem + kOffAbort) = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     __syncthreads();

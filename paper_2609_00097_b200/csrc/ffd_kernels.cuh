@@ -289,6 +289,9 @@ __device__ __forceinline__ float scan_mma(const uint4 (&w)[4], const uint32_t (&
     for (int mt = 0; mt < 4; ++mt)
 #pragma unroll
         for (int x = 0; x < 4; ++x) acc[mt][x] = 0.f;
+    uint4 t[4];   // bits 10..15 of every half moved down to 0..5 (k-steps 5..7)
+#pragma unroll
+    for (int mt = 0; mt < 4; ++mt) t[mt] = make_uint4(w[mt].x >> 10, w[mt].y >> 10, w[mt].z >> 10, w[mt].w >> 10);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const int e = i < 5 ? i : i - 5;
@@ -296,8 +299,8 @@ __device__ __forceinline__ float scan_mma(const uint4 (&w)[4], const uint32_t (&
         const uint32_t one = 0x00010001u << (2 * e);
 #pragma unroll
         for (int mt = 0; mt < 4; ++mt) {
-            uint32_t x0 = w[mt].x, x1 = w[mt].y, x2 = w[mt].z, x3 = w[mt].w;
-            if (i >= 5) { x0 >>= 10; x1 >>= 10; x2 >>= 10; x3 >>= 10; }
+            const uint4 src = i < 5 ? w[mt] : t[mt];
+            const uint32_t x0 = src.x, x1 = src.y, x2 = src.z, x3 = src.w;
             if (PRECISE) {
                 float part[4] = {0.f, 0.f, 0.f, 0.f};
                 mma_f16(part, x0 & mask, x1 & mask, x2 & mask, x3 & mask, bfrag[2 * i], bfrag[2 * i + 1]);
