@@ -36,9 +36,10 @@ METRIC = "sparse_decode_attn_us_per_step"
 UNIT = "us/step"
 CODE_BYTES_PER_TILE = 2048 + 256          # packed 2-bit codes + fp16 scales of one (block, KV head)
 KV_BYTES_PER_TILE = 2 * 64 * 128 * 2      # K tile + V tile of one kept (block, KV head)
-# DRAM bytes per launch of the fused kernel from the ncu capture summarised under profiles/ (None until
-# captured); reported as measured bytes / algorithmic bytes of the captured case times this run's bytes.
-NCU_TRAFFIC_RATIO = None
+# dram__bytes_read + dram__bytes_write of one fused-kernel launch divided by the launch's algorithmic bytes, from
+# the ncu capture summarised in profiles/fused_sparse_kernel_C3_ctx32768.md (same kernel, same workload recipe at
+# context 32768; traffic grows in proportion to the blocks processed): (308.47 + 5.65) MB / 308.28 MB.
+NCU_TRAFFIC_RATIO = 1.019
 
 
 def measured_peaks():
@@ -103,6 +104,16 @@ class ClockSampler:
         return {"sm_mhz": statistics.median([s[1] for s in inside]) if inside else None,
                 "sm_max_mhz": max([s[2] for s in inside]) if inside else None, "samples": len(inside),
                 "window": window, "reasons": reasons}
+
+
+def reduce_max_over_ranks(values, dist, device="cpu"):
+    """Max over ranks of a list of floats (the only exchange of a multi-rank run: the path itself shards over
+    (sequence, KV head) with no collective)."""
+    if dist is None:
+        return [float(v) for v in values]
+    t = torch.tensor(values, device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
 
 
 def union_kept_tiles(kept: np.ndarray, w) -> int:
@@ -321,10 +332,7 @@ def main():
 
     t_step = statistics.mean(step_us)
     t_e2e = statistics.mean(e2e_us)
-    if dist is not None:
-        t = torch.tensor([t_step, t_e2e], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        t_step, t_e2e = float(t[0]), float(t[1])
+    t_step, t_e2e = reduce_max_over_ranks([t_step, t_e2e], dist, "cuda")
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -344,7 +352,7 @@ def main():
         "gpu_launches": 4 * args.steps,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": (None if NCU_TRAFFIC_RATIO is None else sparse_bytes * NCU_TRAFFIC_RATIO),
-                     "peak_source": f"{peak_kind} copy bandwidth (of {peak_kind})", "kernel": "decode_kernel<true>",
+                     "peak_source": f"{peak_kind} copy bandwidth (of {peak_kind})", "kernel": "fused_sparse_kernel",
                      "kernel_us": t_kernel, "algorithmic_bytes": sparse_bytes,
                      "frac_of_nominal_8TBs": achieved / 8000.0},
         "step_us_median": statistics.median(step_us), "step_us_min": min(step_us),
