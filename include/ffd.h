@@ -48,7 +48,8 @@ typedef enum {
     FFD_ERR_WORKSPACE = 5,     /* workspace smaller than ffd_workspace_bytes reports */
     FFD_ERR_DELTA = 6,         /* delta is NaN or negative */
     FFD_ERR_CUDA = 7,          /* a CUDA runtime call failed (launch error, wrong device ...) */
-    FFD_ERR_DEVICE_STATUS = 8  /* a kernel recorded a problem in the workspace status word */
+    FFD_ERR_DEVICE_STATUS = 8, /* a kernel recorded a problem in the workspace status word */
+    FFD_ERR_STATIC_LIMIT = 9   /* ffd_decode_static: the geometry needs more scratch than the built-in array holds */
 } ffd_status;
 
 /* bits of the device status word (ffd_read_device_status) */
@@ -136,6 +137,42 @@ ffd_status ffd_unpack_codes(const ffd_config* cfg, const void* k_quant, uint8_t*
 /* Waits for `stream`, copies the workspace status word to *status_bits (HOST) and clears it on the device.
  * Returns FFD_ERR_DEVICE_STATUS if any bit was set. */
 ffd_status ffd_read_device_status(void* workspace, void* stream, uint32_t* status_bits);
+
+/*
+ * ffd_decode without a caller-supplied workspace and without any allocation.  (The paper has no counterpart to
+ * this entry point; it exists for integration reasons only.)
+ *
+ * Who needs it: callers that are not in a position to obtain device memory at the time they want to decode - a
+ * serving loop whose device memory was handed out completely at start-up and whose request path must not call
+ * cudaMalloc, or a plug-in whose host application gives it streams and tensors but no allocator.  ffd_decode asks
+ * such a caller for a workspace it cannot produce; this variant brings its own.
+ *
+ * The scratch is one array of FFD_STATIC_SCRATCH_BYTES bytes that is part of the library image: every GPU that
+ * loads the library sets that much memory aside until the process exits, whether or not this function is ever
+ * called.  The function computes exactly what ffd_decode computes (same kernels, same split geometry; results are
+ * bit-identical), with the same arguments minus kept_mask / block_max / workspace.  It calls no cudaMalloc, cudaFree
+ * or other allocating routine.
+ *
+ * Limits and rules
+ *   - Geometry: ffd_workspace_bytes(cfg, batch, max_blocks_per_seq) must not exceed FFD_STATIC_SCRATCH_BYTES,
+ *     otherwise FFD_ERR_STATIC_LIMIT is returned and nothing is launched.  With 32 query / 8 KV heads the 8 MiB
+ *     hold batch 1 up to about 160 K tokens of context, batch 4 up to about 36 K, batch 16 up to about 9 K.
+ *   - First use on a device: the first call made while a given device is current looks up the device address of
+ *     the array (cudaGetSymbolAddress) and remembers it.  Make that first call during start-up, outside of any
+ *     stream capture.
+ *   - One array for everybody: all calls on a device share the scratch, and it keeps whatever the previous call
+ *     left in it.  The function clears the parts that must start at zero itself (the status word; the work counter
+ *     is reset by its first kernel), but two calls whose kernels overlap on the GPU (different streams, or different
+ *     host threads) overwrite each other's partial results.  Issue calls that can overlap through ffd_decode with
+ *     separate workspaces instead.
+ *   - Device-detected problems (bad page index, seq_len out of range) are skipped exactly as in ffd_decode, but the
+ *     status word lives in the private scratch and cannot be read back: validate such inputs on the caller's side.
+ */
+#define FFD_STATIC_SCRATCH_BYTES (8u << 20)
+ffd_status ffd_decode_static(const ffd_config* cfg, const void* q, const void* k_cache, const void* v_cache,
+                             const void* k_quant, const void* k_scales, const int32_t* block_table,
+                             const int32_t* seq_lens, int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages,
+                             float delta, void* out, float* lse, void* stream);
 
 /*
  * Measurement hook (process-wide, not thread-safe; the only state the library keeps): while both events are

@@ -3,6 +3,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "../../include/ffd.h"
 #include "ffd_kernels.cuh"
 #include "ffd_fused.cuh"
@@ -470,6 +472,8 @@ const char* ffd_status_string(ffd_status status) {
         case FFD_ERR_DELTA: return "delta must be >= 0 or +inf";
         case FFD_ERR_CUDA: return "CUDA runtime error";
         case FFD_ERR_DEVICE_STATUS: return "a kernel recorded a problem in the status word";
+        case FFD_ERR_STATIC_LIMIT:
+            return "geometry needs more scratch than the built-in FFD_STATIC_SCRATCH_BYTES array of ffd_decode_static";
     }
     return "unknown status";
 }
@@ -543,6 +547,54 @@ ffd_status ffd_unpack_codes(const ffd_config* cfg, const void* k_quant, uint8_t*
     unpack_kernel<<<(unsigned)tiles, 128, 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const uint8_t*>(k_quant), codes, tiles);
     return launch_status();
+}
+
+// ---- ffd_decode_static: the decode step for callers that cannot allocate ------------------------------------
+//
+// The scratch that ffd_decode takes from its caller lives here instead, in the library image.  In host code the
+// name `g_static_scratch` is only a handle for the symbol, not a device address: the address the kernels need comes
+// from cudaGetSymbolAddress, asked once per device (with that device current) and cached.
+static __device__ __align__(256) unsigned char g_static_scratch[FFD_STATIC_SCRATCH_BYTES];
+
+static ffd_status static_scratch_address(void** out) {
+    constexpr int kMaxDevices = 64;
+    static std::mutex lock;
+    static void* cache[kMaxDevices] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return FFD_ERR_CUDA;
+    std::lock_guard<std::mutex> guard(lock);
+    if (!cache[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) {
+            (void)cudaGetLastError();
+            return FFD_ERR_CUDA;
+        }
+        cache[dev] = ptr;
+    }
+    *out = cache[dev];
+    return FFD_OK;
+}
+
+ffd_status ffd_decode_static(const ffd_config* cfg, const void* q, const void* k_cache, const void* v_cache,
+                             const void* k_quant, const void* k_scales, const int32_t* block_table,
+                             const int32_t* seq_lens, int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages,
+                             float delta, void* out, float* lse, void* stream) {
+    // everything that can be refused on the host is refused before the device is touched
+    ffd_status st = check_config(cfg);
+    if (st) return st;
+    st = check_geometry(batch, max_blocks_per_seq, num_pages);
+    if (st) return st;
+    if (make_plan(cfg, batch, max_blocks_per_seq).total > FFD_STATIC_SCRATCH_BYTES) return FFD_ERR_STATIC_LIMIT;
+    if (!q || !k_cache || !v_cache || !k_quant || !k_scales || !seq_lens || !out) return FFD_ERR_NULL;
+    void* scratch = nullptr;
+    st = static_scratch_address(&scratch);
+    if (st) return st;
+    // the array still holds the previous call's contents: the sticky status word has to start from zero
+    clear_status_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<uint32_t*>(scratch));
+    if (cudaGetLastError() != cudaSuccess) return FFD_ERR_CUDA;
+    return run_decode(true, cfg, q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, batch,
+                      max_blocks_per_seq, num_pages, delta, out, lse, nullptr, nullptr, scratch,
+                      FFD_STATIC_SCRATCH_BYTES, stream);
 }
 
 ffd_status ffd_profile_events(void* start_event, void* stop_event) {

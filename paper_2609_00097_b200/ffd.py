@@ -17,12 +17,14 @@ from .build import LIB_PATH
 
 FFD_OK = 0
 STATUS_NAMES = {0: "FFD_OK", 1: "FFD_ERR_NULL", 2: "FFD_ERR_SHAPE", 3: "FFD_ERR_UNSUPPORTED", 4: "FFD_ERR_ALIGN",
-                5: "FFD_ERR_WORKSPACE", 6: "FFD_ERR_DELTA", 7: "FFD_ERR_CUDA", 8: "FFD_ERR_DEVICE_STATUS"}
+                5: "FFD_ERR_WORKSPACE", 6: "FFD_ERR_DELTA", 7: "FFD_ERR_CUDA", 8: "FFD_ERR_DEVICE_STATUS",
+                9: "FFD_ERR_STATIC_LIMIT"}
+STATIC_SCRATCH_BYTES = 8 << 20
 DEV_BAD_PAGE = 1
 DEV_BAD_SEQ_LEN = 2
 
 EXPORTS = ["ffd_status_string", "ffd_workspace_bytes", "ffd_workspace_init", "ffd_quantize_keys", "ffd_decode",
-           "ffd_decode_dense", "ffd_unpack_codes", "ffd_read_device_status", "ffd_profile_events"]
+           "ffd_decode_dense", "ffd_unpack_codes", "ffd_read_device_status", "ffd_profile_events", "ffd_decode_static"]
 
 
 class FfdError(RuntimeError):
@@ -80,6 +82,8 @@ def load_library() -> ctypes.CDLL:
         lib.ffd_unpack_codes.argtypes = [cfgp, _vp, _vp, i32, _vp]
         lib.ffd_read_device_status.argtypes = [_vp, _vp, ctypes.POINTER(ctypes.c_uint32)]
         lib.ffd_profile_events.argtypes = [_vp, _vp]
+        lib.ffd_decode_static.argtypes = [cfgp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, ctypes.c_float, _vp,
+                                          _vp, _vp]
         for name in EXPORTS:
             if name != "ffd_status_string":
                 getattr(lib, name).restype = ctypes.c_int
@@ -133,6 +137,18 @@ def ffd_decode(cfg: Config, q, k_cache, v_cache, k_quant, k_scales, block_table,
                                      _p(k_scales), _p(block_table), _p(seq_lens), q.shape[0], max_blocks_per_seq,
                                      k_cache.shape[0], ctypes.c_float(delta), _p(out), _p(lse), _p(kept_mask),
                                      _p(block_max), _p(workspace), workspace.numel(), _stream(stream)), "ffd_decode")
+
+
+def ffd_decode_static(cfg: Config, q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, delta: float, out,
+                      *, max_blocks_per_seq: int, lse=None, stream=None):
+    """ffd_decode for callers that must not allocate: no workspace argument, the library's built-in scratch array
+    (STATIC_SCRATCH_BYTES, shared by every call on the device) is used.  Raises FfdError(FFD_ERR_STATIC_LIMIT) when the
+    geometry needs more.  Calls on one device must not overlap on the GPU; make the first call outside stream
+    capture (it looks up the array's device address)."""
+    _check(load_library().ffd_decode_static(ctypes.byref(cfg.c()), _p(q), _p(k_cache), _p(v_cache), _p(k_quant),
+                                            _p(k_scales), _p(block_table), _p(seq_lens), q.shape[0],
+                                            max_blocks_per_seq, k_cache.shape[0], ctypes.c_float(delta), _p(out),
+                                            _p(lse), _stream(stream)), "ffd_decode_static")
 
 
 def ffd_decode_dense(cfg: Config, q, k_cache, v_cache, block_table, seq_lens, out, *, max_blocks_per_seq: int,
