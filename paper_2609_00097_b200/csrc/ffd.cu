@@ -101,7 +101,7 @@ __global__ void __launch_bounds__(128) unpack_kernel(const uint8_t* k_quant, uin
         }
 }
 
-constexpr int kPmWarps = 8;
+constexpr int kPmWarps = 20;   // one warp per sink / local block in the default configuration (1 + 16)
 
 // ---- pseudo-max (Sec. 3.2; Alg. 1 "Pseudo-max estimation") ------------------------------------------------
 // One CTA per (KV head, sequence): its warps scan the sink and local blocks and reduce the block maxima.

@@ -470,11 +470,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodePa
 }
 
 // ---- split combine (FlashDecoding-style log-sum-exp merge) -------------------------------------------------
-// One CTA of 512 threads per (query head, sequence).  FUSED: partial e = (work item, attend warp) of the fused
-// kernel; otherwise partial e = split of the dense kernel.  Thread (el, cg) = (tid / 32, tid % 32) sums the
-// partials e = el, el + 16, ... for channels 4cg .. 4cg+3 with eight independent loads in flight; the sixteen
-// partial sums meet in shared memory.  Summation order is fixed, so results are reproducible.
-constexpr int kCombineThreads = 512;
+// One CTA of 1024 threads per (query head, sequence).  FUSED: partial e = (work item, attend warp) of the fused
+// kernel; otherwise partial e = split of the dense kernel.  The (m, l) pairs are read once into shared memory;
+// thread (el, cg) = (tid / 32, tid % 32) sums the partials e = el, el + 32, ... for channels 4cg .. 4cg+3 with
+// eight independent loads in flight; the 32 partial sums meet in shared memory.  Summation order is fixed, so
+// results are reproducible.
+constexpr int kCombineThreads = 1024;
+constexpr int kCombineLanes = kCombineThreads / 32;   // partials summed side by side
 constexpr int kCombineChunk = 1024;
 
 template <bool FUSED>
@@ -499,46 +501,48 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
                               : min((nb + p.blocks_per_split - 1) / p.blocks_per_split, p.splits);
     const float* ml = FUSED ? p.fpart_ml : p.part_ml;
     const float* pacc = FUSED ? p.fpart_acc : p.part_acc;
-    __shared__ float s_w[kCombineChunk];
-    __shared__ float s_red[kCombineThreads / 32];
-    __shared__ float4 s_part[kCombineThreads / 32][32];
+    __shared__ float s_m[kCombineChunk];   // m of the partial, then its weight
+    __shared__ float s_l[kCombineChunk];
+    __shared__ float s_red[kCombineLanes];
+    __shared__ float4 s_part[kCombineLanes][32];
 
-    // global max over the non-empty partials
-    float M = -INFINITY;
-    for (int e = tid; e < entries; e += kCombineThreads) {
-        const float2 v = *reinterpret_cast<const float2*>(ml + combine_slot<FUSED>(p, head, bg, hl, e) * 2);
-        if (v.y > 0.f) M = fmaxf(M, v.x);
-    }
-#pragma unroll
-    for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(kFull, M, o));
-    if (cg == 0) s_red[el] = M;
-    __syncthreads();
-    M = s_red[0];
-#pragma unroll
-    for (int x = 1; x < kCombineThreads / 32; ++x) M = fmaxf(M, s_red[x]);
-
-    float L = 0.f;
+    float Mrun = -INFINITY, L = 0.f;       // running max / sum across chunks (one chunk unless > 1024 partials)
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int base = 0; base < entries && M != -INFINITY; base += kCombineChunk) {
+    for (int base = 0; base < entries; base += kCombineChunk) {
         const int cnt = min(kCombineChunk, entries - base);
         __syncthreads();
+        float M = -INFINITY;
         for (int x = tid; x < cnt; x += kCombineThreads) {
             const float2 v = *reinterpret_cast<const float2*>(ml + combine_slot<FUSED>(p, head, bg, hl, base + x) * 2);
-            float wv = 0.f;
-            if (v.y > 0.f) {
-                wv = exp2f(v.x - M);
-                L += wv * v.y;
-            }
-            s_w[x] = wv;
+            s_m[x] = v.y > 0.f ? v.x : -INFINITY;
+            s_l[x] = v.y;
+            M = fmaxf(M, s_m[x]);
+        }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(kFull, M, o));
+        if (cg == 0) s_red[el] = M;
+        __syncthreads();
+        M = Mrun;
+#pragma unroll
+        for (int x = 0; x < kCombineLanes; ++x) M = fmaxf(M, s_red[x]);
+        if (M == -INFINITY) continue;      // uniform: nothing in this chunk or before it
+        const float rescale = exp2f(Mrun - M);   // 0 for the first non-empty chunk
+        acc.x *= rescale; acc.y *= rescale; acc.z *= rescale; acc.w *= rescale;
+        L *= rescale;
+        Mrun = M;
+        for (int x = tid; x < cnt; x += kCombineThreads) {
+            const float wv = exp2f(s_m[x] - M);  // exp2(-inf) = 0 for empty partials
+            L += wv * s_l[x];
+            s_m[x] = wv;
         }
         __syncthreads();
-        for (int x0 = el; x0 < cnt; x0 += 16 * 8) {
+        for (int x0 = el; x0 < cnt; x0 += kCombineLanes * 8) {
             float4 v[8];
             float wv[8];
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-                const int x = x0 + 16 * u;
-                wv[u] = x < cnt ? s_w[x] : 0.f;
+                const int x = x0 + kCombineLanes * u;
+                wv[u] = x < cnt ? s_m[x] : 0.f;
                 v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (wv[u] != 0.f)
                     v[u] = *reinterpret_cast<const float4*>(pacc + combine_slot<FUSED>(p, head, bg, hl, base + x) * kD +
@@ -560,7 +564,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
         L = 0.f;
         float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int x = 0; x < kCombineThreads / 32; ++x) {
+        for (int x = 0; x < kCombineLanes; ++x) {
             L += s_red[x];
             const float4 v = s_part[x][tid];
             t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
@@ -576,7 +580,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
             pk.y = *reinterpret_cast<uint32_t*>(&hi);
             reinterpret_cast<uint2*>(p.out)[head * (kD / 4) + tid] = pk;
         }
-        if (p.lse && tid == 0) p.lse[head] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
+        if (p.lse && tid == 0) p.lse[head] = L > 0.f ? (Mrun + log2f(L)) * kLn2 : -INFINITY;
     }
 }
 

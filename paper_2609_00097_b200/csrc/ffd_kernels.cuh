@@ -213,17 +213,17 @@ __device__ __forceinline__ void scan_setup(ScanQuery& sq, const __nv_bfloat16* q
     const int head = n >> 1;
     sq.piece = n & 1;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        float v[4] = {0.f, 0.f, 0.f, 0.f};
-        if (head < G) {
-            const __nv_bfloat16* src = q_group + head * kD + 32 * j + 4 * i;
+    for (int x = 0; x < 4; ++x) {   // 8 contiguous channels 32j + 8x .. + 7 = k-steps 2x and 2x + 1
+        uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+        if (head < G) raw = *reinterpret_cast<const uint4*>(q_group + head * kD + 32 * j + 8 * x);
+        const uint32_t wds[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-            for (int u = 0; u < 4; ++u) v[u] = __bfloat162float(src[u]) * scan_pos_scale(i);
+        for (int y = 0; y < 4; ++y) {
+            const float sc = scan_pos_scale(2 * x + (y >> 1));
+            const float lo = __uint_as_float(wds[y] << 16), hi = __uint_as_float(wds[y] & 0xffff0000u);
+            const __half2 v = __floats2half2_rn(lo * sc, hi * sc);
+            sq.qh[4 * x + y] = *reinterpret_cast<const uint32_t*>(&v);
         }
-        __half2 a = __floats2half2_rn(v[0], v[1]);
-        __half2 c = __floats2half2_rn(v[2], v[3]);
-        sq.qh[2 * i] = *reinterpret_cast<uint32_t*>(&a);
-        sq.qh[2 * i + 1] = *reinterpret_cast<uint32_t*>(&c);
     }
 }
 
@@ -320,12 +320,18 @@ __device__ __forceinline__ float scan_mma(const uint4 (&w)[4], const uint32_t (&
         }
     }
     float best = -INFINITY;
+    if (rows == kBlk) {
 #pragma unroll
-    for (int mt = 0; mt < 4; ++mt) {
-        float t0 = acc[mt][0] + acc[mt][1];
-        float t1 = acc[mt][2] + acc[mt][3];
-        if (16 * mt + r < rows) best = fmaxf(best, t0);
-        if (16 * mt + r + 8 < rows) best = fmaxf(best, t1);
+        for (int mt = 0; mt < 4; ++mt)
+            best = fmaxf(best, fmaxf(acc[mt][0] + acc[mt][1], acc[mt][2] + acc[mt][3]));
+    } else {
+#pragma unroll
+        for (int mt = 0; mt < 4; ++mt) {
+            float t0 = acc[mt][0] + acc[mt][1];
+            float t1 = acc[mt][2] + acc[mt][3];
+            if (16 * mt + r < rows) best = fmaxf(best, t0);
+            if (16 * mt + r + 8 < rows) best = fmaxf(best, t1);
+        }
     }
     best = fmaxf(best, __shfl_xor_sync(kFull, best, 4));
     best = fmaxf(best, __shfl_xor_sync(kFull, best, 8));
@@ -427,6 +433,11 @@ __device__ __forceinline__ bool attend_block(AttendState& st, uint32_t kslot, ui
     for (int nt = 0; nt < 16; ++nt) { st.acc[nt][0] *= alpha; st.acc[nt][1] *= alpha; }
     // O += P V
     if (!mbar_wait(vbar, phase & 1u)) return false;
+    if (rows < kBlk) {   // partial tail block: rows past the sequence end must not meet P = 0 as stale NaN / Inf
+        for (int c = lane; c < (kBlk - rows) * 16; c += 32)
+            asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};\n" ::"r"(vslot + rows * 256 + c * 16), "r"(0u) : "memory");
+        __syncwarp();
+    }
 #pragma unroll
     for (int kt = 0; kt < 4; ++kt) {
         const int t0 = 16 * kt + 2 * j;
@@ -438,7 +449,6 @@ __device__ __forceinline__ bool attend_block(AttendState& st, uint32_t kslot, ui
                 const int tok = t0 + (tt & 1) + ((tt >> 1) << 3);
                 const uint32_t swz_v = (uint32_t)(j << 1) ^ ((uint32_t)(tt & 1) << 2);   // = swz(tok)
                 v[tt] = lds128(vslot + tok * 256 + (((8 * hf + r) ^ swz_v) << 4));
-                if (tok >= rows) v[tt] = make_uint4(0u, 0u, 0u, 0u);   // never multiply 0 by stale memory
             }
             const uint32_t* x0 = reinterpret_cast<const uint32_t*>(&v[0]);
             const uint32_t* x1 = reinterpret_cast<const uint32_t*>(&v[1]);
