@@ -101,6 +101,7 @@ __global__ void __launch_bounds__(128) unpack_kernel(const uint8_t* k_quant, uin
         }
 }
 
+constexpr int kPmHintBlocks = 64;
 constexpr int kPmWarps = 20;   // one warp per sink / local block in the default configuration (1 + 16)
 
 // ---- pseudo-max (Sec. 3.2; Alg. 1 "Pseudo-max estimation") ------------------------------------------------
@@ -114,9 +115,12 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
     const int local_begin = max(nb - p.n_local, ns);
     const int count = ns + (nb - local_begin);
     __shared__ float smax[kPmWarps][kMaxG];
+    __shared__ float sbm[kPmHintBlocks][kMaxG];   // block maxima of the first sink / local blocks, for the hint below
+    __shared__ float sthr[kMaxG];
+    for (int x = threadIdx.x; x < kPmHintBlocks * kMaxG; x += kPmWarps * 32) (&sbm[0][0])[x] = -INFINITY;
+    __syncthreads();
     ScanQuery sq;
     scan_setup(sq, p.q + ((size_t)b * p.Hq + (size_t)g * p.G) * kD, p.G, lane);
-    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *p.item_counter = 0u;
     unsigned char* rec = p.qrec + (size_t)(b * p.Hkv + g) * kQrecBytes;
     if (warp == 0) {   // query record of this (sequence, KV head): the fused kernel stages it per work item
         uint4* dst = reinterpret_cast<uint4*>(rec);
@@ -135,7 +139,9 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
         ScanRegs sr;
         scan_load(sr, reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes),
                   reinterpret_cast<const uint4*>(p.k_scales + tile * kD), lane);
-        best = fmaxf(best, scan_compute<true>(sr, sq, lane, rows, p.sm_scale, band));
+        const float bm = scan_compute<true>(sr, sq, lane, rows, p.sm_scale, band);
+        if (lane < kMaxG && s < kPmHintBlocks) sbm[s][lane] = bm;
+        best = fmaxf(best, bm);
     }
     if (lane < kMaxG) smax[warp][lane] = best;
     __syncthreads();
@@ -149,6 +155,21 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
             thr = m - p.delta;
         }
         reinterpret_cast<float*>(rec + 2048)[threadIdx.x] = thr;
+        if (threadIdx.x < kMaxG) sthr[threadIdx.x] = thr;
+    }
+    __syncthreads();
+    // Scheduling hint for the fused kernel: a (sequence, KV head) whose sink / local blocks are mostly kept is
+    // likely to keep much of its cache (a "dense" head), so its work items are expensive and are handed out first.
+    // The hint only orders the work; it never changes a result.
+    const int hinted = min(count, kPmHintBlocks);
+    bool kept_any = false;
+    if ((int)threadIdx.x < hinted)
+        for (int h = 0; h < p.G; ++h) kept_any |= sbm[threadIdx.x][h] >= sthr[h];
+    const int kept = __syncthreads_count(kept_any);
+    if (threadIdx.x == 0) {
+        const int bg = b * p.Hkv + g;
+        if (hinted > 0 && 2 * kept >= hinted) p.unit_list[atomicAdd(&p.class_counts[0], 1u)] = bg;
+        else p.unit_list[p.units - 1 - (int)atomicAdd(&p.class_counts[1], 1u)] = bg;
     }
 }
 
@@ -322,7 +343,7 @@ __global__ void clear_status_kernel(uint32_t* status) { *status = 0u; }
 struct Plan {
     int blocks_per_split, splits;     // dense path
     int total_items;                  // fused path
-    size_t off_mtilde, off_qrec, off_ml, off_acc, off_fml, off_facc, total;
+    size_t off_mtilde, off_units, off_qrec, off_ml, off_acc, off_fml, off_facc, total;
 };
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -340,7 +361,8 @@ static Plan make_plan(const ffd_config* cfg, int batch, int max_blocks) {
     pl.total_items = ((max_blocks + kItemBlocks - 1) / kItemBlocks) * batch * cfg->num_kv_heads;
     const size_t fslots = (size_t)pl.total_items * kNA * kMaxG;
     pl.off_mtilde = 256;
-    pl.off_qrec = align_up(pl.off_mtilde + heads * sizeof(float), 256);
+    pl.off_units = align_up(pl.off_mtilde + heads * sizeof(float), 256);
+    pl.off_qrec = align_up(pl.off_units + (size_t)batch * cfg->num_kv_heads * sizeof(int32_t), 256);
     pl.off_ml = align_up(pl.off_qrec + (size_t)batch * cfg->num_kv_heads * kQrecBytes, 256);
     pl.off_acc = align_up(pl.off_ml + heads * pl.splits * 2 * sizeof(float), 256);
     pl.off_fml = align_up(pl.off_acc + heads * pl.splits * kD * sizeof(float), 256);
@@ -385,7 +407,8 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
     st = check_geometry(batch, max_blocks, num_pages);
     if (st) return st;
     if (cfg->num_kv_heads > 65535 || cfg->num_q_heads > 65535) return FFD_ERR_SHAPE;
-    if ((double)num_pages * cfg->num_kv_heads >= 4294967296.0) return FFD_ERR_SHAPE;
+    if ((double)num_pages * cfg->num_kv_heads >= 2147483648.0) return FFD_ERR_SHAPE;
+    if ((long)batch * cfg->num_kv_heads >= 65536L) return FFD_ERR_SHAPE;   // fast_div: items * units < 2^48
     if (sparse && (isnan(delta) || delta < 0.f)) return FFD_ERR_DELTA;
     const void* ptrs[] = {q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, out, lse, block_max, workspace};
     for (const void* ptr : ptrs)
@@ -424,6 +447,13 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
     p.fpart_acc = reinterpret_cast<float*>(ws + pl.off_facc);
     p.total_items = pl.total_items;
     p.item_counter = reinterpret_cast<uint32_t*>(ws + 64);
+    p.class_counts = reinterpret_cast<uint32_t*>(ws + 68);
+    p.light_counter = reinterpret_cast<uint32_t*>(ws + 76);
+    p.unit_list = reinterpret_cast<int32_t*>(ws + pl.off_units);
+    p.units = batch * cfg->num_kv_heads;
+    p.item_rows = (max_blocks + kItemBlocks - 1) / kItemBlocks;
+    p.units_magic = fast_div_magic((unsigned)p.units);
+    p.hkv_magic = fast_div_magic((unsigned)cfg->num_kv_heads);
     p.kept_mask = kept_mask;
     p.block_max = block_max;
     p.out = out;
@@ -439,6 +469,8 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
             cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
             cudaFuncSetAttribute(fused_sparse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem) != cudaSuccess)
             return FFD_ERR_CUDA;
+        // work counter and class counts start every call from zero
+        if (cudaMemsetAsync(ws + 64, 0, 16, s) != cudaSuccess) return FFD_ERR_CUDA;
         pseudomax_kernel<<<dim3(p.Hkv, batch), kPmWarps * 32, 0, s>>>(p);
         if (prof) cudaEventRecord(g_prof_start, s);
         fused_sparse_kernel<<<min(p.total_items, sms), kFusedThreads, kFusedSmem, s>>>(p);

@@ -19,36 +19,46 @@
 
 namespace ffd {
 
-constexpr int kNS = 12;                // scan warps (three warpgroups)
+constexpr int kNS = 12;                // warps of the scan role (three warpgroups)
+#ifndef FFD_SCHED_WARP
+#define FFD_SCHED_WARP 1
+#endif
+constexpr int kSched = FFD_SCHED_WARP; // 1: warp 0 only draws and publishes items, warps 1..11 scan
+constexpr int kScanners = kNS - kSched;
 constexpr int kNA = 4;                 // attend warps (one warpgroup)
 constexpr int kFusedThreads = (kNS + kNA) * 32;
 constexpr int kScanRegs = 112;         // 12*32*112 + 4*32*176 = 65536 registers
 constexpr int kAttendRegs = (65536 - kNS * 32 * kScanRegs) / (kNA * 32);
 static_assert(kAttendRegs % 8 == 0 && kScanRegs % 8 == 0, "setmaxnreg takes multiples of 8");
-constexpr int kItemBlocks = 24;        // blocks per work item: two per scan warp
+constexpr int kItemBlocks = 2 * kScanners;   // blocks per work item: two per scanning warp
+static_assert(kItemBlocks <= 24, "batch descriptor arrays");
 constexpr int kRing = 3;               // code-ring stages per scan warp
 constexpr int kStageBytes = kCodeBytes + kD * 2;   // 2048 B codes + 256 B scales
-constexpr int kNB = 2;                 // batch descriptors in flight
+#ifndef FFD_NB
+#define FFD_NB 8
+#endif
+constexpr int kNB = FFD_NB;                 // batch descriptors: how far the scan warps may run ahead of the attend warps
+constexpr int kHeavyAhead = 2;         // heavy batches outstanding at most once the attend warps are the bottleneck
+constexpr int kUnitCache = 512;        // entries of the unit list kept in shared memory
 constexpr int kItemRing = 8;           // decoded items published ahead
 constexpr int kQrecRing = 4;           // query records staged ahead
 constexpr int kQrecBytes = 2048 + 32;  // [4][32 lanes] uint4 of fp16 query fragments, then 4 thresholds (+ pad)
 
 struct Item {
-    int item;                          // work item number; < 0: no more work
-    int b, g, blk0, nblk, n;           // sequence, KV head, first block, blocks (1..24), tokens of the sequence
+    int slot;                          // canonical number row * units + bg (names the partial slots); < 0: no more work
+    int b, g, bg, blk0, nblk, n;       // sequence, KV head, b * Hkv + g, first block, blocks (1..24), tokens
 };
 
-struct ItemSlot {                      // entry `seq` of the published-item ring is valid when tag == seq
-    volatile int tag;
-    volatile int item, b, g, blk0, nblk, n;
+struct ItemSlot {                      // entry seq % 8 of the published-item ring; readiness: one mbarrier per entry
+    volatile int slot, b, g, bg, blk0, nblk, n;
     int pad;
 };
 
 struct BatchDesc {
-    int item, b, g, nblk;              // work item of this batch; item < 0: no more work
-    uint32_t tile[kItemBlocks];        // (page, KV head) tile of each block of the item
-    uint8_t keep4[kItemBlocks];        // bit h: query head h of the group keeps the block; 0 = skipped
-    uint8_t rows[kItemBlocks];         // valid tokens
+    int item, b, g, nblk;              // canonical item number (row * units + bg) of this batch; < 0: no more work
+    uint32_t tile[24];                 // (page, KV head) tile of each block of the item (kItemBlocks <= 24 used)
+    uint8_t keep4[24];                 // bit h: query head h of the group keeps the block; 0 = skipped
+    uint8_t rows[24];                  // valid tokens
 };
 
 constexpr int kOffSlots = 0;
@@ -56,27 +66,74 @@ constexpr int kOffRing = kOffSlots + kNA * 2 * kSlotBytes;
 constexpr int kOffQrec = kOffRing + kNS * kRing * kStageBytes;
 constexpr int kOffDesc = kOffQrec + kQrecRing * kQrecBytes;
 constexpr int kOffBars = kOffDesc + kNB * (int)sizeof(BatchDesc);
-constexpr int kNumBars = 2 * kNB + 2 * kNA + kQrecRing;          // full, empty, K/V slots, query records
+constexpr int kNumBars = 2 * kNB + 2 * kNA + kQrecRing + kItemRing;   // full, empty, K/V slots, records, items
 constexpr int kOffItems = kOffBars + kNumBars * 8;               // ring of decoded items
 constexpr int kOffStageTile = kOffItems + kItemRing * (int)sizeof(ItemSlot);   // tile index of each ring stage
 constexpr int kOffAbort = kOffStageTile + kNS * 4 * 4;
-constexpr int kFusedSmem = kOffAbort + 16;
+constexpr int kOffSched = kOffAbort + 16;                        // state of the item scheduler (one thread)
+constexpr int kOffAttendDone = kOffSched + 96;                   // batches finished by each attend warp
+constexpr int kOffUnits = kOffAttendDone + 16;                   // first kUnitCache entries of each end of the unit list
+constexpr int kFusedSmem = kOffUnits + 2 * kUnitCache * 4;
 static_assert(kOffBars % 8 == 0 && kOffRing % 16 == 0 && kOffDesc % 16 == 0 && kOffQrec % 16 == 0, "alignment");
+static_assert(kOffSched % 8 == 0, "alignment");
 static_assert(sizeof(BatchDesc) % 16 == 0 && sizeof(ItemSlot) == 32, "descriptor sizes");
 static_assert(kFusedSmem <= 227 * 1024, "shared memory budget");
 
-// Items are numbered from the END of the sequences backwards: the local window, whose blocks are the most likely
-// to be kept (and therefore the most expensive), is handed out first.
-__device__ __forceinline__ Item decode_item(const DecodeParams& p, int item) {
+// Work is handed out from two global counters, one per class of (sequence, KV head) units.  "Heavy" units are the
+// ones the pseudo-max kernel's hint expects to keep most of their blocks (expensive for the attend warps, memory
+// bound), "light" units the rest (almost pure scan work).  The drawing thread keeps at most kHeavyAhead heavy batches
+// queued ahead of the attend warps and fills the scan warps' remaining time with light items, so the two kinds of
+// work overlap on every SM; what is left over at the end is light, i.e. a short, well-balanced tail.  Within a class,
+// rows count from the END of the sequences backwards (the local window first).
+struct ItemSched {
+    int n_heavy, n_light, total_heavy, total_light;      // units and items per class
+    unsigned long long magic_heavy, magic_light;          // reciprocals of the unit counts
+    int pend_heavy, pend_light;                           // draw of each class already fetched (>= total: none left)
+    int next_pub;                                         // next ring entry to publish
+    int released;                                         // batches the attend warps have finished, in order
+    int heavy_queued;                                     // heavy batches published and not yet released
+    int finished;                                         // the end marker has been published
+    unsigned long long heavy_hist;                        // bit s % 64: batch s is heavy
+};
+static_assert(sizeof(ItemSched) <= 96, "scheduler state");
+
+__device__ __forceinline__ void sched_init(const DecodeParams& p, ItemSched* sc) {
+    sc->n_heavy = min((int)p.class_counts[0], p.units);
+    sc->n_light = p.units - sc->n_heavy;
+    sc->total_heavy = sc->n_heavy * p.item_rows;
+    sc->total_light = sc->n_light * p.item_rows;
+    sc->magic_heavy = fast_div_magic((unsigned)max(sc->n_heavy, 1));
+    sc->magic_light = fast_div_magic((unsigned)max(sc->n_light, 1));
+    sc->pend_heavy = (int)atomicAdd(p.item_counter, 1u);
+    sc->pend_light = (int)atomicAdd(p.light_counter, 1u);
+    sc->next_pub = 0;
+    sc->released = 0;
+    sc->heavy_queued = 0;
+    sc->finished = 0;
+    sc->heavy_hist = 0ull;
+}
+
+// draw number k of a class -> work item
+__device__ __forceinline__ Item decode_item(const DecodeParams& p, const ItemSched* sc, const int* unit_cache,
+                                            bool heavy, int k) {
     Item it;
-    const int units = p.batch * p.Hkv;
-    const int bg = item % units, split = p.total_items / units - 1 - item / units;
-    it.item = item;
-    it.b = bg / p.Hkv;
-    it.g = bg % p.Hkv;
+    int row, bg;
+    if (heavy) {   // heavy units sit at the front of the list, light units at its back (first ones cached in smem)
+        row = (int)fast_div((unsigned)k, sc->magic_heavy);
+        const int u = k - row * sc->n_heavy;
+        bg = u < kUnitCache ? unit_cache[u] : p.unit_list[u];
+    } else {
+        row = (int)fast_div((unsigned)k, sc->magic_light);
+        const int u = k - row * sc->n_light;
+        bg = u < kUnitCache ? unit_cache[kUnitCache + u] : p.unit_list[p.units - 1 - u];
+    }
+    it.slot = row * p.units + bg;
+    it.bg = bg;
+    it.b = (int)fast_div((unsigned)bg, p.hkv_magic);
+    it.g = bg - it.b * p.Hkv;
     it.n = clamped_seq_len(p, it.b);
     const int nb = (it.n + kBlk - 1) / kBlk;
-    it.blk0 = split * kItemBlocks;
+    it.blk0 = (p.item_rows - 1 - row) * kItemBlocks;
     it.nblk = min(nb - it.blk0, kItemBlocks);
     return it;
 }
@@ -95,45 +152,88 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
 }
 
 // ---- published items ---------------------------------------------------------------------------------------
+// Entry seq lives in slot seq % 8 and is announced by one arrival on that slot's mbarrier (phase seq / 8): the
+// arrive releases the entry's fields, a successful test / wait acquires them.  No fence is used on purpose: a CTA
+// fence would also wait for the reader's in-flight cp.async copies and serialise the prefetch ring.  Every scan warp
+// visits every entry in order and never trails the publisher by more than three entries, so a parity test can not
+// alias.
 
-__device__ __forceinline__ bool item_ready(const ItemSlot* ring, int seq) { return ring[seq & (kItemRing - 1)].tag == seq; }
+__device__ __forceinline__ uint32_t item_bar(uint32_t ibars, int seq) { return ibars + (seq & (kItemRing - 1)) * 8; }
+
+__device__ __forceinline__ bool item_ready(uint32_t ibars, int seq) {
+    return mbar_test(item_bar(ibars, seq), (seq / kItemRing) & 1);
+}
+
+__device__ __forceinline__ bool item_wait(uint32_t ibars, int seq) {
+    return mbar_wait(item_bar(ibars, seq), (seq / kItemRing) & 1);
+}
 
 __device__ __forceinline__ Item item_read(const ItemSlot* ring, int seq) {
     const ItemSlot& e = ring[seq & (kItemRing - 1)];
-    __threadfence_block();
     Item it;
-    it.item = e.item; it.b = e.b; it.g = e.g; it.blk0 = e.blk0; it.nblk = e.nblk; it.n = e.n;
+    it.slot = e.slot; it.b = e.b; it.g = e.g; it.bg = e.bg; it.blk0 = e.blk0; it.nblk = e.nblk; it.n = e.n;
     return it;
 }
 
-// bounded wait for entry `seq` (it is normally there long before it is needed)
-__device__ __forceinline__ bool item_wait(const ItemSlot* ring, int seq) {
-    if (item_ready(ring, seq)) return true;
-    const long long t0 = clock64();
-    while (!item_ready(ring, seq)) {
-        __nanosleep(64);
-        if (clock64() - t0 > kSpinCycles) return false;
-    }
-    return true;
-}
-
-// Lane 0 of scan warp 0: draw the next item that has blocks and publish it as entry `seq`.
-// `pend` holds the result of an atomicAdd issued earlier; `done` is set once the counter ran past the last item.
-__device__ __forceinline__ Item item_publish(const DecodeParams& p, ItemSlot* ring, int seq, int& pend, bool& done) {
-    Item it;
-    it.item = -1; it.b = it.g = it.blk0 = it.nblk = it.n = 0;
-    while (!done) {
-        const int cand = pend;
-        if (cand >= p.total_items) { done = true; break; }
-        pend = (int)atomicAdd(p.item_counter, 1u);   // keep the next draw in flight
-        const Item c = decode_item(p, cand);
-        if (c.nblk > 0) { it = c; break; }
-    }
+__device__ __forceinline__ void item_store(ItemSlot* ring, uint32_t ibars, int seq, const Item& it) {
     ItemSlot& e = ring[seq & (kItemRing - 1)];
-    e.item = it.item; e.b = it.b; e.g = it.g; e.blk0 = it.blk0; e.nblk = it.nblk; e.n = it.n;
-    __threadfence_block();
-    e.tag = seq;
-    return it;
+    e.slot = it.slot; e.b = it.b; e.g = it.g; e.bg = it.bg; e.blk0 = it.blk0; e.nblk = it.nblk; e.n = it.n;
+    mbar_arrive(item_bar(ibars, seq));
+}
+
+// Lane 0 of scan warp 0: choose, draw and publish ring entry sc->next_pub.  Returns the item's unit (bg >= 0), -1 when
+// the end marker was published, -2 when nothing could be published yet (heavy work is due but enough of it is
+// already queued, and may_block is false).  may_block is only passed when the caller has itself finished scanning
+// every batch published so far, so that waiting for the attend warps cannot wait for the caller.
+// batches every attend warp has finished (they take the batches in order); a plain monotonic count, because a
+// parity test on the empty barriers could be fooled when a slot completes two phases between two looks
+__device__ __forceinline__ int attend_finished(const volatile int* attend_done) {
+    return min(min(attend_done[0], attend_done[1]), min(attend_done[2], attend_done[3]));
+}
+static_assert(kNA == 4, "attend_finished reads four counters");
+
+__device__ __forceinline__ int item_publish(const DecodeParams& p, ItemSched* sc, const int* unit_cache, ItemSlot* ring,
+                                            uint32_t ibars, const volatile int* attend_done, bool may_block,
+                                            volatile int* abort_flag) {
+    const int seq = sc->next_pub;
+    Item it;
+    it.slot = -1; it.b = it.g = it.bg = it.blk0 = it.nblk = it.n = 0;
+    while (!sc->finished) {
+        // batches the attend warps have released since the last look
+        for (const int rel = min(attend_finished(attend_done), seq); sc->released < rel; ++sc->released)
+            if ((sc->heavy_hist >> (sc->released & 63)) & 1ull) --sc->heavy_queued;
+        const bool heavy_left = sc->pend_heavy < sc->total_heavy, light_left = sc->pend_light < sc->total_light;
+        if (!heavy_left && !light_left) { sc->finished = 1; break; }
+        // Heavy batches published and not yet released.  While the attend warps keep up with the scan (nothing but
+        // the entries published ahead is outstanding) the limit does not bind; once they fall behind, at most
+        // kHeavyAhead heavy batches may be outstanding, so that no CTA sits on heavy work others could have taken
+        // and the scan warps spend their spare time on light items.
+        const int limit = (seq - sc->released <= 3) ? 4 : kHeavyAhead;
+        bool heavy;
+        if (heavy_left && sc->heavy_queued < limit) heavy = true;
+        else if (light_left) heavy = false;
+        else {   // only heavy work is left and enough of it is queued: wait for the attend warps, or come back later
+            if (!may_block) return -2;
+            const long long t0 = clock64();
+            while (attend_finished(attend_done) <= sc->released) {
+                __nanosleep(256);
+                if (clock64() - t0 > kSpinCycles) { *abort_flag = 1; sc->finished = 1; break; }
+            }
+            continue;
+        }
+        int cand;
+        if (heavy) { cand = sc->pend_heavy; sc->pend_heavy = (int)atomicAdd(p.item_counter, 1u); }
+        else { cand = sc->pend_light; sc->pend_light = (int)atomicAdd(p.light_counter, 1u); }
+        const Item c = decode_item(p, sc, unit_cache, heavy, cand);
+        if (c.nblk <= 0) continue;   // the sequence is shorter than the longest one: nothing in this item
+        it = c;
+        if (heavy) { sc->heavy_hist |= 1ull << (seq & 63); ++sc->heavy_queued; }
+        else sc->heavy_hist &= ~(1ull << (seq & 63));
+        break;
+    }
+    item_store(ring, ibars, seq, it);
+    ++sc->next_pub;
+    return it.slot >= 0 ? it.bg : -1;
 }
 
 // ---- scan role ---------------------------------------------------------------------------------------------
@@ -148,14 +248,14 @@ struct ScanCursor {
 
 // Advance to this warp's next block; false when the item it lies in has not been published yet (the cursor then
 // stays where it can resume) or when there is no more work.
-__device__ __forceinline__ bool cursor_next(ScanCursor& c, const ItemSlot* items, int w) {
+__device__ __forceinline__ bool cursor_next(ScanCursor& c, const ItemSlot* items, uint32_t ibars, int w) {
     if (c.end) return false;
-    int lb = c.lb + kNS;
+    int lb = c.lb + kScanners;
     while (lb >= c.it.nblk) {
-        if (!item_ready(items, c.seq + 1)) { c.lb = lb - kNS; return false; }
+        if (!item_ready(ibars, c.seq + 1)) { c.lb = lb - kScanners; return false; }
         c.it = item_read(items, c.seq + 1);
         ++c.seq;
-        if (c.it.item < 0) { c.end = true; c.it.nblk = 0; return false; }
+        if (c.it.slot < 0) { c.end = true; c.it.nblk = 0; return false; }
         lb = w;
     }
     c.lb = lb;
@@ -220,49 +320,53 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
     const uint32_t qrecs = smem_u32(smem) + kOffQrec;
     const uint32_t bars = smem_u32(smem) + kOffBars;
     const uint32_t qbars = bars + (2 * kNB + 2 * kNA) * 8;
+    const uint32_t ibars = qbars + kQrecRing * 8;
     BatchDesc* descs = reinterpret_cast<BatchDesc*>(smem + kOffDesc);
     ItemSlot* items = reinterpret_cast<ItemSlot*>(smem + kOffItems);
     volatile int* stage_tile = reinterpret_cast<volatile int*>(smem + kOffStageTile) + w * 4;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffAbort);
-    const int units = p.batch * p.Hkv;
-
-    // warp 0 publishes items 0 and 1 (and stages their records) before anybody starts
-    int pend = p.total_items;
-    bool done = false;
-    if (w == 0) {
-        int item0 = -1, item1 = -1;
-        if (lane == 0) {
-            pend = (int)atomicAdd(p.item_counter, 1u);
-            item0 = item_publish(p, items, 0, pend, done).item;
-            item1 = item_publish(p, items, 1, pend, done).item;
-        }
-        item0 = __shfl_sync(kFull, item0, 0);
-        item1 = __shfl_sync(kFull, item1, 0);
-        if (item0 >= 0) qrec_issue(p, 0, item0 % units, qrecs, qbars, lane);
-        if (item1 >= 0) qrec_issue(p, 1, item1 % units, qrecs, qbars, lane);
-    }
+    ItemSched* sched = reinterpret_cast<ItemSched*>(smem + kOffSched);
+    const volatile int* attend_done = reinterpret_cast<const volatile int*>(smem + kOffAttendDone);
+    const int* unit_cache = reinterpret_cast<const int*>(smem + kOffUnits);
+    if (w == 0 && lane == 0) sched_init(p, sched);
     ScanCursor ic;
     ic.seq = -1;
     ic.it.nblk = 0;
-    ic.lb = w - kNS;
+    const int w0 = w - kSched;      // index among the scanning warps (-1: the scheduling warp, which scans nothing)
+    ic.lb = w0 - kScanners;
     ic.end = false;
     int issued = 0, consumed = 0;   // this warp's blocks whose copies were started / whose data was taken
 
 #pragma unroll 1
     for (int seq = 0;; ++seq) {     // published item seq = batch seq
-        if (w == 0) {               // publish item seq + 2 and stage its record
-            int item2 = -1;
-            if (lane == 0) item2 = item_publish(p, items, seq + 2, pend, done).item;
-            item2 = __shfl_sync(kFull, item2, 0);
-            if (item2 >= 0) qrec_issue(p, seq + 2, item2 % units, qrecs, qbars, lane);
+        if (w == 0) {
+            // Publish ring entries up to seq + 2 and stage their query records.  Entry e reuses the slots of entries
+            // e - 4 (records) and e - 8 (items): every scan warp must be done with batch e - 4 first, which the
+            // completion of that batch's full barrier shows.
+#pragma unroll 1
+            for (;;) {
+                int bg = -3, pub = 0;
+                if (lane == 0) {
+                    pub = sched->next_pub;
+                    if (pub <= seq + 2) {
+                        const int guard = pub - 4;
+                        if (guard >= 0 && !mbar_wait(bars + (guard & (kNB - 1)) * 8, (guard / kNB) & 1)) *abort_flag = 1;
+                        bg = item_publish(p, sched, unit_cache, items, ibars, attend_done, pub <= seq, abort_flag);
+                    }
+                }
+                bg = __shfl_sync(kFull, bg, 0);
+                pub = __shfl_sync(kFull, pub, 0);
+                if (bg >= 0) qrec_issue(p, pub, bg, qrecs, qbars, lane);
+                if (bg < -1) break;      // -3: published far enough; -2: nothing to publish for now
+            }
         }
-        if (!item_wait(items, seq)) *abort_flag = 1;
+        if (!item_wait(ibars, seq)) *abort_flag = 1;
         const Item it = item_read(items, seq);
-        const int slot = seq & 1, use = seq >> 1;
-        // the attend warps must have released this descriptor (two batches ago)
+        const int slot = seq & (kNB - 1), use = seq / kNB;
+        // the attend warps must have released this descriptor (kNB batches ago)
         if (use > 0 && !mbar_wait(bars + (kNB + slot) * 8, (use - 1) & 1)) *abort_flag = 1;
         BatchDesc& d = descs[slot];
-        if (it.item < 0 || *abort_flag) {   // no more work: tell the attend warps
+        if (it.slot < 0 || *abort_flag) {   // no more work: tell the attend warps
             if (lane == 0) {
                 if (w == 0) d.item = -1;
                 mbar_arrive(bars + slot * 8);
@@ -273,13 +377,14 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
         if (!mbar_wait(qbars + (seq & (kQrecRing - 1)) * 8, (seq / kQrecRing) & 1)) *abort_flag = 1;
         const uint32_t qrec = qrecs + (seq & (kQrecRing - 1)) * kQrecBytes;
         const size_t head0 = (size_t)it.b * p.Hq + (size_t)it.g * p.G;
-        float thr;
+        float thr, thr_col;   // threshold of head lane % 4 (block-max layout) and of head lane / 8 (B-column layout)
         asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(thr) : "r"(qrec + 2048 + j * 4));
-        if (w == 0 && lane == 0) { d.item = it.item; d.b = it.b; d.g = it.g; d.nblk = it.nblk; }
+        asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(thr_col) : "r"(qrec + 2048 + (lane >> 3) * 4));
+        if (w == 0 && lane == 0) { d.item = it.slot; d.b = it.b; d.g = it.g; d.nblk = it.nblk; }
 #pragma unroll 1
-        for (int lb = w; lb < it.nblk; lb += kNS) {
+        for (int lb = w0 >= 0 ? w0 : it.nblk; lb < it.nblk; lb += kScanners) {
             // keep the ring full: blocks consumed .. consumed + kRing - 1 of this warp's stream
-            while (issued < consumed + kRing && cursor_next(ic, items, w)) {
+            while (issued < consumed + kRing && cursor_next(ic, items, ibars, w0)) {
                 ring_issue(p, ic, ring + (issued % kRing) * kStageBytes, stage_tile + issued % kRing, lane);
                 ++issued;
             }
@@ -292,14 +397,15 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
 #pragma unroll
             for (int mt = 0; mt < 4; ++mt) wv[mt] = lds128(stage + (mt * 32 + lane) * 16);
             uint32_t bfrag[16];
+            __half2 sum_a = __floats2half2_rn(0.f, 0.f), sum_b = sum_a;
 #pragma unroll
             for (int x = 0; x < 4; ++x)
-                scan_bfrag4(bfrag + 4 * x, lds128(qrec + (x * 32 + lane) * 16),
-                            lds128(stage + kCodeBytes + (4 * x + j) * 16), r & 1);
+                scan_bfrag4_bound(bfrag + 4 * x, lds128(qrec + (x * 32 + lane) * 16),
+                                  lds128(stage + kCodeBytes + (4 * x + j) * 16), r & 1, 4 * x, sum_a, sum_b);
             const int tile = stage_tile[st];
             __syncwarp();   // the stage is free again
             ++consumed;
-            if (issued < consumed + kRing && cursor_next(ic, items, w)) {
+            if (issued < consumed + kRing && cursor_next(ic, items, ibars, w0)) {
                 ring_issue(p, ic, ring + (issued % kRing) * kStageBytes, stage_tile + issued % kRing, lane);
                 ++issued;
             }
@@ -307,7 +413,13 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
             const int blk = it.blk0 + lb;
             const int rows = min(kBlk, it.n - blk * kBlk);
             unsigned keep4 = 0;
-            if (tile >= 0) {
+            // No token of the block can score above 1.5 * sum |q s| (every level is at most 1.5 in magnitude).  If
+            // that bound stays below the threshold for every head of the group, no head can keep the block and the
+            // MMA work is skipped; the decision is the same as the full scan's.  (Not when the caller asked for the
+            // block maxima themselves.)
+            const bool cannot_keep =
+                __all_sync(kFull, scan_bound(sum_a, sum_b, p.sm_scale) < thr_col) && p.block_max == nullptr;
+            if (tile >= 0 && !cannot_keep) {
                 float band;
                 float bm = scan_mma<false>(wv, bfrag, lane, rows, p.sm_scale, band);
                 // too close to call (rare): a separate, non-inlined routine re-reads the block and redoes it precisely
@@ -323,6 +435,8 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
                     if (p.block_max) p.block_max[o] = bm;
                 }
             }
+            if (cannot_keep && tile >= 0 && p.kept_mask && r == 0 && j < p.G)
+                p.kept_mask[(head0 + j) * p.max_blocks + blk] = 0;
             if (lane == 0) {
                 d.tile[lb] = tile >= 0 ? (uint32_t)tile : 0u;
                 d.keep4[lb] = (uint8_t)keep4;
@@ -365,13 +479,13 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
     bool ok = true;
     AttendState st;
     for (int bi = 0; ok; ++bi) {
-        const int slot = bi & 1, use = bi >> 1;
+        const int slot = bi & (kNB - 1), use = bi / kNB;
         if (!mbar_wait(bars + slot * 8, use & 1)) { ok = false; break; }
         const BatchDesc& d = descs[slot];
         const int item = d.item;
         if (item < 0) break;
         Item it;
-        it.item = item; it.b = d.b; it.g = d.g; it.nblk = d.nblk;
+        it.slot = item; it.b = d.b; it.g = d.g; it.nblk = d.nblk;
         unsigned mine = my_entries(d, it.nblk, a, lane);
         const bool any = mine != 0;
         if (any) attend_setup(st, p.q + ((size_t)it.b * p.Hq + (size_t)it.g * p.G) * kD, p.G, lane);
@@ -392,8 +506,8 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
                 issued_lb = nlb;
             } else {
                 const int bi2 = bi + 1;
-                if (mbar_test(bars + (bi2 & 1) * 8, (bi2 >> 1) & 1)) {
-                    const BatchDesc& d2 = descs[bi2 & 1];
+                if (mbar_test(bars + (bi2 & (kNB - 1)) * 8, (bi2 / kNB) & 1)) {
+                    const BatchDesc& d2 = descs[bi2 & (kNB - 1)];
                     if (d2.item >= 0) {
                         const unsigned mine2 = my_entries(d2, d2.nblk, a, lane);
                         if (mine2) {
@@ -410,7 +524,10 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
                               logit_scale_log2);
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(bars + (kNB + slot) * 8);   // done with this batch descriptor
+        if (lane == 0) {
+            mbar_arrive(bars + (kNB + slot) * 8);   // done with this batch descriptor
+            reinterpret_cast<volatile int*>(smem + kOffAttendDone)[a] = bi + 1;
+        }
         // this warp's partial (m, l, acc) of the item; heads in rows r < 4 (r + 4 holds the bf16 remainder sums)
         const size_t pslot = ((size_t)item * kNA + a) * kMaxG;
         if (any && ok) {
@@ -455,8 +572,18 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodePa
             mbar_init(bars + (kNB + s) * 8, kNA);     // empty: one arrival per attend warp
         }
         for (int a = 0; a < 2 * kNA + kQrecRing; ++a) mbar_init(bars + (2 * kNB + a) * 8, 32);
-        for (int s = 0; s < kItemRing; ++s) reinterpret_cast<ItemSlot*>(smem + kOffItems)[s].tag = -1;
+        for (int s = 0; s < kItemRing; ++s) mbar_init(bars + (2 * kNB + 2 * kNA + kQrecRing + s) * 8, 1);
         *reinterpret_cast<volatile int*>(smem + kOffAbort) = 0;
+        for (int a = 0; a < kNA; ++a) reinterpret_cast<volatile int*>(smem + kOffAttendDone)[a] = 0;
+    }
+    {   // shared-memory copy of both ends of the unit list (heavy units from the front, light units from the back)
+        int* cache = reinterpret_cast<int*>(smem + kOffUnits);
+        for (int u = threadIdx.x; u < min(p.units, kUnitCache); u += kFusedThreads) {
+            cache[u] = p.unit_list[u];
+            cache[kUnitCache + u] = p.unit_list[p.units - 1 - u];
+        }
+    }
+    if (threadIdx.x == 0) {
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     __syncthreads();
@@ -482,8 +609,7 @@ constexpr int kCombineChunk = 1024;
 template <bool FUSED>
 __device__ __forceinline__ size_t combine_slot(const DecodeParams& p, size_t head, int bg, int hl, int e) {
     if (FUSED) {   // item number of split e / kNA (see decode_item), then the attend warp
-        const int units = p.batch * p.Hkv;
-        const int item = (p.total_items / units - 1 - e / kNA) * units + bg;
+        const int item = (p.item_rows - 1 - e / kNA) * p.units + bg;
         return ((size_t)item * kNA + (e % kNA)) * kMaxG + hl;
     }
     return head * p.splits + e;

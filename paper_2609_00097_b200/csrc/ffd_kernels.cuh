@@ -23,7 +23,10 @@ constexpr int kD = 128;            // head_dim
 constexpr int kBlk = 64;           // tokens per block
 constexpr int kTileBytes = kBlk * kD * 2;
 constexpr int kCodeBytes = kBlk * kD / 4;
-constexpr int kWarps = 7;          // warps per decode CTA: 7 x (16 KB K slot + 16 KB V slot) of shared memory
+#ifndef FFD_DENSE_WARPS
+#define FFD_DENSE_WARPS 7
+#endif
+constexpr int kWarps = FFD_DENSE_WARPS;          // warps per decode CTA: 7 x (16 KB K slot + 16 KB V slot) of shared memory
 constexpr int kSlotBytes = kTileBytes;
 constexpr int kDecodeSmem = kWarps * 2 * kSlotBytes + 128;   // + mbarriers
 constexpr uint32_t kSuspendHintNs = 200000u;       // upper bound of one hardware-suspended try_wait
@@ -61,7 +64,13 @@ struct DecodeParams {
     float* fpart_ml;         // fused path: [items, attend warps, 4 heads, 2]
     float* fpart_acc;        // fused path: [items, attend warps, 4 heads, 128]
     int total_items;         // fused path: work items = ceil(max_blocks / 32) * B * Hkv
-    uint32_t* item_counter;  // fused path: next work item to hand out (workspace; zeroed by the pseudo-max kernel)
+    uint32_t* item_counter;  // fused path: next heavy-class draw (workspace; zeroed at the start of every call)
+    uint32_t* light_counter; // fused path: next light-class draw
+    uint32_t* class_counts;  // fused path: [0] heavy units, [1] light units found by the pseudo-max kernel (workspace)
+    int32_t* unit_list;      // fused path: heavy units from the front, light units from the back (workspace)
+    int units;               // batch * Hkv
+    int item_rows;           // fused path: work items per (sequence, KV head) = ceil(max_blocks / 24)
+    unsigned long long units_magic, hkv_magic;   // reciprocals for fast_div
     uint8_t* kept_mask;      // nullable [B, Hq, max_blocks]
     float* block_max;        // nullable [B, Hq, max_blocks]
     void* out;               // [B, Hq, 128] bf16 or fp32
@@ -161,6 +170,14 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 __device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
+
+// n / d for n < 2^32 with magic = 2^48 / d + 1 (host-computed): exact while n * d < 2^48
+__host__ __device__ __forceinline__ unsigned long long fast_div_magic(unsigned d) {
+    return (1ull << 48) / d + 1ull;
+}
+__device__ __forceinline__ unsigned fast_div(unsigned n, unsigned long long magic) {
+    return (unsigned)__umul64hi((unsigned long long)n << 16, magic);
+}
 
 // physical page of logical block `blk`; returns -1 (and flags) when the table entry is out of range
 __device__ __forceinline__ int page_of(const DecodeParams& p, int b, int blk) {
@@ -262,6 +279,39 @@ __device__ __forceinline__ void scan_bfrag4(uint32_t* bfrag, const uint4& qv, co
         const __half2 pick = piece ? lo : hi;
         bfrag[x] = *reinterpret_cast<const uint32_t*>(&pick);
     }
+}
+
+// The same, and also sum_c |q_c * s_c| over the lane's channels (fp16, two running pairs): the ingredient of an
+// upper bound on every approximate score of the block.  base = index of the first of the four registers (0, 4, 8, 12):
+// register idx belongs to k-step idx / 2, whose pre-scaling of q is undone here.
+__device__ __forceinline__ void scan_bfrag4_bound(uint32_t* bfrag, const uint4& qv, const uint4& sv, int piece,
+                                                  int base, __half2& sum_a, __half2& sum_b) {
+    const uint32_t q[4] = {qv.x, qv.y, qv.z, qv.w};
+    const uint32_t sc[4] = {sv.x, sv.y, sv.z, sv.w};
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        const __half2 a = *reinterpret_cast<const __half2*>(&q[x]);
+        const __half2 b = *reinterpret_cast<const __half2*>(&sc[x]);
+        const __half2 hi = __hmul2(a, b);
+        const __half2 lo = __hfma2(a, b, __hneg2(hi));
+        const __half2 pick = piece ? lo : hi;
+        bfrag[x] = *reinterpret_cast<const uint32_t*>(&pick);
+        const float undo = 1.0f / scan_pos_scale((base + x) >> 1);
+        const __half2 u = __floats2half2_rn(undo, undo);
+        if (x & 1) sum_b = __hfma2(__habs2(hi), u, sum_b);
+        else sum_a = __hfma2(__habs2(hi), u, sum_a);
+    }
+}
+
+// Upper bound (in logits) on the approximate score of every token of the block for the head this lane's column
+// belongs to: |sum_c q_c s_c level_c| <= 1.5 sum_c |q_c s_c|.  The factor 1.02 and the constant cover the fp16
+// roundings of the products and of the 16-term running sums (each below 2^-11 relative) and the lo pieces.
+__device__ __forceinline__ float scan_bound(__half2 sum_a, __half2 sum_b, float sm_scale) {
+    const float2 a = __half22float2(sum_a), b = __half22float2(sum_b);
+    float s = (a.x + a.y) + (b.x + b.y);
+    s += __shfl_xor_sync(kFull, s, 1);
+    s += __shfl_xor_sync(kFull, s, 2);
+    return 1.5f * 1.02f * sm_scale * s + 1e-3f;
 }
 
 template <bool PRECISE>

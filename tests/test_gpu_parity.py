@@ -57,8 +57,16 @@ def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None):
     B, Hq, mb = w.B, w.Hq, w.max_blocks
     kept = torch.full((B, Hq, mb), 255, dtype=torch.uint8, device="cuda")
     bm = torch.full((B, Hq, mb), float("nan"), dtype=torch.float32, device="cuda")
+    # without the block-max debug output the kernel may skip the tensor-core work of blocks whose scale-only upper
+    # bound already rules them out: the decisions and the output must not change
+    kept_fast = torch.full((B, Hq, mb), 255, dtype=torch.uint8, device="cuda")
+    dc.decode(delta, kept_mask=kept_fast)
+    assert ffd.ffd_read_device_status(dc.workspace) == 0
+    out_fast = dc.out.clone()
     dc.decode(delta, kept_mask=kept, block_max=bm)
     assert ffd.ffd_read_device_status(dc.workspace) == 0
+    assert torch.equal(kept, kept_fast)
+    assert (dc.out - out_fast).abs().max().item() <= 1e-6
     out = dc.out.cpu().numpy().astype(np.float64)
     lse = dc.lse.cpu().numpy().astype(np.float64)
     kept = kept.cpu().numpy()
