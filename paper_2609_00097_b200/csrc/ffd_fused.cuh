@@ -1,19 +1,22 @@
 // The fused sparse kernel: scan -> top-delta select -> exact attention over kept blocks, in one persistent launch.
 //
-// One CTA per SM, 16 warps in two roles that run concurrently (register budgets set with setmaxnreg):
-//   12 scan warps   stream the 2-bit codes and scales of every block through a private 3-stage cp.async ring
-//                   (3 blocks = 6.9 KB in flight per warp), compute the block maxima of the approximate scores
-//                   on the tensor cores and publish the keep decisions of one work item in a batch descriptor;
-//   4 attend warps  take the kept blocks of a published batch, stage their K and V tiles (16 KB each) through
-//                   private swizzled slots with cp.async + mbarrier and run the exact online-softmax attention.
-// A work item is 24 consecutive blocks of one (sequence, KV head).  Items are handed out dynamically: lane 0 of scan
-// warp 0 draws item numbers from a global counter (the atomic for the next draw is always in flight, so its latency
-// is not waited for), skips items without blocks, decodes the item once and publishes it two items ahead in a tagged
-// ring in shared memory; it also starts the copy of the item's query record (pre-scaled fp16 query fragments +
-// thresholds, written by the pseudo-max kernel).  Readers check the tag; nobody divides or reloads sequence
-// lengths on the per-block path.  Scan warps run up to two batches ahead of the attend warps (two descriptors,
-// full/empty mbarriers), which also keeps all scan warps within one batch of each other.
-// Every wait is bounded; on expiry the warp records kDevTimeout and the CTA winds down.
+// One CTA per SM, 16 warps in three jobs that run concurrently (register budgets set with setmaxnreg):
+//   1 scheduling warp  (warp 0) draws work items from two global counters, decodes them once and publishes them two
+//                      entries ahead in a ring in shared memory (one mbarrier per entry); it also starts the copy of
+//                      the item's query record (pre-scaled fp16 query fragments + thresholds, written by the
+//                      pseudo-max kernel).  The atomic for the next draw of each class is always in flight.
+//   11 scan warps      stream the 2-bit codes and scales of every block through a private 3-stage cp.async ring
+//                      (3 blocks = 6.9 KB in flight per warp), bound the block's scores from its scales alone and,
+//                      unless that already rules the block out, compute the block maxima of the approximate scores
+//                      on the tensor cores; they publish the keep decisions of one work item in a batch descriptor.
+//   4 attend warps     take the kept blocks of a published batch, stage their K and V tiles (16 KB each) through
+//                      private swizzled slots with cp.async + mbarrier and run the exact online-softmax attention.
+// A work item is 22 consecutive blocks of one (sequence, KV head): two per scan warp.  Scan warps may run up to eight
+// batches ahead of the attend warps (eight descriptors, full/empty mbarriers).  Units that the pseudo-max kernel's
+// hint marks as dense ("heavy") are scheduled so that at most a few heavy batches are outstanding per CTA and the
+// scan warps' spare time goes to light items (see ItemSched).
+// Nobody divides or reloads sequence lengths on the per-block path.  Every wait is bounded; on expiry the warp
+// records kDevTimeout and the CTA winds down.
 #pragma once
 #include "ffd_kernels.cuh"
 
@@ -38,7 +41,10 @@ constexpr int kStageBytes = kCodeBytes + kD * 2;   // 2048 B codes + 256 B scale
 #define FFD_NB 8
 #endif
 constexpr int kNB = FFD_NB;                 // batch descriptors: how far the scan warps may run ahead of the attend warps
-constexpr int kHeavyAhead = 2;         // heavy batches outstanding at most once the attend warps are the bottleneck
+#ifndef FFD_HEAVY_AHEAD
+#define FFD_HEAVY_AHEAD 2
+#endif
+constexpr int kHeavyAhead = FFD_HEAVY_AHEAD;         // heavy batches outstanding at most once the attend warps are the bottleneck
 constexpr int kUnitCache = 512;        // entries of the unit list kept in shared memory
 constexpr int kItemRing = 8;           // decoded items published ahead
 constexpr int kQrecRing = 4;           // query records staged ahead
@@ -204,11 +210,11 @@ __device__ __forceinline__ int item_publish(const DecodeParams& p, ItemSched* sc
             if ((sc->heavy_hist >> (sc->released & 63)) & 1ull) --sc->heavy_queued;
         const bool heavy_left = sc->pend_heavy < sc->total_heavy, light_left = sc->pend_light < sc->total_light;
         if (!heavy_left && !light_left) { sc->finished = 1; break; }
-        // Heavy batches published and not yet released.  While the attend warps keep up with the scan (nothing but
-        // the entries published ahead is outstanding) the limit does not bind; once they fall behind, at most
-        // kHeavyAhead heavy batches may be outstanding, so that no CTA sits on heavy work others could have taken
-        // and the scan warps spend their spare time on light items.
-        const int limit = (seq - sc->released <= 3) ? 4 : kHeavyAhead;
+        // Heavy batches published and not yet released: at most four (two of them are the entries published ahead
+        // for prefetching).  Near the end of the heavy work, when the attend warps are the bottleneck, at most
+        // kHeavyAhead, so that no CTA sits on heavy work others could have taken.  Beyond the limit the scan warps
+        // spend their spare time on light items.
+        const int limit = (seq - sc->released <= 3 || sc->total_heavy - sc->pend_heavy > 2 * (int)gridDim.x) ? 4 : kHeavyAhead;
         bool heavy;
         if (heavy_left && sc->heavy_queued < limit) heavy = true;
         else if (light_left) heavy = false;
@@ -486,7 +492,9 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
         if (item < 0) break;
         Item it;
         it.slot = item; it.b = d.b; it.g = d.g; it.nblk = d.nblk;
-        unsigned mine = my_entries(d, it.nblk, a, lane);
+        // the share rotates with the batch number: when the kept count is not a multiple of four, the extra blocks
+        // go to a different warp each time
+        unsigned mine = my_entries(d, it.nblk, (a + bi) & (kNA - 1), lane);
         const bool any = mine != 0;
         if (any) attend_setup(st, p.q + ((size_t)it.b * p.Hq + (size_t)it.g * p.G) * kD, p.G, lane);
         while (mine && ok) {
@@ -509,7 +517,7 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
                 if (mbar_test(bars + (bi2 & (kNB - 1)) * 8, (bi2 / kNB) & 1)) {
                     const BatchDesc& d2 = descs[bi2 & (kNB - 1)];
                     if (d2.item >= 0) {
-                        const unsigned mine2 = my_entries(d2, d2.nblk, a, lane);
+                        const unsigned mine2 = my_entries(d2, d2.nblk, (a + bi2) & (kNA - 1), lane);
                         if (mine2) {
                             const int nlb = __ffs(mine2) - 1;
                             next_k = kbase + (size_t)d2.tile[nlb] * kTileVec;
