@@ -75,8 +75,10 @@ const char* ffd_status_string(ffd_status status);
 /* Bytes of device workspace ffd_decode / ffd_decode_dense need for this geometry (host call, no CUDA). */
 ffd_status ffd_workspace_bytes(const ffd_config* cfg, int32_t batch, int32_t max_blocks_per_seq, size_t* bytes);
 
-/* Zeroes the status word at the head of a freshly allocated workspace.  Call once before the first decode
- * with that workspace (the status word is sticky across calls until ffd_read_device_status clears it). */
+/* Zeroes the header of a freshly allocated workspace (status word, work counters).  Call once before the first
+ * decode with that workspace.  The status word is sticky across calls until ffd_read_device_status clears it; the
+ * work counters are left at zero by every completed ffd_decode.  If a decode call was interrupted (a CUDA error),
+ * call this again before reusing the workspace. */
 ffd_status ffd_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 
 /*

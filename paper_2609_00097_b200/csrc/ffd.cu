@@ -33,6 +33,8 @@ __device__ __forceinline__ uint32_t quant_code(float x, float s) {
 
 __global__ void __launch_bounds__(128) quantize_kernel(QuantParams p) {
     const int g = blockIdx.y, b = blockIdx.z;
+    pdl_launch_dependents();
+    pdl_wait();
     int n = p.seq_lens[b];
     const int cap = p.max_blocks * kBlk;
     n = n < 0 ? 0 : (n > cap ? cap : n);
@@ -109,6 +111,8 @@ constexpr int kPmWarps = 20;   // one warp per sink / local block in the default
 __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p) {
     const int g = blockIdx.x, b = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    pdl_launch_dependents();
+    pdl_wait();
     const int n = clamped_seq_len(p, b);
     const int nb = (n + kBlk - 1) / kBlk;
     const int ns = min(p.n_sink, nb);
@@ -186,6 +190,8 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(DecodeParams p) 
     const int split = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int r = lane >> 2, j = lane & 3;
+    pdl_launch_dependents();
+    pdl_wait();
     const int n = clamped_seq_len(p, b);
     const int nb = (n + kBlk - 1) / kBlk;
     const int blk_begin = split * p.blocks_per_split;
@@ -338,6 +344,9 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(DecodeParams p) 
 
 __global__ void clear_status_kernel(uint32_t* status) { *status = 0u; }
 
+// status word, work counters and class counts: the first 256 bytes of a workspace
+__global__ void clear_header_kernel(uint32_t* header) { header[threadIdx.x] = 0u; }
+
 // ---- host side --------------------------------------------------------------------------------------------
 
 struct Plan {
@@ -392,6 +401,23 @@ static ffd_status check_geometry(int batch, int max_blocks, int num_pages) {
 }
 
 static cudaEvent_t g_prof_start = nullptr, g_prof_stop = nullptr;
+
+// Launch with programmatic stream serialization: the grid may be scheduled while its predecessor in the stream is
+// still running; every kernel of this library calls pdl_wait() before it reads anything a predecessor wrote.
+template <typename... KArgs, typename... Args>
+static void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    (void)cudaLaunchKernelEx(&cfg, kernel, args...);   // errors surface through cudaGetLastError in launch_status
+}
 
 static ffd_status launch_status() { return cudaGetLastError() == cudaSuccess ? FFD_OK : FFD_ERR_CUDA; }
 
@@ -469,20 +495,20 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
             cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
             cudaFuncSetAttribute(fused_sparse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem) != cudaSuccess)
             return FFD_ERR_CUDA;
-        // work counter and class counts start every call from zero
-        if (cudaMemsetAsync(ws + 64, 0, 16, s) != cudaSuccess) return FFD_ERR_CUDA;
-        pseudomax_kernel<<<dim3(p.Hkv, batch), kPmWarps * 32, 0, s>>>(p);
+        // the work counters and class counts at ws + 64 are zero here: ffd_workspace_init zeroes them and the
+        // combine kernel of every call leaves them zeroed for the next one
+        launch_pdl(pseudomax_kernel, dim3(p.Hkv, batch), dim3(kPmWarps * 32), 0, s, p);
         if (prof) cudaEventRecord(g_prof_start, s);
-        fused_sparse_kernel<<<min(p.total_items, sms), kFusedThreads, kFusedSmem, s>>>(p);
+        launch_pdl(fused_sparse_kernel, dim3(min(p.total_items, sms)), dim3(kFusedThreads), kFusedSmem, s, p);
         if (prof) cudaEventRecord(g_prof_stop, s);
-        combine_kernel<true><<<dim3(p.Hq, batch), kCombineThreads, 0, s>>>(p);
+        launch_pdl(combine_kernel<true>, dim3(p.Hq, batch), dim3(kCombineThreads), 0, s, p);
     } else {
         if (cudaFuncSetAttribute(decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem) != cudaSuccess)
             return FFD_ERR_CUDA;
         if (prof) cudaEventRecord(g_prof_start, s);
-        decode_kernel<false><<<grid, kWarps * 32, kDecodeSmem, s>>>(p);
+        launch_pdl(decode_kernel<false>, grid, dim3(kWarps * 32), kDecodeSmem, s, p);
         if (prof) cudaEventRecord(g_prof_stop, s);
-        combine_kernel<false><<<dim3(p.Hq, batch), kCombineThreads, 0, s>>>(p);
+        launch_pdl(combine_kernel<false>, dim3(p.Hq, batch), dim3(kCombineThreads), 0, s, p);
     }
     return launch_status();
 }
@@ -524,7 +550,7 @@ ffd_status ffd_workspace_init(void* workspace, size_t workspace_bytes, void* str
     if (!workspace) return FFD_ERR_NULL;
     if (workspace_bytes < 256) return FFD_ERR_WORKSPACE;
     if (misaligned(workspace)) return FFD_ERR_ALIGN;
-    clear_status_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<uint32_t*>(workspace));
+    clear_header_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<uint32_t*>(workspace));
     return launch_status();
 }
 
@@ -543,8 +569,8 @@ ffd_status ffd_quantize_keys(const ffd_config* cfg, const void* k_cache, void* k
     QuantParams p{static_cast<const __nv_bfloat16*>(k_cache), static_cast<uint8_t*>(k_quant),
                   static_cast<__half*>(k_scales), block_table, seq_lens, first_token,
                   cfg->num_kv_heads, max_blocks_per_seq, num_pages};
-    quantize_kernel<<<dim3(max_blocks_per_seq < 64 ? max_blocks_per_seq : 64, cfg->num_kv_heads, batch), 128, 0,
-                      static_cast<cudaStream_t>(stream)>>>(p);
+    launch_pdl(quantize_kernel, dim3(max_blocks_per_seq < 64 ? max_blocks_per_seq : 64, cfg->num_kv_heads, batch),
+               dim3(128), 0, static_cast<cudaStream_t>(stream), p);
     return launch_status();
 }
 

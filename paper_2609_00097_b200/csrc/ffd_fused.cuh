@@ -584,6 +584,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodePa
         *reinterpret_cast<volatile int*>(smem + kOffAbort) = 0;
         for (int a = 0; a < kNA; ++a) reinterpret_cast<volatile int*>(smem + kOffAttendDone)[a] = 0;
     }
+    pdl_launch_dependents();
+    pdl_wait();   // the pseudo-max kernel's outputs (unit list, class counts, query records) are needed from here on
     {   // shared-memory copy of both ends of the unit list (heavy units from the front, light units from the back)
         int* cache = reinterpret_cast<int*>(smem + kOffUnits);
         for (int u = threadIdx.x; u < min(p.units, kUnitCache); u += kFusedThreads) {
@@ -627,6 +629,14 @@ template <bool FUSED>
 __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p) {
     const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
     const int el = tid >> 5, cg = tid & 31;
+    pdl_launch_dependents();
+    pdl_wait();
+    if (FUSED && h == 0 && b == 0 && tid == 0) {   // the next call's draws and class lists start from zero
+        *p.item_counter = 0u;
+        p.class_counts[0] = 0u;
+        p.class_counts[1] = 0u;
+        *p.light_counter = 0u;
+    }
     const size_t head = (size_t)b * p.Hq + h;
     const int g = h / p.G, hl = h % p.G, bg = b * p.Hkv + g;
     const int n = min(max(p.seq_lens[b], 0), p.max_blocks * kBlk);

@@ -80,6 +80,12 @@ struct DecodeParams {
 
 // ---- small helpers --------------------------------------------------------------------------------------
 
+// Programmatic dependent launch: every kernel of the library lets its successor in the stream be scheduled early
+// (pdl_launch_dependents) and itself waits, before it touches anything a predecessor may have written, until the
+// predecessor grid has completed and its writes are visible (pdl_wait).  This only hides launch latency.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
+
 __device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                         uint32_t b0, uint32_t b1) {
     asm volatile(
