@@ -249,12 +249,14 @@ struct ScanCursor {
     int seq;       // published item the cursor is in (-1 before the first)
     Item it;
     int lb;
+    int pages;     // lane l: physical page of block l of the item (loaded once per item, not per block)
     bool end;      // ran into the end of the work
 };
 
 // Advance to this warp's next block; false when the item it lies in has not been published yet (the cursor then
 // stays where it can resume) or when there is no more work.
-__device__ __forceinline__ bool cursor_next(ScanCursor& c, const ItemSlot* items, uint32_t ibars, int w) {
+__device__ __forceinline__ bool cursor_next(const DecodeParams& p, ScanCursor& c, const ItemSlot* items,
+                                            uint32_t ibars, int w, int lane) {
     if (c.end) return false;
     int lb = c.lb + kScanners;
     while (lb >= c.it.nblk) {
@@ -263,6 +265,12 @@ __device__ __forceinline__ bool cursor_next(ScanCursor& c, const ItemSlot* items
         ++c.seq;
         if (c.it.slot < 0) { c.end = true; c.it.nblk = 0; return false; }
         lb = w;
+        if (lb < c.it.nblk) {   // one coalesced read of the item's page-table entries; used a block-time later
+            const int blk = c.it.blk0 + lane;
+            c.pages = -1;
+            if (lane < c.it.nblk)
+                c.pages = p.block_table ? p.block_table[(size_t)c.it.b * p.max_blocks + blk] : c.it.b * p.max_blocks + blk;
+        }
     }
     c.lb = lb;
     return true;
@@ -271,7 +279,11 @@ __device__ __forceinline__ bool cursor_next(ScanCursor& c, const ItemSlot* items
 // start the copy of one block's codes + scales into a ring stage (one commit group); remembers the block's tile
 __device__ __forceinline__ void ring_issue(const DecodeParams& p, const ScanCursor& c, uint32_t stage,
                                            volatile int* stage_tile, int lane) {
-    const int page = page_of(p, c.it.b, c.it.blk0 + c.lb);
+    int page = __shfl_sync(kFull, c.pages, c.lb);
+    if (page < 0 || page >= p.num_pages) {   // bad table entry: reported, the block is skipped
+        if (lane == 0) atomicOr(p.status, kDevBadPage);
+        page = -1;
+    }
     const int tile = page >= 0 ? page * p.Hkv + c.it.g : -1;
     if (tile >= 0) {
         const uint4* codes = reinterpret_cast<const uint4*>(p.k_quant + (size_t)tile * kCodeBytes);
@@ -341,6 +353,7 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
     const int w0 = w - kSched;      // index among the scanning warps (-1: the scheduling warp, which scans nothing)
     ic.lb = w0 - kScanners;
     ic.end = false;
+    ic.pages = -1;
     int issued = 0, consumed = 0;   // this warp's blocks whose copies were started / whose data was taken
 
 #pragma unroll 1
@@ -390,7 +403,7 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
 #pragma unroll 1
         for (int lb = w0 >= 0 ? w0 : it.nblk; lb < it.nblk; lb += kScanners) {
             // keep the ring full: blocks consumed .. consumed + kRing - 1 of this warp's stream
-            while (issued < consumed + kRing && cursor_next(ic, items, ibars, w0)) {
+            while (issued < consumed + kRing && cursor_next(p, ic, items, ibars, w0, lane)) {
                 ring_issue(p, ic, ring + (issued % kRing) * kStageBytes, stage_tile + issued % kRing, lane);
                 ++issued;
             }
@@ -411,7 +424,7 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
             const int tile = stage_tile[st];
             __syncwarp();   // the stage is free again
             ++consumed;
-            if (issued < consumed + kRing && cursor_next(ic, items, ibars, w0)) {
+            if (issued < consumed + kRing && cursor_next(p, ic, items, ibars, w0, lane)) {
                 ring_issue(p, ic, ring + (issued % kRing) * kStageBytes, stage_tile + issued % kRing, lane);
                 ++issued;
             }
