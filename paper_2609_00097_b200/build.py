@@ -8,7 +8,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "libffd_b200.so")
 SOURCES = [os.path.join(CSRC, "ffd.cu")]
-HEADERS = [os.path.join(CSRC, "ffd_kernels.cuh"), os.path.join(os.path.dirname(_HERE), "include", "ffd.h")]
+HEADERS = [os.path.join(CSRC, "ffd_kernels.cuh"), os.path.join(CSRC, "ffd_fused.cuh"),
+           os.path.join(os.path.dirname(_HERE), "include", "ffd.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-shared",
               "-Xcompiler", "-fPIC"]
 

@@ -104,7 +104,8 @@ __global__ void __launch_bounds__(128) unpack_kernel(const uint8_t* k_quant, uin
 }
 
 constexpr int kPmHintBlocks = 64;
-constexpr int kPmWarps = 20;   // one warp per sink / local block in the default configuration (1 + 16)
+constexpr int kPmWarps = 24;   // one warp per sink / local block in the default configuration (1 + 16), the rest sample
+constexpr int kPmSamples = 7;  // blocks sampled between the sink and the local window for the scheduling hint
 
 // ---- pseudo-max (Sec. 3.2; Alg. 1 "Pseudo-max estimation") ------------------------------------------------
 // One CTA per (KV head, sequence): its warps scan the sink and local blocks and reduce the block maxima.
@@ -132,9 +133,15 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
         for (int x = 0; x < 4; ++x)
             dst[x * 32 + lane] = make_uint4(sq.qh[4 * x], sq.qh[4 * x + 1], sq.qh[4 * x + 2], sq.qh[4 * x + 3]);
     }
+    // Besides the sink and local blocks, a few blocks spread evenly over the middle of the sequence are scanned.
+    // They never enter m_tilde: they only tell the scheduler below how dense this unit's selection will be.
+    const int middle = local_begin - ns;
+    const int nsamp = min(kPmSamples, middle);
     float best = -INFINITY;
-    for (int s = warp; s < count; s += kPmWarps) {
-        const int blk = s < ns ? s : local_begin + (s - ns);
+    for (int s = warp; s < count + nsamp; s += kPmWarps) {
+        const bool sample = s >= count;
+        const int blk = sample ? ns + (int)(((long long)(2 * (s - count) + 1) * middle) / (2 * nsamp))
+                               : (s < ns ? s : local_begin + (s - ns));
         const int page = page_of(p, b, blk);
         if (page < 0) continue;
         const size_t tile = (size_t)page * p.Hkv + g;
@@ -145,7 +152,7 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
                   reinterpret_cast<const uint4*>(p.k_scales + tile * kD), lane);
         const float bm = scan_compute<true>(sr, sq, lane, rows, p.sm_scale, band);
         if (lane < kMaxG && s < kPmHintBlocks) sbm[s][lane] = bm;
-        best = fmaxf(best, bm);
+        if (!sample) best = fmaxf(best, bm);
     }
     if (lane < kMaxG) smax[warp][lane] = best;
     __syncthreads();
@@ -162,18 +169,21 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
         if (threadIdx.x < kMaxG) sthr[threadIdx.x] = thr;
     }
     __syncthreads();
-    // Scheduling hint for the fused kernel: a (sequence, KV head) whose sink / local blocks are mostly kept is
-    // likely to keep much of its cache (a "dense" head), so its work items are expensive and are handed out first.
-    // The hint only orders the work; it never changes a result.
-    const int hinted = min(count, kPmHintBlocks);
+    // Scheduling hint for the fused kernel: a (sequence, KV head) that keeps at least half of the sampled middle
+    // blocks (of its sink / local blocks, when the sequence has no middle) is a "dense" unit: its work items are
+    // expensive for the attend warps and are handed out first.  The hint only orders the work; it never changes a
+    // result.
+    int h_begin = 0, hinted = min(count, kPmHintBlocks);
+    if (nsamp > 0 && count + nsamp <= kPmHintBlocks) { h_begin = count; hinted = nsamp; }
     bool kept_any = false;
     if ((int)threadIdx.x < hinted)
-        for (int h = 0; h < p.G; ++h) kept_any |= sbm[threadIdx.x][h] >= sthr[h];
+        for (int h = 0; h < p.G; ++h) kept_any |= sbm[h_begin + threadIdx.x][h] >= sthr[h];
     const int kept = __syncthreads_count(kept_any);
     if (threadIdx.x == 0) {
         const int bg = b * p.Hkv + g;
         if (hinted > 0 && 2 * kept >= hinted) p.unit_list[atomicAdd(&p.class_counts[0], 1u)] = bg;
         else p.unit_list[p.units - 1 - (int)atomicAdd(&p.class_counts[1], 1u)] = bg;
+        FFD_TL(14, blockIdx.y == 0);
     }
 }
 
@@ -367,7 +377,7 @@ static Plan make_plan(const ffd_config* cfg, int batch, int max_blocks) {
     pl.blocks_per_split = bps;
     pl.splits = max_blocks > 0 ? (max_blocks + bps - 1) / bps : 1;
     const size_t heads = (size_t)batch * cfg->num_q_heads;
-    pl.total_items = ((max_blocks + kItemBlocks - 1) / kItemBlocks) * batch * cfg->num_kv_heads;
+    pl.total_items = item_geometry(units, max_blocks).item_rows * batch * cfg->num_kv_heads;
     const size_t fslots = (size_t)pl.total_items * kNA * kMaxG;
     pl.off_mtilde = 256;
     pl.off_units = align_up(pl.off_mtilde + heads * sizeof(float), 256);
@@ -477,7 +487,8 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
     p.light_counter = reinterpret_cast<uint32_t*>(ws + 76);
     p.unit_list = reinterpret_cast<int32_t*>(ws + pl.off_units);
     p.units = batch * cfg->num_kv_heads;
-    p.item_rows = (max_blocks + kItemBlocks - 1) / kItemBlocks;
+    p.item_rows = item_geometry(p.units, max_blocks).item_rows;
+    p.rows_small = item_geometry(p.units, max_blocks).rows_small;
     p.units_magic = fast_div_magic((unsigned)p.units);
     p.hkv_magic = fast_div_magic((unsigned)cfg->num_kv_heads);
     p.kept_mask = kept_mask;
@@ -677,3 +688,16 @@ ffd_status ffd_read_device_status(void* workspace, void* stream, uint32_t* statu
 }
 
 }  // extern "C"
+
+// Diagnostic build only: copies the probe tables to the host ([160][16] first-hit timestamps in ns, then [160][8]
+// clock buckets) and clears the timestamps.  Not part of the library's interface.
+#ifdef FFD_TIMELINE
+extern "C" int ffd_debug_timeline(unsigned long long* host) {
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(host, g_tl, sizeof(unsigned long long) * 160 * 16);
+    static unsigned long long zeros[160 * 16];
+    cudaMemcpyToSymbol(g_tl, zeros, sizeof(zeros));
+    cudaMemcpyFromSymbol(host + 160 * 16, g_acc, sizeof(long long) * 160 * 8);
+    return 0;
+}
+#endif

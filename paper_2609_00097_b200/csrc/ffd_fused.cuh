@@ -35,6 +35,41 @@ constexpr int kAttendRegs = (65536 - kNS * 32 * kScanRegs) / (kNA * 32);
 static_assert(kAttendRegs % 8 == 0 && kScanRegs % 8 == 0, "setmaxnreg takes multiples of 8");
 constexpr int kItemBlocks = 2 * kScanners;   // blocks per work item: two per scanning warp
 static_assert(kItemBlocks <= 24, "batch descriptor arrays");
+// The sequence is cut into items from block 0 upwards: first rows_small half-size items (one block per scanning
+// warp), then full items.  Items are drawn from the sequence END backwards, so the half-size ones are drawn last and
+// the CTAs run out of work within half an item's time of each other.
+constexpr int kSmallBlocks = kScanners;
+
+struct ItemGeom { int rows_small, item_rows; };
+
+// pure function of the launch geometry (the workspace layout depends on it)
+__host__ __device__ inline ItemGeom item_geometry(long units, int max_blocks) {
+    ItemGeom g;
+    const int full_rows = (max_blocks + kItemBlocks - 1) / kItemBlocks;
+    const int all_small = (max_blocks + kSmallBlocks - 1) / kSmallBlocks;
+    if (units * full_rows < 2 * 148) {
+        g.rows_small = all_small;        // few items per SM: halve them all
+    } else {
+        const long want = (6 * 148 + units - 1) / units;             // about three half-size heavy items per SM
+        const long cap = all_small / 3;                              // at most a third of the blocks
+        g.rows_small = (int)(want < cap ? want : cap);
+    }
+    const int rest = max_blocks - g.rows_small * kSmallBlocks;
+    g.item_rows = g.rows_small + (rest > 0 ? (rest + kItemBlocks - 1) / kItemBlocks : 0);
+    return g;
+}
+
+// item number idx of a sequence, counted from block 0: first block and capacity
+__device__ __forceinline__ void item_span(const DecodeParams& p, int idx, int& blk0, int& cap) {
+    if (idx < p.rows_small) { blk0 = idx * kSmallBlocks; cap = kSmallBlocks; }
+    else { blk0 = p.rows_small * kSmallBlocks + (idx - p.rows_small) * kItemBlocks; cap = kItemBlocks; }
+}
+
+// items a sequence of nb blocks is cut into
+__device__ __forceinline__ int item_count(const DecodeParams& p, int nb) {
+    const int s = p.rows_small * kSmallBlocks;
+    return nb <= s ? (nb + kSmallBlocks - 1) / kSmallBlocks : p.rows_small + (nb - s + kItemBlocks - 1) / kItemBlocks;
+}
 constexpr int kRing = 3;               // code-ring stages per scan warp
 constexpr int kStageBytes = kCodeBytes + kD * 2;   // 2048 B codes + 256 B scales
 #ifndef FFD_NB
@@ -139,8 +174,9 @@ __device__ __forceinline__ Item decode_item(const DecodeParams& p, const ItemSch
     it.g = bg - it.b * p.Hkv;
     it.n = clamped_seq_len(p, it.b);
     const int nb = (it.n + kBlk - 1) / kBlk;
-    it.blk0 = (p.item_rows - 1 - row) * kItemBlocks;
-    it.nblk = min(nb - it.blk0, kItemBlocks);
+    int cap;
+    item_span(p, p.item_rows - 1 - row, it.blk0, cap);
+    it.nblk = min(nb - it.blk0, cap);
     return it;
 }
 
@@ -214,7 +250,7 @@ __device__ __forceinline__ int item_publish(const DecodeParams& p, ItemSched* sc
         // for prefetching).  Near the end of the heavy work, when the attend warps are the bottleneck, at most
         // kHeavyAhead, so that no CTA sits on heavy work others could have taken.  Beyond the limit the scan warps
         // spend their spare time on light items.
-        const int limit = (seq - sc->released <= 3 || sc->total_heavy - sc->pend_heavy > 2 * (int)gridDim.x) ? 4 : kHeavyAhead;
+        const int limit = sc->total_heavy - sc->pend_heavy > 2 * (int)gridDim.x ? 4 : kHeavyAhead;
         bool heavy;
         if (heavy_left && sc->heavy_queued < limit) heavy = true;
         else if (light_left) heavy = false;
@@ -347,6 +383,7 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
     const volatile int* attend_done = reinterpret_cast<const volatile int*>(smem + kOffAttendDone);
     const int* unit_cache = reinterpret_cast<const int*>(smem + kOffUnits);
     if (w == 0 && lane == 0) sched_init(p, sched);
+    FFD_TL(3, w == 0 && lane == 0);
     ScanCursor ic;
     ic.seq = -1;
     ic.it.nblk = 0;
@@ -375,12 +412,14 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
                 }
                 bg = __shfl_sync(kFull, bg, 0);
                 pub = __shfl_sync(kFull, pub, 0);
+                FFD_TL(4, lane == 0 && bg >= 0);
                 if (bg >= 0) qrec_issue(p, pub, bg, qrecs, qbars, lane);
                 if (bg < -1) break;      // -3: published far enough; -2: nothing to publish for now
             }
         }
         if (!item_wait(ibars, seq)) *abort_flag = 1;
         const Item it = item_read(items, seq);
+        FFD_TL(5, w == 1 && lane == 0 && it.slot >= 0);
         const int slot = seq & (kNB - 1), use = seq / kNB;
         // the attend warps must have released this descriptor (kNB batches ago)
         if (use > 0 && !mbar_wait(bars + (kNB + slot) * 8, (use - 1) & 1)) *abort_flag = 1;
@@ -395,6 +434,7 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
         // the item's query record must have landed
         if (!mbar_wait(qbars + (seq & (kQrecRing - 1)) * 8, (seq / kQrecRing) & 1)) *abort_flag = 1;
         const uint32_t qrec = qrecs + (seq & (kQrecRing - 1)) * kQrecBytes;
+        FFD_TL(6, w == 1 && lane == 0);
         const size_t head0 = (size_t)it.b * p.Hq + (size_t)it.g * p.G;
         float thr, thr_col;   // threshold of head lane % 4 (block-max layout) and of head lane / 8 (B-column layout)
         asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(thr) : "r"(qrec + 2048 + j * 4));
@@ -409,8 +449,10 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
             }
             const int st = consumed % kRing;
             const uint32_t stage = ring + st * kStageBytes;
+            FFD_TL(7, w == 1 && lane == 0);
             ring_wait(issued - consumed - 1);
             __syncwarp();
+            FFD_TL(8, w == 1 && lane == 0);
             // codes into registers; B operand straight from the staged scales and the item's query record
             uint4 wv[4];
 #pragma unroll
@@ -464,6 +506,7 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(bars + slot * 8);   // this warp's share of the batch is published
+        FFD_TL(9, w == 1 && lane == 0);
     }
     cp_async_drain();
     if (*abort_flag && w == 0 && lane == 0) atomicOr(p.status, kDevTimeout);
@@ -473,12 +516,10 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
 
 // bits of the blocks of a published batch that attend warp `a` processes: every kNA-th kept block
 __device__ __forceinline__ unsigned my_entries(const BatchDesc& d, int nblk, int a, int lane) {
-    const unsigned kept = __ballot_sync(kFull, lane < nblk && d.keep4[lane] != 0);
-    unsigned mine = 0;
-    int rank = 0;
-    for (unsigned m = kept; m; m &= m - 1, ++rank)
-        if (rank % kNA == a) mine |= m & (0u - m);
-    return mine;
+    const bool is_kept = lane < nblk && d.keep4[lane] != 0;
+    const unsigned kept = __ballot_sync(kFull, is_kept);
+    const int rank = __popc(kept & ((1u << lane) - 1u));   // kept blocks before this lane's
+    return __ballot_sync(kFull, is_kept && (rank & (kNA - 1)) == a);
 }
 
 __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char* smem, int a, int lane) {
@@ -497,19 +538,26 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
     int issued_bi = -1, issued_lb = -1;   // block whose K/V copies are already in flight
     bool ok = true;
     AttendState st;
+    FFD_ACC_DECL;
     for (int bi = 0; ok; ++bi) {
         const int slot = bi & (kNB - 1), use = bi / kNB;
+        FFD_ACC(0);
         if (!mbar_wait(bars + slot * 8, use & 1)) { ok = false; break; }
+        FFD_ACC(1);
         const BatchDesc& d = descs[slot];
         const int item = d.item;
         if (item < 0) break;
+        FFD_TL(10, a == 0 && lane == 0);
         Item it;
         it.slot = item; it.b = d.b; it.g = d.g; it.nblk = d.nblk;
         // the share rotates with the batch number: when the kept count is not a multiple of four, the extra blocks
         // go to a different warp each time
         unsigned mine = my_entries(d, it.nblk, (a + bi) & (kNA - 1), lane);
         const bool any = mine != 0;
+        FFD_ACC(6);
         if (any) attend_setup(st, p.q + ((size_t)it.b * p.Hq + (size_t)it.g * p.G) * kD, p.G, lane);
+        FFD_TL(11, a == 0 && lane == 0 && any);
+        FFD_ACC(2);
         while (mine && ok) {
             const int lb = __ffs(mine) - 1;
             mine &= mine - 1;
@@ -545,6 +593,8 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
                               logit_scale_log2);
         }
         __syncwarp();
+        FFD_ACC(3);
+        FFD_TL(12, a == 0 && lane == 0 && any);
         if (lane == 0) {
             mbar_arrive(bars + (kNB + slot) * 8);   // done with this batch descriptor
             reinterpret_cast<volatile int*>(smem + kOffAttendDone)[a] = bi + 1;
@@ -580,12 +630,15 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
         }
     }
     cp_async_drain();
+    FFD_ACC_OUT(a == 0 && lane == 0);
+    FFD_TL(13, a == 0 && lane == 0);
     if (!ok && lane == 0) atomicOr(p.status, kDevTimeout);
 }
 
 __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodeParams p) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    FFD_TL(0, threadIdx.x == 0);
     if (threadIdx.x == 0) {
         const uint32_t bars = smem_u32(smem) + kOffBars;
         for (int s = 0; s < kNB; ++s) {
@@ -599,6 +652,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodePa
     }
     pdl_launch_dependents();
     pdl_wait();   // the pseudo-max kernel's outputs (unit list, class counts, query records) are needed from here on
+    FFD_TL(1, threadIdx.x == 0);
     {   // shared-memory copy of both ends of the unit list (heavy units from the front, light units from the back)
         int* cache = reinterpret_cast<int*>(smem + kOffUnits);
         for (int u = threadIdx.x; u < min(p.units, kUnitCache); u += kFusedThreads) {
@@ -610,6 +664,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodePa
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     __syncthreads();
+    FFD_TL(2, threadIdx.x == 0);
     if (warp < kNS) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kScanRegs));
         scan_role(p, smem, warp, lane);
@@ -644,6 +699,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
     const int el = tid >> 5, cg = tid & 31;
     pdl_launch_dependents();
     pdl_wait();
+    FFD_TL(15, FUSED && tid == 0 && blockIdx.y == 0);
     if (FUSED && h == 0 && b == 0 && tid == 0) {   // the next call's draws and class lists start from zero
         *p.item_counter = 0u;
         p.class_counts[0] = 0u;
@@ -654,7 +710,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
     const int g = h / p.G, hl = h % p.G, bg = b * p.Hkv + g;
     const int n = min(max(p.seq_lens[b], 0), p.max_blocks * kBlk);
     const int nb = (n + kBlk - 1) / kBlk;
-    const int entries = FUSED ? ((nb + kItemBlocks - 1) / kItemBlocks) * kNA
+    const int entries = FUSED ? item_count(p, nb) * kNA
                               : min((nb + p.blocks_per_split - 1) / p.blocks_per_split, p.splits);
     const float* ml = FUSED ? p.fpart_ml : p.part_ml;
     const float* pacc = FUSED ? p.fpart_acc : p.part_acc;

@@ -33,6 +33,25 @@ constexpr uint32_t kSuspendHintNs = 200000u;       // upper bound of one hardwar
 constexpr long long kSpinCycles = 2000000000LL;   // bounded mbarrier wait (~1 s of SM clocks); then report and stop
 constexpr int kMaxG = 4;           // query heads per KV head handled by one warp
 constexpr unsigned kFull = 0xffffffffu;
+
+// Diagnostic build only (-DFFD_TIMELINE): FFD_TL(i, cond) stores the global timer the first time CTA blockIdx.x
+// reaches probe i; FFD_ACC(i) adds the SM clocks since the previous FFD_ACC to bucket i of a per-thread table that
+// FFD_ACC_OUT writes out.  The normal build compiles all of them to nothing.
+#ifdef FFD_TIMELINE
+__device__ unsigned long long g_tl[160 * 16];
+#define FFD_TL(i, cond) do { if (cond) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); \
+    if (g_tl[blockIdx.x * 16 + (i)] == 0) g_tl[blockIdx.x * 16 + (i)] = t_; } } while (0)
+__device__ long long g_acc[160 * 8];
+#define FFD_ACC_DECL long long acc_t_[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long acc_c_ = clock64()
+#define FFD_ACC(i) do { const long long n_ = clock64(); acc_t_[i] += n_ - acc_c_; acc_c_ = n_; } while (0)
+#define FFD_ACC_OUT(cond) do { if (cond) for (int i_ = 0; i_ < 8; ++i_) g_acc[blockIdx.x * 8 + i_] = acc_t_[i_]; } while (0)
+#else
+#define FFD_TL(i, cond)
+#define FFD_ACC_DECL
+#define FFD_ACC(i)
+#define FFD_ACC_OUT(cond)
+#endif
+
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -69,7 +88,8 @@ struct DecodeParams {
     uint32_t* class_counts;  // fused path: [0] heavy units, [1] light units found by the pseudo-max kernel (workspace)
     int32_t* unit_list;      // fused path: heavy units from the front, light units from the back (workspace)
     int units;               // batch * Hkv
-    int item_rows;           // fused path: work items per (sequence, KV head) = ceil(max_blocks / 24)
+    int item_rows;           // fused path: work items per (sequence, KV head)
+    int rows_small;          // fused path: how many of them, counted from block 0, are half-size items
     unsigned long long units_magic, hkv_magic;   // reciprocals for fast_div
     uint8_t* kept_mask;      // nullable [B, Hq, max_blocks]
     float* block_max;        // nullable [B, Hq, max_blocks]
@@ -415,19 +435,28 @@ struct AttendState {
     float acc[16][2];  // O fragments: n-tile nt, columns 2j, 2j+1
 };
 
-__device__ __forceinline__ void attend_setup(AttendState& st, const __nv_bfloat16* q_group, int G, int lane) {
+// A fragments of the group's queries (rows r < 4 and their duplicates r + 4; heads >= G are zero)
+__device__ __forceinline__ void attend_load_q(uint32_t (&qa)[16], const __nv_bfloat16* q_group, int G, int lane) {
     const int r = lane >> 2, j = lane & 3;
     const int head = r & 3;
 #pragma unroll
     for (int l4 = 0; l4 < 4; ++l4) {
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
         if (head < G) v = *reinterpret_cast<const uint4*>(q_group + head * kD + 32 * l4 + 8 * j);
-        st.qa[4 * l4 + 0] = v.x; st.qa[4 * l4 + 1] = v.y; st.qa[4 * l4 + 2] = v.z; st.qa[4 * l4 + 3] = v.w;
+        qa[4 * l4 + 0] = v.x; qa[4 * l4 + 1] = v.y; qa[4 * l4 + 2] = v.z; qa[4 * l4 + 3] = v.w;
     }
+}
+
+__device__ __forceinline__ void attend_reset(AttendState& st) {
     st.m = -INFINITY;
     st.l = 0.f;
 #pragma unroll
     for (int nt = 0; nt < 16; ++nt) st.acc[nt][0] = st.acc[nt][1] = 0.f;
+}
+
+__device__ __forceinline__ void attend_setup(AttendState& st, const __nv_bfloat16* q_group, int G, int lane) {
+    attend_load_q(st.qa, q_group, G, lane);
+    attend_reset(st);
 }
 
 // keep4: bit h set when head h attends to this block.  rows: valid tokens in the block (1..64).
