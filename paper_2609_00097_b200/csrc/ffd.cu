@@ -112,8 +112,11 @@ constexpr int kPmSamples = 7;  // blocks sampled between the sink and the local 
 __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p) {
     const int g = blockIdx.x, b = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    pdl_launch_dependents();
+    // Wait first, then let the fused kernel start: whatever the fused kernel does ahead of its own dependency wait
+    // (it draws its first work tickets there) then runs after everything that precedes this kernel has finished,
+    // the previous call's reset of the work counters included.
     pdl_wait();
+    pdl_launch_dependents();
     const int n = clamped_seq_len(p, b);
     const int nb = (n + kBlk - 1) / kBlk;
     const int ns = min(p.n_sink, nb);
@@ -690,7 +693,7 @@ ffd_status ffd_read_device_status(void* workspace, void* stream, uint32_t* statu
 }  // extern "C"
 
 // Diagnostic build only: copies the probe tables to the host ([160][16] first-hit timestamps in ns, then [160][8]
-// clock buckets) and clears the timestamps.  Not part of the library's interface.
+// clock buckets of an attend warp, then [160][8] of a scan warp) and clears the timestamps.  Not part of the library's interface.
 #ifdef FFD_TIMELINE
 extern "C" int ffd_debug_timeline(unsigned long long* host) {
     cudaDeviceSynchronize();
@@ -698,6 +701,7 @@ extern "C" int ffd_debug_timeline(unsigned long long* host) {
     static unsigned long long zeros[160 * 16];
     cudaMemcpyToSymbol(g_tl, zeros, sizeof(zeros));
     cudaMemcpyFromSymbol(host + 160 * 16, g_acc, sizeof(long long) * 160 * 8);
+    cudaMemcpyFromSymbol(host + 160 * 24, g_acc2, sizeof(long long) * 160 * 8);
     return 0;
 }
 #endif

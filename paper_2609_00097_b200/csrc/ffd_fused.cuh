@@ -28,6 +28,7 @@ constexpr int kNS = 12;                // warps of the scan role (three warpgrou
 #endif
 constexpr int kSched = FFD_SCHED_WARP; // 1: warp 0 only draws and publishes items, warps 1..11 scan
 constexpr int kScanners = kNS - kSched;
+static_assert(kSched == 1, "warp 0 schedules, warps 1 .. kNS - 1 scan");
 constexpr int kNA = 4;                 // attend warps (one warpgroup)
 constexpr int kFusedThreads = (kNS + kNA) * 32;
 constexpr int kScanRegs = 112;         // 12*32*112 + 4*32*176 = 65536 registers
@@ -93,6 +94,7 @@ struct Item {
 struct ItemSlot {                      // entry seq % 8 of the published-item ring; readiness: one mbarrier per entry
     volatile int slot, b, g, bg, blk0, nblk, n;
     int pad;
+    volatile int pages[24];            // physical page of each block of the item (-1: bad page-table entry)
 };
 
 struct BatchDesc {
@@ -104,20 +106,18 @@ struct BatchDesc {
 
 constexpr int kOffSlots = 0;
 constexpr int kOffRing = kOffSlots + kNA * 2 * kSlotBytes;
-constexpr int kOffQrec = kOffRing + kNS * kRing * kStageBytes;
+constexpr int kOffQrec = kOffRing + kScanners * kRing * kStageBytes;
 constexpr int kOffDesc = kOffQrec + kQrecRing * kQrecBytes;
 constexpr int kOffBars = kOffDesc + kNB * (int)sizeof(BatchDesc);
 constexpr int kNumBars = 2 * kNB + 2 * kNA + kQrecRing + kItemRing;   // full, empty, K/V slots, records, items
 constexpr int kOffItems = kOffBars + kNumBars * 8;               // ring of decoded items
 constexpr int kOffStageTile = kOffItems + kItemRing * (int)sizeof(ItemSlot);   // tile index of each ring stage
 constexpr int kOffAbort = kOffStageTile + kNS * 4 * 4;
-constexpr int kOffSched = kOffAbort + 16;                        // state of the item scheduler (one thread)
-constexpr int kOffAttendDone = kOffSched + 96;                   // batches finished by each attend warp
+constexpr int kOffAttendDone = kOffAbort + 16;                   // batches finished by each attend warp
 constexpr int kOffUnits = kOffAttendDone + 16;                   // first kUnitCache entries of each end of the unit list
 constexpr int kFusedSmem = kOffUnits + 2 * kUnitCache * 4;
 static_assert(kOffBars % 8 == 0 && kOffRing % 16 == 0 && kOffDesc % 16 == 0 && kOffQrec % 16 == 0, "alignment");
-static_assert(kOffSched % 8 == 0, "alignment");
-static_assert(sizeof(BatchDesc) % 16 == 0 && sizeof(ItemSlot) == 32, "descriptor sizes");
+static_assert(sizeof(BatchDesc) % 16 == 0 && sizeof(ItemSlot) == 128, "descriptor sizes");
 static_assert(kFusedSmem <= 227 * 1024, "shared memory budget");
 
 // Work is handed out from two global counters, one per class of (sequence, KV head) units.  "Heavy" units are the
@@ -126,46 +126,27 @@ static_assert(kFusedSmem <= 227 * 1024, "shared memory budget");
 // queued ahead of the attend warps and fills the scan warps' remaining time with light items, so the two kinds of
 // work overlap on every SM; what is left over at the end is light, i.e. a short, well-balanced tail.  Within a class,
 // rows count from the END of the sequences backwards (the local window first).
-struct ItemSched {
+struct ItemSched {                                        // lives in the registers of the scheduling warp's lane 0
     int n_heavy, n_light, total_heavy, total_light;      // units and items per class
     unsigned long long magic_heavy, magic_light;          // reciprocals of the unit counts
     int pend_heavy, pend_light;                           // draw of each class already fetched (>= total: none left)
-    int next_pub;                                         // next ring entry to publish
     int released;                                         // batches the attend warps have finished, in order
     int heavy_queued;                                     // heavy batches published and not yet released
-    int finished;                                         // the end marker has been published
     unsigned long long heavy_hist;                        // bit s % 64: batch s is heavy
 };
-static_assert(sizeof(ItemSched) <= 96, "scheduler state");
-
-__device__ __forceinline__ void sched_init(const DecodeParams& p, ItemSched* sc) {
-    sc->n_heavy = min((int)p.class_counts[0], p.units);
-    sc->n_light = p.units - sc->n_heavy;
-    sc->total_heavy = sc->n_heavy * p.item_rows;
-    sc->total_light = sc->n_light * p.item_rows;
-    sc->magic_heavy = fast_div_magic((unsigned)max(sc->n_heavy, 1));
-    sc->magic_light = fast_div_magic((unsigned)max(sc->n_light, 1));
-    sc->pend_heavy = (int)atomicAdd(p.item_counter, 1u);
-    sc->pend_light = (int)atomicAdd(p.light_counter, 1u);
-    sc->next_pub = 0;
-    sc->released = 0;
-    sc->heavy_queued = 0;
-    sc->finished = 0;
-    sc->heavy_hist = 0ull;
-}
 
 // draw number k of a class -> work item
-__device__ __forceinline__ Item decode_item(const DecodeParams& p, const ItemSched* sc, const int* unit_cache,
+__device__ __forceinline__ Item decode_item(const DecodeParams& p, const ItemSched& sc, const int* unit_cache,
                                             bool heavy, int k) {
     Item it;
     int row, bg;
     if (heavy) {   // heavy units sit at the front of the list, light units at its back (first ones cached in smem)
-        row = (int)fast_div((unsigned)k, sc->magic_heavy);
-        const int u = k - row * sc->n_heavy;
+        row = (int)fast_div((unsigned)k, sc.magic_heavy);
+        const int u = k - row * sc.n_heavy;
         bg = u < kUnitCache ? unit_cache[u] : p.unit_list[u];
     } else {
-        row = (int)fast_div((unsigned)k, sc->magic_light);
-        const int u = k - row * sc->n_light;
+        row = (int)fast_div((unsigned)k, sc.magic_light);
+        const int u = k - row * sc.n_light;
         bg = u < kUnitCache ? unit_cache[kUnitCache + u] : p.unit_list[p.units - 1 - u];
     }
     it.slot = row * p.units + bg;
@@ -217,16 +198,6 @@ __device__ __forceinline__ Item item_read(const ItemSlot* ring, int seq) {
     return it;
 }
 
-__device__ __forceinline__ void item_store(ItemSlot* ring, uint32_t ibars, int seq, const Item& it) {
-    ItemSlot& e = ring[seq & (kItemRing - 1)];
-    e.slot = it.slot; e.b = it.b; e.g = it.g; e.bg = it.bg; e.blk0 = it.blk0; e.nblk = it.nblk; e.n = it.n;
-    mbar_arrive(item_bar(ibars, seq));
-}
-
-// Lane 0 of scan warp 0: choose, draw and publish ring entry sc->next_pub.  Returns the item's unit (bg >= 0), -1 when
-// the end marker was published, -2 when nothing could be published yet (heavy work is due but enough of it is
-// already queued, and may_block is false).  may_block is only passed when the caller has itself finished scanning
-// every batch published so far, so that waiting for the attend warps cannot wait for the caller.
 // batches every attend warp has finished (they take the batches in order); a plain monotonic count, because a
 // parity test on the empty barriers could be fooled when a slot completes two phases between two looks
 __device__ __forceinline__ int attend_finished(const volatile int* attend_done) {
@@ -234,48 +205,107 @@ __device__ __forceinline__ int attend_finished(const volatile int* attend_done) 
 }
 static_assert(kNA == 4, "attend_finished reads four counters");
 
-__device__ __forceinline__ int item_publish(const DecodeParams& p, ItemSched* sc, const int* unit_cache, ItemSlot* ring,
-                                            uint32_t ibars, const volatile int* attend_done, bool may_block,
-                                            volatile int* abort_flag) {
-    const int seq = sc->next_pub;
-    Item it;
-    it.slot = -1; it.b = it.g = it.bg = it.blk0 = it.nblk = it.n = 0;
-    while (!sc->finished) {
-        // batches the attend warps have released since the last look
-        for (const int rel = min(attend_finished(attend_done), seq); sc->released < rel; ++sc->released)
-            if ((sc->heavy_hist >> (sc->released & 63)) & 1ull) --sc->heavy_queued;
-        const bool heavy_left = sc->pend_heavy < sc->total_heavy, light_left = sc->pend_light < sc->total_light;
-        if (!heavy_left && !light_left) { sc->finished = 1; break; }
-        // Heavy batches published and not yet released: at most four (two of them are the entries published ahead
-        // for prefetching).  Near the end of the heavy work, when the attend warps are the bottleneck, at most
-        // kHeavyAhead, so that no CTA sits on heavy work others could have taken.  Beyond the limit the scan warps
-        // spend their spare time on light items.
-        const int limit = sc->total_heavy - sc->pend_heavy > 2 * (int)gridDim.x ? 4 : kHeavyAhead;
-        bool heavy;
-        if (heavy_left && sc->heavy_queued < limit) heavy = true;
-        else if (light_left) heavy = false;
-        else {   // only heavy work is left and enough of it is queued: wait for the attend warps, or come back later
-            if (!may_block) return -2;
-            const long long t0 = clock64();
-            while (attend_finished(attend_done) <= sc->released) {
-                __nanosleep(256);
-                if (clock64() - t0 > kSpinCycles) { *abort_flag = 1; sc->finished = 1; break; }
+__device__ __forceinline__ void qrec_issue(const DecodeParams& p, int seq, int bg, uint32_t qrecs, uint32_t qbars,
+                                           int lane);
+
+// ---- scheduling role (warp 0) ------------------------------------------------------------------------------
+// Publishes ring entry after ring entry: chooses the class, takes the class's pending ticket (the next one is
+// fetched at once and not looked at until the next entry, so the atomic's latency is hidden), decodes it, looks the
+// item's pages up, writes the item and the header of its batch descriptor, announces it and starts the copy of its
+// query record.  Entry e reuses the record slot of entry e - 4 and the item slot of entry e - 8, so every scan warp
+// must have finished batch e - 4 (its full barrier) and the attend warps batch e - 8 (its empty barrier) first.
+// pend_heavy / pend_light: the first tickets, drawn by the caller.
+__device__ __forceinline__ void sched_role(const DecodeParams& p, unsigned char* smem, int lane, int pend_heavy,
+                                           int pend_light) {
+    const uint32_t qrecs = smem_u32(smem) + kOffQrec;
+    const uint32_t bars = smem_u32(smem) + kOffBars;
+    const uint32_t qbars = bars + (2 * kNB + 2 * kNA) * 8;
+    const uint32_t ibars = qbars + kQrecRing * 8;
+    BatchDesc* descs = reinterpret_cast<BatchDesc*>(smem + kOffDesc);
+    ItemSlot* items = reinterpret_cast<ItemSlot*>(smem + kOffItems);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffAbort);
+    const volatile int* attend_done = reinterpret_cast<const volatile int*>(smem + kOffAttendDone);
+    const int* unit_cache = reinterpret_cast<const int*>(smem + kOffUnits);
+    ItemSched sc;
+    sc.n_heavy = min((int)p.class_counts[0], p.units);
+    sc.n_light = p.units - sc.n_heavy;
+    sc.total_heavy = sc.n_heavy * p.item_rows;
+    sc.total_light = sc.n_light * p.item_rows;
+    sc.magic_heavy = fast_div_magic((unsigned)max(sc.n_heavy, 1));
+    sc.magic_light = fast_div_magic((unsigned)max(sc.n_light, 1));
+    sc.pend_heavy = pend_heavy;
+    sc.pend_light = pend_light;
+    sc.released = 0;
+    sc.heavy_queued = 0;
+    sc.heavy_hist = 0ull;
+    FFD_TL(3, lane == 0);
+#pragma unroll 1
+    for (int pub = 0;; ++pub) {
+        bool ok = true;
+        if (pub >= 4) ok = mbar_wait(bars + ((pub - 4) & (kNB - 1)) * 8, ((pub - 4) / kNB) & 1);
+        if (ok && pub >= kNB) ok = mbar_wait(bars + (kNB + (pub & (kNB - 1))) * 8, (pub / kNB - 1) & 1);
+        ItemSlot& e = items[pub & (kItemRing - 1)];
+        BatchDesc& d = descs[pub & (kNB - 1)];
+        if (!ok) *abort_flag = 1;
+        Item it;
+        it.slot = -1; it.b = it.g = it.bg = it.blk0 = it.nblk = it.n = 0;
+#pragma unroll 1
+        while (!*abort_flag) {
+            int kind = -1, cand = 0;      // -1: no work left, 0: light, 1: heavy
+            if (lane == 0) {
+                // batches the attend warps have released since the last look
+                for (const int rel = min(attend_finished(attend_done), pub); sc.released < rel; ++sc.released)
+                    if ((sc.heavy_hist >> (sc.released & 63)) & 1ull) --sc.heavy_queued;
+                const bool heavy_left = sc.pend_heavy < sc.total_heavy, light_left = sc.pend_light < sc.total_light;
+                // Heavy batches published and not yet released: at most four.  Near the end of the heavy work, when
+                // the attend warps are the bottleneck, at most kHeavyAhead, so that no CTA sits on heavy work others
+                // could have taken.  Beyond the limit the scan warps spend their spare time on light items.
+                const int limit = sc.total_heavy - sc.pend_heavy > 2 * (int)gridDim.x ? 4 : kHeavyAhead;
+                if (heavy_left && sc.heavy_queued < limit) kind = 1;
+                else if (light_left) kind = 0;
+                else if (heavy_left) {   // only heavy work is left and enough of it is queued: wait for the attend warps
+                    kind = 2;
+                    const long long t0 = clock64();
+                    while (attend_finished(attend_done) <= sc.released) {
+                        __nanosleep(256);
+                        if (clock64() - t0 > kSpinCycles) { *abort_flag = 1; break; }
+                    }
+                }
+                if (kind == 1) { cand = sc.pend_heavy; sc.pend_heavy = (int)atomicAdd(p.item_counter, 1u); }
+                if (kind == 0) { cand = sc.pend_light; sc.pend_light = (int)atomicAdd(p.light_counter, 1u); }
             }
-            continue;
+            kind = __shfl_sync(kFull, kind, 0);
+            cand = __shfl_sync(kFull, cand, 0);
+            if (kind == 2) continue;
+            if (kind < 0) break;
+            // every lane decodes the same item (the class sizes and reciprocals are the same in all lanes)
+            const Item c = decode_item(p, sc, unit_cache, kind == 1, cand);
+            if (c.nblk <= 0) continue;   // the sequence is shorter than the longest one: nothing in this item
+            it = c;
+            if (lane == 0) {
+                if (kind == 1) { sc.heavy_hist |= 1ull << (pub & 63); ++sc.heavy_queued; }
+                else sc.heavy_hist &= ~(1ull << (pub & 63));
+            }
+            break;
         }
-        int cand;
-        if (heavy) { cand = sc->pend_heavy; sc->pend_heavy = (int)atomicAdd(p.item_counter, 1u); }
-        else { cand = sc->pend_light; sc->pend_light = (int)atomicAdd(p.light_counter, 1u); }
-        const Item c = decode_item(p, sc, unit_cache, heavy, cand);
-        if (c.nblk <= 0) continue;   // the sequence is shorter than the longest one: nothing in this item
-        it = c;
-        if (heavy) { sc->heavy_hist |= 1ull << (seq & 63); ++sc->heavy_queued; }
-        else sc->heavy_hist &= ~(1ull << (seq & 63));
-        break;
+        if (it.slot >= 0) qrec_issue(p, pub, it.bg, qrecs, qbars, lane);   // lands while the pages are looked up
+        if (it.slot >= 0 && lane < it.nblk) {   // the item's page-table entries: one coalesced read
+            const int blk = it.blk0 + lane;
+            int page = p.block_table ? p.block_table[(size_t)it.b * p.max_blocks + blk] : it.b * p.max_blocks + blk;
+            if (page < 0 || page >= p.num_pages) { atomicOr(p.status, kDevBadPage); page = -1; }
+            e.pages[lane] = page;
+        }
+        if (lane == 0) {
+            e.slot = it.slot; e.b = it.b; e.g = it.g; e.bg = it.bg; e.blk0 = it.blk0; e.nblk = it.nblk; e.n = it.n;
+            d.item = it.slot; d.b = it.b; d.g = it.g; d.nblk = it.nblk;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(item_bar(ibars, pub));
+        FFD_TL(4, lane == 0 && it.slot >= 0);
+        if (it.slot < 0) break;
     }
-    item_store(ring, ibars, seq, it);
-    ++sc->next_pub;
-    return it.slot >= 0 ? it.bg : -1;
+    cp_async_drain();
+    if (*abort_flag && lane == 0) atomicOr(p.status, kDevTimeout);
 }
 
 // ---- scan role ---------------------------------------------------------------------------------------------
@@ -301,12 +331,7 @@ __device__ __forceinline__ bool cursor_next(const DecodeParams& p, ScanCursor& c
         ++c.seq;
         if (c.it.slot < 0) { c.end = true; c.it.nblk = 0; return false; }
         lb = w;
-        if (lb < c.it.nblk) {   // one coalesced read of the item's page-table entries; used a block-time later
-            const int blk = c.it.blk0 + lane;
-            c.pages = -1;
-            if (lane < c.it.nblk)
-                c.pages = p.block_table ? p.block_table[(size_t)c.it.b * p.max_blocks + blk] : c.it.b * p.max_blocks + blk;
-        }
+        if (lb < c.it.nblk) c.pages = lane < c.it.nblk ? items[c.seq & (kItemRing - 1)].pages[lane] : -1;
     }
     c.lb = lb;
     return true;
@@ -315,11 +340,7 @@ __device__ __forceinline__ bool cursor_next(const DecodeParams& p, ScanCursor& c
 // start the copy of one block's codes + scales into a ring stage (one commit group); remembers the block's tile
 __device__ __forceinline__ void ring_issue(const DecodeParams& p, const ScanCursor& c, uint32_t stage,
                                            volatile int* stage_tile, int lane) {
-    int page = __shfl_sync(kFull, c.pages, c.lb);
-    if (page < 0 || page >= p.num_pages) {   // bad table entry: reported, the block is skipped
-        if (lane == 0) atomicOr(p.status, kDevBadPage);
-        page = -1;
-    }
+    const int page = __shfl_sync(kFull, c.pages, c.lb);   // -1: bad table entry (reported by the scheduler), skipped
     const int tile = page >= 0 ? page * p.Hkv + c.it.g : -1;
     if (tile >= 0) {
         const uint4* codes = reinterpret_cast<const uint4*>(p.k_quant + (size_t)tile * kCodeBytes);
@@ -370,7 +391,8 @@ __device__ __noinline__ float scan_block_precise(const uint4* codes_tile, const 
 
 __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* smem, int w, int lane) {
     const int r = lane >> 2, j = lane & 3;
-    const uint32_t ring = smem_u32(smem) + kOffRing + w * kRing * kStageBytes;
+    const int w0 = w - kSched;      // index among the scanning warps
+    const uint32_t ring = smem_u32(smem) + kOffRing + w0 * kRing * kStageBytes;
     const uint32_t qrecs = smem_u32(smem) + kOffQrec;
     const uint32_t bars = smem_u32(smem) + kOffBars;
     const uint32_t qbars = bars + (2 * kNB + 2 * kNA) * 8;
@@ -379,59 +401,40 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
     ItemSlot* items = reinterpret_cast<ItemSlot*>(smem + kOffItems);
     volatile int* stage_tile = reinterpret_cast<volatile int*>(smem + kOffStageTile) + w * 4;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffAbort);
-    ItemSched* sched = reinterpret_cast<ItemSched*>(smem + kOffSched);
-    const volatile int* attend_done = reinterpret_cast<const volatile int*>(smem + kOffAttendDone);
-    const int* unit_cache = reinterpret_cast<const int*>(smem + kOffUnits);
-    if (w == 0 && lane == 0) sched_init(p, sched);
-    FFD_TL(3, w == 0 && lane == 0);
     ScanCursor ic;
     ic.seq = -1;
     ic.it.nblk = 0;
-    const int w0 = w - kSched;      // index among the scanning warps (-1: the scheduling warp, which scans nothing)
     ic.lb = w0 - kScanners;
     ic.end = false;
     ic.pages = -1;
     int issued = 0, consumed = 0;   // this warp's blocks whose copies were started / whose data was taken
+    FFD_ACC_DECL;
 
 #pragma unroll 1
     for (int seq = 0;; ++seq) {     // published item seq = batch seq
-        if (w == 0) {
-            // Publish ring entries up to seq + 2 and stage their query records.  Entry e reuses the slots of entries
-            // e - 4 (records) and e - 8 (items): every scan warp must be done with batch e - 4 first, which the
-            // completion of that batch's full barrier shows.
-#pragma unroll 1
-            for (;;) {
-                int bg = -3, pub = 0;
-                if (lane == 0) {
-                    pub = sched->next_pub;
-                    if (pub <= seq + 2) {
-                        const int guard = pub - 4;
-                        if (guard >= 0 && !mbar_wait(bars + (guard & (kNB - 1)) * 8, (guard / kNB) & 1)) *abort_flag = 1;
-                        bg = item_publish(p, sched, unit_cache, items, ibars, attend_done, pub <= seq, abort_flag);
-                    }
-                }
-                bg = __shfl_sync(kFull, bg, 0);
-                pub = __shfl_sync(kFull, pub, 0);
-                FFD_TL(4, lane == 0 && bg >= 0);
-                if (bg >= 0) qrec_issue(p, pub, bg, qrecs, qbars, lane);
-                if (bg < -1) break;      // -3: published far enough; -2: nothing to publish for now
-            }
-        }
+        FFD_ACC(0);
         if (!item_wait(ibars, seq)) *abort_flag = 1;
+        FFD_ACC(5);
         const Item it = item_read(items, seq);
         FFD_TL(5, w == 1 && lane == 0 && it.slot >= 0);
-        const int slot = seq & (kNB - 1), use = seq / kNB;
-        // the attend warps must have released this descriptor (kNB batches ago)
-        if (use > 0 && !mbar_wait(bars + (kNB + slot) * 8, (use - 1) & 1)) *abort_flag = 1;
+        // (the scheduling warp made sure, before it published the item, that the attend warps have released this
+        // descriptor and wrote its header)
+        const int slot = seq & (kNB - 1);
         BatchDesc& d = descs[slot];
+        FFD_ACC(6);
         if (it.slot < 0 || *abort_flag) {   // no more work: tell the attend warps
             if (lane == 0) {
-                if (w == 0) d.item = -1;
+                if (w0 == 0) d.item = -1;
                 mbar_arrive(bars + slot * 8);
             }
             break;
         }
-        // the item's query record must have landed
+        // start this warp's copies of the item's blocks, then wait for the item's query record
+        if (w0 < it.nblk)
+            while (issued < consumed + kRing && cursor_next(p, ic, items, ibars, w0, lane)) {
+                ring_issue(p, ic, ring + (issued % kRing) * kStageBytes, stage_tile + issued % kRing, lane);
+                ++issued;
+            }
         if (!mbar_wait(qbars + (seq & (kQrecRing - 1)) * 8, (seq / kQrecRing) & 1)) *abort_flag = 1;
         const uint32_t qrec = qrecs + (seq & (kQrecRing - 1)) * kQrecBytes;
         FFD_TL(6, w == 1 && lane == 0);
@@ -439,9 +442,10 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
         float thr, thr_col;   // threshold of head lane % 4 (block-max layout) and of head lane / 8 (B-column layout)
         asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(thr) : "r"(qrec + 2048 + j * 4));
         asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(thr_col) : "r"(qrec + 2048 + (lane >> 3) * 4));
-        if (w == 0 && lane == 0) { d.item = it.slot; d.b = it.b; d.g = it.g; d.nblk = it.nblk; }
+        FFD_ACC(7);
 #pragma unroll 1
-        for (int lb = w0 >= 0 ? w0 : it.nblk; lb < it.nblk; lb += kScanners) {
+        for (int lb = w0; lb < it.nblk; lb += kScanners) {
+            FFD_ACC(0);
             // keep the ring full: blocks consumed .. consumed + kRing - 1 of this warp's stream
             while (issued < consumed + kRing && cursor_next(p, ic, items, ibars, w0, lane)) {
                 ring_issue(p, ic, ring + (issued % kRing) * kStageBytes, stage_tile + issued % kRing, lane);
@@ -453,6 +457,7 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
             ring_wait(issued - consumed - 1);
             __syncwarp();
             FFD_TL(8, w == 1 && lane == 0);
+            FFD_ACC(1);
             // codes into registers; B operand straight from the staged scales and the item's query record
             uint4 wv[4];
 #pragma unroll
@@ -480,6 +485,7 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
             // block maxima themselves.)
             const bool cannot_keep =
                 __all_sync(kFull, scan_bound(sum_a, sum_b, p.sm_scale) < thr_col) && p.block_max == nullptr;
+            FFD_ACC(2);
             if (tile >= 0 && !cannot_keep) {
                 float band;
                 float bm = scan_mma<false>(wv, bfrag, lane, rows, p.sm_scale, band);
@@ -496,6 +502,7 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
                     if (p.block_max) p.block_max[o] = bm;
                 }
             }
+            FFD_ACC(3);
             if (cannot_keep && tile >= 0 && p.kept_mask && r == 0 && j < p.G)
                 p.kept_mask[(head0 + j) * p.max_blocks + blk] = 0;
             if (lane == 0) {
@@ -503,13 +510,15 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
                 d.keep4[lb] = (uint8_t)keep4;
                 d.rows[lb] = (uint8_t)rows;
             }
+            FFD_ACC(4);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(bars + slot * 8);   // this warp's share of the batch is published
         FFD_TL(9, w == 1 && lane == 0);
     }
     cp_async_drain();
-    if (*abort_flag && w == 0 && lane == 0) atomicOr(p.status, kDevTimeout);
+    FFD_ACC_OUT2(w == 1 && lane == 0);
+    if (*abort_flag && w0 == 0 && lane == 0) atomicOr(p.status, kDevTimeout);
 }
 
 // ---- attend role -------------------------------------------------------------------------------------------
@@ -642,7 +651,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodePa
     if (threadIdx.x == 0) {
         const uint32_t bars = smem_u32(smem) + kOffBars;
         for (int s = 0; s < kNB; ++s) {
-            mbar_init(bars + s * 8, kNS);             // full: one arrival per scan warp
+            mbar_init(bars + s * 8, kScanners);       // full: one arrival per scanning warp
             mbar_init(bars + (kNB + s) * 8, kNA);     // empty: one arrival per attend warp
         }
         for (int a = 0; a < 2 * kNA + kQrecRing; ++a) mbar_init(bars + (2 * kNB + a) * 8, 32);
@@ -651,6 +660,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodePa
         for (int a = 0; a < kNA; ++a) reinterpret_cast<volatile int*>(smem + kOffAttendDone)[a] = 0;
     }
     pdl_launch_dependents();
+    // First draw of each class.  The counters were reset by the previous call's combine kernel, and the pseudo-max
+    // kernel lets this kernel start only once everything before it has finished, so this need not wait.
+    int pend_heavy = 0, pend_light = 0;
+    if (threadIdx.x == 0) {
+        pend_heavy = (int)atomicAdd(p.item_counter, 1u);
+        pend_light = (int)atomicAdd(p.light_counter, 1u);
+    }
     pdl_wait();   // the pseudo-max kernel's outputs (unit list, class counts, query records) are needed from here on
     FFD_TL(1, threadIdx.x == 0);
     {   // shared-memory copy of both ends of the unit list (heavy units from the front, light units from the back)
@@ -667,7 +683,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodePa
     FFD_TL(2, threadIdx.x == 0);
     if (warp < kNS) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kScanRegs));
-        scan_role(p, smem, warp, lane);
+        if (warp < kSched) sched_role(p, smem, lane, pend_heavy, pend_light);
+        else scan_role(p, smem, warp, lane);
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kAttendRegs));
         attend_role(p, smem, warp - kNS, lane);

@@ -45,11 +45,16 @@ __device__ long long g_acc[160 * 8];
 #define FFD_ACC_DECL long long acc_t_[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long acc_c_ = clock64()
 #define FFD_ACC(i) do { const long long n_ = clock64(); acc_t_[i] += n_ - acc_c_; acc_c_ = n_; } while (0)
 #define FFD_ACC_OUT(cond) do { if (cond) for (int i_ = 0; i_ < 8; ++i_) g_acc[blockIdx.x * 8 + i_] = acc_t_[i_]; } while (0)
+__device__ long long g_acc2[160 * 8];
+#define FFD_ACC_OUT2(cond) do { if (cond) for (int i_ = 0; i_ < 8; ++i_) g_acc2[blockIdx.x * 8 + i_] = acc_t_[i_]; } while (0)
+#define FFD_CNT(i) (acc_t_[i] += 1)
 #else
 #define FFD_TL(i, cond)
 #define FFD_ACC_DECL
 #define FFD_ACC(i)
 #define FFD_ACC_OUT(cond)
+#define FFD_ACC_OUT2(cond)
+#define FFD_CNT(i)
 #endif
 
 constexpr float kLog2e = 1.4426950408889634f;
