@@ -135,6 +135,20 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
 #pragma unroll
         for (int x = 0; x < 4; ++x)
             dst[x * 32 + lane] = make_uint4(sq.qh[4 * x], sq.qh[4 * x + 1], sq.qh[4 * x + 2], sq.qh[4 * x + 3]);
+        // |q| in the same fragment layout, with the pre-scaling of the k-steps undone (exact: powers of four)
+        uint4* dst_abs = reinterpret_cast<uint4*>(rec + kQrecAbs);
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            uint32_t a[4];
+#pragma unroll
+            for (int y = 0; y < 4; ++y) {
+                const float undo = 1.0f / scan_pos_scale(2 * x + (y >> 1));
+                const __half2 v = __hmul2(__habs2(*reinterpret_cast<const __half2*>(&sq.qh[4 * x + y])),
+                                          __floats2half2_rn(undo, undo));
+                a[y] = *reinterpret_cast<const uint32_t*>(&v);
+            }
+            dst_abs[x * 32 + lane] = make_uint4(a[0], a[1], a[2], a[3]);
+        }
     }
     // Besides the sink and local blocks, a few blocks spread evenly over the middle of the sequence are scanned.
     // They never enter m_tilde: they only tell the scheduler below how dense this unit's selection will be.
@@ -168,7 +182,7 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
             p.mtilde[(size_t)b * p.Hq + g * p.G + threadIdx.x] = m;
             thr = m - p.delta;
         }
-        reinterpret_cast<float*>(rec + 2048)[threadIdx.x] = thr;
+        reinterpret_cast<float*>(rec + kQrecThr)[threadIdx.x] = thr;
         if (threadIdx.x < kMaxG) sthr[threadIdx.x] = thr;
     }
     __syncthreads();

@@ -84,7 +84,9 @@ constexpr int kHeavyAhead = FFD_HEAVY_AHEAD;         // heavy batches outstandin
 constexpr int kUnitCache = 512;        // entries of the unit list kept in shared memory
 constexpr int kItemRing = 8;           // decoded items published ahead
 constexpr int kQrecRing = 4;           // query records staged ahead
-constexpr int kQrecBytes = 2048 + 32;  // [4][32 lanes] uint4 of fp16 query fragments, then 4 thresholds (+ pad)
+constexpr int kQrecAbs = 2048;         // query record: [4][32 lanes] uint4 of pre-scaled fp16 query fragments, ...
+constexpr int kQrecThr = 4096;         // ... the same fragments of |q| (not pre-scaled), then 4 thresholds (+ pad)
+constexpr int kQrecBytes = kQrecThr + 32;
 
 struct Item {
     int slot;                          // canonical number row * units + bg (names the partial slots); < 0: no more work
@@ -408,6 +410,7 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
     ic.end = false;
     ic.pages = -1;
     int issued = 0, consumed = 0;   // this warp's blocks whose copies were started / whose data was taken
+    int bound_state = 0;            // >= 0: failures of the scale-only bound in a row; < 0: blocks until it is tried again
     FFD_ACC_DECL;
 
 #pragma unroll 1
@@ -440,8 +443,8 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
         FFD_TL(6, w == 1 && lane == 0);
         const size_t head0 = (size_t)it.b * p.Hq + (size_t)it.g * p.G;
         float thr, thr_col;   // threshold of head lane % 4 (block-max layout) and of head lane / 8 (B-column layout)
-        asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(thr) : "r"(qrec + 2048 + j * 4));
-        asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(thr_col) : "r"(qrec + 2048 + (lane >> 3) * 4));
+        asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(thr) : "r"(qrec + kQrecThr + j * 4));
+        asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(thr_col) : "r"(qrec + kQrecThr + (lane >> 3) * 4));
         FFD_ACC(7);
 #pragma unroll 1
         for (int lb = w0; lb < it.nblk; lb += kScanners) {
@@ -458,35 +461,45 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
             __syncwarp();
             FFD_TL(8, w == 1 && lane == 0);
             FFD_ACC(1);
-            // codes into registers; B operand straight from the staged scales and the item's query record
-            uint4 wv[4];
+            // No token of the block can score above 1.5 * sum |q s| (every level is at most 1.5 in magnitude).  If
+            // that bound stays below the threshold for every head of the group, no head can keep the block: its
+            // codes are not even read from shared memory, and the decision is the same as the full scan's.  (Not when
+            // the caller asked for the block maxima themselves, and not while the bound keeps failing.)
+            uint4 sv[4];
 #pragma unroll
-            for (int mt = 0; mt < 4; ++mt) wv[mt] = lds128(stage + (mt * 32 + lane) * 16);
-            uint32_t bfrag[16];
-            __half2 sum_a = __floats2half2_rn(0.f, 0.f), sum_b = sum_a;
-#pragma unroll
-            for (int x = 0; x < 4; ++x)
-                scan_bfrag4_bound(bfrag + 4 * x, lds128(qrec + (x * 32 + lane) * 16),
-                                  lds128(stage + kCodeBytes + (4 * x + j) * 16), r & 1, 4 * x, sum_a, sum_b);
+            for (int x = 0; x < 4; ++x) sv[x] = lds128(stage + kCodeBytes + (4 * x + j) * 16);
             const int tile = stage_tile[st];
-            __syncwarp();   // the stage is free again
-            ++consumed;
-            if (issued < consumed + kRing && cursor_next(p, ic, items, ibars, w0, lane)) {
-                ring_issue(p, ic, ring + (issued % kRing) * kStageBytes, stage_tile + issued % kRing, lane);
-                ++issued;
+            bool cannot_keep = false;
+            if (p.block_max == nullptr && bound_state >= 0) {
+                __half2 sum_a = __floats2half2_rn(0.f, 0.f), sum_b = sum_a;
+#pragma unroll
+                for (int x = 0; x < 4; ++x) scan_abs_sum(lds128(qrec + kQrecAbs + (x * 32 + lane) * 16), sv[x], sum_a, sum_b);
+                cannot_keep = __all_sync(kFull, scan_bound(sum_a, sum_b, p.sm_scale) < thr_col);
+                // a bound that fails 16 times in a row (a dense head) is left out for the next 48 blocks
+                bound_state = cannot_keep ? 0 : bound_state + 1;
+                if (bound_state == 16) bound_state = -48;
+            } else if (bound_state < 0) {
+                ++bound_state;
             }
-
             const int blk = it.blk0 + lb;
             const int rows = min(kBlk, it.n - blk * kBlk);
             unsigned keep4 = 0;
-            // No token of the block can score above 1.5 * sum |q s| (every level is at most 1.5 in magnitude).  If
-            // that bound stays below the threshold for every head of the group, no head can keep the block and the
-            // MMA work is skipped; the decision is the same as the full scan's.  (Not when the caller asked for the
-            // block maxima themselves.)
-            const bool cannot_keep =
-                __all_sync(kFull, scan_bound(sum_a, sum_b, p.sm_scale) < thr_col) && p.block_max == nullptr;
+            bool refilled = false;
             FFD_ACC(2);
-            if (tile >= 0 && !cannot_keep) {
+            if (tile >= 0 && !cannot_keep) {   // codes into registers; B operand from the staged scales and the record
+                uint4 wv[4];
+                uint32_t bfrag[16];
+#pragma unroll
+                for (int mt = 0; mt < 4; ++mt) wv[mt] = lds128(stage + (mt * 32 + lane) * 16);
+#pragma unroll
+                for (int x = 0; x < 4; ++x) scan_bfrag4(bfrag + 4 * x, lds128(qrec + (x * 32 + lane) * 16), sv[x], r & 1);
+                __syncwarp();   // the stage is free again: refill it before the tensor-core work, not after
+                ++consumed;
+                if (issued < consumed + kRing && cursor_next(p, ic, items, ibars, w0, lane)) {
+                    ring_issue(p, ic, ring + (issued % kRing) * kStageBytes, stage_tile + issued % kRing, lane);
+                    ++issued;
+                }
+                refilled = true;
                 float band;
                 float bm = scan_mma<false>(wv, bfrag, lane, rows, p.sm_scale, band);
                 // too close to call (rare): a separate, non-inlined routine re-reads the block and redoes it precisely
@@ -501,6 +514,12 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
                     if (p.kept_mask) p.kept_mask[o] = keep ? 1 : 0;
                     if (p.block_max) p.block_max[o] = bm;
                 }
+            }
+            __syncwarp();
+            if (!refilled) ++consumed;   // the stage is free again (what was read from it has been used)
+            if (!refilled && issued < consumed + kRing && cursor_next(p, ic, items, ibars, w0, lane)) {
+                ring_issue(p, ic, ring + (issued % kRing) * kStageBytes, stage_tile + issued % kRing, lane);
+                ++issued;
             }
             FFD_ACC(3);
             if (cannot_keep && tile >= 0 && p.kept_mask && r == 0 && j < p.G)

@@ -334,6 +334,20 @@ __device__ __forceinline__ void scan_bfrag4_bound(uint32_t* bfrag, const uint4& 
     }
 }
 
+// sum_c |q_c| s_c over four registers of the lane's channels (fp16, two running pairs; the products are exact
+// inside the fused multiply-add)
+__device__ __forceinline__ void scan_abs_sum(const uint4& qabs, const uint4& sv, __half2& sum_a, __half2& sum_b) {
+    const uint32_t q[4] = {qabs.x, qabs.y, qabs.z, qabs.w};
+    const uint32_t sc[4] = {sv.x, sv.y, sv.z, sv.w};
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        const __half2 a = *reinterpret_cast<const __half2*>(&q[x]);
+        const __half2 b = *reinterpret_cast<const __half2*>(&sc[x]);
+        if (x & 1) sum_b = __hfma2(a, b, sum_b);
+        else sum_a = __hfma2(a, b, sum_a);
+    }
+}
+
 // Upper bound (in logits) on the approximate score of every token of the block for the head this lane's column
 // belongs to: |sum_c q_c s_c level_c| <= 1.5 sum_c |q_c s_c|.  The factor 1.02 and the constant cover the fp16
 // roundings of the products and of the 16-term running sums (each below 2^-11 relative) and the lo pieces.
