@@ -57,7 +57,9 @@ __global__ void __launch_bounds__(128) quantize_kernel(QuantParams p) {
         __syncthreads();
         {
             float a = 0.f;
-            for (int r = 0; r < rows; ++r) a = fmaxf(a, fabsf(__bfloat162float(sk[r * kD + tid])));
+#pragma unroll 16
+            for (int r = 0; r < kBlk; ++r)   // (independent reads; rows past the sequence's end do not count)
+                if (r < rows) a = fmaxf(a, fabsf(__bfloat162float(sk[r * kD + tid])));
             float s32 = __fdiv_rn(a, 1.5f);
             s32 = fminf(s32, 65504.f);
             const __half s = __float2half_rn(s32);
@@ -427,6 +429,12 @@ static ffd_status check_geometry(int batch, int max_blocks, int num_pages) {
     return FFD_OK;
 }
 
+// Threads per combine CTA (two CTAs per head): as many as still let all of them be resident at once.
+static int combine_threads(long heads) {
+    const long ctas = 2 * heads;
+    return ctas <= 2 * 148 ? 1024 : ctas <= 4 * 148 ? 512 : 256;
+}
+
 static cudaEvent_t g_prof_start = nullptr, g_prof_stop = nullptr;
 
 // Launch with programmatic stream serialization: the grid may be scheduled while its predecessor in the stream is
@@ -529,14 +537,14 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
         if (prof) cudaEventRecord(g_prof_start, s);
         launch_pdl(fused_sparse_kernel, dim3(min(p.total_items, sms)), dim3(kFusedThreads), kFusedSmem, s, p);
         if (prof) cudaEventRecord(g_prof_stop, s);
-        launch_pdl(combine_kernel<true>, dim3(p.Hq, batch), dim3(kCombineThreads), 0, s, p);
+        launch_pdl(combine_kernel<true>, dim3(p.Hq, batch, 2), dim3(combine_threads(p.Hq * batch)), 0, s, p);
     } else {
         if (cudaFuncSetAttribute(decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem) != cudaSuccess)
             return FFD_ERR_CUDA;
         if (prof) cudaEventRecord(g_prof_start, s);
         launch_pdl(decode_kernel<false>, grid, dim3(kWarps * 32), kDecodeSmem, s, p);
         if (prof) cudaEventRecord(g_prof_stop, s);
-        launch_pdl(combine_kernel<false>, dim3(p.Hq, batch), dim3(kCombineThreads), 0, s, p);
+        launch_pdl(combine_kernel<false>, dim3(p.Hq, batch, 2), dim3(combine_threads(p.Hq * batch)), 0, s, p);
     }
     return launch_status();
 }
@@ -597,8 +605,12 @@ ffd_status ffd_quantize_keys(const ffd_config* cfg, const void* k_cache, void* k
     QuantParams p{static_cast<const __nv_bfloat16*>(k_cache), static_cast<uint8_t*>(k_quant),
                   static_cast<__half*>(k_scales), block_table, seq_lens, first_token,
                   cfg->num_kv_heads, max_blocks_per_seq, num_pages};
-    launch_pdl(quantize_kernel, dim3(max_blocks_per_seq < 64 ? max_blocks_per_seq : 64, cfg->num_kv_heads, batch),
-               dim3(128), 0, static_cast<cudaStream_t>(stream), p);
+    // CTAs per (sequence, KV head): every CTA walks its share of the blocks, so any number is correct.  With
+    // first_token (decode steps re-quantize the block the new token fell into) two are plenty and a wide grid
+    // would only launch thousands of CTAs that find nothing to do.
+    const int wide = max_blocks_per_seq < 64 ? max_blocks_per_seq : 64;
+    launch_pdl(quantize_kernel, dim3(first_token ? (wide < 2 ? wide : 2) : wide, cfg->num_kv_heads, batch), dim3(128), 0,
+               static_cast<cudaStream_t>(stream), p);
     return launch_status();
 }
 

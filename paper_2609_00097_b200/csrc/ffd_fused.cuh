@@ -713,11 +713,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodePa
 // ---- split combine (FlashDecoding-style log-sum-exp merge) -------------------------------------------------
 // One CTA of 1024 threads per (query head, sequence).  FUSED: partial e = (work item, attend warp) of the fused
 // kernel; otherwise partial e = split of the dense kernel.  The (m, l) pairs are read once into shared memory;
-// thread (el, cg) = (tid / 32, tid % 32) sums the partials e = el, el + 32, ... for channels 4cg .. 4cg+3 with
-// eight independent loads in flight; the 32 partial sums meet in shared memory.  Summation order is fixed, so
+// two CTAs share a head (blockIdx.z = channel half); thread (el, cg) = (tid / 16, tid % 16) sums the partials
+// e = el, el + 64, ... for channels 64z + 4cg .. + 3 with eight independent loads in flight; the partial sums meet
+// in shared memory.  Summation order is fixed, so
 // results are reproducible.
 constexpr int kCombineThreads = 1024;
-constexpr int kCombineLanes = kCombineThreads / 32;   // partials summed side by side
+constexpr int kCombineWarps = kCombineThreads / 32;   // (at most; the launch may use 256 or 512 threads)
 constexpr int kCombineChunk = 1024;
 
 template <bool FUSED>
@@ -731,12 +732,13 @@ __device__ __forceinline__ size_t combine_slot(const DecodeParams& p, size_t hea
 
 template <bool FUSED>
 __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p) {
-    const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
-    const int el = tid >> 5, cg = tid & 31;
+    const int h = blockIdx.x, b = blockIdx.y, half = blockIdx.z, tid = threadIdx.x;
+    const int el = tid >> 4, cg = tid & 15, warp = tid >> 5, lane = tid & 31;
+    const int threads = blockDim.x, warps = threads >> 5, lanes = threads >> 4;   // lanes: partials summed side by side
     pdl_launch_dependents();
     pdl_wait();
-    FFD_TL(15, FUSED && tid == 0 && blockIdx.y == 0);
-    if (FUSED && h == 0 && b == 0 && tid == 0) {   // the next call's draws and class lists start from zero
+    FFD_TL(15, FUSED && tid == 0 && blockIdx.y == 0 && half == 0);
+    if (FUSED && h == 0 && b == 0 && half == 0 && tid == 0) {   // the next call's draws and class lists start from zero
         *p.item_counter = 0u;
         p.class_counts[0] = 0u;
         p.class_counts[1] = 0u;
@@ -752,8 +754,8 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
     const float* pacc = FUSED ? p.fpart_acc : p.part_acc;
     __shared__ float s_m[kCombineChunk];   // m of the partial, then its weight
     __shared__ float s_l[kCombineChunk];
-    __shared__ float s_red[kCombineLanes];
-    __shared__ float4 s_part[kCombineLanes][32];
+    __shared__ float s_red[kCombineWarps];
+    __shared__ float4 s_part[kCombineWarps][16];
 
     float Mrun = -INFINITY, L = 0.f;       // running max / sum across chunks (one chunk unless > 1024 partials)
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -761,7 +763,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
         const int cnt = min(kCombineChunk, entries - base);
         __syncthreads();
         float M = -INFINITY;
-        for (int x = tid; x < cnt; x += kCombineThreads) {
+        for (int x = tid; x < cnt; x += threads) {
             const float2 v = *reinterpret_cast<const float2*>(ml + combine_slot<FUSED>(p, head, bg, hl, base + x) * 2);
             s_m[x] = v.y > 0.f ? v.x : -INFINITY;
             s_l[x] = v.y;
@@ -769,33 +771,34 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
         }
 #pragma unroll
         for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(kFull, M, o));
-        if (cg == 0) s_red[el] = M;
+        if (lane == 0) s_red[warp] = M;
         __syncthreads();
         M = Mrun;
 #pragma unroll
-        for (int x = 0; x < kCombineLanes; ++x) M = fmaxf(M, s_red[x]);
+        for (int x = 0; x < kCombineWarps; ++x)
+            if (x < warps) M = fmaxf(M, s_red[x]);
         if (M == -INFINITY) continue;      // uniform: nothing in this chunk or before it
         const float rescale = exp2f(Mrun - M);   // 0 for the first non-empty chunk
         acc.x *= rescale; acc.y *= rescale; acc.z *= rescale; acc.w *= rescale;
         L *= rescale;
         Mrun = M;
-        for (int x = tid; x < cnt; x += kCombineThreads) {
+        for (int x = tid; x < cnt; x += threads) {
             const float wv = exp2f(s_m[x] - M);  // exp2(-inf) = 0 for empty partials
             L += wv * s_l[x];
             s_m[x] = wv;
         }
         __syncthreads();
-        for (int x0 = el; x0 < cnt; x0 += kCombineLanes * 8) {
+        for (int x0 = el; x0 < cnt; x0 += lanes * 8) {
             float4 v[8];
             float wv[8];
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-                const int x = x0 + kCombineLanes * u;
+                const int x = x0 + lanes * u;
                 wv[u] = x < cnt ? s_m[x] : 0.f;
                 v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (wv[u] != 0.f)
                     v[u] = *reinterpret_cast<const float4*>(pacc + combine_slot<FUSED>(p, head, bg, hl, base + x) * kD +
-                                                            4 * cg);
+                                                            64 * half + 4 * cg);
             }
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
@@ -805,15 +808,18 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
     }
 #pragma unroll
     for (int o = 16; o; o >>= 1) L += __shfl_xor_sync(kFull, L, o);
+    // the two partial lanes of a warp (lanes cg and cg + 16) first
+    acc.x += __shfl_xor_sync(kFull, acc.x, 16); acc.y += __shfl_xor_sync(kFull, acc.y, 16);
+    acc.z += __shfl_xor_sync(kFull, acc.z, 16); acc.w += __shfl_xor_sync(kFull, acc.w, 16);
     __syncthreads();
-    if (cg == 0) s_red[el] = L;
-    s_part[el][cg] = acc;
+    if (lane == 0) s_red[warp] = L;
+    if (lane < 16) s_part[warp][lane] = acc;
     __syncthreads();
-    if (tid < 32) {
+    if (tid < 16) {
         L = 0.f;
         float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int x = 0; x < kCombineLanes; ++x) {
+        for (int x = 0; x < warps; ++x) {
             L += s_red[x];
             const float4 v = s_part[x][tid];
             t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
@@ -821,15 +827,15 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
         const float inv = L > 0.f ? 1.f / L : 0.f;
         const float4 o = make_float4(t.x * inv, t.y * inv, t.z * inv, t.w * inv);
         if (p.out_fp32) {
-            reinterpret_cast<float4*>(p.out)[head * (kD / 4) + tid] = o;
+            reinterpret_cast<float4*>(p.out)[head * (kD / 4) + 16 * half + tid] = o;
         } else {
             __nv_bfloat162 lo = __floats2bfloat162_rn(o.x, o.y), hi = __floats2bfloat162_rn(o.z, o.w);
             uint2 pk;
             pk.x = *reinterpret_cast<uint32_t*>(&lo);
             pk.y = *reinterpret_cast<uint32_t*>(&hi);
-            reinterpret_cast<uint2*>(p.out)[head * (kD / 4) + tid] = pk;
+            reinterpret_cast<uint2*>(p.out)[head * (kD / 4) + 16 * half + tid] = pk;
         }
-        if (p.lse && tid == 0) p.lse[head] = L > 0.f ? (Mrun + log2f(L)) * kLn2 : -INFINITY;
+        if (p.lse && tid == 0 && half == 0) p.lse[head] = L > 0.f ? (Mrun + log2f(L)) * kLn2 : -INFINITY;
     }
 }
 
