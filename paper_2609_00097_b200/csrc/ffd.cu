@@ -429,11 +429,11 @@ static ffd_status check_geometry(int batch, int max_blocks, int num_pages) {
     return FFD_OK;
 }
 
-// Threads per combine CTA (two CTAs per head): as many as still let all of them be resident at once.
-static int combine_threads(long heads) {
-    const long ctas = 2 * heads;
-    return ctas <= 2 * 148 ? 1024 : ctas <= 4 * 148 ? 512 : 256;
-}
+// Threads per combine CTA (one CTA per head): as many as still let all CTAs be resident at once.
+static int combine_threads(long heads) { return heads <= 2 * 148 ? 1024 : heads <= 4 * 148 ? 512 : 256; }
+// CTAs per head (each takes a share of the channels): more when there are few heads, so that a long sequence's
+// partials are not summed by a handful of SMs.
+static int combine_split(long heads) { return heads >= 128 ? 1 : heads >= 64 ? 2 : 4; }
 
 static cudaEvent_t g_prof_start = nullptr, g_prof_stop = nullptr;
 
@@ -537,14 +537,14 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
         if (prof) cudaEventRecord(g_prof_start, s);
         launch_pdl(fused_sparse_kernel, dim3(min(p.total_items, sms)), dim3(kFusedThreads), kFusedSmem, s, p);
         if (prof) cudaEventRecord(g_prof_stop, s);
-        launch_pdl(combine_kernel<true>, dim3(p.Hq, batch, 2), dim3(combine_threads(p.Hq * batch)), 0, s, p);
+        launch_pdl(combine_kernel<true>, dim3(p.Hq, batch, combine_split(p.Hq * batch)), dim3(combine_threads(p.Hq * batch)), 0, s, p);
     } else {
         if (cudaFuncSetAttribute(decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem) != cudaSuccess)
             return FFD_ERR_CUDA;
         if (prof) cudaEventRecord(g_prof_start, s);
         launch_pdl(decode_kernel<false>, grid, dim3(kWarps * 32), kDecodeSmem, s, p);
         if (prof) cudaEventRecord(g_prof_stop, s);
-        launch_pdl(combine_kernel<false>, dim3(p.Hq, batch, 2), dim3(combine_threads(p.Hq * batch)), 0, s, p);
+        launch_pdl(combine_kernel<false>, dim3(p.Hq, batch, combine_split(p.Hq * batch)), dim3(combine_threads(p.Hq * batch)), 0, s, p);
     }
     return launch_status();
 }

@@ -713,12 +713,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodePa
 // ---- split combine (FlashDecoding-style log-sum-exp merge) -------------------------------------------------
 // One CTA of 1024 threads per (query head, sequence).  FUSED: partial e = (work item, attend warp) of the fused
 // kernel; otherwise partial e = split of the dense kernel.  The (m, l) pairs are read once into shared memory;
-// two CTAs share a head (blockIdx.z = channel half); thread (el, cg) = (tid / 16, tid % 16) sums the partials
-// e = el, el + 64, ... for channels 64z + 4cg .. + 3 with eight independent loads in flight; the partial sums meet
-// in shared memory.  Summation order is fixed, so
+// thread (el, cg) = (tid / 32, tid % 32) sums the partials e = el, el + 32, ... for channels 4cg .. 4cg+3 with
+// eight independent loads in flight; the 32 partial sums meet in shared memory.  Summation order is fixed, so
 // results are reproducible.
 constexpr int kCombineThreads = 1024;
-constexpr int kCombineWarps = kCombineThreads / 32;   // (at most; the launch may use 256 or 512 threads)
+constexpr int kCombineLanes = kCombineThreads / 32;   // partials summed side by side (at most: the launch may use fewer threads)
 constexpr int kCombineChunk = 1024;
 
 template <bool FUSED>
@@ -732,13 +731,16 @@ __device__ __forceinline__ size_t combine_slot(const DecodeParams& p, size_t hea
 
 template <bool FUSED>
 __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p) {
-    const int h = blockIdx.x, b = blockIdx.y, half = blockIdx.z, tid = threadIdx.x;
-    const int el = tid >> 4, cg = tid & 15, warp = tid >> 5, lane = tid & 31;
-    const int threads = blockDim.x, warps = threads >> 5, lanes = threads >> 4;   // lanes: partials summed side by side
+    // gridDim.z = 1, 2 or 4 CTAs share a head, each taking 128 / gridDim.z channels (few heads: more CTAs)
+    const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int cgn = 32 / (int)gridDim.z;          // groups of four channels per CTA
+    const int el = tid / cgn, cg = tid % cgn;
+    const int threads = blockDim.x, warps = threads >> 5, lanes = threads / cgn;
+    const int chan0 = (int)blockIdx.z * 4 * cgn;
     pdl_launch_dependents();
     pdl_wait();
-    FFD_TL(15, FUSED && tid == 0 && blockIdx.y == 0 && half == 0);
-    if (FUSED && h == 0 && b == 0 && half == 0 && tid == 0) {   // the next call's draws and class lists start from zero
+    FFD_TL(15, FUSED && tid == 0 && blockIdx.y == 0 && blockIdx.z == 0);
+    if (FUSED && h == 0 && b == 0 && blockIdx.z == 0 && tid == 0) {   // the next call's draws and class lists start from zero
         *p.item_counter = 0u;
         p.class_counts[0] = 0u;
         p.class_counts[1] = 0u;
@@ -754,8 +756,8 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
     const float* pacc = FUSED ? p.fpart_acc : p.part_acc;
     __shared__ float s_m[kCombineChunk];   // m of the partial, then its weight
     __shared__ float s_l[kCombineChunk];
-    __shared__ float s_red[kCombineWarps];
-    __shared__ float4 s_part[kCombineWarps][16];
+    __shared__ float s_red[kCombineLanes];
+    __shared__ float4 s_part[kCombineLanes][32];
 
     float Mrun = -INFINITY, L = 0.f;       // running max / sum across chunks (one chunk unless > 1024 partials)
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -775,7 +777,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
         __syncthreads();
         M = Mrun;
 #pragma unroll
-        for (int x = 0; x < kCombineWarps; ++x)
+        for (int x = 0; x < kCombineLanes; ++x)
             if (x < warps) M = fmaxf(M, s_red[x]);
         if (M == -INFINITY) continue;      // uniform: nothing in this chunk or before it
         const float rescale = exp2f(Mrun - M);   // 0 for the first non-empty chunk
@@ -798,7 +800,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
                 v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (wv[u] != 0.f)
                     v[u] = *reinterpret_cast<const float4*>(pacc + combine_slot<FUSED>(p, head, bg, hl, base + x) * kD +
-                                                            64 * half + 4 * cg);
+                                                            chan0 + 4 * cg);
             }
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
@@ -808,17 +810,17 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
     }
 #pragma unroll
     for (int o = 16; o; o >>= 1) L += __shfl_xor_sync(kFull, L, o);
-    // the two partial lanes of a warp (lanes cg and cg + 16) first
-    acc.x += __shfl_xor_sync(kFull, acc.x, 16); acc.y += __shfl_xor_sync(kFull, acc.y, 16);
-    acc.z += __shfl_xor_sync(kFull, acc.z, 16); acc.w += __shfl_xor_sync(kFull, acc.w, 16);
+    for (int o = cgn; o < 32; o <<= 1) {   // the partial lanes that share a warp
+        acc.x += __shfl_xor_sync(kFull, acc.x, o); acc.y += __shfl_xor_sync(kFull, acc.y, o);
+        acc.z += __shfl_xor_sync(kFull, acc.z, o); acc.w += __shfl_xor_sync(kFull, acc.w, o);
+    }
     __syncthreads();
     if (lane == 0) s_red[warp] = L;
-    if (lane < 16) s_part[warp][lane] = acc;
+    if (lane < cgn) s_part[warp][lane] = acc;
     __syncthreads();
-    if (tid < 16) {
+    if (tid < cgn) {
         L = 0.f;
         float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
         for (int x = 0; x < warps; ++x) {
             L += s_red[x];
             const float4 v = s_part[x][tid];
@@ -827,15 +829,15 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
         const float inv = L > 0.f ? 1.f / L : 0.f;
         const float4 o = make_float4(t.x * inv, t.y * inv, t.z * inv, t.w * inv);
         if (p.out_fp32) {
-            reinterpret_cast<float4*>(p.out)[head * (kD / 4) + 16 * half + tid] = o;
+            reinterpret_cast<float4*>(p.out)[head * (kD / 4) + chan0 / 4 + tid] = o;
         } else {
             __nv_bfloat162 lo = __floats2bfloat162_rn(o.x, o.y), hi = __floats2bfloat162_rn(o.z, o.w);
             uint2 pk;
             pk.x = *reinterpret_cast<uint32_t*>(&lo);
             pk.y = *reinterpret_cast<uint32_t*>(&hi);
-            reinterpret_cast<uint2*>(p.out)[head * (kD / 4) + 16 * half + tid] = pk;
+            reinterpret_cast<uint2*>(p.out)[head * (kD / 4) + chan0 / 4 + tid] = pk;
         }
-        if (p.lse && tid == 0 && half == 0) p.lse[head] = L > 0.f ? (Mrun + log2f(L)) * kLn2 : -INFINITY;
+        if (p.lse && tid == 0 && blockIdx.z == 0) p.lse[head] = L > 0.f ? (Mrun + log2f(L)) * kLn2 : -INFINITY;
     }
 }
 
