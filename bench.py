@@ -39,7 +39,7 @@ KV_BYTES_PER_TILE = 2 * 64 * 128 * 2      # K tile + V tile of one kept (block, 
 # dram__bytes_read + dram__bytes_write of one fused-kernel launch divided by the launch's algorithmic bytes, from
 # the ncu capture summarised in profiles/fused_sparse_kernel_C3_ctx32768.md (same kernel, same workload recipe at
 # context 32768; traffic grows in proportion to the blocks processed): (308.47 + 5.65) MB / 308.28 MB.
-NCU_TRAFFIC_RATIO = 1.019
+NCU_TRAFFIC_RATIO = 1.024
 
 
 def measured_peaks():
@@ -281,12 +281,13 @@ def main():
         dc.quantize(first_token=first_token)
         dc.decode(delta)
 
-    def timed_loop(fn, n, profile_kernel):
+    def timed_loop(fn, n, profile_kernel, cold=True):
         """n steps, each bracketed by CUDA events on the launching stream, L2 flushed (untimed) before each."""
         total, kernel = [], []
         for _ in range(n):
-            flush.fill_(1)          # evicts every input line from L2 ...
-            drain.sum()             # ... and this read sweep pushes the fill's dirty lines out to HBM, so that their
+            if cold:
+                flush.fill_(1)      # evicts every input line from L2 ...
+                drain.sum()         # ... and this read sweep pushes the fill's dirty lines out to HBM, so that their
                                     # write-back (an artefact of the flush, not of the workload) ends before the timing starts
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record(stream)
@@ -319,6 +320,28 @@ def main():
     # the same step without the event pair around the fused kernel (the records sit between the step's kernels and
     # cost their programmatic-launch overlap): what a caller who does not profile sees
     plain_us, _ = timed_loop(step, min(args.steps, 200), False)
+    # the same without the flush (whatever of the previous step is still in L2 stays there) ...
+    warm_us, _ = timed_loop(step, min(args.steps, 200), False, cold=False)
+    # ... submitted as one CUDA graph (cold L2) ...
+    graph_us = None
+    try:
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            step()
+            torch.cuda.synchronize()
+            with torch.cuda.graph(graph, stream=side):
+                step()
+        torch.cuda.synchronize()
+        graph_us, _ = timed_loop(graph.replay, min(args.steps, 200), False)
+    except Exception as exc:   # reported, not fatal: the graph number is an extra
+        graph_us = None
+        print(f"bench: CUDA graph capture failed: {exc}", file=sys.stderr)
+    # ... and a pure-read calibration: a sum over 1 GiB (torch's reduction kernel), cold
+    calib = torch.zeros(128 << 20, dtype=torch.int64, device="cuda")
+    calib_us, _ = timed_loop(calib.sum, 13, False)
+    read_gbs = calib.numel() * 8 / (statistics.median(calib_us[3:]) * 1e-6) / 1e9
+    del calib
 
     # end to end through the public API with HOST buffers: q comes from pinned host memory every step and the
     # output goes back to the host; the KV cache itself is resident (it is a cache), as in a serving loop
@@ -364,6 +387,9 @@ def main():
                      "frac_of_nominal_8TBs": achieved / 8000.0},
         "step_us_median": statistics.median(step_us), "step_us_min": min(step_us),
         "step_us_without_kernel_events": statistics.mean(plain_us),
+        "step_us_warm_l2": statistics.mean(warm_us),
+        "step_us_cuda_graph": None if graph_us is None else statistics.mean(graph_us),
+        "read_calibration_gbs": read_gbs,
         "effective_hbm_gbs_step": sparse_bytes / (t_step * 1e-6) / 1e9,
         "sparsity": {"skipped_fraction_per_head": 1.0 - kept_head_blocks / head_blocks,
                      "skipped_fraction_per_loaded_block": 1.0 - kept_tiles / total_tiles,
@@ -374,6 +400,9 @@ def main():
     }
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(w, delta)
+        one = cpu_baseline(w, delta, threads=1, seconds_target=5.0)
+        line["cpu_baseline"]["value_1_thread"] = one["value"]
+        line["cpu_baseline"]["sample_1_thread"] = one["sample"]
     else:
         line["cpu_baseline"] = None
     print(json.dumps(line), flush=True)

@@ -122,6 +122,8 @@ SMALL = [
     ("C2", dict(N=6000, sink=False), None),                 # no-sink variant: everything kept
     ("C3", dict(N=8192, B=8), None),                        # enough units for long splits: several blocks per warp
     ("C5", dict(B=16, lens=(2000, 4200)), None),
+    ("C5", dict(B=3, lens=(700, 3000)), None),              # 96 heads: two combine CTAs per head
+    ("C5", dict(B=20, lens=(300, 1500)), None),             # 640 heads: the smallest combine CTAs
 ]
 
 
@@ -217,6 +219,44 @@ def test_bad_page_index_sets_status_and_does_not_fault(ffd, oracle):
     assert ffd.ffd_read_device_status(dc.workspace) == ffd.DEV_BAD_PAGE
     assert ffd.ffd_read_device_status(dc.workspace) == 0       # reading clears it
     assert torch.isfinite(dc.out).all()
+
+
+def test_step_replays_from_a_cuda_graph(ffd, oracle):
+    """A whole step (tail re-quantize + decode) captured once and replayed gives the eager step's result; every
+    step-varying argument (q, seq_lens, first_token, block_table) lives on the device (Sec. 3.3)."""
+    w = make_workload("C5", B=4, lens=(1000, 5000))
+    dc = ffd.DeviceCache(w)
+    dc.quantize()
+    first = torch.from_numpy(np.maximum(w.seq_lens - 1, 0).astype(np.int32)).cuda()
+
+    def step():
+        dc.quantize(first_token=first)
+        dc.decode(6.0)
+
+    step()
+    torch.cuda.synchronize()
+    eager = dc.out.clone()
+    graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        step()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            step()
+    torch.cuda.synchronize()
+    for _ in range(3):
+        dc.out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert ffd.ffd_read_device_status(dc.workspace) == 0
+        assert (dc.out - eager).abs().max().item() <= 1e-6
+    # a new query through the same graph: only device memory changes
+    dc.q.copy_(torch.roll(dc.q, 1, dims=1))
+    graph.replay()
+    torch.cuda.synchronize()
+    replayed = dc.out.clone()
+    step()
+    torch.cuda.synchronize()
+    assert (dc.out - replayed).abs().max().item() <= 1e-6
 
 
 # full-size configurations: the oracle checks a sample of (sequence, head) rows one by one
