@@ -96,6 +96,23 @@ ffd_status ffd_quantize_keys(const ffd_config* cfg, const void* k_cache, void* k
                              int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages, void* stream);
 
 /*
+ * Cache append for one decode step, all indices on the device (Sec. 3.3: a cache that a captured graph can replay
+ * needs tensor indices instead of host-side lengths; App. A.1 for the quantizer).  For every sequence b with
+ * pos = seq_lens[b] < max_blocks_per_seq*64: the rows k_new[b, g, :] and v_new[b, g, :] (bf16 [B, Hkv, 128], device)
+ * are written to token position pos of k_cache / v_cache (block pos/64 through block_table, row pos%64), that
+ * block's thumbnails (k_quant, k_scales) are re-quantized over its rows 0 .. pos%64 exactly as ffd_quantize_keys
+ * would, and seq_lens[b] becomes pos + 1.  A sequence with no room left, or whose block_table entry for the block is
+ * outside [0, num_pages), is left untouched and reported in the status word (FFD_DEV_BAD_SEQ_LEN / FFD_DEV_BAD_PAGE).
+ * workspace: device memory of at least 256 bytes whose first word is the status word (a decode workspace will do).
+ * Asynchronous on `stream`; two kernel launches; allocates nothing; may be captured in a CUDA graph together with
+ * the decode call that follows it.  Host errors as for ffd_quantize_keys (FFD_ERR_WORKSPACE if workspace_bytes < 256).
+ */
+ffd_status ffd_append_kv(const ffd_config* cfg, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                         void* k_quant, void* k_scales, const int32_t* block_table, int32_t* seq_lens, int32_t batch,
+                         int32_t max_blocks_per_seq, int32_t num_pages, void* workspace, size_t workspace_bytes,
+                         void* stream);
+
+/*
  * One sparse decode step (Alg. 1; Sec. 3.2 Eq. 1 and the pseudo-max equation; Sec. 3.3 kernel steps).
  * Per query head h of sequence b, with sm = sm_scale and khat = (code - 1.5) * scale:
  *   approx[t]  = sm * sum_c q[c] * khat[t,c]                      every valid token t

@@ -31,6 +31,40 @@ __device__ __forceinline__ uint32_t quant_code(float x, float s) {
     return neg ? (big ? 0u : 1u) : (big ? 3u : 2u);
 }
 
+// One (page, KV head) tile, staged in shared memory as sk[64][128], by 128 threads: per-channel scale over the first
+// `rows` rows (App. A.1), then the packed 2-bit codes.  Contains a __syncthreads().
+__device__ __forceinline__ void quantize_tile(const __nv_bfloat16* sk, float* ss, int rows, __half* scales_out,
+                                              uint8_t* codes_out, int tid) {
+    {
+        float a = 0.f;
+#pragma unroll 16
+        for (int r = 0; r < kBlk; ++r)   // (independent reads; rows past the sequence's end do not count)
+            if (r < rows) a = fmaxf(a, fabsf(__bfloat162float(sk[r * kD + tid])));
+        float s32 = __fdiv_rn(a, 1.5f);
+        s32 = fminf(s32, 65504.f);
+        const __half s = __float2half_rn(s32);
+        scales_out[tid] = s;
+        ss[tid] = __half2float(s);
+    }
+    __syncthreads();
+    const int mt = tid >> 5, lane = tid & 31, r = lane >> 2, j = lane & 3;
+    uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int c = 32 * j + 4 * i + u;
+            const float s = ss[c];
+            const uint32_t lo_row = quant_code(__bfloat162float(sk[(16 * mt + r) * kD + c]), s);
+            const uint32_t hi_row = quant_code(__bfloat162float(sk[(16 * mt + r + 8) * kD + c]), s);
+            const int shift = 2 * i + 16 * (u & 1);
+            w[(u >> 1) * 2 + 0] |= lo_row << shift;   // W0 / W2: token r
+            w[(u >> 1) * 2 + 1] |= hi_row << shift;   // W1 / W3: token r + 8
+        }
+    }
+    reinterpret_cast<uint4*>(codes_out)[mt * 32 + lane] = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
 __global__ void __launch_bounds__(128) quantize_kernel(QuantParams p) {
     const int g = blockIdx.y, b = blockIdx.z;
     pdl_launch_dependents();
@@ -55,35 +89,65 @@ __global__ void __launch_bounds__(128) quantize_kernel(QuantParams p) {
 #pragma unroll
         for (int x = 0; x < 8; ++x) dst[tid + 128 * x] = ldg_stream(src + tid + 128 * x);
         __syncthreads();
-        {
-            float a = 0.f;
-#pragma unroll 16
-            for (int r = 0; r < kBlk; ++r)   // (independent reads; rows past the sequence's end do not count)
-                if (r < rows) a = fmaxf(a, fabsf(__bfloat162float(sk[r * kD + tid])));
-            float s32 = __fdiv_rn(a, 1.5f);
-            s32 = fminf(s32, 65504.f);
-            const __half s = __float2half_rn(s32);
-            p.k_scales[tile * kD + tid] = s;
-            ss[tid] = __half2float(s);
-        }
-        __syncthreads();
-        const int mt = tid >> 5, lane = tid & 31, r = lane >> 2, j = lane & 3;
-        uint32_t w[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int c = 32 * j + 4 * i + u;
-                const float s = ss[c];
-                const uint32_t lo_row = quant_code(__bfloat162float(sk[(16 * mt + r) * kD + c]), s);
-                const uint32_t hi_row = quant_code(__bfloat162float(sk[(16 * mt + r + 8) * kD + c]), s);
-                const int shift = 2 * i + 16 * (u & 1);
-                w[(u >> 1) * 2 + 0] |= lo_row << shift;   // W0 / W2: token r
-                w[(u >> 1) * 2 + 1] |= hi_row << shift;   // W1 / W3: token r + 8
-            }
-        }
-        uint4* out = reinterpret_cast<uint4*>(p.k_quant + tile * kCodeBytes);
-        out[mt * 32 + lane] = make_uint4(w[0], w[1], w[2], w[3]);
+        quantize_tile(sk, ss, rows, p.k_scales + tile * kD, p.k_quant + tile * kCodeBytes, tid);
+    }
+}
+
+// ---- cache append (Sec. 3.3: every step-varying index lives on the device) ---------------------------------
+struct AppendParams {
+    const __nv_bfloat16* k_new;   // [B, Hkv, 128]
+    const __nv_bfloat16* v_new;
+    __nv_bfloat16* k_cache;
+    __nv_bfloat16* v_cache;
+    uint8_t* k_quant;
+    __half* k_scales;
+    const int32_t* block_table;
+    int32_t* seq_lens;
+    uint32_t* status;
+    int Hkv, max_blocks, num_pages;
+};
+
+// One CTA of 128 threads (one per channel) per (KV head, sequence): the new token's K and V rows go to position
+// seq_lens[b] of the cache, and the block they fall into is re-quantized over its rows up to and including the new one.
+__global__ void __launch_bounds__(128) append_kernel(AppendParams p) {
+    const int g = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+    pdl_launch_dependents();
+    pdl_wait();
+    const int pos = p.seq_lens[b];
+    if (pos < 0 || pos >= p.max_blocks * kBlk) {   // no room (or a corrupt length): reported, nothing written
+        if (tid == 0) atomicOr(p.status, kDevBadSeqLen);
+        return;
+    }
+    const int blk = pos / kBlk, row = pos % kBlk;
+    const int page = p.block_table ? p.block_table[(size_t)b * p.max_blocks + blk] : b * p.max_blocks + blk;
+    if (page < 0 || page >= p.num_pages) {
+        if (tid == 0) atomicOr(p.status, kDevBadPage);
+        return;
+    }
+    __shared__ __align__(16) __nv_bfloat16 sk[kBlk * kD];
+    __shared__ float ss[kD];
+    const size_t tile = (size_t)page * p.Hkv + g;
+    const size_t unit = (size_t)b * p.Hkv + g;
+    const __nv_bfloat16 kn = p.k_new[unit * kD + tid];
+    p.v_cache[(tile * kBlk + row) * kD + tid] = p.v_new[unit * kD + tid];
+    p.k_cache[(tile * kBlk + row) * kD + tid] = kn;
+    // the rows before the new one (16-byte vectors: 16 per row)
+    const uint4* src = reinterpret_cast<const uint4*>(p.k_cache + tile * kBlk * kD);
+    uint4* dst = reinterpret_cast<uint4*>(sk);
+    for (int x = tid; x < row * (kD / 8); x += 128) dst[x] = src[x];
+    sk[row * kD + tid] = kn;
+    __syncthreads();
+    quantize_tile(sk, ss, row + 1, p.k_scales + tile * kD, p.k_quant + tile * kCodeBytes, tid);
+}
+
+// after every CTA of append_kernel has read the lengths: one more token per sequence that had room
+__global__ void __launch_bounds__(256) bump_lengths_kernel(int32_t* seq_lens, int batch, int cap) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < batch) {
+        const int n = seq_lens[b];
+        if (n >= 0 && n < cap) seq_lens[b] = n + 1;
     }
 }
 
@@ -611,6 +675,31 @@ ffd_status ffd_quantize_keys(const ffd_config* cfg, const void* k_cache, void* k
     const int wide = max_blocks_per_seq < 64 ? max_blocks_per_seq : 64;
     launch_pdl(quantize_kernel, dim3(first_token ? (wide < 2 ? wide : 2) : wide, cfg->num_kv_heads, batch), dim3(128), 0,
                static_cast<cudaStream_t>(stream), p);
+    return launch_status();
+}
+
+ffd_status ffd_append_kv(const ffd_config* cfg, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                         void* k_quant, void* k_scales, const int32_t* block_table, int32_t* seq_lens, int32_t batch,
+                         int32_t max_blocks_per_seq, int32_t num_pages, void* workspace, size_t workspace_bytes,
+                         void* stream) {
+    ffd_status st = check_config(cfg);
+    if (st) return st;
+    if (!k_new || !v_new || !k_cache || !v_cache || !k_quant || !k_scales || !seq_lens || !workspace) return FFD_ERR_NULL;
+    st = check_geometry(batch, max_blocks_per_seq, num_pages);
+    if (st) return st;
+    if (cfg->num_kv_heads > 65535) return FFD_ERR_SHAPE;
+    if (workspace_bytes < 256) return FFD_ERR_WORKSPACE;
+    const void* ptrs[] = {k_new, v_new, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, workspace};
+    for (const void* ptr : ptrs)
+        if (ptr && misaligned(ptr)) return FFD_ERR_ALIGN;
+    AppendParams p{static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
+                   static_cast<__nv_bfloat16*>(k_cache), static_cast<__nv_bfloat16*>(v_cache),
+                   static_cast<uint8_t*>(k_quant), static_cast<__half*>(k_scales), block_table, seq_lens,
+                   static_cast<uint32_t*>(workspace), cfg->num_kv_heads, max_blocks_per_seq, num_pages};
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    launch_pdl(append_kernel, dim3(cfg->num_kv_heads, batch), dim3(128), 0, s, p);
+    launch_pdl(bump_lengths_kernel, dim3((batch + 255) / 256), dim3(256), 0, s, seq_lens, (int)batch,
+               (int)(max_blocks_per_seq * kBlk));
     return launch_status();
 }
 

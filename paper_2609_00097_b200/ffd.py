@@ -24,7 +24,8 @@ DEV_BAD_PAGE = 1
 DEV_BAD_SEQ_LEN = 2
 
 EXPORTS = ["ffd_status_string", "ffd_workspace_bytes", "ffd_workspace_init", "ffd_quantize_keys", "ffd_decode",
-           "ffd_decode_dense", "ffd_unpack_codes", "ffd_read_device_status", "ffd_profile_events", "ffd_decode_static"]
+           "ffd_decode_dense", "ffd_unpack_codes", "ffd_read_device_status", "ffd_profile_events", "ffd_decode_static",
+           "ffd_append_kv"]
 
 
 class FfdError(RuntimeError):
@@ -84,6 +85,8 @@ def load_library() -> ctypes.CDLL:
         lib.ffd_profile_events.argtypes = [_vp, _vp]
         lib.ffd_decode_static.argtypes = [cfgp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, ctypes.c_float, _vp,
                                           _vp, _vp]
+        lib.ffd_append_kv.argtypes = [cfgp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, _vp, ctypes.c_size_t,
+                                      _vp]
         for name in EXPORTS:
             if name != "ffd_status_string":
                 getattr(lib, name).restype = ctypes.c_int
@@ -129,6 +132,16 @@ def ffd_quantize_keys(cfg: Config, k_cache, k_quant, k_scales, block_table, seq_
     _check(load_library().ffd_quantize_keys(ctypes.byref(cfg.c()), _p(k_cache), _p(k_quant), _p(k_scales),
                                             _p(block_table), _p(seq_lens), _p(first_token), seq_lens.numel(),
                                             max_blocks_per_seq, num_pages, _stream(stream)), "ffd_quantize_keys")
+
+
+def ffd_append_kv(cfg: Config, k_new, v_new, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, *,
+                  max_blocks_per_seq: int, workspace, stream=None):
+    num_pages = k_cache.shape[0]
+    _check(load_library().ffd_append_kv(ctypes.byref(cfg.c()), _p(k_new), _p(v_new), _p(k_cache), _p(v_cache),
+                                        _p(k_quant), _p(k_scales), _p(block_table), _p(seq_lens), seq_lens.numel(),
+                                        max_blocks_per_seq, num_pages, _p(workspace),
+                                        ctypes.c_size_t(workspace.numel() * workspace.element_size()),
+                                        _stream(stream)), "ffd_append_kv")
 
 
 def ffd_decode(cfg: Config, q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, delta: float, out, *,
@@ -205,6 +218,10 @@ class DeviceCache:
     def quantize(self, first_token=None):
         ffd_quantize_keys(self.cfg, self.k_cache, self.k_quant, self.k_scales, self.block_table, self.seq_lens,
                           first_token, max_blocks_per_seq=self.w.max_blocks)
+
+    def append(self, k_new, v_new):
+        ffd_append_kv(self.cfg, k_new, v_new, self.k_cache, self.v_cache, self.k_quant, self.k_scales,
+                      self.block_table, self.seq_lens, max_blocks_per_seq=self.w.max_blocks, workspace=self.workspace)
 
     def decode(self, delta, kept_mask=None, block_max=None):
         ffd_decode(self.cfg, self.q, self.k_cache, self.v_cache, self.k_quant, self.k_scales, self.block_table,

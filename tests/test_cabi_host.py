@@ -79,6 +79,13 @@ def test_null_and_range_arguments_are_rejected_before_any_launch(lib):
                                 1 << 30, None) == 2
     assert lib.ffd_quantize_keys(ctypes.byref(cfg), None, fake, fake, None, fake, None, 1, 16, 16, None) == 1
     assert lib.ffd_unpack_codes(ctypes.byref(cfg), fake, fake, 0, None) == 2
+    # append: NULL new rows, workspace below 256 bytes, misaligned lengths
+    assert lib.ffd_append_kv(ctypes.byref(cfg), None, fake, fake, fake, fake, fake, None, fake, 1, 16, 16, fake, 256,
+                             None) == 1
+    assert lib.ffd_append_kv(ctypes.byref(cfg), fake, fake, fake, fake, fake, fake, None, fake, 1, 16, 16, fake, 128,
+                             None) == 5
+    assert lib.ffd_append_kv(ctypes.byref(cfg), fake, fake, fake, fake, fake, fake, None, odd, 1, 16, 16, fake, 256,
+                             None) == 4
     assert lib.ffd_read_device_status(None, None, None) == 1
 
 

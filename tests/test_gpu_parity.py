@@ -259,6 +259,102 @@ def test_step_replays_from_a_cuda_graph(ffd, oracle):
     assert (dc.out - replayed).abs().max().item() <= 1e-6
 
 
+def test_append_writes_the_token_requantizes_its_block_and_bumps_the_length(ffd, oracle):
+    """Tokens appended one at a time through ffd_append_kv (Sec. 3.3) must leave exactly the cache, thumbnails and
+    lengths of the workload that already holds them: rows bit for bit, codes and scales as the oracle quantizer gives
+    them.  Lengths are chosen so that some sequences cross a block boundary and one starts a block at row 0."""
+    w = make_workload("C5", B=4, lens=(1000, 5000))
+    steps = 5
+    full = w.seq_lens.copy()
+    full[0] = 64 * ((full[0] - 3) // 64) + 2            # sequence 0 crosses into a new block during the appends
+    full[1] = 64 * ((full[1] - steps - 1) // 64) + steps    # sequence 1 starts its last block at row 0
+    dc = ffd.DeviceCache(w)
+    k_all, v_all = dc.k_cache.clone(), dc.v_cache.clone()
+    start = (full - steps).astype(np.int32)
+    dc.seq_lens.copy_(torch.from_numpy(start))
+    # wipe what the appends must restore
+    for b in range(w.B):
+        for t in range(int(start[b]), int(full[b])):
+            page = int(w.block_table[b, t // 64])
+            dc.k_cache[page, :, t % 64, :] = 7.0
+            dc.v_cache[page, :, t % 64, :] = -7.0
+    ffd.ffd_quantize_keys(dc.cfg, dc.k_cache, dc.k_quant, dc.k_scales, dc.block_table, dc.seq_lens,
+                          max_blocks_per_seq=w.max_blocks)
+    for s in range(steps):
+        k_new = torch.empty(w.B, w.Hkv, 128, dtype=torch.bfloat16, device="cuda")
+        v_new = torch.empty_like(k_new)
+        for b in range(w.B):
+            t = int(start[b]) + s
+            page = int(w.block_table[b, t // 64])
+            k_new[b] = k_all[page, :, t % 64, :]
+            v_new[b] = v_all[page, :, t % 64, :]
+        dc.append(k_new, v_new)
+    torch.cuda.synchronize()
+    assert ffd.ffd_read_device_status(dc.workspace) == 0
+    assert np.array_equal(dc.seq_lens.cpu().numpy(), full)
+    w.seq_lens[:] = full
+    vm, mapped = valid_row_mask(w)
+    sel = torch.from_numpy(np.broadcast_to(vm, tuple(k_all.shape)).copy()).cuda()
+    assert torch.equal(dc.k_cache.view(torch.int16)[sel], k_all.view(torch.int16)[sel])
+    assert torch.equal(dc.v_cache.view(torch.int16)[sel], v_all.view(torch.int16)[sel])
+    codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
+    g_codes = dc.canonical_codes().cpu().numpy()
+    g_scales = dc.k_scales.cpu().view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(g_scales[mapped], scales[mapped])
+    csel = np.broadcast_to(vm, codes.shape)
+    assert np.array_equal(g_codes[csel], codes[csel])
+    check_decode(ffd, oracle, w, dc, codes, scales, 6.0)
+    # a full sequence is reported and left alone
+    dc.seq_lens[2] = w.max_blocks * 64
+    dc.append(k_new, v_new)
+    torch.cuda.synchronize()
+    assert ffd.ffd_read_device_status(dc.workspace) == ffd.DEV_BAD_SEQ_LEN
+    assert int(dc.seq_lens[2]) == w.max_blocks * 64
+    for b in (0, 1, 3):
+        assert int(dc.seq_lens[b]) == int(full[b]) + 1
+
+
+def test_serving_loop_append_and_decode_from_one_graph(ffd, oracle):
+    """append + decode captured once; every replay advances the lengths on the device and must give what the same
+    calls give when issued eagerly on a second copy of the cache."""
+    w = make_workload("C5", B=4, lens=(1000, 5000))
+    w.seq_lens[:] = w.seq_lens - 8                      # room for the appended tokens inside the mapped blocks
+    a, b = ffd.DeviceCache(w), ffd.DeviceCache(w)
+    a.quantize(), b.quantize()
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    k_new = torch.randn(w.B, w.Hkv, 128, device="cuda", generator=gen).to(torch.bfloat16)
+    v_new = torch.randn(w.B, w.Hkv, 128, device="cuda", generator=gen).to(torch.bfloat16)
+
+    def step(dc):
+        dc.append(k_new, v_new)
+        dc.decode(6.0)
+
+    graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        step(a)                                         # warm-up outside the capture (token 1)
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            step(a)                                     # capturing does not run it
+    step(b)
+    for i in range(3):
+        k_new.copy_(torch.randn(w.B, w.Hkv, 128, device="cuda", generator=gen).to(torch.bfloat16))
+        v_new.copy_(torch.randn(w.B, w.Hkv, 128, device="cuda", generator=gen).to(torch.bfloat16))
+        graph.replay()
+        step(b)
+        torch.cuda.synchronize()
+        assert ffd.ffd_read_device_status(a.workspace) == 0 and ffd.ffd_read_device_status(b.workspace) == 0
+        assert torch.equal(a.seq_lens, b.seq_lens)
+        assert int(a.seq_lens[0]) == int(w.seq_lens[0]) + 2 + i
+        assert torch.equal(a.k_scales.view(torch.int16), b.k_scales.view(torch.int16))
+        assert (a.out - b.out).abs().max().item() <= 1e-6
+    # codes of the valid rows (those past a sequence's end are unspecified)
+    w.seq_lens[:] = a.seq_lens.cpu().numpy()
+    vm, _ = valid_row_mask(w)
+    ca, cb = a.canonical_codes().cpu().numpy(), b.canonical_codes().cpu().numpy()
+    sel = np.broadcast_to(vm, ca.shape)
+    assert np.array_equal(ca[sel], cb[sel])
+
+
 # full-size configurations: the oracle checks a sample of (sequence, head) rows one by one
 FULL = [
     ("C2", dict(), 8),
