@@ -264,6 +264,10 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
     const int kept = __syncthreads_count(kept_any);
     if (threadIdx.x == 0) {
         const int bg = b * p.Hkv + g;
+        // the longest and the shortest sequence of the batch, for the fused kernel's draw plan
+        atomicMax(&p.len_stats[0], (unsigned)nb);
+        atomicMax(&p.len_stats[1], (unsigned)(p.max_blocks - nb));
+        atomicAdd(&p.len_stats[2], (unsigned)item_count(p, nb));   // work items that exist
         if (hinted > 0 && 2 * kept >= hinted) p.unit_list[atomicAdd(&p.class_counts[0], 1u)] = bg;
         else p.unit_list[p.units - 1 - (int)atomicAdd(&p.class_counts[1], 1u)] = bg;
         FFD_TL(14, blockIdx.y == 0);
@@ -574,6 +578,7 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
     p.item_counter = reinterpret_cast<uint32_t*>(ws + 64);
     p.class_counts = reinterpret_cast<uint32_t*>(ws + 68);
     p.light_counter = reinterpret_cast<uint32_t*>(ws + 76);
+    p.len_stats = reinterpret_cast<uint32_t*>(ws + 80);
     p.unit_list = reinterpret_cast<int32_t*>(ws + pl.off_units);
     p.units = batch * cfg->num_kv_heads;
     p.item_rows = item_geometry(p.units, max_blocks).item_rows;

@@ -131,6 +131,7 @@ static_assert(kFusedSmem <= 227 * 1024, "shared memory budget");
 struct ItemSched {                                        // lives in the registers of the scheduling warp's lane 0
     int n_heavy, n_light, total_heavy, total_light;      // units and items per class
     unsigned long long magic_heavy, magic_light;          // reciprocals of the unit counts
+    int row_off;                                          // leading rows that no sequence of the batch reaches
     int pend_heavy, pend_light;                           // draw of each class already fetched (>= total: none left)
     int released;                                         // batches the attend warps have finished, in order
     int heavy_queued;                                     // heavy batches published and not yet released
@@ -151,6 +152,7 @@ __device__ __forceinline__ Item decode_item(const DecodeParams& p, const ItemSch
         const int u = k - row * sc.n_light;
         bg = u < kUnitCache ? unit_cache[kUnitCache + u] : p.unit_list[p.units - 1 - u];
     }
+    row += sc.row_off;
     it.slot = row * p.units + bg;
     it.bg = bg;
     it.b = (int)fast_div((unsigned)bg, p.hkv_magic);
@@ -231,8 +233,12 @@ __device__ __forceinline__ void sched_role(const DecodeParams& p, unsigned char*
     ItemSched sc;
     sc.n_heavy = min((int)p.class_counts[0], p.units);
     sc.n_light = p.units - sc.n_heavy;
-    sc.total_heavy = sc.n_heavy * p.item_rows;
-    sc.total_light = sc.n_light * p.item_rows;
+    // Rows in use: up to the longest sequence of the batch (a cache sized for longer contexts than it holds would
+    // otherwise spend most tickets on rows no sequence reaches).
+    const int rows = item_count(p, min((int)p.len_stats[0], p.max_blocks));
+    sc.row_off = p.item_rows - rows;
+    sc.total_heavy = sc.n_heavy * rows;
+    sc.total_light = sc.n_light * rows;
     sc.magic_heavy = fast_div_magic((unsigned)max(sc.n_heavy, 1));
     sc.magic_light = fast_div_magic((unsigned)max(sc.n_light, 1));
     sc.pend_heavy = pend_heavy;
@@ -745,6 +751,9 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
         p.class_counts[0] = 0u;
         p.class_counts[1] = 0u;
         *p.light_counter = 0u;
+        p.len_stats[0] = 0u;
+        p.len_stats[1] = 0u;
+        p.len_stats[2] = 0u;
     }
     const size_t head = (size_t)b * p.Hq + h;
     const int g = h / p.G, hl = h % p.G, bg = b * p.Hkv + g;

@@ -91,6 +91,7 @@ struct DecodeParams {
     uint32_t* item_counter;  // fused path: next heavy-class draw (workspace; zeroed at the start of every call)
     uint32_t* light_counter; // fused path: next light-class draw
     uint32_t* class_counts;  // fused path: [0] heavy units, [1] light units found by the pseudo-max kernel (workspace)
+    uint32_t* len_stats;     // fused path: [0] largest block count of the batch, [1] largest (max_blocks - block count), [2] items
     int32_t* unit_list;      // fused path: heavy units from the front, light units from the back (workspace)
     int units;               // batch * Hkv
     int item_rows;           // fused path: work items per (sequence, KV head)

@@ -221,6 +221,18 @@ def test_bad_page_index_sets_status_and_does_not_fault(ffd, oracle):
     assert torch.isfinite(dc.out).all()
 
 
+def test_cache_with_room_for_much_longer_sequences(ffd, oracle):
+    """max_blocks_per_seq is a capacity: sequences far shorter than it (the usual state of a serving cache) must
+    give the same results, and the work items of the rows nobody reaches must not be handed out."""
+    w = make_workload("C5", B=4, lens=(3000, 5000))
+    w.seq_lens[:] = np.array([700, 64, 1, 333], dtype=np.int32)       # capacity stays ~79 blocks
+    dc = ffd.DeviceCache(w)
+    codes, scales = check_quantize(ffd, oracle, w, dc)
+    check_decode(ffd, oracle, w, dc, codes, scales, 6.0)
+    check_decode(ffd, oracle, w, dc, codes, scales, INF)
+    check_dense(ffd, oracle, w, dc)
+
+
 def test_step_replays_from_a_cuda_graph(ffd, oracle):
     """A whole step (tail re-quantize + decode) captured once and replayed gives the eager step's result; every
     step-varying argument (q, seq_lens, first_token, block_table) lives on the device (Sec. 3.3)."""
