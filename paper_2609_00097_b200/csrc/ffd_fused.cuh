@@ -81,7 +81,8 @@ constexpr int kNB = FFD_NB;                 // batch descriptors: how far the sc
 #define FFD_HEAVY_AHEAD 2
 #endif
 constexpr int kHeavyAhead = FFD_HEAVY_AHEAD;         // heavy batches outstanding at most once the attend warps are the bottleneck
-constexpr int kUnitCache = 512;        // entries of the unit list kept in shared memory
+constexpr int kUnitCache = 256;        // entries of each end of the unit list kept in shared memory
+constexpr int kRowCap = 256;           // item rows up to which the table of existing items is built (ragged batches)
 constexpr int kItemRing = 8;           // decoded items published ahead
 constexpr int kQrecRing = 4;           // query records staged ahead
 constexpr int kQrecAbs = 2048;         // query record: [4][32 lanes] uint4 of pre-scaled fp16 query fragments, ...
@@ -117,7 +118,9 @@ constexpr int kOffStageTile = kOffItems + kItemRing * (int)sizeof(ItemSlot);   /
 constexpr int kOffAbort = kOffStageTile + kNS * 4 * 4;
 constexpr int kOffAttendDone = kOffAbort + 16;                   // batches finished by each attend warp
 constexpr int kOffUnits = kOffAttendDone + 16;                   // first kUnitCache entries of each end of the unit list
-constexpr int kFusedSmem = kOffUnits + 2 * kUnitCache * 4;
+constexpr int kOffStart = kOffUnits + 2 * kUnitCache * 4;        // first row (16 bit) in which each cached unit has an item
+constexpr int kOffRowPref = kOffStart + 2 * kUnitCache * 2;      // per class: draws before each row, then the total
+constexpr int kFusedSmem = kOffRowPref + 2 * (kRowCap + 1) * 4;
 static_assert(kOffBars % 8 == 0 && kOffRing % 16 == 0 && kOffDesc % 16 == 0 && kOffQrec % 16 == 0, "alignment");
 static_assert(sizeof(BatchDesc) % 16 == 0 && sizeof(ItemSlot) == 128, "descriptor sizes");
 static_assert(kFusedSmem <= 227 * 1024, "shared memory budget");
@@ -132,18 +135,111 @@ struct ItemSched {                                        // lives in the regist
     int n_heavy, n_light, total_heavy, total_light;      // units and items per class
     unsigned long long magic_heavy, magic_light;          // reciprocals of the unit counts
     int row_off;                                          // leading rows that no sequence of the batch reaches
+    int table;                                            // 1: draws go through the row tables (see plan_tables)
     int pend_heavy, pend_light;                           // draw of each class already fetched (>= total: none left)
     int released;                                         // batches the attend warps have finished, in order
     int heavy_queued;                                     // heavy batches published and not yet released
     unsigned long long heavy_hist;                        // bit s % 64: batch s is heavy
 };
 
+// Row tables for batches whose sequences differ much in length.  A sequence shorter than the longest one has no
+// item in the first rows; when more than half of the (row, unit) grid is empty (and the batch fits: kUnitCache
+// units per class, kRowCap rows) the scheduling warp builds, per class, the number of draws before each row
+// counting only items that exist, so that no ticket is spent on a missing item.  Kept out of line: the scheduling
+// loop of the common case stays small.
+__device__ __noinline__ int2 plan_tables(const int32_t* seq_lens, int max_blocks, int units, int rows_small,
+                                         unsigned long long hkv_magic, unsigned char* smem, int n_heavy, int rows,
+                                         int lane) {
+    int total_heavy = 0, total_light = 0;
+    const int* cache = reinterpret_cast<const int*>(smem + kOffUnits);
+    unsigned short* ustart = reinterpret_cast<unsigned short*>(smem + kOffStart);
+    int* pref = reinterpret_cast<int*>(smem + kOffRowPref);
+    for (int x = lane; x <= rows; x += 32) pref[x] = pref[kRowCap + 1 + x] = 0;
+    __syncwarp();
+    for (int c = 0; c < 2; ++c) {
+        const int n_class = c == 0 ? n_heavy : units - n_heavy;
+        for (int u = lane; u < n_class; u += 32) {
+            const int b = (int)fast_div((unsigned)cache[c * kUnitCache + u], hkv_magic);
+            const int nb = (min(max(seq_lens[b], 0), max_blocks * kBlk) + kBlk - 1) / kBlk;
+            const int s = rows_small * kSmallBlocks;
+            const int items = nb <= s ? (nb + kSmallBlocks - 1) / kSmallBlocks
+                                      : rows_small + (nb - s + kItemBlocks - 1) / kItemBlocks;   // item_count
+            const int start = max(rows - items, 0);   // == rows: the sequence is empty
+            ustart[c * kUnitCache + u] = (unsigned short)start;
+            if (start < rows) atomicAdd(&pref[c * (kRowCap + 1) + start], 1);
+        }
+    }
+    __syncwarp();
+    for (int c = 0; c < 2; ++c) {   // units starting in row r -> units present in row r -> draws before row r
+        int* pc = pref + c * (kRowCap + 1);
+        int started = 0, before = 0;
+        for (int base = 0; base < rows; base += 32) {
+            const int r = base + lane;
+            int v = r < rows ? pc[r] : 0;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(kFull, v, o);
+                if (lane >= o) v += t;
+            }
+            const int here = r < rows ? started + v : 0;
+            int w = here;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(kFull, w, o);
+                if (lane >= o) w += t;
+            }
+            if (r < rows) pc[r] = before + w - here;
+            started += __shfl_sync(kFull, v, 31);
+            before += __shfl_sync(kFull, w, 31);
+        }
+        if (lane == 0) pc[rows] = before;
+        if (c == 0) total_heavy = before; else total_light = before;
+    }
+    __syncwarp();
+    return make_int2(total_heavy, total_light);
+}
+
+// draw number k of a class -> row (among the rows in use) and index within the class, through the row tables;
+// all lanes, same arguments
+__device__ __forceinline__ int2 table_lookup(const unsigned char* smem, int c, int n_class, int rows, int k, int lane) {
+    const int* pc = reinterpret_cast<const int*>(smem + kOffRowPref) + c * (kRowCap + 1);
+    const unsigned short* ustart = reinterpret_cast<const unsigned short*>(smem + kOffStart) + c * kUnitCache;
+    // the last row whose first draw is <= k: 32-way search, the lanes probing evenly spaced rows (pc is monotone and
+    // pc[0] = 0 <= k, so the lanes that pass form a prefix)
+    int lo = 0, span = rows;
+    while (span > 1) {
+        const int step = (span + 31) >> 5;
+        const int r = lo + lane * step;
+        const unsigned pass = __ballot_sync(kFull, r < lo + span && pc[r] <= k);
+        const int seg = __popc(pass) - 1;
+        span = min(step, span - seg * step);
+        lo += seg * step;
+    }
+    int j = k - pc[lo], sel = 0;               // the j-th unit, in list order, that has an item in this row
+    for (int i0 = 0; i0 < n_class; i0 += 32) {
+        const int i = i0 + lane;
+        const bool present = i < n_class && (int)ustart[i] <= lo;
+        const unsigned m = __ballot_sync(kFull, present);
+        const int cnt = __popc(m);
+        if (j < cnt) {   // the lane whose unit is present and has exactly j present units before it
+            const unsigned hit = __ballot_sync(kFull, present && __popc(m & ((1u << lane) - 1u)) == j);
+            sel = i0 + __ffs(hit) - 1;
+            break;
+        }
+        j -= cnt;
+    }
+    return make_int2(lo, sel);
+}
+
 // draw number k of a class -> work item
 __device__ __forceinline__ Item decode_item(const DecodeParams& p, const ItemSched& sc, const int* unit_cache,
-                                            bool heavy, int k) {
+                                            bool heavy, int k, int2 via_table) {
     Item it;
     int row, bg;
-    if (heavy) {   // heavy units sit at the front of the list, light units at its back (first ones cached in smem)
+    if (sc.table) {
+        row = via_table.x;
+        bg = unit_cache[(heavy ? 0 : kUnitCache) + via_table.y];
+    } else if (heavy) {   // heavy units sit at the front of the list, light units at its back (first ones cached in smem)
         row = (int)fast_div((unsigned)k, sc.magic_heavy);
         const int u = k - row * sc.n_heavy;
         bg = u < kUnitCache ? unit_cache[u] : p.unit_list[u];
@@ -239,6 +335,14 @@ __device__ __forceinline__ void sched_role(const DecodeParams& p, unsigned char*
     sc.row_off = p.item_rows - rows;
     sc.total_heavy = sc.n_heavy * rows;
     sc.total_light = sc.n_light * rows;
+    sc.table = 2ll * (long long)p.len_stats[2] < (long long)p.units * rows && rows <= kRowCap &&
+               sc.n_heavy <= kUnitCache && sc.n_light <= kUnitCache;
+    if (sc.table) {
+        const int2 totals = plan_tables(p.seq_lens, p.max_blocks, p.units, p.rows_small, p.hkv_magic, smem, sc.n_heavy,
+                                        rows, lane);
+        sc.total_heavy = totals.x;
+        sc.total_light = totals.y;
+    }
     sc.magic_heavy = fast_div_magic((unsigned)max(sc.n_heavy, 1));
     sc.magic_light = fast_div_magic((unsigned)max(sc.n_light, 1));
     sc.pend_heavy = pend_heavy;
@@ -287,7 +391,9 @@ __device__ __forceinline__ void sched_role(const DecodeParams& p, unsigned char*
             if (kind == 2) continue;
             if (kind < 0) break;
             // every lane decodes the same item (the class sizes and reciprocals are the same in all lanes)
-            const Item c = decode_item(p, sc, unit_cache, kind == 1, cand);
+            int2 via_table = make_int2(0, 0);
+            if (sc.table) via_table = table_lookup(smem, kind == 1 ? 0 : 1, kind == 1 ? sc.n_heavy : sc.n_light, rows, cand, lane);
+            const Item c = decode_item(p, sc, unit_cache, kind == 1, cand, via_table);
             if (c.nblk <= 0) continue;   // the sequence is shorter than the longest one: nothing in this item
             it = c;
             if (lane == 0) {

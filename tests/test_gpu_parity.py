@@ -233,6 +233,17 @@ def test_cache_with_room_for_much_longer_sequences(ffd, oracle):
     check_dense(ffd, oracle, w, dc)
 
 
+def test_one_long_sequence_among_short_ones(ffd, oracle):
+    """Most of the (row, unit) grid of work items is empty: the scheduler hands the tickets out through its table of
+    existing items.  Same results as ever."""
+    w = make_workload("C5", B=6, lens=(4000, 5000))
+    w.seq_lens[:] = np.array([int(w.seq_lens[0]), 200, 130, 64, 1, 2049], dtype=np.int32)
+    dc = ffd.DeviceCache(w)
+    codes, scales = check_quantize(ffd, oracle, w, dc)
+    for delta in (6.0, 0.0, INF):
+        check_decode(ffd, oracle, w, dc, codes, scales, delta)
+
+
 def test_step_replays_from_a_cuda_graph(ffd, oracle):
     """A whole step (tail re-quantize + decode) captured once and replayed gives the eager step's result; every
     step-varying argument (q, seq_lens, first_token, block_table) lives on the device (Sec. 3.3)."""
