@@ -202,10 +202,16 @@ class DeviceCache:
         self.w = w
         self.cfg = cfg or Config(w.Hq, w.Hkv)
         self.device = device
-        self.q = w.q.to(device)
+        # q and seq_lens, the two inputs that change every step, share one allocation (q first, both 16-byte
+        # aligned) so that a serving loop can bring them over with a single host-to-device copy into `step_in`
+        qb = w.q.numel() * 2
+        self.step_in = torch.zeros(qb + (4 * w.B + 15) // 16 * 16, dtype=torch.uint8, device=device)
+        self.q = self.step_in[:qb].view(torch.bfloat16).view(w.q.shape)
+        self.q.copy_(w.q)
+        self.seq_lens = self.step_in[qb:qb + 4 * w.B].view(torch.int32)
+        self.seq_lens.copy_(torch.from_numpy(w.seq_lens))
         self.k_cache = w.k_cache.to(device)
         self.v_cache = w.v_cache.to(device)
-        self.seq_lens = torch.from_numpy(w.seq_lens).to(device)
         self.block_table = None if w.block_table is None else torch.from_numpy(w.block_table).to(device)
         P, Hkv = w.num_pages, w.Hkv
         self.k_quant = torch.zeros(P, Hkv, 2048, dtype=torch.uint8, device=device)
