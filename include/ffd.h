@@ -87,7 +87,8 @@ ffd_status ffd_workspace_init(void* workspace, size_t workspace_bytes, void* str
  * (re)quantized over its valid rows r < min(64, seq_lens[b] - 64*blk): per channel
  *   s = fp16_rne(min(fp32(max_r |K[r,c]|) / 1.5f, 65504)),  code = x<0 ? (|x|>=s ? 0 : 1) : (|x|>=s ? 3 : 2)
  * (the nearest level of {-1.5,-0.5,+0.5,+1.5}*s; ties go outward, +-0 to +0.5).  Codes of rows past the
- * sequence end are unspecified.  first_token NULL means 0 (quantize everything).
+ * sequence end are unspecified.  first_token NULL means 0 (quantize everything).  K must be finite (no NaN: the
+ * whole-cache path and the first_token path would code a NaN differently; +-inf is handled like a large value).
  * Writes k_quant and k_scales of the touched (page, head) tiles only.  Blocks whose block_table entry is
  * outside [0, num_pages) are skipped; a seq_len outside [0, max_blocks_per_seq*64] is clamped.
  */

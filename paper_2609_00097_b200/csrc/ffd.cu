@@ -641,9 +641,14 @@ static ffd_status check_geometry(int batch, int max_blocks, int num_pages) {
 
 // Threads per combine CTA (one CTA per head): as many as still let all CTAs be resident at once.
 static int combine_threads(long heads) { return heads <= 2 * 148 ? 1024 : heads <= 4 * 148 ? 512 : 256; }
-// CTAs per head (each takes a share of the channels): more when there are few heads, so that a long sequence's
-// partials are not summed by a handful of SMs.
-static int combine_split(long heads) { return heads >= 128 ? 1 : heads >= 64 ? 2 : 4; }
+// CTAs per head (each takes a share of the channels): more when there are few heads with many partials each, so
+// that a long sequence's partials are not summed by a handful of SMs; never so many that a CTA is left with fewer
+// than 128 partials (its fixed cost would dominate) or that the grid exceeds two CTAs per SM.
+static int combine_split(long heads, long max_partials) {
+    for (int z = 4; z > 1; z >>= 1)
+        if (heads * z <= 2 * 148 + 32 && max_partials / z >= 128) return z;
+    return 1;
+}
 
 static cudaEvent_t g_prof_start = nullptr, g_prof_stop = nullptr;
 
@@ -748,14 +753,16 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
         if (prof) cudaEventRecord(g_prof_start, s);
         launch_pdl(fused_sparse_kernel, dim3(min(p.total_items, sms)), dim3(kFusedThreads), kFusedSmem, s, p);
         if (prof) cudaEventRecord(g_prof_stop, s);
-        launch_pdl(combine_kernel<true>, dim3(p.Hq, batch, combine_split(p.Hq * batch)), dim3(combine_threads(p.Hq * batch)), 0, s, p);
+        launch_pdl(combine_kernel<true>, dim3(p.Hq, batch, combine_split(p.Hq * batch, (long)p.item_rows * kNA)),
+                   dim3(combine_threads(p.Hq * batch)), 0, s, p);
     } else {
         if (cudaFuncSetAttribute(decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem) != cudaSuccess)
             return FFD_ERR_CUDA;
         if (prof) cudaEventRecord(g_prof_start, s);
         launch_pdl(decode_kernel<false>, grid, dim3(kWarps * 32), kDecodeSmem, s, p);
         if (prof) cudaEventRecord(g_prof_stop, s);
-        launch_pdl(combine_kernel<false>, dim3(p.Hq, batch, combine_split(p.Hq * batch)), dim3(combine_threads(p.Hq * batch)), 0, s, p);
+        launch_pdl(combine_kernel<false>, dim3(p.Hq, batch, combine_split(p.Hq * batch, p.splits)),
+                   dim3(combine_threads(p.Hq * batch)), 0, s, p);
     }
     return launch_status();
 }
