@@ -111,7 +111,7 @@ constexpr int kQbStages = 1;
 constexpr int kQbSmem = kQbStages * kTileBytes + 8 * 16 * 16 + 2 * kD * 2;
 
 __device__ __forceinline__ uint32_t qb_chunk(int row, int chunk) {   // byte offset of a 16-byte chunk in a staged tile
-    return (uint32_t)(row * 256 + ((chunk ^ (row & 1)) << 4));
+    return (uint32_t)(row * 256 + ((chunk ^ ((row & 1) << 1)) << 4));   // (with the read order below: conflict-free)
 }
 
 __global__ void __launch_bounds__(kQbThreads) quantize_bulk_kernel(QuantParams p) {
@@ -208,7 +208,10 @@ __global__ void __launch_bounds__(kQbThreads) quantize_bulk_kernel(QuantParams p
             const __nv_bfloat162 bias = __floats2bfloat162_rn(128.f, 128.f);
             uint32_t w[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
+            for (int kk = 0; kk < 4; ++kk) {
+                // lanes j = 2, 3 take their four chunks one step ahead of lanes j = 0, 1: the chunks 4j + k and
+                // 4(j + 2) + k lie 128 bytes apart, i.e. in the same banks
+                const int k = (kk + (j >> 1)) & 3;
                 const uint4 v0 = lds128(stage + qb_chunk(r0, 4 * j + k));
                 const uint4 v1 = lds128(stage + qb_chunk(r1, 4 * j + k));
                 const uint4 tv = *reinterpret_cast<const uint4*>(tq + 32 * j + 8 * k);
