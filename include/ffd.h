@@ -102,8 +102,9 @@ ffd_status ffd_quantize_keys(const ffd_config* cfg, const void* k_cache, void* k
  * pos = seq_lens[b] < max_blocks_per_seq*64: the rows k_new[b, g, :] and v_new[b, g, :] (bf16 [B, Hkv, 128], device)
  * are written to token position pos of k_cache / v_cache (block pos/64 through block_table, row pos%64), that
  * block's thumbnails (k_quant, k_scales) are re-quantized over its rows 0 .. pos%64 exactly as ffd_quantize_keys
- * would, and seq_lens[b] becomes pos + 1.  A sequence with no room left, or whose block_table entry for the block is
- * outside [0, num_pages), is left untouched and reported in the status word (FFD_DEV_BAD_SEQ_LEN / FFD_DEV_BAD_PAGE).
+ * would, and seq_lens[b] becomes pos + 1.  A sequence with no room left is left untouched and reported in the status
+ * word (FFD_DEV_BAD_SEQ_LEN); if the block_table entry for the block is outside [0, num_pages) the rows are not
+ * written and FFD_DEV_BAD_PAGE is reported, but the length still advances (a decode skips such a block anyway).
  * workspace: device memory of at least 256 bytes whose first word is the status word (a decode workspace will do).
  * Asynchronous on `stream`; two kernel launches; allocates nothing; may be captured in a CUDA graph together with
  * the decode call that follows it.  Host errors as for ffd_quantize_keys (FFD_ERR_WORKSPACE if workspace_bytes < 256).
@@ -137,6 +138,21 @@ ffd_status ffd_decode(const ffd_config* cfg, const void* q, const void* k_cache,
                       const int32_t* seq_lens, int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages,
                       float delta, void* out, float* lse, uint8_t* kept_mask, float* block_max, void* workspace,
                       size_t workspace_bytes, void* stream);
+
+/*
+ * One serving step in a single call: ffd_append_kv followed by ffd_decode on the lengthened sequences, with the
+ * append folded into the first kernel of the decode (three launches instead of five; Sec. 3.3).  Arguments as for
+ * those two calls; k_cache, v_cache, k_quant, k_scales are written (the new rows, the re-quantized tail block) and
+ * seq_lens[b] becomes seq_lens[b] + 1 for every sequence that had room.  While the call runs, its kernels take the
+ * new lengths from the workspace; the caller's seq_lens array is updated by the last kernel.  A sequence without
+ * room is decoded at its old length and reported (FFD_DEV_BAD_SEQ_LEN).  Results equal those of the two separate
+ * calls.  Asynchronous, allocation-free, capturable in a CUDA graph.
+ */
+ffd_status ffd_append_decode(const ffd_config* cfg, const void* k_new, const void* v_new, const void* q, void* k_cache,
+                             void* v_cache, void* k_quant, void* k_scales, const int32_t* block_table,
+                             int32_t* seq_lens, int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages,
+                             float delta, void* out, float* lse, uint8_t* kept_mask, float* block_max, void* workspace,
+                             size_t workspace_bytes, void* stream);
 
 /*
  * Dense decode attention over every valid token (the exact baseline the paper compares against in

@@ -33,6 +33,8 @@ __device__ __forceinline__ uint32_t quant_code(float x, float s) {
 
 // One (page, KV head) tile, staged in shared memory as sk[64][128], by 128 threads: per-channel scale over the first
 // `rows` rows (App. A.1), then the packed 2-bit codes.  Contains a __syncthreads().
+// GROUP: the 128 calling threads are part of a larger CTA and meet at named barrier 1 instead of the CTA's.
+template <bool GROUP = false>
 __device__ __forceinline__ void quantize_tile(const __nv_bfloat16* sk, float* ss, int rows, __half* scales_out,
                                               uint8_t* codes_out, int tid) {
     {
@@ -46,7 +48,8 @@ __device__ __forceinline__ void quantize_tile(const __nv_bfloat16* sk, float* ss
         scales_out[tid] = s;
         ss[tid] = __half2float(s);
     }
-    __syncthreads();
+    if (GROUP) asm volatile("bar.sync 1, 128;\n" ::: "memory");
+    else __syncthreads();
     const int mt = tid >> 5, lane = tid & 31, r = lane >> 2, j = lane & 3;
     uint32_t w[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
@@ -320,7 +323,11 @@ constexpr int kPmSamples = 7;  // blocks sampled between the sink and the local 
 
 // ---- pseudo-max (Sec. 3.2; Alg. 1 "Pseudo-max estimation") ------------------------------------------------
 // One CTA per (KV head, sequence): its warps scan the sink and local blocks and reduce the block maxima.
-__global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p) {
+// APPEND (ffd_append_decode): the CTA first appends the new token of its (sequence, KV head) as append_kernel does
+// — rows written, tail block re-quantized — and works with the new length; new_lens[b] receives that length for
+// the kernels that follow (the caller's seq_lens is only read here; the combine kernel updates it at the end).
+template <bool APPEND>
+__global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p, AppendParams ap, int32_t* new_lens) {
     const int g = blockIdx.x, b = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // Wait first, then let the fused kernel start: whatever the fused kernel does ahead of its own dependency wait
@@ -328,7 +335,41 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
     // the previous call's reset of the work counters included.
     pdl_wait();
     pdl_launch_dependents();
-    const int n = clamped_seq_len(p, b);
+    int n = clamped_seq_len(p, b);
+    int tail_blk = -1;   // APPEND: the block whose thumbnails warps 0..3 of this CTA rewrite (warp 0 scans it)
+    if (APPEND) {
+        __shared__ __align__(16) __nv_bfloat16 sk[kBlk * kD];
+        __shared__ float ss[kD];
+        const int tid = threadIdx.x;
+        const int pos = n;
+        const bool room = pos < p.max_blocks * kBlk;
+        if (!room && tid == 0) atomicOr(p.status, kDevBadSeqLen);   // reported, nothing appended
+        int page = -1;
+        if (room) {
+            n = pos + 1;
+            page = page_of(p, b, pos / kBlk);   // (reports a bad entry; the rows are then not written)
+        }
+        if (g == 0 && tid == 0) new_lens[b] = n;
+        if (page >= 0) {   // (uniform over the CTA)
+            tail_blk = pos / kBlk;
+            if (tid < kD) {   // warps 0..3 append and re-quantize while the other warps already scan
+                const int row = pos % kBlk;
+                const size_t tile = (size_t)page * p.Hkv + g;
+                const size_t unit = (size_t)b * p.Hkv + g;
+                const __nv_bfloat16 kn = ap.k_new[unit * kD + tid];
+                ap.v_cache[(tile * kBlk + row) * kD + tid] = ap.v_new[unit * kD + tid];
+                ap.k_cache[(tile * kBlk + row) * kD + tid] = kn;
+                sk[row * kD + tid] = kn;
+                const uint4* src = reinterpret_cast<const uint4*>(ap.k_cache + tile * kBlk * kD);
+                uint4* dst = reinterpret_cast<uint4*>(sk);
+                for (int x = tid; x < row * (kD / 8); x += kD) dst[x] = src[x];
+                asm volatile("bar.sync 1, 128;\n" ::: "memory");
+                quantize_tile<true>(sk, ss, row + 1, ap.k_scales + tile * kD, ap.k_quant + tile * kCodeBytes, tid);
+                __threadfence_block();
+                asm volatile("bar.sync 1, 128;\n" ::: "memory");   // warp 0 may now read the new thumbnails
+            }
+        }
+    }
     const int nb = (n + kBlk - 1) / kBlk;
     const int ns = min(p.n_sink, nb);
     const int local_begin = max(nb - p.n_local, ns);
@@ -366,7 +407,18 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
     const int middle = local_begin - ns;
     const int nsamp = min(kPmSamples, middle);
     float best = -INFINITY;
-    for (int s = warp; s < count + nsamp; s += kPmWarps) {
+    // blocks s = 0 .. count + nsamp - 1 are dealt to the warps round-robin; with a tail block being rewritten
+    // (APPEND) warp 0 takes that one (it is s = count - 1, the last local block) after its part in rewriting it,
+    // warps 1..3 join once they are done with theirs, and the other warps never touch it
+    const bool special = APPEND && tail_blk >= 0;
+    const int first_s = special ? (warp == 0 ? count - 1 : warp - 1) : warp;
+    const int step_s = special ? kPmWarps - 1 : kPmWarps;
+    for (int s0 = first_s; s0 < count + nsamp; s0 += step_s) {
+        int s = s0;
+        if (special && warp != 0) {          // skip over the tail block's slot
+            if (s >= count - 1) ++s;
+            if (s >= count + nsamp) break;
+        } else if (special && s0 != count - 1) break;   // warp 0: the tail block only
         const bool sample = s >= count;
         const int blk = sample ? ns + (int)(((long long)(2 * (s - count) + 1) * middle) / (2 * nsamp))
                                : (s < ns ? s : local_begin + (s - ns));
@@ -376,8 +428,12 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
         const int rows = min(kBlk, n - blk * kBlk);
         float band;
         ScanRegs sr;
-        scan_load(sr, reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes),
-                  reinterpret_cast<const uint4*>(p.k_scales + tile * kD), lane);
+        if (APPEND && blk == tail_blk)
+            scan_load_plain(sr, reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes),
+                            reinterpret_cast<const uint4*>(p.k_scales + tile * kD), lane);
+        else
+            scan_load(sr, reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes),
+                      reinterpret_cast<const uint4*>(p.k_scales + tile * kD), lane);
         const float bm = scan_compute<true>(sr, sq, lane, rows, p.sm_scale, band);
         if (lane < kMaxG && s < kPmHintBlocks) sbm[s][lane] = bm;
         if (!sample) best = fmaxf(best, bm);
@@ -594,7 +650,7 @@ __global__ void clear_header_kernel(uint32_t* header) { header[threadIdx.x] = 0u
 struct Plan {
     int blocks_per_split, splits;     // dense path
     int total_items;                  // fused path
-    size_t off_mtilde, off_units, off_qrec, off_ml, off_acc, off_fml, off_facc, total;
+    size_t off_mtilde, off_lens, off_units, off_qrec, off_ml, off_acc, off_fml, off_facc, total;
 };
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -612,7 +668,8 @@ static Plan make_plan(const ffd_config* cfg, int batch, int max_blocks) {
     pl.total_items = item_geometry(units, max_blocks).item_rows * batch * cfg->num_kv_heads;
     const size_t fslots = (size_t)pl.total_items * kNA * kMaxG;
     pl.off_mtilde = 256;
-    pl.off_units = align_up(pl.off_mtilde + heads * sizeof(float), 256);
+    pl.off_lens = align_up(pl.off_mtilde + heads * sizeof(float), 256);
+    pl.off_units = align_up(pl.off_lens + (size_t)batch * sizeof(int32_t), 256);
     pl.off_qrec = align_up(pl.off_units + (size_t)batch * cfg->num_kv_heads * sizeof(int32_t), 256);
     pl.off_ml = align_up(pl.off_qrec + (size_t)batch * cfg->num_kv_heads * kQrecBytes, 256);
     pl.off_acc = align_up(pl.off_ml + heads * pl.splits * 2 * sizeof(float), 256);
@@ -678,7 +735,8 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
                              const void* v_cache, const void* k_quant, const void* k_scales,
                              const int32_t* block_table, const int32_t* seq_lens, int batch, int max_blocks,
                              int num_pages, float delta, void* out, float* lse, uint8_t* kept_mask,
-                             float* block_max, void* workspace, size_t workspace_bytes, void* stream) {
+                             float* block_max, void* workspace, size_t workspace_bytes, void* stream,
+                             const AppendParams* append = nullptr) {
     ffd_status st = check_config(cfg);
     if (st) return st;
     if (!q || !k_cache || !v_cache || !seq_lens || !out || !workspace) return FFD_ERR_NULL;
@@ -752,7 +810,16 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
             return FFD_ERR_CUDA;
         // the work counters and class counts at ws + 64 are zero here: ffd_workspace_init zeroes them and the
         // combine kernel of every call leaves them zeroed for the next one
-        launch_pdl(pseudomax_kernel, dim3(p.Hkv, batch), dim3(kPmWarps * 32), 0, s, p);
+        if (append) {
+            // the kernels after the first one read the lengths it leaves in the workspace
+            int32_t* new_lens = reinterpret_cast<int32_t*>(ws + pl.off_lens);
+            launch_pdl(pseudomax_kernel<true>, dim3(p.Hkv, batch), dim3(kPmWarps * 32), 0, s, p, *append, new_lens);
+            p.seq_lens = new_lens;
+            p.bump_lens = append->seq_lens;
+        } else {
+            launch_pdl(pseudomax_kernel<false>, dim3(p.Hkv, batch), dim3(kPmWarps * 32), 0, s, p, AppendParams{},
+                       static_cast<int32_t*>(nullptr));
+        }
         if (prof) cudaEventRecord(g_prof_start, s);
         launch_pdl(fused_sparse_kernel, dim3(min(p.total_items, sms)), dim3(kFusedThreads), kFusedSmem, s, p);
         if (prof) cudaEventRecord(g_prof_stop, s);
@@ -879,6 +946,22 @@ ffd_status ffd_decode(const ffd_config* cfg, const void* q, const void* k_cache,
     return run_decode(true, cfg, q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, batch,
                       max_blocks_per_seq, num_pages, delta, out, lse, kept_mask, block_max, workspace,
                       workspace_bytes, stream);
+}
+
+ffd_status ffd_append_decode(const ffd_config* cfg, const void* k_new, const void* v_new, const void* q, void* k_cache,
+                             void* v_cache, void* k_quant, void* k_scales, const int32_t* block_table,
+                             int32_t* seq_lens, int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages,
+                             float delta, void* out, float* lse, uint8_t* kept_mask, float* block_max, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+    if (!k_new || !v_new) return FFD_ERR_NULL;
+    if (misaligned(k_new) || misaligned(v_new)) return FFD_ERR_ALIGN;
+    AppendParams ap{static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
+                    static_cast<__nv_bfloat16*>(k_cache), static_cast<__nv_bfloat16*>(v_cache),
+                    static_cast<uint8_t*>(k_quant), static_cast<__half*>(k_scales), block_table, seq_lens,
+                    static_cast<uint32_t*>(workspace), cfg ? cfg->num_kv_heads : 0, max_blocks_per_seq, num_pages};
+    return run_decode(true, cfg, q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, batch,
+                      max_blocks_per_seq, num_pages, delta, out, lse, kept_mask, block_max, workspace, workspace_bytes,
+                      stream, &ap);
 }
 
 ffd_status ffd_decode_dense(const ffd_config* cfg, const void* q, const void* k_cache, const void* v_cache,

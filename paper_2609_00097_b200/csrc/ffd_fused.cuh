@@ -861,6 +861,8 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
         p.len_stats[1] = 0u;
         p.len_stats[2] = 0u;
     }
+    // append + decode: the caller's lengths take the new values now that nothing of this call reads them any more
+    if (FUSED && p.bump_lens && h == 0 && blockIdx.z == 0 && tid == 0) p.bump_lens[b] = p.seq_lens[b];
     const size_t head = (size_t)b * p.Hq + h;
     const int g = h / p.G, hl = h % p.G, bg = b * p.Hkv + g;
     const int n = min(max(p.seq_lens[b], 0), p.max_blocks * kBlk);

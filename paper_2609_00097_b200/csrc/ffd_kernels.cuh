@@ -91,6 +91,7 @@ struct DecodeParams {
     uint32_t* item_counter;  // fused path: next heavy-class draw (workspace; zeroed at the start of every call)
     uint32_t* light_counter; // fused path: next light-class draw
     uint32_t* class_counts;  // fused path: [0] heavy units, [1] light units found by the pseudo-max kernel (workspace)
+    int32_t* bump_lens;      // append + decode: the caller's seq_lens, set to the new lengths by the combine kernel
     uint32_t* len_stats;     // fused path: [0] largest block count of the batch, [1] largest (max_blocks - block count), [2] items
     int32_t* unit_list;      // fused path: heavy units from the front, light units from the back (workspace)
     int units;               // batch * Hkv
@@ -128,6 +129,13 @@ __device__ __forceinline__ void mma_bf16_top(float& c0, float& c1, uint32_t a0, 
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
         : "+f"(c0), "+f"(c1), "+f"(z0), "+f"(z1)
         : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+}
+
+// an ordinary (coherent) 16-byte global load
+__device__ __forceinline__ uint4 ldg_plain(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
 }
 
 __device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
@@ -289,6 +297,15 @@ struct ScanRegs {
     uint4 w[4];   // packed codes of the four 16-token groups
     uint4 s[4];   // this lane's 32 scales
 };
+
+// the same through ordinary loads: for a tile this kernel has itself just written
+__device__ __forceinline__ void scan_load_plain(ScanRegs& sr, const uint4* codes_tile, const uint4* scales_tile,
+                                                int lane) {
+#pragma unroll
+    for (int mt = 0; mt < 4; ++mt) sr.w[mt] = ldg_plain(codes_tile + mt * 32 + lane);
+#pragma unroll
+    for (int x = 0; x < 4; ++x) sr.s[x] = ldg_plain(scales_tile + 4 * (lane & 3) + x);
+}
 
 __device__ __forceinline__ void scan_load(ScanRegs& sr, const uint4* __restrict__ codes_tile,
                                           const uint4* __restrict__ scales_tile, int lane) {

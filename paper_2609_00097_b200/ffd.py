@@ -25,7 +25,7 @@ DEV_BAD_SEQ_LEN = 2
 
 EXPORTS = ["ffd_status_string", "ffd_workspace_bytes", "ffd_workspace_init", "ffd_quantize_keys", "ffd_decode",
            "ffd_decode_dense", "ffd_unpack_codes", "ffd_read_device_status", "ffd_profile_events", "ffd_decode_static",
-           "ffd_append_kv"]
+           "ffd_append_kv", "ffd_append_decode"]
 
 
 class FfdError(RuntimeError):
@@ -87,6 +87,8 @@ def load_library() -> ctypes.CDLL:
                                           _vp, _vp]
         lib.ffd_append_kv.argtypes = [cfgp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, _vp, ctypes.c_size_t,
                                       _vp]
+        lib.ffd_append_decode.argtypes = [cfgp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32,
+                                          ctypes.c_float, _vp, _vp, _vp, _vp, _vp, ctypes.c_size_t, _vp]
         for name in EXPORTS:
             if name != "ffd_status_string":
                 getattr(lib, name).restype = ctypes.c_int
@@ -150,6 +152,16 @@ def ffd_decode(cfg: Config, q, k_cache, v_cache, k_quant, k_scales, block_table,
                                      _p(k_scales), _p(block_table), _p(seq_lens), q.shape[0], max_blocks_per_seq,
                                      k_cache.shape[0], ctypes.c_float(delta), _p(out), _p(lse), _p(kept_mask),
                                      _p(block_max), _p(workspace), workspace.numel(), _stream(stream)), "ffd_decode")
+
+
+def ffd_append_decode(cfg: Config, k_new, v_new, q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens,
+                      delta: float, out, *, max_blocks_per_seq: int, workspace, lse=None, kept_mask=None,
+                      block_max=None, stream=None):
+    _check(load_library().ffd_append_decode(ctypes.byref(cfg.c()), _p(k_new), _p(v_new), _p(q), _p(k_cache),
+                                            _p(v_cache), _p(k_quant), _p(k_scales), _p(block_table), _p(seq_lens),
+                                            q.shape[0], max_blocks_per_seq, k_cache.shape[0], ctypes.c_float(delta),
+                                            _p(out), _p(lse), _p(kept_mask), _p(block_max), _p(workspace),
+                                            workspace.numel(), _stream(stream)), "ffd_append_decode")
 
 
 def ffd_decode_static(cfg: Config, q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, delta: float, out,
@@ -228,6 +240,11 @@ class DeviceCache:
     def append(self, k_new, v_new):
         ffd_append_kv(self.cfg, k_new, v_new, self.k_cache, self.v_cache, self.k_quant, self.k_scales,
                       self.block_table, self.seq_lens, max_blocks_per_seq=self.w.max_blocks, workspace=self.workspace)
+
+    def append_decode(self, k_new, v_new, delta, kept_mask=None, block_max=None):
+        ffd_append_decode(self.cfg, k_new, v_new, self.q, self.k_cache, self.v_cache, self.k_quant, self.k_scales,
+                          self.block_table, self.seq_lens, delta, self.out, max_blocks_per_seq=self.w.max_blocks,
+                          workspace=self.workspace, lse=self.lse, kept_mask=kept_mask, block_max=block_max)
 
     def decode(self, delta, kept_mask=None, block_max=None):
         ffd_decode(self.cfg, self.q, self.k_cache, self.v_cache, self.k_quant, self.k_scales, self.block_table,

@@ -378,6 +378,54 @@ def test_serving_loop_append_and_decode_from_one_graph(ffd, oracle):
     assert np.array_equal(ca[sel], cb[sel])
 
 
+def test_append_decode_equals_append_then_decode(ffd, oracle):
+    """The single-call step must leave the cache, the thumbnails, the lengths and the output exactly as
+    ffd_append_kv followed by ffd_decode does, step after step, across block boundaries and at a full cache."""
+    w = make_workload("C5", B=4, lens=(1000, 5000))
+    w.seq_lens[:] = w.seq_lens - 70                      # the appends below cross at least one block boundary
+    w.seq_lens[1] = 64 * (int(w.seq_lens[1]) // 64)      # sequence 1 starts a block with its first append
+    a, b = ffd.DeviceCache(w), ffd.DeviceCache(w)
+    a.quantize(), b.quantize()
+    gen = torch.Generator(device="cuda").manual_seed(9)
+    kept_a = torch.zeros(w.B, w.Hq, w.max_blocks, dtype=torch.uint8, device="cuda")
+    kept_b = torch.zeros_like(kept_a)
+    for i in range(70):
+        k_new = torch.randn(w.B, w.Hkv, 128, device="cuda", generator=gen).to(torch.bfloat16)
+        v_new = torch.randn(w.B, w.Hkv, 128, device="cuda", generator=gen).to(torch.bfloat16)
+        a.append_decode(k_new, v_new, 6.0, kept_mask=kept_a)
+        b.append(k_new, v_new)
+        b.decode(6.0, kept_mask=kept_b)
+        if i % 23 == 0 or i == 69:
+            torch.cuda.synchronize()
+            assert ffd.ffd_read_device_status(a.workspace) == 0 and ffd.ffd_read_device_status(b.workspace) == 0
+            assert torch.equal(a.seq_lens, b.seq_lens)
+            assert torch.equal(a.k_scales.view(torch.int16), b.k_scales.view(torch.int16))
+            assert torch.equal(kept_a, kept_b)
+            assert (a.out - b.out).abs().max().item() <= 1e-6
+            assert (a.lse - b.lse).abs().max().item() <= 1e-5
+    assert int(a.seq_lens[0]) == int(w.seq_lens[0]) + 70
+    w.seq_lens[:] = a.seq_lens.cpu().numpy()
+    vm, _ = valid_row_mask(w)
+    sel = torch.from_numpy(np.broadcast_to(vm, tuple(a.k_cache.shape)).copy()).cuda()
+    assert torch.equal(a.k_cache.view(torch.int16)[sel], b.k_cache.view(torch.int16)[sel])
+    assert torch.equal(a.v_cache.view(torch.int16)[sel], b.v_cache.view(torch.int16)[sel])
+    ca, cb = a.canonical_codes().cpu().numpy(), b.canonical_codes().cpu().numpy()
+    csel = np.broadcast_to(vm, ca.shape)
+    assert np.array_equal(ca[csel], cb[csel])
+    # and against the oracle on the final state
+    w.k_cache = a.k_cache.cpu()
+    w.v_cache = a.v_cache.cpu()
+    codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
+    check_decode(ffd, oracle, w, a, codes, scales, 6.0)
+    # a sequence at capacity: decoded at its old length, reported, left alone
+    a.seq_lens[2] = w.max_blocks * 64
+    b.seq_lens[2] = w.max_blocks * 64
+    a.append_decode(k_new, v_new, 6.0)
+    torch.cuda.synchronize()
+    assert ffd.ffd_read_device_status(a.workspace) & ffd.DEV_BAD_SEQ_LEN
+    assert int(a.seq_lens[2]) == w.max_blocks * 64 and int(a.seq_lens[0]) == int(w.seq_lens[0]) + 1
+
+
 # full-size configurations: the oracle checks a sample of (sequence, head) rows one by one
 FULL = [
     ("C2", dict(), 8),
