@@ -426,6 +426,39 @@ def test_append_decode_equals_append_then_decode(ffd, oracle):
     assert int(a.seq_lens[2]) == w.max_blocks * 64 and int(a.seq_lens[0]) == int(w.seq_lens[0]) + 1
 
 
+def test_randomised_geometries(ffd, oracle):
+    """A seeded sweep over what the five configurations do not vary: query heads per KV head (1, 2, 4), odd head
+    counts, batch sizes, sink / local set sizes (including none of one kind and more local blocks than the pseudo-max
+    kernel has warps), lengths from one token to a few hundred blocks, paging, thresholds."""
+    import paper_2609_00097_b200.workloads as W
+    rng = np.random.default_rng(20260101)
+    try:
+        for case in range(24):
+            G, Hkv = int(rng.choice([1, 2, 4])), int(rng.choice([1, 2, 3, 8]))
+            lo = int(rng.choice([1, 40, 64, 65, 700, 1500, 9000]))
+            hi = lo + int(rng.choice([0, 1, 63, 500, 3000, 20000]))
+            recipe = dict(seed=int(rng.integers(1 << 20)), B=int(rng.choice([1, 2, 3, 5, 9])), Hq=G * Hkv, Hkv=Hkv,
+                          lens=(lo, hi), frac=float(rng.choice([0.0, 0.01, 0.05])), amp=float(rng.choice([2.0, 3.0, 4.0])),
+                          sink=bool(rng.integers(2)), deltas=(6.0,))
+            if rng.integers(2):
+                recipe.update(paged=True, spare_pages=int(rng.integers(0, 9)))
+            if rng.integers(2) and Hkv > 1:
+                recipe.update(flat_odd_heads=True)
+            if rng.integers(4) == 0:
+                recipe.update(recency_tokens=int(rng.choice([64, 300])), recency_amp=2.0)
+            n_sink = int(rng.choice([0, 1, 2]))
+            n_local = int(rng.choice([1, 4, 16, 40])) if n_sink == 0 else int(rng.choice([0, 1, 4, 16, 40]))
+            delta = float(rng.choice([0.0, 0.5, 3.0, 6.0, 12.0, np.inf]))
+            W.CONFIGS["sweep"] = recipe
+            w = make_workload("sweep")
+            dc = ffd.DeviceCache(w, ffd.Config(G * Hkv, Hkv, n_sink_blocks=n_sink, n_local_blocks=n_local))
+            codes, scales = check_quantize(ffd, oracle, w, dc)
+            check_decode(ffd, oracle, w, dc, codes, scales, delta)
+            check_dense(ffd, oracle, w, dc)
+    finally:
+        W.CONFIGS.pop("sweep", None)
+
+
 # full-size configurations: the oracle checks a sample of (sequence, head) rows one by one
 FULL = [
     ("C2", dict(), 8),
