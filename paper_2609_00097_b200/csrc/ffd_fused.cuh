@@ -71,7 +71,7 @@ __device__ __forceinline__ int item_count(const DecodeParams& p, int nb) {
     const int s = p.rows_small * kSmallBlocks;
     return nb <= s ? (nb + kSmallBlocks - 1) / kSmallBlocks : p.rows_small + (nb - s + kItemBlocks - 1) / kItemBlocks;
 }
-constexpr int kRing = 3;               // code-ring stages per scan warp
+constexpr int kRing = 2;               // code-ring stages per scan warp (a third stage measured no faster)
 constexpr int kStageBytes = kCodeBytes + kD * 2;   // 2048 B codes + 256 B scales
 #ifndef FFD_NB
 #define FFD_NB 8
@@ -81,8 +81,8 @@ constexpr int kNB = FFD_NB;                 // batch descriptors: how far the sc
 #define FFD_HEAVY_AHEAD 2
 #endif
 constexpr int kHeavyAhead = FFD_HEAVY_AHEAD;         // heavy batches outstanding at most once the attend warps are the bottleneck
-constexpr int kUnitCache = 256;        // entries of each end of the unit list kept in shared memory
-constexpr int kRowCap = 256;           // item rows up to which the table of existing items is built (ragged batches)
+constexpr int kUnitCache = 512;        // entries of each end of the unit list kept in shared memory
+constexpr int kRowCap = 512;           // item rows up to which the table of existing items is built (ragged batches)
 constexpr int kItemRing = 8;           // decoded items published ahead
 constexpr int kQrecRing = 4;           // query records staged ahead
 constexpr int kQrecAbs = 2048;         // query record: [4][32 lanes] uint4 of pre-scaled fp16 query fragments, ...
