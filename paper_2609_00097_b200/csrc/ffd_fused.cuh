@@ -1,18 +1,21 @@
 // The fused sparse kernel: scan -> top-delta select -> exact attention over kept blocks, in one persistent launch.
 //
 // One CTA per SM, 16 warps in three jobs that run concurrently (register budgets set with setmaxnreg):
-//   1 scheduling warp  (warp 0) draws work items from two global counters, decodes them once and publishes them two
-//                      entries ahead in a ring in shared memory (one mbarrier per entry); it also starts the copy of
-//                      the item's query record (pre-scaled fp16 query fragments + thresholds, written by the
-//                      pseudo-max kernel).  The atomic for the next draw of each class is always in flight.
-//   11 scan warps      stream the 2-bit codes and scales of every block through a private 3-stage cp.async ring
-//                      (3 blocks = 6.9 KB in flight per warp), bound the block's scores from its scales alone and,
-//                      unless that already rules the block out, compute the block maxima of the approximate scores
-//                      on the tensor cores; they publish the keep decisions of one work item in a batch descriptor.
+//   1 scheduling warp  (warp 0) draws work items from two global counters, decodes them once and publishes them up to
+//                      four entries ahead in a ring in shared memory (one mbarrier per entry) together with the
+//                      item's page-table entries and the header of its batch descriptor; it also starts the copy
+//                      of the item's query record (pre-scaled fp16 query fragments, |q| fragments and thresholds,
+//                      written by the pseudo-max kernel).  The atomic for the next draw of each class is always in
+//                      flight.
+//   11 scan warps      stream the 2-bit codes and scales of every block through a private 2-stage cp.async ring,
+//                      bound the block's scores from its scales alone and, unless that already rules the block out,
+//                      compute the block maxima of the approximate scores on the tensor cores; they publish the
+//                      keep decisions of one work item in a batch descriptor.
 //   4 attend warps     take the kept blocks of a published batch, stage their K and V tiles (16 KB each) through
 //                      private swizzled slots with cp.async + mbarrier and run the exact online-softmax attention.
-// A work item is 22 consecutive blocks of one (sequence, KV head): two per scan warp.  Scan warps may run up to eight
-// batches ahead of the attend warps (eight descriptors, full/empty mbarriers).  Units that the pseudo-max kernel's
+// A work item is 22 consecutive blocks of one (sequence, KV head), two per scan warp (11 for the half-size items at
+// the start of a sequence, which are handed out last).  Scan warps may run up to eight batches ahead of the attend
+// warps (eight descriptors, full/empty mbarriers).  Units that the pseudo-max kernel's
 // hint marks as dense ("heavy") are scheduled so that at most a few heavy batches are outstanding per CTA and the
 // scan warps' spare time goes to light items (see ItemSched).
 // Nobody divides or reloads sequence lengths on the per-block path.  Every wait is bounded; on expiry the warp
@@ -22,7 +25,7 @@
 
 namespace ffd {
 
-constexpr int kNS = 12;                // warps of the scan role (three warpgroups)
+constexpr int kNS = 12;                // warps of the scheduling + scan roles (three warpgroups)
 #ifndef FFD_SCHED_WARP
 #define FFD_SCHED_WARP 1
 #endif
@@ -424,7 +427,7 @@ __device__ __forceinline__ void sched_role(const DecodeParams& p, unsigned char*
 
 // ---- scan role ---------------------------------------------------------------------------------------------
 
-// Position of a scan warp in its stream of blocks: published item after published item, local blocks w and w + 12.
+// Position of a scan warp in its stream of blocks: published item after published item, local blocks w and w + 11.
 struct ScanCursor {
     int seq;       // published item the cursor is in (-1 before the first)
     Item it;
@@ -475,7 +478,7 @@ __device__ __forceinline__ void ring_wait(int younger) {
     else asm volatile("cp.async.wait_group 0;\n" ::: "memory");
 }
 
-// Warp 0 only: copy the query record of published item `seq` into slot seq % 4 of the record ring and report
+// Scheduling warp: copy the query record of published item `seq` into slot seq % 4 of the record ring and report
 // completion on that slot's mbarrier.  Every scan warp waits for every record, in order, so a parity wait can
 // never see a stale phase.
 __device__ __forceinline__ void qrec_issue(const DecodeParams& p, int seq, int bg, uint32_t qrecs, uint32_t qbars,
@@ -834,7 +837,7 @@ constexpr int kCombineChunk = 1024;
 
 template <bool FUSED>
 __device__ __forceinline__ size_t combine_slot(const DecodeParams& p, size_t head, int bg, int hl, int e) {
-    if (FUSED) {   // item number of split e / kNA (see decode_item), then the attend warp
+    if (FUSED) {   // item number of split e / kNA (items count from block 0, see item_span), then the attend warp
         const int item = (p.item_rows - 1 - e / kNA) * p.units + bg;
         return ((size_t)item * kNA + (e % kNA)) * kMaxG + hl;
     }
