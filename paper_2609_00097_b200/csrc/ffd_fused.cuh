@@ -132,8 +132,8 @@ static_assert(kFusedSmem <= 227 * 1024, "shared memory budget");
 // ones the pseudo-max kernel's hint expects to keep most of their blocks (expensive for the attend warps, memory
 // bound), "light" units the rest (almost pure scan work).  The drawing thread keeps at most kHeavyAhead heavy batches
 // queued ahead of the attend warps and fills the scan warps' remaining time with light items, so the two kinds of
-// work overlap on every SM; what is left over at the end is light, i.e. a short, well-balanced tail.  Within a class,
-// rows count from the END of the sequences backwards (the local window first).
+// work overlap on every SM.  Within a class,
+// rows count from the END of the sequences backwards (the local window first, the half-size items last).
 struct ItemSched {                                        // lives in the registers of the scheduling warp's lane 0
     int n_heavy, n_light, total_heavy, total_light;      // units and items per class
     unsigned long long magic_heavy, magic_light;          // reciprocals of the unit counts
@@ -281,8 +281,8 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
 // Entry seq lives in slot seq % 8 and is announced by one arrival on that slot's mbarrier (phase seq / 8): the
 // arrive releases the entry's fields, a successful test / wait acquires them.  No fence is used on purpose: a CTA
 // fence would also wait for the reader's in-flight cp.async copies and serialise the prefetch ring.  Every scan warp
-// visits every entry in order and never trails the publisher by more than three entries, so a parity test can not
-// alias.
+// visits every entry in order and the publisher is never more than four entries ahead of the slowest of them (it
+// waits for the full barrier of entry e - 4 before publishing e), so a parity test can not alias.
 
 __device__ __forceinline__ uint32_t item_bar(uint32_t ibars, int seq) { return ibars + (seq & (kItemRing - 1)) * 8; }
 
@@ -826,11 +826,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodePa
 }
 
 // ---- split combine (FlashDecoding-style log-sum-exp merge) -------------------------------------------------
-// One CTA of 1024 threads per (query head, sequence).  FUSED: partial e = (work item, attend warp) of the fused
-// kernel; otherwise partial e = split of the dense kernel.  The (m, l) pairs are read once into shared memory;
-// thread (el, cg) = (tid / 32, tid % 32) sums the partials e = el, el + 32, ... for channels 4cg .. 4cg+3 with
-// eight independent loads in flight; the 32 partial sums meet in shared memory.  Summation order is fixed, so
-// results are reproducible.
+// One, two or four CTAs of 256 .. 1024 threads per (query head, sequence), each taking a share of the channels.
+// FUSED: partial e = (work item, attend warp) of the fused kernel; otherwise partial e = split of the dense kernel.
+// The (m, l) pairs are read once into shared memory; thread (el, cg) sums the partials e = el, el + lanes, ... for
+// four channels with eight independent loads in flight; the partial sums meet in shared memory.  For a given launch
+// shape the summation order is fixed.
 constexpr int kCombineThreads = 1024;
 constexpr int kCombineLanes = kCombineThreads / 32;   // partials summed side by side (at most: the launch may use fewer threads)
 constexpr int kCombineChunk = 1024;
