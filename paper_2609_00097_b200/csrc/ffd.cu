@@ -791,6 +791,7 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
     p.units = batch * cfg->num_kv_heads;
     p.item_rows = item_geometry(p.units, max_blocks).item_rows;
     p.rows_small = item_geometry(p.units, max_blocks).rows_small;
+    p.item_blocks = item_geometry(p.units, max_blocks).item_blocks;
     p.units_magic = fast_div_magic((unsigned)p.units);
     p.hkv_magic = fast_div_magic((unsigned)cfg->num_kv_heads);
     p.kept_mask = kept_mask;

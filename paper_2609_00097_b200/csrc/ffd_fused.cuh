@@ -37,21 +37,30 @@ constexpr int kFusedThreads = (kNS + kNA) * 32;
 constexpr int kScanRegs = 112;         // 12*32*112 + 4*32*176 = 65536 registers
 constexpr int kAttendRegs = (65536 - kNS * 32 * kScanRegs) / (kNA * 32);
 static_assert(kAttendRegs % 8 == 0 && kScanRegs % 8 == 0, "setmaxnreg takes multiples of 8");
-// Blocks per work item: as many as the one-lane-per-block ballots allow.  Every batch costs its scan warps a round
-// of waits (item, query record, ring refill); 32 blocks per batch instead of 22 made the scan-bound workloads up to
-// 9 % faster.  Scan warp w takes blocks w, w + 11, w + 22.
-constexpr int kItemBlocks = 32;
-static_assert(kItemBlocks <= 32, "batch descriptor arrays; one lane per block in the ballots");
+// Blocks per full work item: 32 — as many as the one-lane-per-block ballots allow — when the launch has plenty of
+// items per SM, else 22.  Every batch costs its scan warps a round of waits (item, query record, ring refill), so
+// big batches are cheaper per block (C5: 9 % faster with 32 than with 22); but with only a few items per SM the
+// coarser items leave the SMs unevenly loaded (C3 at context 32768: 10 % slower).  Scan warp w takes blocks w,
+// w + 11, w + 22.
+constexpr int kItemBlocksMax = 32;
+constexpr int kItemBlocksMin = 2 * kScanners;
+static_assert(kItemBlocksMax <= 32, "batch descriptor arrays; one lane per block in the ballots");
 // The sequence is cut into items from block 0 upwards: first rows_small small items (one block per scanning
 // warp), then full items.  Items are drawn from the sequence END backwards, so the small ones are drawn last and
 // the CTAs run out of work within a small item's time of each other.
 constexpr int kSmallBlocks = kScanners;
 
-struct ItemGeom { int rows_small, item_rows; };
+struct ItemGeom { int rows_small, item_rows, item_blocks; };
 
 // pure function of the launch geometry (the workspace layout depends on it)
 __host__ __device__ inline ItemGeom item_geometry(long units, int max_blocks) {
     ItemGeom g;
+#ifdef FFD_DBG_ITEM_BLOCKS
+    g.item_blocks = FFD_DBG_ITEM_BLOCKS;
+#else
+    g.item_blocks = units * ((max_blocks + kItemBlocksMax - 1) / kItemBlocksMax) >= 6 * 148 ? kItemBlocksMax : kItemBlocksMin;
+#endif
+    const int kItemBlocks = g.item_blocks;
     const int full_rows = (max_blocks + kItemBlocks - 1) / kItemBlocks;
     const int all_small = (max_blocks + kSmallBlocks - 1) / kSmallBlocks;
     if (units * full_rows < 2 * 148) {
@@ -69,13 +78,13 @@ __host__ __device__ inline ItemGeom item_geometry(long units, int max_blocks) {
 // item number idx of a sequence, counted from block 0: first block and capacity
 __device__ __forceinline__ void item_span(const DecodeParams& p, int idx, int& blk0, int& cap) {
     if (idx < p.rows_small) { blk0 = idx * kSmallBlocks; cap = kSmallBlocks; }
-    else { blk0 = p.rows_small * kSmallBlocks + (idx - p.rows_small) * kItemBlocks; cap = kItemBlocks; }
+    else { blk0 = p.rows_small * kSmallBlocks + (idx - p.rows_small) * p.item_blocks; cap = p.item_blocks; }
 }
 
 // items a sequence of nb blocks is cut into
 __device__ __forceinline__ int item_count(const DecodeParams& p, int nb) {
     const int s = p.rows_small * kSmallBlocks;
-    return nb <= s ? (nb + kSmallBlocks - 1) / kSmallBlocks : p.rows_small + (nb - s + kItemBlocks - 1) / kItemBlocks;
+    return nb <= s ? (nb + kSmallBlocks - 1) / kSmallBlocks : p.rows_small + (nb - s + p.item_blocks - 1) / p.item_blocks;
 }
 constexpr int kRing = 2;               // code-ring stages per scan warp (a third stage measured no faster)
 constexpr int kStageBytes = kCodeBytes + kD * 2;   // 2048 B codes + 256 B scales
@@ -108,7 +117,7 @@ struct ItemSlot {                      // entry seq % 8 of the published-item ri
 
 struct BatchDesc {
     int item, b, g, nblk;              // canonical item number (row * units + bg) of this batch; < 0: no more work
-    uint32_t tile[32];                 // (page, KV head) tile of each block of the item (kItemBlocks <= 24 used)
+    uint32_t tile[32];                 // (page, KV head) tile of each block of the item (at most kItemBlocksMax used)
     uint8_t keep4[32];                 // bit h: query head h of the group keeps the block; 0 = skipped
     uint8_t rows[32];                  // valid tokens
 };
@@ -153,7 +162,7 @@ struct ItemSched {                                        // lives in the regist
 // units per class, kRowCap rows) the scheduling warp builds, per class, the number of draws before each row
 // counting only items that exist, so that no ticket is spent on a missing item.  Kept out of line: the scheduling
 // loop of the common case stays small.
-__device__ __noinline__ int2 plan_tables(const int32_t* seq_lens, int max_blocks, int units, int rows_small,
+__device__ __noinline__ int2 plan_tables(const int32_t* seq_lens, int max_blocks, int units, int rows_small, int item_blocks,
                                          unsigned long long hkv_magic, unsigned char* smem, int n_heavy, int rows,
                                          int lane) {
     int total_heavy = 0, total_light = 0;
@@ -169,7 +178,7 @@ __device__ __noinline__ int2 plan_tables(const int32_t* seq_lens, int max_blocks
             const int nb = (min(max(seq_lens[b], 0), max_blocks * kBlk) + kBlk - 1) / kBlk;
             const int s = rows_small * kSmallBlocks;
             const int items = nb <= s ? (nb + kSmallBlocks - 1) / kSmallBlocks
-                                      : rows_small + (nb - s + kItemBlocks - 1) / kItemBlocks;   // item_count
+                                      : rows_small + (nb - s + item_blocks - 1) / item_blocks;   // item_count
             const int start = max(rows - items, 0);   // == rows: the sequence is empty
             ustart[c * kUnitCache + u] = (unsigned short)start;
             if (start < rows) atomicAdd(&pref[c * (kRowCap + 1) + start], 1);
@@ -344,7 +353,7 @@ __device__ __forceinline__ void sched_role(const DecodeParams& p, unsigned char*
     sc.table = 2ll * (long long)p.len_stats[2] < (long long)p.units * rows && rows <= kRowCap &&
                sc.n_heavy <= kUnitCache && sc.n_light <= kUnitCache;
     if (sc.table) {
-        const int2 totals = plan_tables(p.seq_lens, p.max_blocks, p.units, p.rows_small, p.hkv_magic, smem, sc.n_heavy,
+        const int2 totals = plan_tables(p.seq_lens, p.max_blocks, p.units, p.rows_small, p.item_blocks, p.hkv_magic, smem, sc.n_heavy,
                                         rows, lane);
         sc.total_heavy = totals.x;
         sc.total_light = totals.y;

@@ -96,6 +96,7 @@ struct DecodeParams {
     int32_t* unit_list;      // fused path: heavy units from the front, light units from the back (workspace)
     int units;               // batch * Hkv
     int item_rows;           // fused path: work items per (sequence, KV head)
+    int item_blocks;         // fused path: blocks per full-size item (22 or 32)
     int rows_small;          // fused path: how many of them, counted from block 0, are half-size items
     unsigned long long units_magic, hkv_magic;   // reciprocals for fast_div
     uint8_t* kept_mask;      // nullable [B, Hq, max_blocks]
