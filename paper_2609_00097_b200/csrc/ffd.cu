@@ -469,8 +469,8 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
         atomicMax(&p.len_stats[0], (unsigned)nb);
         atomicMax(&p.len_stats[1], (unsigned)(p.max_blocks - nb));
         atomicAdd(&p.len_stats[2], (unsigned)item_count(p, nb));   // work items that exist
-        if (hinted > 0 && 2 * kept >= hinted) p.unit_list[atomicAdd(&p.class_counts[0], 1u)] = bg;
-        else p.unit_list[p.units - 1 - (int)atomicAdd(&p.class_counts[1], 1u)] = bg;
+        if (hinted > 0 && 2 * kept >= hinted) p.unit_list[atomicAdd(&p.class_counts[0], 1u)] = make_int2(bg, n);
+        else p.unit_list[p.units - 1 - (int)atomicAdd(&p.class_counts[1], 1u)] = make_int2(bg, n);
         FFD_TL(14, blockIdx.y == 0);
     }
 }
@@ -670,7 +670,7 @@ static Plan make_plan(const ffd_config* cfg, int batch, int max_blocks) {
     pl.off_mtilde = 256;
     pl.off_lens = align_up(pl.off_mtilde + heads * sizeof(float), 256);
     pl.off_units = align_up(pl.off_lens + (size_t)batch * sizeof(int32_t), 256);
-    pl.off_qrec = align_up(pl.off_units + (size_t)batch * cfg->num_kv_heads * sizeof(int32_t), 256);
+    pl.off_qrec = align_up(pl.off_units + (size_t)batch * cfg->num_kv_heads * sizeof(int2), 256);
     pl.off_ml = align_up(pl.off_qrec + (size_t)batch * cfg->num_kv_heads * kQrecBytes, 256);
     pl.off_acc = align_up(pl.off_ml + heads * pl.splits * 2 * sizeof(float), 256);
     pl.off_fml = align_up(pl.off_acc + heads * pl.splits * kD * sizeof(float), 256);
@@ -787,7 +787,7 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
     p.class_counts = reinterpret_cast<uint32_t*>(ws + 68);
     p.light_counter = reinterpret_cast<uint32_t*>(ws + 76);
     p.len_stats = reinterpret_cast<uint32_t*>(ws + 80);
-    p.unit_list = reinterpret_cast<int32_t*>(ws + pl.off_units);
+    p.unit_list = reinterpret_cast<int2*>(ws + pl.off_units);
     p.units = batch * cfg->num_kv_heads;
     p.item_rows = item_geometry(p.units, max_blocks).item_rows;
     p.rows_small = item_geometry(p.units, max_blocks).rows_small;

@@ -133,7 +133,7 @@ constexpr int kOffStageTile = kOffItems + kItemRing * (int)sizeof(ItemSlot);   /
 constexpr int kOffAbort = kOffStageTile + kNS * 4 * 4;
 constexpr int kOffAttendDone = kOffAbort + 16;                   // batches finished by each attend warp
 constexpr int kOffUnits = kOffAttendDone + 16;                   // first kUnitCache entries of each end of the unit list
-constexpr int kOffStart = kOffUnits + 2 * kUnitCache * 4;        // first row (16 bit) in which each cached unit has an item
+constexpr int kOffStart = kOffUnits + 2 * kUnitCache * 8;        // first row (16 bit) in which each cached unit has an item
 constexpr int kOffRowPref = kOffStart + 2 * kUnitCache * 2;      // per class: draws before each row, then the total
 constexpr int kFusedSmem = kOffRowPref + 2 * (kRowCap + 1) * 4;
 static_assert(kOffBars % 8 == 0 && kOffRing % 16 == 0 && kOffDesc % 16 == 0 && kOffQrec % 16 == 0, "alignment");
@@ -162,11 +162,10 @@ struct ItemSched {                                        // lives in the regist
 // units per class, kRowCap rows) the scheduling warp builds, per class, the number of draws before each row
 // counting only items that exist, so that no ticket is spent on a missing item.  Kept out of line: the scheduling
 // loop of the common case stays small.
-__device__ __noinline__ int2 plan_tables(const int32_t* seq_lens, int max_blocks, int units, int rows_small, int item_blocks,
-                                         unsigned long long hkv_magic, unsigned char* smem, int n_heavy, int rows,
-                                         int lane) {
+__device__ __noinline__ int2 plan_tables(int units, int rows_small, int item_blocks, unsigned char* smem, int n_heavy,
+                                         int rows, int lane) {
     int total_heavy = 0, total_light = 0;
-    const int* cache = reinterpret_cast<const int*>(smem + kOffUnits);
+    const int2* cache = reinterpret_cast<const int2*>(smem + kOffUnits);
     unsigned short* ustart = reinterpret_cast<unsigned short*>(smem + kOffStart);
     int* pref = reinterpret_cast<int*>(smem + kOffRowPref);
     for (int x = lane; x <= rows; x += 32) pref[x] = pref[kRowCap + 1 + x] = 0;
@@ -174,8 +173,7 @@ __device__ __noinline__ int2 plan_tables(const int32_t* seq_lens, int max_blocks
     for (int c = 0; c < 2; ++c) {
         const int n_class = c == 0 ? n_heavy : units - n_heavy;
         for (int u = lane; u < n_class; u += 32) {
-            const int b = (int)fast_div((unsigned)cache[c * kUnitCache + u], hkv_magic);
-            const int nb = (min(max(seq_lens[b], 0), max_blocks * kBlk) + kBlk - 1) / kBlk;
+            const int nb = (cache[c * kUnitCache + u].y + kBlk - 1) / kBlk;
             const int s = rows_small * kSmallBlocks;
             const int items = nb <= s ? (nb + kSmallBlocks - 1) / kSmallBlocks
                                       : rows_small + (nb - s + item_blocks - 1) / item_blocks;   // item_count
@@ -247,28 +245,31 @@ __device__ __forceinline__ int2 table_lookup(const unsigned char* smem, int c, i
 }
 
 // draw number k of a class -> work item
-__device__ __forceinline__ Item decode_item(const DecodeParams& p, const ItemSched& sc, const int* unit_cache,
+// (a unit-list entry is the pair (unit, clamped sequence length), so no length is fetched per item)
+__device__ __forceinline__ Item decode_item(const DecodeParams& p, const ItemSched& sc, const int2* unit_cache,
                                             bool heavy, int k, int2 via_table) {
     Item it;
-    int row, bg;
+    int row;
+    int2 un;
     if (sc.table) {
         row = via_table.x;
-        bg = unit_cache[(heavy ? 0 : kUnitCache) + via_table.y];
+        un = unit_cache[(heavy ? 0 : kUnitCache) + via_table.y];
     } else if (heavy) {   // heavy units sit at the front of the list, light units at its back (first ones cached in smem)
         row = (int)fast_div((unsigned)k, sc.magic_heavy);
         const int u = k - row * sc.n_heavy;
-        bg = u < kUnitCache ? unit_cache[u] : p.unit_list[u];
+        un = u < kUnitCache ? unit_cache[u] : p.unit_list[u];
     } else {
         row = (int)fast_div((unsigned)k, sc.magic_light);
         const int u = k - row * sc.n_light;
-        bg = u < kUnitCache ? unit_cache[kUnitCache + u] : p.unit_list[p.units - 1 - u];
+        un = u < kUnitCache ? unit_cache[kUnitCache + u] : p.unit_list[p.units - 1 - u];
     }
+    const int bg = un.x;
     row += sc.row_off;
     it.slot = row * p.units + bg;
     it.bg = bg;
     it.b = (int)fast_div((unsigned)bg, p.hkv_magic);
     it.g = bg - it.b * p.Hkv;
-    it.n = clamped_seq_len(p, it.b);
+    it.n = un.y;
     const int nb = (it.n + kBlk - 1) / kBlk;
     int cap;
     item_span(p, p.item_rows - 1 - row, it.blk0, cap);
@@ -340,7 +341,7 @@ __device__ __forceinline__ void sched_role(const DecodeParams& p, unsigned char*
     ItemSlot* items = reinterpret_cast<ItemSlot*>(smem + kOffItems);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffAbort);
     const volatile int* attend_done = reinterpret_cast<const volatile int*>(smem + kOffAttendDone);
-    const int* unit_cache = reinterpret_cast<const int*>(smem + kOffUnits);
+    const int2* unit_cache = reinterpret_cast<const int2*>(smem + kOffUnits);
     ItemSched sc;
     sc.n_heavy = min((int)p.class_counts[0], p.units);
     sc.n_light = p.units - sc.n_heavy;
@@ -353,8 +354,7 @@ __device__ __forceinline__ void sched_role(const DecodeParams& p, unsigned char*
     sc.table = 2ll * (long long)p.len_stats[2] < (long long)p.units * rows && rows <= kRowCap &&
                sc.n_heavy <= kUnitCache && sc.n_light <= kUnitCache;
     if (sc.table) {
-        const int2 totals = plan_tables(p.seq_lens, p.max_blocks, p.units, p.rows_small, p.item_blocks, p.hkv_magic, smem, sc.n_heavy,
-                                        rows, lane);
+        const int2 totals = plan_tables(p.units, p.rows_small, p.item_blocks, smem, sc.n_heavy, rows, lane);
         sc.total_heavy = totals.x;
         sc.total_light = totals.y;
     }
@@ -816,7 +816,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodePa
     pdl_wait();   // the pseudo-max kernel's outputs (unit list, class counts, query records) are needed from here on
     FFD_TL(1, threadIdx.x == 0);
     {   // shared-memory copy of both ends of the unit list (heavy units from the front, light units from the back)
-        int* cache = reinterpret_cast<int*>(smem + kOffUnits);
+        int2* cache = reinterpret_cast<int2*>(smem + kOffUnits);
         for (int u = threadIdx.x; u < min(p.units, kUnitCache); u += kFusedThreads) {
             cache[u] = p.unit_list[u];
             cache[kUnitCache + u] = p.unit_list[p.units - 1 - u];

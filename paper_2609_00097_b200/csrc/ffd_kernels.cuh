@@ -93,7 +93,8 @@ struct DecodeParams {
     uint32_t* class_counts;  // fused path: [0] heavy units, [1] light units found by the pseudo-max kernel (workspace)
     int32_t* bump_lens;      // append + decode: the caller's seq_lens, set to the new lengths by the combine kernel
     uint32_t* len_stats;     // fused path: [0] largest block count of the batch, [1] largest (max_blocks - block count), [2] items
-    int32_t* unit_list;      // fused path: heavy units from the front, light units from the back (workspace)
+    int2* unit_list;         // fused path: (unit, its clamped sequence length); heavy units from the front, light units
+                             // from the back (workspace)
     int units;               // batch * Hkv
     int item_rows;           // fused path: work items per (sequence, KV head)
     int item_blocks;         // fused path: blocks per full-size item (22 or 32)
