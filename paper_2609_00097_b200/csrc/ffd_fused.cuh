@@ -559,6 +559,15 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
             }
             break;
         }
+        // The prefetch cursor only moves when this warp has a block to fetch, so after items too short to reach the
+        // warp it lags behind; an entry more than a ring behind has been overwritten.  Everything of this warp's
+        // stream before this item has been issued, so the cursor may jump to the item's start.
+        if (ic.seq < seq) {
+            ic.seq = seq;
+            ic.it = it;
+            ic.lb = w0 - kScanners;
+            if (w0 < it.nblk) ic.pages = lane < it.nblk ? items[seq & (kItemRing - 1)].pages[lane] : -1;
+        }
         // start this warp's copies of the item's blocks, then wait for the item's query record
         if (w0 < it.nblk)
             while (issued < consumed + kRing && cursor_next(p, ic, items, ibars, w0, lane)) {

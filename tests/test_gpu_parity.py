@@ -459,6 +459,32 @@ def test_randomised_geometries(ffd, oracle):
         W.CONFIGS.pop("sweep", None)
 
 
+@pytest.mark.parametrize("B,Hkv,G,lens,paged", [
+    (600, 2, 2, (1, 300), True),      # most items end before scan warp 4's block, a few reach it
+    (1100, 1, 1, (64, 64), False),    # one-block items only
+    (300, 8, 1, (1, 700), True),      # items that end anywhere among the scan warps
+])
+def test_many_short_sequences(ffd, oracle, B, Hkv, G, lens, paged):
+    """Serving-size batches of short sequences: more (sequence, KV head) units than the scheduler caches in shared
+    memory, and more work items per CTA than its ring of published items holds, most of them too short to give every
+    scan warp a block (a warp that sits out a ring's worth of items must not look back at overwritten entries)."""
+    import paper_2609_00097_b200.workloads as W
+    recipe = dict(seed=77, B=B, Hq=G * Hkv, Hkv=Hkv, lens=lens, frac=0.02, amp=3.0, sink=True, deltas=(6.0,))
+    if paged:
+        recipe.update(paged=True, spare_pages=5)
+    try:
+        W.CONFIGS["many_short"] = recipe
+        w = make_workload("many_short")
+        dc = ffd.DeviceCache(w, ffd.Config(G * Hkv, Hkv))
+        codes, scales = check_quantize(ffd, oracle, w, dc)
+        for delta in (6.0, INF):
+            check_decode(ffd, oracle, w, dc, codes, scales, delta)
+            check_decode(ffd, oracle, w, dc, codes, scales, delta)   # a second pass sees a different ticket order
+        check_dense(ffd, oracle, w, dc)
+    finally:
+        W.CONFIGS.pop("many_short", None)
+
+
 # full-size configurations: the oracle checks a sample of (sequence, head) rows one by one
 FULL = [
     ("C2", dict(), 8),
