@@ -29,12 +29,20 @@
  *                                                                              (parity unpinned)
  *   - refinement uses the full 16-bit K (the two-term form of Sec. 3.3 equals q.k when the residual
  *     is exact), softmax over the kept tokens only
+ *   - optional 8-bit residual format (Sec. 3.1 "k -> {k^quant, k^res}", Alg. 1 Dequant, Sec. 3.3 two-term
+ *     score): the paper does not print the residual quantizer.  Reading: symmetric int8 on the grid
+ *     s/254 of the channel's own 2-bit scale s (the residual of a mid-rise level lies in [-s/2, s/2]),
+ *     code8 = clamp(rint(r * (254/s)), -127, 127), r = x - level*s, all three operations in IEEE
+ *     binary32 (the precision the code is decided in); refinement then uses
+ *     K^full = level*s + code8*s/254 in place of the 16-bit K                  (parity unpinned: the
+ *     grid is this file's choice; what is pinned is the error bound and the two-term identity)
  *
  * Layouts (all host pointers, row-major, innermost last):
  *   q        bf16 bits  [B, Hq, D]
  *   k_cache  bf16 bits  [num_pages, Hkv, BLK, D]      v_cache the same
  *   codes    u8 0..3    [num_pages, Hkv, BLK, D]      level = code - 1.5
  *   scales   fp16 bits  [num_pages, Hkv, D]
+ *   k_res    int8       [num_pages, Hkv, BLK, D]      residual in units of scale/254
  *   block_table int32   [B, max_blocks]  logical block -> physical page; NULL = b*max_blocks + blk
  *   seq_lens int32      [B]
  *   query head h belongs to KV head h / (Hq/Hkv).
@@ -172,6 +180,60 @@ int ffd_oracle_quantize(const uint16_t* k_cache, uint8_t* codes, uint16_t* scale
     return 0;
 }
 
+/* ---- Sec. 3.1: the 8-bit residual ------------------------------------------------------------- */
+
+/* Residual code of one element: x (bf16 bits), its 2-bit code and the channel's scale (fp16 bits).
+ * Every operation is a single IEEE binary32 operation (level*s is exact in binary32). */
+static int8_t residual_code(uint16_t xbits, uint8_t code, uint16_t sbits) {
+    float s = (float)fp16_value(sbits);
+    if (s == 0.0f) return 0;                      /* all-zero channel: nothing to refine */
+    float x = (float)bf16_value(xbits);
+    float level_s = ((float)code - 1.5f) * s;     /* exact: 11 significant bits times 1.5 or 0.5 */
+    float r = x - level_s;
+    float inv = 254.0f / s;
+    float t = rintf(r * inv);                     /* to nearest, ties to even */
+    if (t > 127.0f) t = 127.0f;
+    if (t < -127.0f) t = -127.0f;
+    return (int8_t)t;
+}
+
+/* Residual codes of every valid token, given the 2-bit codes and scales; padding rows get 0. */
+int ffd_oracle_quantize_residual(const uint16_t* k_cache, const uint8_t* codes, const uint16_t* scales, int8_t* k_res,
+                                 const int32_t* block_table, const int32_t* seq_lens, int B, int Hkv, int D, int BLK,
+                                 int max_blocks, int num_pages) {
+    for (int b = 0; b < B; ++b) {
+        int nb = (seq_lens[b] + BLK - 1) / BLK;
+        if (seq_lens[b] < 0 || nb > max_blocks) return 2;
+        for (int blk = 0; blk < nb; ++blk) {
+            int64_t page = page_of(block_table, b, blk, max_blocks);
+            if (page < 0 || page >= num_pages) return 3;
+        }
+    }
+    for (int b = 0; b < B; ++b) {
+        int nb = (seq_lens[b] + BLK - 1) / BLK;
+#pragma omp parallel for schedule(static) num_threads(g_threads)
+        for (int blk = 0; blk < nb; ++blk) {
+            int64_t page = page_of(block_table, b, blk, max_blocks);
+            int rows = valid_rows(seq_lens[b], blk, BLK);
+            for (int g = 0; g < Hkv; ++g) {
+                int64_t tile = page * Hkv + g;
+                for (int r = 0; r < BLK; ++r)
+                    for (int c = 0; c < D; ++c) {
+                        int64_t e = (tile * BLK + r) * D + c;
+                        k_res[e] = r < rows ? residual_code(k_cache[e], codes[e], scales[tile * D + c]) : 0;
+                    }
+            }
+        }
+    }
+    return 0;
+}
+
+/* Alg. 1 "Dequant": the key the refinement sees in the residual format. */
+static double dequant_full(uint8_t code, int8_t res, uint16_t sbits) {
+    double s = fp16_value(sbits);
+    return ((double)code - 1.5) * s + (double)res * s / 254.0;
+}
+
 /* ---- Alg. 1 for one (sequence, query head) ---------------------------------------------------- */
 
 typedef struct {
@@ -183,6 +245,7 @@ typedef struct {
     const uint8_t* forced_mask; /* nullable [B,Hq,max_blocks]: use these decisions instead of top-delta */
     double *out, *lse, *block_max, *mtilde;
     uint8_t* kept;
+    const int8_t* k_res;        /* nullable: refine from Dequant(codes, k_res) instead of the 16-bit K */
 } decode_args;
 
 static void softmax_attention_over_mask(const decode_args* a, int b, int h, const uint8_t* keep, double* out,
@@ -199,7 +262,12 @@ static void softmax_attention_over_mask(const decode_args* a, int b, int h, cons
         int rows = valid_rows(N, blk, BLK);
         for (int r = 0; r < rows; ++r) {
             double dot = 0.0;
-            for (int c = 0; c < D; ++c) dot += bf16_value(qv[c]) * bf16_value(a->k_cache[(tile * BLK + r) * D + c]);
+            for (int c = 0; c < D; ++c) {
+                int64_t e = (tile * BLK + r) * D + c;
+                double k = a->k_res ? dequant_full(a->codes[e], a->k_res[e], a->scales[tile * D + c])
+                                    : bf16_value(a->k_cache[e]);
+                dot += bf16_value(qv[c]) * k;
+            }
             s[blk * BLK + r] = a->sm_scale * dot;
             if (s[blk * BLK + r] > M) M = s[blk * BLK + r];
         }
@@ -279,14 +347,16 @@ static int check_geometry(const decode_args* a) {
 }
 
 /* Sparse decode step.  Rows of kept / block_max beyond a sequence's block count are left untouched.
+ * k_res: NULL = refine from the 16-bit K; else from the 2-bit + 8-bit reconstruction (k_cache is then unused).
  * units: nullable list of n_units (b, h) pairs to compute; NULL = all B*Hq pairs. */
 int ffd_oracle_decode(const uint16_t* q, const uint16_t* k_cache, const uint16_t* v_cache, const uint8_t* codes,
                       const uint16_t* scales, const int32_t* block_table, const int32_t* seq_lens, int B, int Hq,
                       int Hkv, int D, int BLK, int max_blocks, int num_pages, int n_sink, int n_local,
                       double sm_scale, double delta, const uint8_t* forced_mask, const int32_t* units, int n_units,
-                      double* out, double* lse, uint8_t* kept, double* block_max, double* mtilde) {
+                      double* out, double* lse, uint8_t* kept, double* block_max, double* mtilde, const int8_t* k_res) {
     decode_args a = {q, k_cache, v_cache, scales, codes, block_table, seq_lens, B, Hq, Hkv, D, BLK, max_blocks,
-                     num_pages, n_sink, n_local, sm_scale, delta, forced_mask, out, lse, block_max, mtilde, kept};
+                     num_pages, n_sink, n_local, sm_scale, delta, forced_mask, out, lse, block_max, mtilde, kept,
+                     k_res};
     int rc = check_geometry(&a);
     if (rc) return rc;
     if (isnan(delta) || delta < 0.0) return 4;
@@ -305,7 +375,7 @@ int ffd_oracle_dense(const uint16_t* q, const uint16_t* k_cache, const uint16_t*
                      const int32_t* seq_lens, int B, int Hq, int Hkv, int D, int BLK, int max_blocks, int num_pages,
                      double sm_scale, const int32_t* units, int n_units, double* out, double* lse) {
     decode_args a = {q, k_cache, v_cache, NULL, NULL, block_table, seq_lens, B, Hq, Hkv, D, BLK, max_blocks,
-                     num_pages, 0, 0, sm_scale, INFINITY, NULL, out, lse, NULL, NULL, NULL};
+                     num_pages, 0, 0, sm_scale, INFINITY, NULL, out, lse, NULL, NULL, NULL, NULL};
     int rc = check_geometry(&a);
     if (rc) return rc;
     int total = units ? n_units : B * Hq;

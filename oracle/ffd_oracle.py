@@ -99,6 +99,25 @@ def quantize(k_cache, block_table, seq_lens, max_blocks):
     return codes, scales
 
 
+def quantize_residual(k_cache, codes, scales, block_table, seq_lens, max_blocks):
+    """Sec. 3.1 residual: int8 [pages,Hkv,BLK,D], the part of K the 2-bit level misses, in units of scale/254
+    (this file's reading; the paper prints no residual quantizer).  Padding rows and unmapped tiles are 0."""
+    k_cache = _u16(k_cache)
+    scales = _u16(scales)
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    P, Hkv, BLK, D = k_cache.shape
+    seq_lens = _i32(seq_lens)
+    block_table = _i32(block_table)
+    k_res = np.zeros((P, Hkv, BLK, D), dtype=np.int8)
+    rc = lib().ffd_oracle_quantize_residual(
+        _ptr(k_cache, ctypes.c_uint16), _ptr(codes, ctypes.c_uint8), _ptr(scales, ctypes.c_uint16),
+        _ptr(k_res, ctypes.c_int8), _ptr(block_table, ctypes.c_int32), _ptr(seq_lens, ctypes.c_int32), len(seq_lens),
+        Hkv, D, BLK, int(max_blocks), P)
+    if rc:
+        raise ValueError(f"ffd_oracle_quantize_residual: geometry error {rc}")
+    return k_res
+
+
 @dataclass
 class DecodeResult:
     out: np.ndarray        # float64 [B, Hq, D]
@@ -118,8 +137,10 @@ def _units(units):
 
 
 def decode(q, k_cache, v_cache, codes, scales, block_table, seq_lens, max_blocks, delta, *, n_sink=1, n_local=16,
-           sm_scale=None, forced_mask=None, units=None) -> DecodeResult:
+           sm_scale=None, forced_mask=None, units=None, k_res=None) -> DecodeResult:
     """Alg. 1: approximate scores -> pseudo-max -> top-delta -> exact attention over kept blocks.
+
+    ``k_res`` (int8, from ``quantize_residual``): refine from Dequant(codes, k_res) instead of the 16-bit K.
 
     ``units``: optional list of (b, h) pairs; only those rows of the result are computed (others stay at
     their fill values: out 0, lse nan, block_max -inf).  ``forced_mask`` replaces the top-delta decisions.
@@ -142,13 +163,15 @@ def decode(q, k_cache, v_cache, codes, scales, block_table, seq_lens, max_blocks
     mt = np.full((B, Hq), np.nan, dtype=np.float64)
     fm = None if forced_mask is None else np.ascontiguousarray(forced_mask, dtype=np.uint8)
     u, nu = _units(units)
+    kr = None if k_res is None else np.ascontiguousarray(k_res, dtype=np.int8)
+    assert kr is None or kr.shape == k_cache.shape
     rc = lib().ffd_oracle_decode(
         _ptr(q, ctypes.c_uint16), _ptr(k_cache, ctypes.c_uint16), _ptr(v_cache, ctypes.c_uint16),
         _ptr(codes, ctypes.c_uint8), _ptr(scales, ctypes.c_uint16), _ptr(block_table, ctypes.c_int32),
         _ptr(seq_lens, ctypes.c_int32), B, Hq, Hkv, D, BLK, int(max_blocks), P, int(n_sink), int(n_local),
         ctypes.c_double(sm_scale), ctypes.c_double(delta), _ptr(fm, ctypes.c_uint8), _ptr(u, ctypes.c_int32), nu,
         _ptr(out, ctypes.c_double), _ptr(lse, ctypes.c_double), _ptr(kept, ctypes.c_uint8),
-        _ptr(bm, ctypes.c_double), _ptr(mt, ctypes.c_double))
+        _ptr(bm, ctypes.c_double), _ptr(mt, ctypes.c_double), _ptr(kr, ctypes.c_int8))
     if rc:
         raise ValueError(f"ffd_oracle_decode: error {rc}")
     return DecodeResult(out, lse, kept, bm, mt)

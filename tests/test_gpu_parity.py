@@ -485,6 +485,34 @@ def test_many_short_sequences(ffd, oracle, B, Hkv, G, lens, paged):
         W.CONFIGS.pop("many_short", None)
 
 
+@pytest.mark.parametrize("lens,short", [((1048576, 1048576), None), ((700000, 700000), 77)])
+def test_very_long_contexts_on_sampled_heads(ffd, oracle, lens, short):
+    """A million-token sequence (16384 blocks, four times the longest configuration), and a two-sequence paged batch
+    of 700000 and 77 tokens; sampled heads against the oracle, scales of the whole cache bit for bit."""
+    import paper_2609_00097_b200.workloads as W
+    recipe = dict(seed=91, B=1 if short is None else 2, Hq=32, Hkv=8, lens=lens, frac=0.005, amp=3.0, sink=True,
+                  deltas=(6.0,))
+    if short is not None:
+        recipe.update(paged=True, spare_pages=3)
+    try:
+        W.CONFIGS["very_long"] = recipe
+        w = make_workload("very_long")
+    finally:
+        W.CONFIGS.pop("very_long", None)
+    if short is not None:
+        w.seq_lens[1] = short
+    dc = ffd.DeviceCache(w)
+    dc.quantize()
+    codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
+    _, mapped = valid_row_mask(w)
+    assert np.array_equal(dc.k_scales.cpu().view(torch.int16).numpy().view(np.uint16)[mapped], scales[mapped])
+    units = [(0, 0), (0, 13), (w.B - 1, 31)]
+    for delta in (6.0, INF):
+        check_decode(ffd, oracle, w, dc, codes, scales, delta, units=units)
+    check_dense(ffd, oracle, w, dc, units=units[:1])
+    assert ffd.ffd_read_device_status(dc.workspace) == 0
+
+
 # full-size configurations: the oracle checks a sample of (sequence, head) rows one by one
 FULL = [
     ("C2", dict(), 8),

@@ -159,6 +159,123 @@ def test_padding_rows_do_not_move_the_scale(oracle):
 # hand-worked example (tests/golden/worked_example.json)
 # ---------------------------------------------------------------------------------------------------------
 
+# ---------------------------------------------------------------------------------------------------------
+# Sec. 3.1 / Alg. 1 Dequant / Sec. 3.3 two-term score: the 8-bit residual
+# ---------------------------------------------------------------------------------------------------------
+
+def _full_key(codes, scales, k_res):
+    """Alg. 1 Dequant, by numpy: level * s + residual * s / 254."""
+    S = scales.view(np.float16).astype(np.float64)[:, :, None, :]
+    return (codes.astype(np.float64) - 1.5) * S + k_res.astype(np.float64) * S / 254.0
+
+
+def test_residual_brings_the_key_back_to_half_a_step(oracle):
+    """Sec. 3.1: kept keys are rebuilt to near-16-bit precision.  With an 8-bit symmetric grid over the 2-bit cell
+    [-s/2, s/2] every valid element comes back to within half a step, s/508 (+ the binary32 roundings, 1e-6 s):
+    about 1/760 of the block's largest key, 250 times closer than the 2-bit level alone.  A wrong sign, channel or
+    token index in the residual breaks the bound at once."""
+    w = make_workload("C1", N=1024, tail=13)
+    codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
+    k_res = oracle.quantize_residual(w.bits("k_cache"), codes, scales, w.block_table, w.seq_lens, w.max_blocks)
+    assert k_res.dtype == np.int8 and k_res.min() >= -127
+    K = bits_to_f64(w.bits("k_cache"))
+    full = _full_key(codes, scales, k_res)
+    S = np.broadcast_to(scales.view(np.float16).astype(np.float64)[:, :, None, :], K.shape)
+    n = int(w.seq_lens[0])
+    for blk in range(w.num_blocks(0)):
+        rows = min(64, n - 64 * blk)
+        err = np.abs(full[blk, :, :rows] - K[blk, :, :rows])
+        assert np.all(err <= S[blk, :, :rows] * (1.0 / 508.0 + 1e-6))
+        assert np.all(k_res[blk, :, rows:] == 0)                          # padding rows
+        # the grid is used: codes reach the ends of the range and are not all tiny
+        if rows == 64:
+            assert np.abs(k_res[blk]).max() >= 120
+    # and the residual really is the finer part: the 2-bit level alone is ~ s/4 off on average
+    lvl_err = np.abs((codes.astype(np.float64) - 1.5) * S - K)[: w.num_blocks(0) - 1]
+    res_err = np.abs(full - K)[: w.num_blocks(0) - 1]
+    assert res_err.mean() < lvl_err.mean() / 100
+
+
+def test_two_term_score_equals_the_exact_score_when_the_residual_is_exact(oracle):
+    """Sec. 3.3: s_final = (q.k_quant + q.k_res) / sqrt(d) is the Dequant form of Alg. 1, and it equals q.k / sqrt(d)
+    when the residual loses nothing.  Construction: every channel's largest key is +-0.75, so s = 0.5 and the levels
+    are +-0.25, +-0.75; every key is a level plus -127, 0 or +127 residual steps of s / 254, i.e. a multiple of 0.25
+    (a bf16 value).  The test checks these premises itself, then asks for identical results from both refinements."""
+    rng = np.random.default_rng(12)
+    P, Hkv, G = 6, 2, 2
+    s = 0.5
+    level = rng.choice(CODEBOOK, size=(P, Hkv, 64, 128)) * s
+    steps = rng.choice(np.array([-127, 0, 127]), size=(P, Hkv, 64, 128))
+    K = np.clip(level + steps * s / 254.0, -0.75, 0.75)
+    rows = rng.integers(0, 64, size=(P, Hkv, 128))
+    pp, hh, cc = np.meshgrid(np.arange(P), np.arange(Hkv), np.arange(128), indexing="ij")
+    K[pp, hh, rows, cc] = 0.75 * rng.choice([-1.0, 1.0], size=(P, Hkv, 128))
+    kb = bf16_bits(K)
+    assert np.array_equal(bits_to_f64(kb), K)                  # premise: every key is a bf16 value
+    seq = np.array([64 * P], dtype=np.int32)
+    codes, scales = oracle.quantize(kb, None, seq, P)
+    assert np.all(scales.view(np.float16) == np.float16(0.5))  # premise: s = 0.5 in every channel
+    k_res = oracle.quantize_residual(kb, codes, scales, None, seq, P)
+    assert set(np.unique(k_res).tolist()) == {-127, 0, 127}
+    assert np.array_equal(_full_key(codes, scales, k_res), K)  # premise: the residual is exact
+    q = bf16_bits(rng.standard_normal((1, Hkv * G, 128)) * 4.0)
+    v = bf16_bits(rng.standard_normal((P, Hkv, 64, 128)))
+    for delta in (0.5, 6.0, INF):
+        a = oracle.decode(q, kb, v, codes, scales, None, seq, P, delta, n_sink=1, n_local=1)
+        b = oracle.decode(q, kb, v, codes, scales, None, seq, P, delta, n_sink=1, n_local=1, k_res=k_res)
+        assert np.array_equal(a.kept, b.kept)
+        assert np.abs(a.out - b.out).max() < 1e-12 and np.abs(a.lse - b.lse).max() < 1e-12
+    # and a residual that is wrong by one step in one element is seen
+    k_bad = k_res.copy()
+    k_bad[0, 0, 0, 0] += 1 if k_bad[0, 0, 0, 0] < 127 else -1
+    c = oracle.decode(q, kb, v, codes, scales, None, seq, P, INF, n_sink=1, n_local=1, k_res=k_bad)
+    assert np.abs(c.lse[0, :G] - a.lse[0, :G]).max() > 0
+
+
+def test_residual_refinement_stays_within_its_logit_bound_of_the_exact_one(oracle):
+    """With an inexact residual every refined logit moves by at most sm * sum_c |q_c| s_c / 508 (half a step per
+    channel); softmax weights then move by at most a factor exp(2 * that), so the output stays close."""
+    w = make_workload("C1", N=2048, tail=7)
+    codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
+    k_res = oracle.quantize_residual(w.bits("k_cache"), codes, scales, w.block_table, w.seq_lens, w.max_blocks)
+    a = oracle.decode(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), codes, scales, w.block_table, w.seq_lens,
+                      w.max_blocks, 6.0)
+    b = oracle.decode(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), codes, scales, w.block_table, w.seq_lens,
+                      w.max_blocks, 6.0, k_res=k_res)
+    assert np.array_equal(a.kept, b.kept) and np.array_equal(a.block_max, b.block_max)   # selection is untouched
+    q = np.abs(bits_to_f64(w.bits("q")))[0]                                              # [Hq, D]
+    S = scales.view(np.float16).astype(np.float64)                                       # [pages, Hkv, D]
+    G = w.Hq // w.Hkv
+    bound = max(float((q[h] * S[:, h // G].max(axis=0)).sum()) for h in range(w.Hq)) / 508.0 / math.sqrt(128)
+    assert bound < 0.1                                     # worst case; errors of random sign stay far below it
+    vmax = np.abs(bits_to_f64(w.bits("v_cache"))).max()
+    assert np.abs(a.lse - b.lse).max() <= bound + 1e-12
+    assert np.abs(a.lse - b.lse).max() <= bound / 10
+    assert np.abs(a.out - b.out).max() <= (math.exp(2 * bound) - 1) * vmax
+    assert np.abs(a.out - b.out).max() > 0                                               # and it is not the same path
+
+
+def test_residual_worked_column_zero_channel_and_saturation(oracle):
+    """One column by hand.  Largest key a = 3.015625: s = fp16(a / 1.5) = 2.009765625 (rounded down), step s / 254.
+    a -> level 1.5 s = 3.0146484, 0.12 steps short: 0.  2.0 < s -> level 0.5 s = 1.0048828, 125.77 steps: 126.
+    0 -> level +0.5 s, exactly -127 steps.  0.125 -> -111.2 steps: -111.  An all-zero channel has s = 0: residual 0.
+    A key beyond the saturated scale (|x| > 1.5 * 65504) pins the residual at +-127 instead of wrapping."""
+    col = bf16_bits(np.array([3.015625, -3.015625, 2.0, -2.0, 0.0] + [0.125] * 59))
+    k, seq = _one_column(col)
+    codes, scales = oracle.quantize(k, None, seq, 1)
+    assert float(scales.view(np.float16)[0, 0, 0]) == 2.009765625
+    res = oracle.quantize_residual(k, codes, scales, None, seq, 1)[0, 0, :, 0]
+    assert res[:5].tolist() == [0, 0, 126, -126, -127] and np.all(res[5:] == -111)
+    k, seq = _one_column(bf16_bits(np.zeros(64)))
+    codes, scales = oracle.quantize(k, None, seq, 1)
+    assert np.all(oracle.quantize_residual(k, codes, scales, None, seq, 1) == 0)
+    k, seq = _one_column(bf16_bits(np.array([1.0e6, -1.0e6, 98304.0, 1.0] + [0.0] * 60)))
+    codes, scales = oracle.quantize(k, None, seq, 1)
+    assert float(scales.view(np.float16)[0, 0, 0]) == 65504.0
+    res = oracle.quantize_residual(k, codes, scales, None, seq, 1)[0, 0, :, 0]
+    assert res[0] == 127 and res[1] == -127 and res[2] == 0     # 98304 - 98256 = 48 = 0.19 steps of 65504 / 254
+
+
 @pytest.fixture(scope="module")
 def golden():
     with open(os.path.join(HERE, "golden", "worked_example.json")) as f:
