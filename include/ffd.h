@@ -97,6 +97,23 @@ ffd_status ffd_quantize_keys(const ffd_config* cfg, const void* k_cache, void* k
                              int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages, void* stream);
 
 /*
+ * 8-bit residual of the keys (Sec. 3.1: the key cache is split into 2-bit thumbnails k_quant and 8-bit residuals
+ * k_res; Alg. 1 "Dequant").  The paper prints no residual quantizer; this one puts the remainder of every valid
+ * element on a symmetric 8-bit grid over the cell of its 2-bit level, whose half-width is s/2 (s = the channel's
+ * scale in k_scales):
+ *   r = x - (code - 1.5) * s,   k_res = clamp(rint(r * (254 / s)), -127, 127),   0 when s = 0
+ * with every operation one IEEE binary32 operation (round to nearest even).  The rebuilt key
+ * (code - 1.5) * s + k_res * s / 254 is within s/508 of x.  Rows past the sequence end get 0.
+ *   k_res  int8 [num_pages, num_kv_heads, 64, 128] (device, row-major, same indexing as k_cache)
+ * Call after ffd_quantize_keys on the same stream with the same block_table / seq_lens / first_token: it reads
+ * k_cache and k_scales and (re)writes k_res of the blocks that hold a token in [first_token[b], seq_lens[b]).
+ * Other arguments, skipped pages, clamping and host errors as for ffd_quantize_keys.
+ */
+ffd_status ffd_quantize_residual(const ffd_config* cfg, const void* k_cache, const void* k_scales, void* k_res,
+                                 const int32_t* block_table, const int32_t* seq_lens, const int32_t* first_token,
+                                 int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages, void* stream);
+
+/*
  * Cache append for one decode step, all indices on the device (Sec. 3.3: a cache that a captured graph can replay
  * needs tensor indices instead of host-side lengths; App. A.1 for the quantizer).  For every sequence b with
  * pos = seq_lens[b] < max_blocks_per_seq*64: the rows k_new[b, g, :] and v_new[b, g, :] (bf16 [B, Hkv, 128], device)
@@ -138,6 +155,23 @@ ffd_status ffd_decode(const ffd_config* cfg, const void* q, const void* k_cache,
                       const int32_t* seq_lens, int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages,
                       float delta, void* out, float* lse, uint8_t* kept_mask, float* block_max, void* workspace,
                       size_t workspace_bytes, void* stream);
+
+/*
+ * The same step on the 2 + 8 bit key format (Sec. 3.3, "Fine-grained refinement": a block that passes the filter
+ * loads its 8-bit residual keys and its values; s_final = (q . k_quant + q . k_res) / sqrt(d), both dot products
+ * accumulated without a full-precision key).  Selection is exactly ffd_decode's; the refined logit of a kept token is
+ *   sm * sum_c q[c] * ((code - 1.5) * s[c] + k_res[t,c] * s[c] / 254)
+ * so a kept block costs 8 KB of k_res + 16 KB of V (plus its 2.3 KB of thumbnails, normally still in L2) instead of
+ * 32 KB, and the 16-bit keys are not read at all.  k_res as written by ffd_quantize_residual; every other argument,
+ * the outputs and the error behaviour as for ffd_decode.  Arithmetic: q . k_quant on the tensor cores as in the
+ * scan (exact fp16 products, fp32 accumulation); q . k_res with int8 tensor-core products of k_res and q[c] * s[c]
+ * split into two 8-bit digits (relative error below 2^-15 of the largest |q[c] * s[c]| per channel).
+ */
+ffd_status ffd_decode_residual(const ffd_config* cfg, const void* q, const void* k_res, const void* v_cache,
+                               const void* k_quant, const void* k_scales, const int32_t* block_table,
+                               const int32_t* seq_lens, int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages,
+                               float delta, void* out, float* lse, uint8_t* kept_mask, float* block_max,
+                               void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * One serving step in a single call: ffd_append_kv followed by ffd_decode on the lengthened sequences, with the

@@ -96,6 +96,75 @@ __global__ void __launch_bounds__(128) quantize_kernel(QuantParams p) {
     }
 }
 
+// ---- 8-bit residual (Sec. 3.1: k -> {k_quant, k_res}) ------------------------------------------------------
+// For every valid element: the part of the key its 2-bit level misses, on the grid s / 254 of the channel's own
+// scale (a mid-rise level leaves a remainder in [-s/2, s/2]): code8 = clamp(rint((x - level * s) * (254 / s))),
+// each operation one IEEE binary32 operation; s = 0 (all-zero channel) and padding rows give 0.  The level is
+// recomputed from x and the stored scale with the quantizer's own comparison, so the codes need not be unpacked.
+// Runs after the quantizer (it reads the scales); row-major int8 [page][KV head][64][128].
+struct ResidualParams {
+    const __nv_bfloat16* k_cache;
+    const __half* k_scales;
+    int8_t* k_res;
+    const int32_t* block_table;
+    const int32_t* seq_lens;
+    const int32_t* first_token;
+    int Hkv, max_blocks, num_pages;
+};
+
+__device__ __forceinline__ int residual_code(float x, float s, float inv) {
+    const float level_s = __fmul_rn((float)quant_code(x, s) - 1.5f, s);   // exact
+    float t = rintf(__fmul_rn(__fsub_rn(x, level_s), inv));
+    t = fminf(fmaxf(t, -127.f), 127.f);
+    return s == 0.f ? 0 : (int)t;
+}
+
+__global__ void __launch_bounds__(128) residual_kernel(ResidualParams p) {
+    const int g = blockIdx.y, b = blockIdx.z;
+    pdl_launch_dependents();
+    pdl_wait();
+    int n = p.seq_lens[b];
+    const int cap = p.max_blocks * kBlk;
+    n = n < 0 ? 0 : (n > cap ? cap : n);
+    const int nb = (n + kBlk - 1) / kBlk;
+    const int first = p.first_token ? max(p.first_token[b], 0) / kBlk : 0;
+    __shared__ __align__(16) __nv_bfloat16 sk[kBlk * kD];
+    __shared__ float ss[kD], sinv[kD];
+    const int tid = threadIdx.x;
+    for (int blk = first + blockIdx.x; blk < nb; blk += gridDim.x) {
+        const int page = p.block_table ? p.block_table[(size_t)b * p.max_blocks + blk] : b * p.max_blocks + blk;
+        if (page < 0 || page >= p.num_pages) continue;
+        const int rows = min(kBlk, n - blk * kBlk);
+        const size_t tile = (size_t)page * p.Hkv + g;
+        const uint4* src = reinterpret_cast<const uint4*>(p.k_cache + tile * kBlk * kD);
+        uint4* dst = reinterpret_cast<uint4*>(sk);
+        __syncthreads();   // the previous block's tile is no longer needed
+#pragma unroll
+        for (int x = 0; x < 8; ++x) dst[tid + 128 * x] = ldg_stream(src + tid + 128 * x);
+        {
+            const float s = __half2float(p.k_scales[tile * kD + tid]);
+            ss[tid] = s;
+            sinv[tid] = __fdiv_rn(254.f, s);
+        }
+        __syncthreads();
+        uint4* out = reinterpret_cast<uint4*>(p.k_res + tile * kBlk * kD);
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {   // 16 consecutive channels of one token per thread and pass
+            const int chunk = tid + 128 * x, row = chunk >> 3, c0 = (chunk & 7) * 16;
+            uint32_t w[4] = {0u, 0u, 0u, 0u};
+            if (row < rows) {
+#pragma unroll
+                for (int u = 0; u < 16; ++u) {
+                    const int c = c0 + u;
+                    const int code = residual_code(__bfloat162float(sk[row * kD + c]), ss[c], sinv[c]);
+                    w[u >> 2] |= (uint32_t)(code & 0xff) << (8 * (u & 3));
+                }
+            }
+            out[chunk] = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+    }
+}
+
 // ---- whole-cache quantizer ---------------------------------------------------------------------------------
 // The same arithmetic as quantize_tile, organised for bandwidth: per element the plain routine spends ~9
 // instructions (16-bit shared-memory reads, conversions, two compares, selects, shifts) and is instruction-bound at
@@ -736,10 +805,10 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
                              const int32_t* block_table, const int32_t* seq_lens, int batch, int max_blocks,
                              int num_pages, float delta, void* out, float* lse, uint8_t* kept_mask,
                              float* block_max, void* workspace, size_t workspace_bytes, void* stream,
-                             const AppendParams* append = nullptr) {
+                             const AppendParams* append = nullptr, const void* k_res = nullptr) {
     ffd_status st = check_config(cfg);
     if (st) return st;
-    if (!q || !k_cache || !v_cache || !seq_lens || !out || !workspace) return FFD_ERR_NULL;
+    if (!q || (!k_cache && !k_res) || !v_cache || !seq_lens || !out || !workspace) return FFD_ERR_NULL;
     if (sparse && (!k_quant || !k_scales)) return FFD_ERR_NULL;
     st = check_geometry(batch, max_blocks, num_pages);
     if (st) return st;
@@ -747,7 +816,8 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
     if ((double)num_pages * cfg->num_kv_heads >= 2147483648.0) return FFD_ERR_SHAPE;
     if ((long)batch * cfg->num_kv_heads >= 65536L) return FFD_ERR_SHAPE;   // fast_div: items * units < 2^48
     if (sparse && (isnan(delta) || delta < 0.f)) return FFD_ERR_DELTA;
-    const void* ptrs[] = {q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, out, lse, block_max, workspace};
+    const void* ptrs[] = {q, k_cache, k_res, v_cache, k_quant, k_scales, block_table, seq_lens, out, lse, block_max,
+                          workspace};
     for (const void* ptr : ptrs)
         if (ptr && misaligned(ptr)) return FFD_ERR_ALIGN;
     const Plan pl = make_plan(cfg, batch, max_blocks);
@@ -757,6 +827,7 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
     memset(&p, 0, sizeof p);
     p.q = static_cast<const __nv_bfloat16*>(q);
     p.k_cache = static_cast<const __nv_bfloat16*>(k_cache);
+    p.k_res = static_cast<const int8_t*>(k_res);
     p.v_cache = static_cast<const __nv_bfloat16*>(v_cache);
     p.k_quant = static_cast<const uint8_t*>(k_quant);
     p.k_scales = static_cast<const __half*>(k_scales);
@@ -807,7 +878,8 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
         int dev = 0, sms = 0;
         if (cudaGetDevice(&dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-            cudaFuncSetAttribute(fused_sparse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem) != cudaSuccess)
+            cudaFuncSetAttribute(fused_sparse_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem) != cudaSuccess ||
+            cudaFuncSetAttribute(fused_sparse_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem) != cudaSuccess)
             return FFD_ERR_CUDA;
         // the work counters and class counts at ws + 64 are zero here: ffd_workspace_init zeroes them and the
         // combine kernel of every call leaves them zeroed for the next one
@@ -822,7 +894,8 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
                        static_cast<int32_t*>(nullptr));
         }
         if (prof) cudaEventRecord(g_prof_start, s);
-        launch_pdl(fused_sparse_kernel, dim3(min(p.total_items, sms)), dim3(kFusedThreads), kFusedSmem, s, p);
+        launch_pdl(k_res ? fused_sparse_kernel<true> : fused_sparse_kernel<false>, dim3(min(p.total_items, sms)),
+                   dim3(kFusedThreads), kFusedSmem, s, p);
         if (prof) cudaEventRecord(g_prof_stop, s);
         launch_pdl(combine_kernel<true>, dim3(p.Hq, batch, combine_split(p.Hq * batch, (long)p.item_rows * kNA)),
                    dim3(combine_threads(p.Hq * batch)), 0, s, p);
@@ -914,6 +987,31 @@ ffd_status ffd_quantize_keys(const ffd_config* cfg, const void* k_cache, void* k
     return launch_status();
 }
 
+ffd_status ffd_quantize_residual(const ffd_config* cfg, const void* k_cache, const void* k_scales, void* k_res,
+                                 const int32_t* block_table, const int32_t* seq_lens, const int32_t* first_token,
+                                 int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages, void* stream) {
+    ffd_status st = check_config(cfg);
+    if (st) return st;
+    if (!k_cache || !k_scales || !k_res || !seq_lens) return FFD_ERR_NULL;
+    st = check_geometry(batch, max_blocks_per_seq, num_pages);
+    if (st) return st;
+    if (cfg->num_kv_heads > 65535) return FFD_ERR_SHAPE;
+    const void* ptrs[] = {k_cache, k_scales, k_res, block_table, seq_lens, first_token};
+    for (const void* ptr : ptrs)
+        if (ptr && misaligned(ptr)) return FFD_ERR_ALIGN;
+    ResidualParams p{static_cast<const __nv_bfloat16*>(k_cache), static_cast<const __half*>(k_scales),
+                     static_cast<int8_t*>(k_res), block_table, seq_lens, first_token,
+                     cfg->num_kv_heads, max_blocks_per_seq, num_pages};
+    // as in ffd_quantize_keys: every CTA walks its share of the blocks; two per (sequence, KV head) when only the
+    // tail block is redone, else enough to fill the GPU several times over
+    long x = first_token ? 2 : (16 * 148 + (long)batch * cfg->num_kv_heads - 1) / ((long)batch * cfg->num_kv_heads);
+    if (x > max_blocks_per_seq) x = max_blocks_per_seq;
+    if (x < 1) x = 1;
+    launch_pdl(residual_kernel, dim3((unsigned)x, cfg->num_kv_heads, batch), dim3(128), 0,
+               static_cast<cudaStream_t>(stream), p);
+    return launch_status();
+}
+
 ffd_status ffd_append_kv(const ffd_config* cfg, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
                          void* k_quant, void* k_scales, const int32_t* block_table, int32_t* seq_lens, int32_t batch,
                          int32_t max_blocks_per_seq, int32_t num_pages, void* workspace, size_t workspace_bytes,
@@ -947,6 +1045,17 @@ ffd_status ffd_decode(const ffd_config* cfg, const void* q, const void* k_cache,
     return run_decode(true, cfg, q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, batch,
                       max_blocks_per_seq, num_pages, delta, out, lse, kept_mask, block_max, workspace,
                       workspace_bytes, stream);
+}
+
+ffd_status ffd_decode_residual(const ffd_config* cfg, const void* q, const void* k_res, const void* v_cache,
+                               const void* k_quant, const void* k_scales, const int32_t* block_table,
+                               const int32_t* seq_lens, int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages,
+                               float delta, void* out, float* lse, uint8_t* kept_mask, float* block_max,
+                               void* workspace, size_t workspace_bytes, void* stream) {
+    if (!k_res) return FFD_ERR_NULL;
+    return run_decode(true, cfg, q, nullptr, v_cache, k_quant, k_scales, block_table, seq_lens, batch,
+                      max_blocks_per_seq, num_pages, delta, out, lse, kept_mask, block_max, workspace,
+                      workspace_bytes, stream, nullptr, k_res);
 }
 
 ffd_status ffd_append_decode(const ffd_config* cfg, const void* k_new, const void* v_new, const void* q, void* k_cache,

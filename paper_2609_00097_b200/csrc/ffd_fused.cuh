@@ -686,6 +686,9 @@ __device__ __forceinline__ unsigned my_entries(const BatchDesc& d, int nblk, int
     return __ballot_sync(kFull, is_kept && (rank & (kNA - 1)) == a);
 }
 
+// RES: the 2 + 8 bit key format -- the K slot receives the block's residual tile, codes and scales instead of its
+// 16-bit keys
+template <bool RES>
 __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char* smem, int a, int lane) {
     const int r = lane >> 2, j = lane & 3;
     const uint32_t kslot = smem_u32(smem) + kOffSlots + a * 2 * kSlotBytes;
@@ -702,6 +705,7 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
     int issued_bi = -1, issued_lb = -1;   // block whose K/V copies are already in flight
     bool ok = true;
     AttendState st;
+    uint32_t qb[RES ? 16 : 1];
     FFD_ACC_DECL;
     for (int bi = 0; ok; ++bi) {
         const int slot = bi & (kNB - 1), use = bi / kNB;
@@ -719,20 +723,28 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
         unsigned mine = my_entries(d, it.nblk, (a + bi) & (kNA - 1), lane);
         const bool any = mine != 0;
         FFD_ACC(6);
-        if (any) attend_setup(st, p.q + ((size_t)it.b * p.Hq + (size_t)it.g * p.G) * kD, p.G, lane);
+        if (any) {
+            if constexpr (RES)
+                attend_setup_res(st, qb, p, it.b, it.g,
+                                 reinterpret_cast<const uint4*>(p.qrec + (size_t)(it.b * p.Hkv + it.g) * kQrecBytes), lane);
+            else attend_setup(st, p.q + ((size_t)it.b * p.Hq + (size_t)it.g * p.G) * kD, p.G, lane);
+        }
         FFD_TL(11, a == 0 && lane == 0 && any);
         FFD_ACC(2);
         while (mine && ok) {
             const int lb = __ffs(mine) - 1;
             mine &= mine - 1;
             if (!(issued_bi == bi && issued_lb == lb)) {
-                tile_copy_async(kslot, kbase + (size_t)d.tile[lb] * kTileVec, lane, kbar);
+                if constexpr (RES) res_copy_async(kslot, p, d.tile[lb], lane, kbar);
+                else tile_copy_async(kslot, kbase + (size_t)d.tile[lb] * kTileVec, lane, kbar);
                 tile_copy_async(vslot, vbase + (size_t)d.tile[lb] * kTileVec, lane, vbar);
             }
             // the next block this warp will attend: in this batch, else in the next one if it is already published
             const uint4 *next_k = nullptr, *next_v = nullptr;
+            int next_tile = -1;
             if (mine) {
                 const int nlb = __ffs(mine) - 1;
+                next_tile = (int)d.tile[nlb];
                 next_k = kbase + (size_t)d.tile[nlb] * kTileVec;
                 next_v = vbase + (size_t)d.tile[nlb] * kTileVec;
                 issued_bi = bi;
@@ -745,6 +757,7 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
                         const unsigned mine2 = my_entries(d2, d2.nblk, (a + bi2) & (kNA - 1), lane);
                         if (mine2) {
                             const int nlb = __ffs(mine2) - 1;
+                            next_tile = (int)d2.tile[nlb];
                             next_k = kbase + (size_t)d2.tile[nlb] * kTileVec;
                             next_v = vbase + (size_t)d2.tile[nlb] * kTileVec;
                             issued_bi = bi2;
@@ -753,8 +766,12 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
                     }
                 }
             }
-            ok = attend_block(st, kslot, vslot, kbar, vbar, phase, next_k, next_v, lane, d.rows[lb], d.keep4[lb],
-                              logit_scale_log2);
+            if constexpr (RES)
+                ok = attend_block_res(st, qb, p, kslot, vslot, kbar, vbar, phase, next_tile, next_v, lane, d.rows[lb],
+                                      d.keep4[lb], logit_scale_log2);
+            else
+                ok = attend_block(st, kslot, vslot, kbar, vbar, phase, next_k, next_v, lane, d.rows[lb], d.keep4[lb],
+                                  logit_scale_log2);
         }
         __syncwarp();
         FFD_ACC(3);
@@ -799,6 +816,7 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
     if (!ok && lane == 0) atomicOr(p.status, kDevTimeout);
 }
 
+template <bool RES>
 __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodeParams p) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -842,7 +860,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodePa
         else scan_role(p, smem, warp, lane);
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kAttendRegs));
-        attend_role(p, smem, warp - kNS, lane);
+        attend_role<RES>(p, smem, warp - kNS, lane);
     }
 }
 

@@ -70,6 +70,8 @@ constexpr uint32_t kDevTimeout = 4u;
 struct DecodeParams {
     const __nv_bfloat16* q;
     const __nv_bfloat16* k_cache;
+    const int8_t* k_res;      // 2 + 8 bit key format: residuals of the keys (k_cache is then unused)
+    float* res_scores;        // 2 + 8 bit key format: per-token approximate scores of maybe-kept blocks, scan -> attend
     const __nv_bfloat16* v_cache;
     const uint8_t* k_quant;
     const __half* k_scales;
@@ -130,6 +132,24 @@ __device__ __forceinline__ void mma_bf16_top(float& c0, float& c1, uint32_t a0, 
     asm volatile(
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
         : "+f"(c0), "+f"(c1), "+f"(z0), "+f"(z1)
+        : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+}
+
+// the same with fp16 operands
+__device__ __forceinline__ void mma_f16_top(float& c0, float& c1, uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+    float z0 = 0.f, z1 = 0.f;
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+        : "+f"(c0), "+f"(c1), "+f"(z0), "+f"(z1)
+        : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+}
+
+// signed 8-bit operands, K = 32, 32-bit integer accumulation; rows 8..15 of A are zero
+__device__ __forceinline__ void mma_s8_top(int& c0, int& c1, uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+    int z0 = 0, z1 = 0;
+    asm volatile(
+        "mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+        : "+r"(c0), "+r"(c1), "+r"(z0), "+r"(z1)
         : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
 }
 
@@ -498,6 +518,10 @@ __device__ __forceinline__ void attend_setup(AttendState& st, const __nv_bfloat1
     attend_reset(st);
 }
 
+__device__ __forceinline__ bool attend_finish(AttendState& st, float (&s)[8][2], uint32_t vslot, uint32_t vbar,
+                                              uint32_t& phase, const uint4* next_v, int lane, int rows, bool mine,
+                                              float logit_scale_log2);
+
 // keep4: bit h set when head h attends to this block.  rows: valid tokens in the block (1..64).
 // The block's K and V tiles are (being) copied into kslot / vslot; kbar / vbar complete when they have landed.
 // next_k / next_v: global tiles of the next kept block (nullptr = none); their copies are issued as soon as
@@ -525,7 +549,15 @@ __device__ __forceinline__ bool attend_block(AttendState& st, uint32_t kslot, ui
     }
     __syncwarp();   // every lane is done reading the K slot
     if (next_k) tile_copy_async(kslot, next_k, lane, kbar);
-    // online softmax (log2 domain)
+    return attend_finish(st, s, vslot, vbar, phase, next_v, lane, rows, mine, logit_scale_log2);
+}
+
+// Second half of a block: s[nt][x] = q . k of head r % 4 and token 8 nt + 2j + x (rows r and r + 4 hold the same
+// values) -> online softmax (log2 domain) -> O += P V.  Issues the copy of the next V tile when the slot is free.
+__device__ __forceinline__ bool attend_finish(AttendState& st, float (&s)[8][2], uint32_t vslot, uint32_t vbar,
+                                              uint32_t& phase, const uint4* next_v, int lane, int rows, bool mine,
+                                              float logit_scale_log2) {
+    const int r = lane >> 2, j = lane & 3;
     float mx = -INFINITY;
 #pragma unroll
     for (int nt = 0; nt < 8; ++nt)
@@ -592,6 +624,165 @@ __device__ __forceinline__ bool attend_block(AttendState& st, uint32_t kslot, ui
     if (next_v) tile_copy_async(vslot, next_v, lane, vbar);
     phase ^= 1u;
     return true;
+}
+
+// ---- attend on the 2 + 8 bit key format (Sec. 3.3: s_final = (q . k_quant + q . k_res) / sqrt(d)) -------------
+//
+// The K slot of a kept block holds, instead of the 16 KB bf16 tile: the 8 KB int8 residual tile (token rows of
+// 128 bytes, the two 64-byte halves of odd rows swapped so that a quarter-warp's reads cover all banks), the block's
+// 2 KB of packed codes and its 256 bytes of scales.
+//
+// q . k_quant, tokens as MMA columns: the packed code words serve as B fragments exactly as they serve as A
+// fragments in the scan (word x / z of a lane = token lane/4, channels k = 2j.. / 2j+8.. of every k-step; words
+// y / w the token eight further on), and the scan's B fragments (hi / lo piece of pre-scaled q times scale) become
+// the A fragments: row r < 4 = hi piece of head r, row r + 4 = its lo piece.
+//
+// q . k_res: int8 MMA, K = 32.  A lane's B fragments are its two 16-byte reads of token lane/4 (channels 16j..16j+15
+// and 64+16j..64+16j+15); the A operand is v_c = q_c * s_c written with two signed 8-bit digits,
+// v_c ~ (vmax / 127) * (d0 + d1 / 254): row r < 4 = digit d0 of head r, row r + 4 = digit d1.
+constexpr uint32_t kResOffCodes = 8192, kResOffScales = kResOffCodes + kCodeBytes;
+
+__device__ __forceinline__ void res_copy_async(uint32_t slot, const DecodeParams& p, uint32_t tile, int lane,
+                                               uint32_t bar) {
+    const uint4* res = reinterpret_cast<const uint4*>(p.k_res + (size_t)tile * (kBlk * kD));
+#pragma unroll
+    for (int x = 0; x < 16; ++x) {
+        const uint32_t idx = x * 32 + lane, t = idx >> 3, c = idx & 7;
+        cp_async16(slot + t * 128 + ((c ^ ((t & 1u) << 2)) << 4), res + idx);
+    }
+    const uint4* codes = reinterpret_cast<const uint4*>(p.k_quant + (size_t)tile * kCodeBytes);
+#pragma unroll
+    for (int x = 0; x < 4; ++x) cp_async16(slot + kResOffCodes + (x * 32 + lane) * 16, codes + x * 32 + lane);
+    if (lane < 16)
+        cp_async16(slot + kResOffScales + lane * 16, reinterpret_cast<const uint4*>(p.k_scales + (size_t)tile * kD) + lane);
+    cp_async_arrive(bar);
+}
+
+// Per batch: st.qa = the pre-scaled fp16 fragments of head r % 4 from the unit's query record (the scan's B-fragment
+// owner of that head), qb = the head's bf16 q for this lane's 32 residual channels.
+__device__ __forceinline__ void attend_setup_res(AttendState& st, uint32_t (&qb)[16], const DecodeParams& p, int b, int g,
+                                                 const uint4* rec /* the unit's query record */, int lane) {
+    const int r = lane >> 2, j = lane & 3, head = r & 3;
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        const uint4 v = ldg_plain(rec + x * 32 + 8 * head + j);
+        st.qa[4 * x + 0] = v.x; st.qa[4 * x + 1] = v.y; st.qa[4 * x + 2] = v.z; st.qa[4 * x + 3] = v.w;
+    }
+    const __nv_bfloat16* qh = p.q + ((size_t)b * p.Hq + (size_t)g * p.G + head) * kD;
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (head < p.G) v = *reinterpret_cast<const uint4*>(qh + 64 * (x >> 1) + 16 * j + 8 * (x & 1));
+        qb[4 * x + 0] = v.x; qb[4 * x + 1] = v.y; qb[4 * x + 2] = v.z; qb[4 * x + 3] = v.w;
+    }
+    attend_reset(st);
+}
+
+// v = q * s of the two channels held in one bf16 pair / fp16 pair
+__device__ __forceinline__ float2 res_qs(uint32_t q2, uint32_t s2) {
+    const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
+    return make_float2(__uint_as_float(q2 << 16) * sf.x, __uint_as_float(q2 & 0xffff0000u) * sf.y);
+}
+
+__device__ __forceinline__ bool attend_block_res(AttendState& st, const uint32_t (&qb)[16], const DecodeParams& p,
+                                                 uint32_t kslot, uint32_t vslot, uint32_t kbar, uint32_t vbar,
+                                                 uint32_t& phase, int next_tile, const uint4* next_v, int lane, int rows,
+                                                 unsigned keep4, float logit_scale_log2) {
+    const int r = lane >> 2, j = lane & 3;
+    const bool mine = (keep4 >> (r & 3)) & 1u;
+    const int piece = r >> 2;
+    if (!mbar_wait(kbar, phase & 1u)) return false;
+    float s[8][2];
+    // ---- q . k_quant ----
+    {
+        uint32_t afrag[16];
+#pragma unroll
+        for (int x = 0; x < 4; ++x)
+            scan_bfrag4(afrag + 4 * x, make_uint4(st.qa[4 * x], st.qa[4 * x + 1], st.qa[4 * x + 2], st.qa[4 * x + 3]),
+                        lds128(kslot + kResOffScales + (4 * j + x) * 16), piece);
+        float off0 = 0.f, off1 = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t one = 0x00010001u << (2 * (i < 5 ? i : i - 5));
+            mma_f16_top(off0, off1, afrag[2 * i], afrag[2 * i + 1], one, one);
+        }
+#pragma unroll
+        for (int mt = 0; mt < 4; ++mt) {
+            const uint4 w = lds128(kslot + kResOffCodes + (mt * 32 + lane) * 16);
+            const uint4 t = make_uint4(w.x >> 10, w.y >> 10, w.z >> 10, w.w >> 10);
+            float c00 = 0.f, c01 = 0.f, c10 = 0.f, c11 = 0.f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t mask = 0x00030003u << (2 * (i < 5 ? i : i - 5));
+                const uint4 src = i < 5 ? w : t;
+                mma_f16_top(c00, c01, afrag[2 * i], afrag[2 * i + 1], src.x & mask, src.z & mask);   // tokens 16 mt + lane/4
+                mma_f16_top(c10, c11, afrag[2 * i], afrag[2 * i + 1], src.y & mask, src.w & mask);   // eight further on
+            }
+            // sum_c (code - 1.5) q s = 2^20 * (acc - 1.5 * off): this row's piece of it
+            s[2 * mt][0] = (c00 - 1.5f * off0) * 1048576.0f;
+            s[2 * mt][1] = (c01 - 1.5f * off1) * 1048576.0f;
+            s[2 * mt + 1][0] = (c10 - 1.5f * off0) * 1048576.0f;
+            s[2 * mt + 1][1] = (c11 - 1.5f * off1) * 1048576.0f;
+        }
+    }
+    // ---- q . k_res ----
+    {
+        // this lane's 32 scales: channels 16j..16j+15 and 64+16j..64+16j+15
+        uint4 sv[4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) sv[x] = lds128(kslot + kResOffScales + (8 * (x >> 1) + 2 * j + (x & 1)) * 16);
+        const uint32_t* s2 = reinterpret_cast<const uint32_t*>(sv);
+        float vmax = 0.f;
+#pragma unroll
+        for (int y = 0; y < 16; ++y) {
+            const float2 v = res_qs(qb[y], s2[y]);
+            vmax = fmaxf(vmax, fmaxf(fabsf(v.x), fabsf(v.y)));
+        }
+        vmax = fmaxf(vmax, __shfl_xor_sync(kFull, vmax, 1));
+        vmax = fmaxf(vmax, __shfl_xor_sync(kFull, vmax, 2));
+        const float inv = vmax > 0.f ? 127.f / vmax : 0.f, step = vmax * (1.f / 127.f);
+        const float inv1 = inv * 254.f;
+        constexpr float kMagic = 12582912.f;   // 1.5 * 2^23: adding it leaves rint(x) in the low mantissa bits
+        uint32_t adig[8];   // register rho: channels 4 rho .. 4 rho + 3 of the lane's 32, one digit per byte
+#pragma unroll
+        for (int rho = 0; rho < 8; ++rho) {
+            uint32_t bits[4];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const float2 v = res_qs(qb[2 * rho + h], s2[2 * rho + h]);
+                const float t0x = fmaf(v.x, inv, kMagic), t0y = fmaf(v.y, inv, kMagic);
+                const float t1x = fmaf(fmaf(-(t0x - kMagic), step, v.x), inv1, kMagic);
+                const float t1y = fmaf(fmaf(-(t0y - kMagic), step, v.y), inv1, kMagic);
+                bits[2 * h] = __float_as_uint(piece ? t1x : t0x);
+                bits[2 * h + 1] = __float_as_uint(piece ? t1y : t0y);
+            }
+            adig[rho] = __byte_perm(__byte_perm(bits[0], bits[1], 0x0040), __byte_perm(bits[2], bits[3], 0x0040), 0x5410);
+        }
+        // digits -> logits: v ~ step * (d0 + d1 / 254); a residual step is s / 254 (s is inside v)
+        const float unit = step * (1.f / 254.f) * (piece ? 1.f / 254.f : 1.f);
+        const uint32_t flip = (uint32_t)(r & 1) << 2;   // token 8 nt + r: odd rows have their halves swapped
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) {
+            const uint32_t row = kslot + (8 * nt + r) * 128;
+            const uint4 k0 = lds128(row + ((j ^ flip) << 4)), k1 = lds128(row + (((j + 4) ^ flip) << 4));
+            int d0 = 0, d1 = 0;
+            mma_s8_top(d0, d1, adig[0], adig[1], k0.x, k0.y);
+            mma_s8_top(d0, d1, adig[2], adig[3], k0.z, k0.w);
+            mma_s8_top(d0, d1, adig[4], adig[5], k1.x, k1.y);
+            mma_s8_top(d0, d1, adig[6], adig[7], k1.z, k1.w);
+            s[nt][0] = fmaf((float)d0, unit, s[nt][0]);
+            s[nt][1] = fmaf((float)d1, unit, s[nt][1]);
+        }
+    }
+    __syncwarp();   // every lane is done reading the K slot
+    if (next_tile >= 0) res_copy_async(kslot, p, (uint32_t)next_tile, lane, kbar);
+    // rows r and r + 4 hold the two pieces of the same head: both get the sum
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+        s[nt][0] += __shfl_xor_sync(kFull, s[nt][0], 16);
+        s[nt][1] += __shfl_xor_sync(kFull, s[nt][1], 16);
+    }
+    return attend_finish(st, s, vslot, vbar, phase, next_v, lane, rows, mine, logit_scale_log2);
 }
 
 // output channel of O fragment (n-tile nt, column n)

@@ -25,7 +25,7 @@ DEV_BAD_SEQ_LEN = 2
 
 EXPORTS = ["ffd_status_string", "ffd_workspace_bytes", "ffd_workspace_init", "ffd_quantize_keys", "ffd_decode",
            "ffd_decode_dense", "ffd_unpack_codes", "ffd_read_device_status", "ffd_profile_events", "ffd_decode_static",
-           "ffd_append_kv", "ffd_append_decode"]
+           "ffd_append_kv", "ffd_append_decode", "ffd_quantize_residual", "ffd_decode_residual"]
 
 
 class FfdError(RuntimeError):
@@ -89,6 +89,8 @@ def load_library() -> ctypes.CDLL:
                                       _vp]
         lib.ffd_append_decode.argtypes = [cfgp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32,
                                           ctypes.c_float, _vp, _vp, _vp, _vp, _vp, ctypes.c_size_t, _vp]
+        lib.ffd_quantize_residual.argtypes = [cfgp, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, _vp]
+        lib.ffd_decode_residual.argtypes = lib.ffd_decode.argtypes
         for name in EXPORTS:
             if name != "ffd_status_string":
                 getattr(lib, name).restype = ctypes.c_int
@@ -134,6 +136,23 @@ def ffd_quantize_keys(cfg: Config, k_cache, k_quant, k_scales, block_table, seq_
     _check(load_library().ffd_quantize_keys(ctypes.byref(cfg.c()), _p(k_cache), _p(k_quant), _p(k_scales),
                                             _p(block_table), _p(seq_lens), _p(first_token), seq_lens.numel(),
                                             max_blocks_per_seq, num_pages, _stream(stream)), "ffd_quantize_keys")
+
+
+def ffd_quantize_residual(cfg: Config, k_cache, k_scales, k_res, block_table, seq_lens, first_token=None, *,
+                          max_blocks_per_seq: int, stream=None):
+    _check(load_library().ffd_quantize_residual(ctypes.byref(cfg.c()), _p(k_cache), _p(k_scales), _p(k_res),
+                                                _p(block_table), _p(seq_lens), _p(first_token), seq_lens.numel(),
+                                                max_blocks_per_seq, k_cache.shape[0], _stream(stream)),
+           "ffd_quantize_residual")
+
+
+def ffd_decode_residual(cfg: Config, q, k_res, v_cache, k_quant, k_scales, block_table, seq_lens, delta: float, out, *,
+                        max_blocks_per_seq: int, workspace, lse=None, kept_mask=None, block_max=None, stream=None):
+    _check(load_library().ffd_decode_residual(ctypes.byref(cfg.c()), _p(q), _p(k_res), _p(v_cache), _p(k_quant),
+                                              _p(k_scales), _p(block_table), _p(seq_lens), q.shape[0],
+                                              max_blocks_per_seq, k_res.shape[0], ctypes.c_float(delta), _p(out),
+                                              _p(lse), _p(kept_mask), _p(block_max), _p(workspace), workspace.numel(),
+                                              _stream(stream)), "ffd_decode_residual")
 
 
 def ffd_append_kv(cfg: Config, k_new, v_new, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, *,
@@ -236,6 +255,18 @@ class DeviceCache:
     def quantize(self, first_token=None):
         ffd_quantize_keys(self.cfg, self.k_cache, self.k_quant, self.k_scales, self.block_table, self.seq_lens,
                           first_token, max_blocks_per_seq=self.w.max_blocks)
+
+    def quantize_residual(self, first_token=None):
+        """The 8-bit residuals of the keys (after ``quantize``); allocates ``k_res`` on first use."""
+        if getattr(self, "k_res", None) is None:
+            self.k_res = torch.zeros(self.w.num_pages, self.w.Hkv, 64, 128, dtype=torch.int8, device=self.device)
+        ffd_quantize_residual(self.cfg, self.k_cache, self.k_scales, self.k_res, self.block_table, self.seq_lens,
+                              first_token, max_blocks_per_seq=self.w.max_blocks)
+
+    def decode_residual(self, delta, kept_mask=None, block_max=None):
+        ffd_decode_residual(self.cfg, self.q, self.k_res, self.v_cache, self.k_quant, self.k_scales, self.block_table,
+                            self.seq_lens, delta, self.out, max_blocks_per_seq=self.w.max_blocks,
+                            workspace=self.workspace, lse=self.lse, kept_mask=kept_mask, block_max=block_max)
 
     def append(self, k_new, v_new):
         ffd_append_kv(self.cfg, k_new, v_new, self.k_cache, self.v_cache, self.k_quant, self.k_scales,

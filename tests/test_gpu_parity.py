@@ -53,17 +53,28 @@ def check_quantize(ffd, oracle, w, dc):
     return codes, scales
 
 
-def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None):
+def check_residual(ffd, oracle, w, dc, codes, scales):
+    """8-bit residuals (after check_quantize): bit for bit on every mapped tile, padding rows included (zero)."""
+    dc.quantize_residual()
+    k_res = oracle.quantize_residual(w.bits("k_cache"), codes, scales, w.block_table, w.seq_lens, w.max_blocks)
+    _, mapped = valid_row_mask(w)
+    assert np.array_equal(dc.k_res.cpu().numpy()[mapped], k_res[mapped])
+    return k_res
+
+
+def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None, k_res=None):
+    """k_res (the oracle's residuals): check the 2 + 8 bit format's decode against the oracle's Dequant refinement."""
     B, Hq, mb = w.B, w.Hq, w.max_blocks
+    gpu_decode = dc.decode if k_res is None else dc.decode_residual
     kept = torch.full((B, Hq, mb), 255, dtype=torch.uint8, device="cuda")
     bm = torch.full((B, Hq, mb), float("nan"), dtype=torch.float32, device="cuda")
     # without the block-max debug output the kernel may skip the tensor-core work of blocks whose scale-only upper
     # bound already rules them out: the decisions and the output must not change
     kept_fast = torch.full((B, Hq, mb), 255, dtype=torch.uint8, device="cuda")
-    dc.decode(delta, kept_mask=kept_fast)
+    gpu_decode(delta, kept_mask=kept_fast)
     assert ffd.ffd_read_device_status(dc.workspace) == 0
     out_fast = dc.out.clone()
-    dc.decode(delta, kept_mask=kept, block_max=bm)
+    gpu_decode(delta, kept_mask=kept, block_max=bm)
     assert ffd.ffd_read_device_status(dc.workspace) == 0
     assert torch.equal(kept, kept_fast)
     assert (dc.out - out_fast).abs().max().item() <= 1e-6
@@ -72,7 +83,7 @@ def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None):
     kept = kept.cpu().numpy()
     bm = bm.cpu().numpy()
     r = oracle.decode(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), codes, scales, w.block_table, w.seq_lens,
-                      mb, delta, n_sink=dc.cfg.n_sink_blocks, n_local=dc.cfg.n_local_blocks, units=units)
+                      mb, delta, n_sink=dc.cfg.n_sink_blocks, n_local=dc.cfg.n_local_blocks, units=units, k_res=k_res)
     rows = units if units is not None else [(b, h) for b in range(B) for h in range(Hq)]
     differs = False
     for b, h in rows:
@@ -88,7 +99,7 @@ def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None):
     if differs:   # compare the output against the oracle's attention over the GPU's (equally valid) mask
         forced = np.where(kept == 255, 0, kept).astype(np.uint8)
         r = oracle.decode(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), codes, scales, w.block_table,
-                          w.seq_lens, mb, delta, forced_mask=forced, units=units)
+                          w.seq_lens, mb, delta, forced_mask=forced, units=units, k_res=k_res)
     idx = tuple(np.array(rows).T)
     err = np.abs(out[idx] - r.out[idx])
     assert err.max() < OUT_MAX and err.mean() < OUT_MEAN
@@ -136,6 +147,19 @@ def test_small_configs_element_by_element(ffd, oracle, name, kw, _):
         check_decode(ffd, oracle, w, dc, codes, scales, delta)
     check_decode(ffd, oracle, w, dc, codes, scales, 0.0)
     check_dense(ffd, oracle, w, dc)
+
+
+@pytest.mark.parametrize("name,kw,_", SMALL)
+def test_small_configs_residual_key_format(ffd, oracle, name, kw, _):
+    """Sec. 3.1 / 3.3: the 2 + 8 bit key format.  Residual codes bit for bit; the decode that refines from
+    k_quant + k_res (two-term score) against the oracle's Dequant refinement at the same bars as the 16-bit path."""
+    w = make_workload(name, **kw)
+    dc = ffd.DeviceCache(w)
+    codes, scales = check_quantize(ffd, oracle, w, dc)
+    k_res = check_residual(ffd, oracle, w, dc, codes, scales)
+    dc.k_cache = None   # the residual decode must not need the 16-bit keys
+    for delta in w.deltas:
+        check_decode(ffd, oracle, w, dc, codes, scales, delta, k_res=k_res)
 
 
 def test_bf16_output_is_rounding_of_fp32_output(ffd, oracle):
