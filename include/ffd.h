@@ -75,6 +75,12 @@ const char* ffd_status_string(ffd_status status);
 /* Bytes of device workspace ffd_decode / ffd_decode_dense need for this geometry (host call, no CUDA). */
 ffd_status ffd_workspace_bytes(const ffd_config* cfg, int32_t batch, int32_t max_blocks_per_seq, size_t* bytes);
 
+/* The same for ffd_decode_residual: the workspace of ffd_decode for this geometry followed by the tiles in which the
+ * scan leaves the approximate scores of kept blocks for the refinement (about 57 MB, independent of the geometry).
+ * Such a workspace serves every other call too. */
+ffd_status ffd_workspace_bytes_residual(const ffd_config* cfg, int32_t batch, int32_t max_blocks_per_seq,
+                                        size_t* bytes);
+
 /* Zeroes the header of a freshly allocated workspace (status word, work counters).  Call once before the first
  * decode with that workspace.  The status word is sticky across calls until ffd_read_device_status clears it; the
  * work counters are left at zero by every completed ffd_decode.  If a decode call was interrupted (a CUDA error),
@@ -161,11 +167,14 @@ ffd_status ffd_decode(const ffd_config* cfg, const void* q, const void* k_cache,
  * loads its 8-bit residual keys and its values; s_final = (q . k_quant + q . k_res) / sqrt(d), both dot products
  * accumulated without a full-precision key).  Selection is exactly ffd_decode's; the refined logit of a kept token is
  *   sm * sum_c q[c] * ((code - 1.5) * s[c] + k_res[t,c] * s[c] / 254)
- * so a kept block costs 8 KB of k_res + 16 KB of V (plus its 2.3 KB of thumbnails, normally still in L2) instead of
- * 32 KB, and the 16-bit keys are not read at all.  k_res as written by ffd_quantize_residual; every other argument,
- * the outputs and the error behaviour as for ffd_decode.  Arithmetic: q . k_quant on the tensor cores as in the
- * scan (exact fp16 products, fp32 accumulation); q . k_res with int8 tensor-core products of k_res and q[c] * s[c]
- * split into two 8-bit digits (relative error below 2^-15 of the largest |q[c] * s[c]| per channel).
+ * so a kept block costs 8 KB of k_res + 16 KB of V instead of 32 KB, and the 16-bit keys are not read at all.  The
+ * q . k_quant term is the scan's own per-token result, handed from the scanning to the refining warps through
+ * score tiles in the workspace (1.1 KB per kept block, L2-resident), as Sec. 3 describes ("the computer reuses the
+ * selector's estimation results").  k_res as written by ffd_quantize_residual; workspace_bytes at least
+ * ffd_workspace_bytes_residual (FFD_ERR_WORKSPACE otherwise; FFD_ERR_UNSUPPORTED on a GPU with more than 192 SMs);
+ * every other argument, the outputs and the error behaviour as for ffd_decode.  Arithmetic: q . k_quant as in the
+ * scan (exact fp16 tensor-core products, fp32 accumulation); q . k_res with int8 tensor-core products of k_res and
+ * q[c] * s[c] split into two 8-bit digits (relative error below 2^-15 of the largest |q[c] * s[c]| per channel).
  */
 ffd_status ffd_decode_residual(const ffd_config* cfg, const void* q, const void* k_res, const void* v_cache,
                                const void* k_quant, const void* k_scales, const int32_t* block_table,

@@ -720,7 +720,12 @@ struct Plan {
     int blocks_per_split, splits;     // dense path
     int total_items;                  // fused path
     size_t off_mtilde, off_lens, off_units, off_qrec, off_ml, off_acc, off_fml, off_facc, total;
+    size_t off_scores, total_residual;   // 2 + 8 bit key format: the score tiles follow everything else
 };
+
+// score tiles of the 2 + 8 bit format: one ring of (batch descriptors x blocks per item) tiles per CTA of the fused
+// kernel, which runs one CTA per SM; sized for GPUs of up to this many SMs
+constexpr int kResMaxCtas = 192;
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -745,6 +750,8 @@ static Plan make_plan(const ffd_config* cfg, int batch, int max_blocks) {
     pl.off_fml = align_up(pl.off_acc + heads * pl.splits * kD * sizeof(float), 256);
     pl.off_facc = align_up(pl.off_fml + fslots * 2 * sizeof(float), 256);
     pl.total = align_up(pl.off_facc + fslots * kD * sizeof(float), 256);
+    pl.off_scores = pl.total;
+    pl.total_residual = pl.off_scores + (size_t)kResMaxCtas * kNB * kItemBlocksMax * kScoreTileFloats * sizeof(float);
     return pl;
 }
 
@@ -821,7 +828,7 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
     for (const void* ptr : ptrs)
         if (ptr && misaligned(ptr)) return FFD_ERR_ALIGN;
     const Plan pl = make_plan(cfg, batch, max_blocks);
-    if (workspace_bytes < pl.total) return FFD_ERR_WORKSPACE;
+    if (workspace_bytes < (k_res ? pl.total_residual : pl.total)) return FFD_ERR_WORKSPACE;
 
     DecodeParams p;
     memset(&p, 0, sizeof p);
@@ -859,6 +866,7 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
     p.light_counter = reinterpret_cast<uint32_t*>(ws + 76);
     p.len_stats = reinterpret_cast<uint32_t*>(ws + 80);
     p.unit_list = reinterpret_cast<int2*>(ws + pl.off_units);
+    p.res_scores = reinterpret_cast<float*>(ws + pl.off_scores);
     p.units = batch * cfg->num_kv_heads;
     p.item_rows = item_geometry(p.units, max_blocks).item_rows;
     p.rows_small = item_geometry(p.units, max_blocks).rows_small;
@@ -881,6 +889,7 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
             cudaFuncSetAttribute(fused_sparse_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem) != cudaSuccess ||
             cudaFuncSetAttribute(fused_sparse_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem) != cudaSuccess)
             return FFD_ERR_CUDA;
+        if (k_res && sms > kResMaxCtas) return FFD_ERR_UNSUPPORTED;
         // the work counters and class counts at ws + 64 are zero here: ffd_workspace_init zeroes them and the
         // combine kernel of every call leaves them zeroed for the next one
         if (append) {
@@ -941,6 +950,16 @@ ffd_status ffd_workspace_bytes(const ffd_config* cfg, int32_t batch, int32_t max
     st = check_geometry(batch, max_blocks_per_seq, 1);
     if (st) return st;
     *bytes = make_plan(cfg, batch, max_blocks_per_seq).total;
+    return FFD_OK;
+}
+
+ffd_status ffd_workspace_bytes_residual(const ffd_config* cfg, int32_t batch, int32_t max_blocks_per_seq, size_t* bytes) {
+    ffd_status st = check_config(cfg);
+    if (st) return st;
+    if (!bytes) return FFD_ERR_NULL;
+    st = check_geometry(batch, max_blocks_per_seq, 1);
+    if (st) return st;
+    *bytes = make_plan(cfg, batch, max_blocks_per_seq).total_residual;
     return FFD_OK;
 }
 

@@ -518,6 +518,10 @@ __device__ __noinline__ float scan_block_precise(const uint4* codes_tile, const 
     return scan_compute<true>(sr, sq, lane, rows, sm_scale, band);
 }
 
+// RES (2 + 8 bit key format): the per-token approximate logits of every block that may be kept are left in the
+// CTA's ring of score tiles in global memory (tile (batch slot, block) -- free again when the attend warps have
+// released the batch slot, which the scheduler waits for before it publishes into it).
+template <bool RES>
 __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* smem, int w, int lane) {
     const int r = lane >> 2, j = lane & 3;
     const int w0 = w - kSched;      // index among the scanning warps
@@ -637,7 +641,19 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
                 }
                 refilled = true;
                 float band;
-                float bm = scan_mma<false>(wv, bfrag, lane, rows, p.sm_scale, band);
+                float tok[8];
+                float bm = scan_mma<false>(wv, bfrag, lane, rows, p.sm_scale, band, RES ? tok : nullptr);
+                if constexpr (RES) {
+                    if (__any_sync(kFull, (j < p.G) && bm >= thr - band)) {
+                        float* dst = p.res_scores + ((size_t)(blockIdx.x * kNB + slot) * kItemBlocksMax + lb) * kScoreTileFloats +
+                                     j * kScoreStride + r;
+#pragma unroll
+                        for (int mt = 0; mt < 4; ++mt) {
+                            dst[16 * mt] = tok[2 * mt];
+                            dst[16 * mt + 8] = tok[2 * mt + 1];
+                        }
+                    }
+                }
                 // too close to call (rare): a separate, non-inlined routine re-reads the block and redoes it precisely
                 if (__any_sync(kFull, (j < p.G) && fabsf(bm - thr) <= band))
                     bm = scan_block_precise(reinterpret_cast<const uint4*>(p.k_quant + (size_t)tile * kCodeBytes),
@@ -686,6 +702,11 @@ __device__ __forceinline__ unsigned my_entries(const BatchDesc& d, int nblk, int
     return __ballot_sync(kFull, is_kept && (rank & (kNA - 1)) == a);
 }
 
+// score tile of block lb of the batch in descriptor slot `slot` of this CTA
+__device__ __forceinline__ float* score_tile(const DecodeParams& p, int slot, int lb) {
+    return p.res_scores + ((size_t)(blockIdx.x * kNB + slot) * kItemBlocksMax + lb) * kScoreTileFloats;
+}
+
 // RES: the 2 + 8 bit key format -- the K slot receives the block's residual tile, codes and scales instead of its
 // 16-bit keys
 template <bool RES>
@@ -724,9 +745,7 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
         const bool any = mine != 0;
         FFD_ACC(6);
         if (any) {
-            if constexpr (RES)
-                attend_setup_res(st, qb, p, it.b, it.g,
-                                 reinterpret_cast<const uint4*>(p.qrec + (size_t)(it.b * p.Hkv + it.g) * kQrecBytes), lane);
+            if constexpr (RES) attend_setup_res(st, qb, p, it.b, it.g, lane);
             else attend_setup(st, p.q + ((size_t)it.b * p.Hq + (size_t)it.g * p.G) * kD, p.G, lane);
         }
         FFD_TL(11, a == 0 && lane == 0 && any);
@@ -735,16 +754,18 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
             const int lb = __ffs(mine) - 1;
             mine &= mine - 1;
             if (!(issued_bi == bi && issued_lb == lb)) {
-                if constexpr (RES) res_copy_async(kslot, p, d.tile[lb], lane, kbar);
+                if constexpr (RES) res_copy_async(kslot, p, d.tile[lb], score_tile(p, slot, lb), lane, kbar);
                 else tile_copy_async(kslot, kbase + (size_t)d.tile[lb] * kTileVec, lane, kbar);
                 tile_copy_async(vslot, vbase + (size_t)d.tile[lb] * kTileVec, lane, vbar);
             }
             // the next block this warp will attend: in this batch, else in the next one if it is already published
             const uint4 *next_k = nullptr, *next_v = nullptr;
             int next_tile = -1;
+            const float* next_scores = nullptr;
             if (mine) {
                 const int nlb = __ffs(mine) - 1;
                 next_tile = (int)d.tile[nlb];
+                if constexpr (RES) next_scores = score_tile(p, slot, nlb);
                 next_k = kbase + (size_t)d.tile[nlb] * kTileVec;
                 next_v = vbase + (size_t)d.tile[nlb] * kTileVec;
                 issued_bi = bi;
@@ -758,6 +779,7 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
                         if (mine2) {
                             const int nlb = __ffs(mine2) - 1;
                             next_tile = (int)d2.tile[nlb];
+                            if constexpr (RES) next_scores = score_tile(p, bi2 & (kNB - 1), nlb);
                             next_k = kbase + (size_t)d2.tile[nlb] * kTileVec;
                             next_v = vbase + (size_t)d2.tile[nlb] * kTileVec;
                             issued_bi = bi2;
@@ -767,8 +789,8 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
                 }
             }
             if constexpr (RES)
-                ok = attend_block_res(st, qb, p, kslot, vslot, kbar, vbar, phase, next_tile, next_v, lane, d.rows[lb],
-                                      d.keep4[lb], logit_scale_log2);
+                ok = attend_block_res(st, qb, p, kslot, vslot, kbar, vbar, phase, next_tile, next_scores, next_v, lane,
+                                      d.rows[lb], d.keep4[lb]);
             else
                 ok = attend_block(st, kslot, vslot, kbar, vbar, phase, next_k, next_v, lane, d.rows[lb], d.keep4[lb],
                                   logit_scale_log2);
@@ -857,7 +879,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodePa
     if (warp < kNS) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kScanRegs));
         if (warp < kSched) sched_role(p, smem, lane, pend_heavy, pend_light);
-        else scan_role(p, smem, warp, lane);
+        else scan_role<RES>(p, smem, warp, lane);
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kAttendRegs));
         attend_role<RES>(p, smem, warp - kNS, lane);

@@ -401,7 +401,7 @@ __device__ __forceinline__ float scan_bound(__half2 sum_a, __half2 sum_b, float 
 
 template <bool PRECISE>
 __device__ __forceinline__ float scan_mma(const uint4 (&w)[4], const uint32_t (&bfrag)[16], int lane, int rows,
-                                          float sm_scale, float& band);
+                                          float sm_scale, float& band, float* tok = nullptr);
 
 template <bool PRECISE>
 __device__ __forceinline__ float scan_compute(const ScanRegs& sr, const ScanQuery& sq, int lane, int rows,
@@ -414,9 +414,11 @@ __device__ __forceinline__ float scan_compute(const ScanRegs& sr, const ScanQuer
     return scan_mma<PRECISE>(sr.w, bfrag, lane, rows, sm_scale, band);
 }
 
+// tok (optional): the approximate logits themselves, tok[2 mt] for token 16 mt + lane/4 and tok[2 mt + 1] for the
+// token eight further on, head lane % 4 (rows past `rows` included: the caller masks them).
 template <bool PRECISE>
 __device__ __forceinline__ float scan_mma(const uint4 (&w)[4], const uint32_t (&bfrag)[16], int lane, int rows,
-                                          float sm_scale, float& band) {
+                                          float sm_scale, float& band, float* tok) {
     const int r = lane >> 2;
     float acc[4][4];
     float off[4] = {0.f, 0.f, 0.f, 0.f};
@@ -475,6 +477,13 @@ __device__ __forceinline__ float scan_mma(const uint4 (&w)[4], const uint32_t (&
     const float o = 1.5f * (off[0] + off[1]);
     const float unit = 1048576.0f * sm_scale;
     band = kScanBandRel * (fabsf(best) + fabsf(o)) * unit;
+    if (tok) {
+#pragma unroll
+        for (int mt = 0; mt < 4; ++mt) {
+            tok[2 * mt] = (acc[mt][0] + acc[mt][1] - o) * unit;
+            tok[2 * mt + 1] = (acc[mt][2] + acc[mt][3] - o) * unit;
+        }
+    }
     return (best - o) * unit;
 }
 
@@ -628,46 +637,44 @@ __device__ __forceinline__ bool attend_finish(AttendState& st, float (&s)[8][2],
 
 // ---- attend on the 2 + 8 bit key format (Sec. 3.3: s_final = (q . k_quant + q . k_res) / sqrt(d)) -------------
 //
-// The K slot of a kept block holds, instead of the 16 KB bf16 tile: the 8 KB int8 residual tile (token rows of
-// 128 bytes, the two 64-byte halves of odd rows swapped so that a quarter-warp's reads cover all banks), the block's
-// 2 KB of packed codes and its 256 bytes of scales.
-//
-// q . k_quant, tokens as MMA columns: the packed code words serve as B fragments exactly as they serve as A
-// fragments in the scan (word x / z of a lane = token lane/4, channels k = 2j.. / 2j+8.. of every k-step; words
-// y / w the token eight further on), and the scan's B fragments (hi / lo piece of pre-scaled q times scale) become
-// the A fragments: row r < 4 = hi piece of head r, row r + 4 = its lo piece.
+// q . k_quant is not computed again: the scan warp that judged the block wrote its per-token approximate logits
+// (all four heads, 64 tokens) to a score tile in global memory, which stays in L2, and the attend warp copies that
+// tile along with the residuals ("the computer reuses the selector's estimation results", Sec. 3).  The K slot of a
+// kept block holds, instead of the 16 KB bf16 tile: the 8 KB int8 residual tile (token rows of 128 bytes, the two
+// 64-byte halves of odd rows swapped so that a quarter-warp's reads cover all banks), the 1152-byte score tile
+// (head h, token t at float h * 72 + t: the padding spreads the four heads over the banks) and the 256 bytes of
+// scales.
 //
 // q . k_res: int8 MMA, K = 32.  A lane's B fragments are its two 16-byte reads of token lane/4 (channels 16j..16j+15
 // and 64+16j..64+16j+15); the A operand is v_c = q_c * s_c written with two signed 8-bit digits,
 // v_c ~ (vmax / 127) * (d0 + d1 / 254): row r < 4 = digit d0 of head r, row r + 4 = digit d1.
-constexpr uint32_t kResOffCodes = 8192, kResOffScales = kResOffCodes + kCodeBytes;
+constexpr int kScoreStride = 72;                          // floats per head in a score tile
+constexpr int kScoreTileFloats = 4 * kScoreStride;        // 1152 bytes
+constexpr uint32_t kResOffScores = 8192, kResOffScales = kResOffScores + kScoreTileFloats * 4;
 
-__device__ __forceinline__ void res_copy_async(uint32_t slot, const DecodeParams& p, uint32_t tile, int lane,
-                                               uint32_t bar) {
+__device__ __forceinline__ void res_copy_async(uint32_t slot, const DecodeParams& p, uint32_t tile, const float* scores,
+                                               int lane, uint32_t bar) {
     const uint4* res = reinterpret_cast<const uint4*>(p.k_res + (size_t)tile * (kBlk * kD));
 #pragma unroll
     for (int x = 0; x < 16; ++x) {
         const uint32_t idx = x * 32 + lane, t = idx >> 3, c = idx & 7;
         cp_async16(slot + t * 128 + ((c ^ ((t & 1u) << 2)) << 4), res + idx);
     }
-    const uint4* codes = reinterpret_cast<const uint4*>(p.k_quant + (size_t)tile * kCodeBytes);
-#pragma unroll
-    for (int x = 0; x < 4; ++x) cp_async16(slot + kResOffCodes + (x * 32 + lane) * 16, codes + x * 32 + lane);
-    if (lane < 16)
-        cp_async16(slot + kResOffScales + lane * 16, reinterpret_cast<const uint4*>(p.k_scales + (size_t)tile * kD) + lane);
+    const uint4* sc = reinterpret_cast<const uint4*>(scores);
+    cp_async16(slot + kResOffScores + lane * 16, sc + lane);
+    cp_async16(slot + kResOffScores + (32 + lane) * 16, sc + 32 + lane);
+    if (lane < kScoreTileFloats / 4 - 64) cp_async16(slot + kResOffScores + (64 + lane) * 16, sc + 64 + lane);
+    if (lane >= 16)
+        cp_async16(slot + kResOffScales + (lane - 16) * 16,
+                   reinterpret_cast<const uint4*>(p.k_scales + (size_t)tile * kD) + (lane - 16));
     cp_async_arrive(bar);
 }
+static_assert(kScoreTileFloats / 4 - 64 <= 16, "score tile: at most 80 chunks");
 
-// Per batch: st.qa = the pre-scaled fp16 fragments of head r % 4 from the unit's query record (the scan's B-fragment
-// owner of that head), qb = the head's bf16 q for this lane's 32 residual channels.
+// Per batch: qb = bf16 q of head r % 4 for this lane's 32 residual channels.
 __device__ __forceinline__ void attend_setup_res(AttendState& st, uint32_t (&qb)[16], const DecodeParams& p, int b, int g,
-                                                 const uint4* rec /* the unit's query record */, int lane) {
+                                                 int lane) {
     const int r = lane >> 2, j = lane & 3, head = r & 3;
-#pragma unroll
-    for (int x = 0; x < 4; ++x) {
-        const uint4 v = ldg_plain(rec + x * 32 + 8 * head + j);
-        st.qa[4 * x + 0] = v.x; st.qa[4 * x + 1] = v.y; st.qa[4 * x + 2] = v.z; st.qa[4 * x + 3] = v.w;
-    }
     const __nv_bfloat16* qh = p.q + ((size_t)b * p.Hq + (size_t)g * p.G + head) * kD;
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
@@ -686,46 +693,13 @@ __device__ __forceinline__ float2 res_qs(uint32_t q2, uint32_t s2) {
 
 __device__ __forceinline__ bool attend_block_res(AttendState& st, const uint32_t (&qb)[16], const DecodeParams& p,
                                                  uint32_t kslot, uint32_t vslot, uint32_t kbar, uint32_t vbar,
-                                                 uint32_t& phase, int next_tile, const uint4* next_v, int lane, int rows,
-                                                 unsigned keep4, float logit_scale_log2) {
+                                                 uint32_t& phase, int next_tile, const float* next_scores,
+                                                 const uint4* next_v, int lane, int rows, unsigned keep4) {
     const int r = lane >> 2, j = lane & 3;
     const bool mine = (keep4 >> (r & 3)) & 1u;
     const int piece = r >> 2;
     if (!mbar_wait(kbar, phase & 1u)) return false;
     float s[8][2];
-    // ---- q . k_quant ----
-    {
-        uint32_t afrag[16];
-#pragma unroll
-        for (int x = 0; x < 4; ++x)
-            scan_bfrag4(afrag + 4 * x, make_uint4(st.qa[4 * x], st.qa[4 * x + 1], st.qa[4 * x + 2], st.qa[4 * x + 3]),
-                        lds128(kslot + kResOffScales + (4 * j + x) * 16), piece);
-        float off0 = 0.f, off1 = 0.f;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const uint32_t one = 0x00010001u << (2 * (i < 5 ? i : i - 5));
-            mma_f16_top(off0, off1, afrag[2 * i], afrag[2 * i + 1], one, one);
-        }
-#pragma unroll
-        for (int mt = 0; mt < 4; ++mt) {
-            const uint4 w = lds128(kslot + kResOffCodes + (mt * 32 + lane) * 16);
-            const uint4 t = make_uint4(w.x >> 10, w.y >> 10, w.z >> 10, w.w >> 10);
-            float c00 = 0.f, c01 = 0.f, c10 = 0.f, c11 = 0.f;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const uint32_t mask = 0x00030003u << (2 * (i < 5 ? i : i - 5));
-                const uint4 src = i < 5 ? w : t;
-                mma_f16_top(c00, c01, afrag[2 * i], afrag[2 * i + 1], src.x & mask, src.z & mask);   // tokens 16 mt + lane/4
-                mma_f16_top(c10, c11, afrag[2 * i], afrag[2 * i + 1], src.y & mask, src.w & mask);   // eight further on
-            }
-            // sum_c (code - 1.5) q s = 2^20 * (acc - 1.5 * off): this row's piece of it
-            s[2 * mt][0] = (c00 - 1.5f * off0) * 1048576.0f;
-            s[2 * mt][1] = (c01 - 1.5f * off1) * 1048576.0f;
-            s[2 * mt + 1][0] = (c10 - 1.5f * off0) * 1048576.0f;
-            s[2 * mt + 1][1] = (c11 - 1.5f * off1) * 1048576.0f;
-        }
-    }
-    // ---- q . k_res ----
     {
         // this lane's 32 scales: channels 16j..16j+15 and 64+16j..64+16j+15
         uint4 sv[4];
@@ -759,8 +733,9 @@ __device__ __forceinline__ bool attend_block_res(AttendState& st, const uint32_t
             adig[rho] = __byte_perm(__byte_perm(bits[0], bits[1], 0x0040), __byte_perm(bits[2], bits[3], 0x0040), 0x5410);
         }
         // digits -> logits: v ~ step * (d0 + d1 / 254); a residual step is s / 254 (s is inside v)
-        const float unit = step * (1.f / 254.f) * (piece ? 1.f / 254.f : 1.f);
+        const float unit = p.sm_scale * step * (1.f / 254.f) * (piece ? 1.f / 254.f : 1.f);
         const uint32_t flip = (uint32_t)(r & 1) << 2;   // token 8 nt + r: odd rows have their halves swapped
+        const uint32_t score_row = kslot + kResOffScores + ((r & 3) * kScoreStride + 2 * j) * 4;
 #pragma unroll
         for (int nt = 0; nt < 8; ++nt) {
             const uint32_t row = kslot + (8 * nt + r) * 128;
@@ -770,19 +745,22 @@ __device__ __forceinline__ bool attend_block_res(AttendState& st, const uint32_t
             mma_s8_top(d0, d1, adig[2], adig[3], k0.z, k0.w);
             mma_s8_top(d0, d1, adig[4], adig[5], k1.x, k1.y);
             mma_s8_top(d0, d1, adig[6], adig[7], k1.z, k1.w);
-            s[nt][0] = fmaf((float)d0, unit, s[nt][0]);
-            s[nt][1] = fmaf((float)d1, unit, s[nt][1]);
+            // the scan's approximate logit (the q . k_quant term) is added once, in the rows of the first digit
+            float a0, a1;
+            asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];\n" : "=f"(a0), "=f"(a1) : "r"(score_row + nt * 32));
+            s[nt][0] = fmaf((float)d0, unit, piece ? 0.f : a0);
+            s[nt][1] = fmaf((float)d1, unit, piece ? 0.f : a1);
         }
     }
     __syncwarp();   // every lane is done reading the K slot
-    if (next_tile >= 0) res_copy_async(kslot, p, (uint32_t)next_tile, lane, kbar);
-    // rows r and r + 4 hold the two pieces of the same head: both get the sum
+    if (next_tile >= 0) res_copy_async(kslot, p, (uint32_t)next_tile, next_scores, lane, kbar);
+    // rows r and r + 4 hold the two digits' shares of the same head: both get the sum
 #pragma unroll
     for (int nt = 0; nt < 8; ++nt) {
         s[nt][0] += __shfl_xor_sync(kFull, s[nt][0], 16);
         s[nt][1] += __shfl_xor_sync(kFull, s[nt][1], 16);
     }
-    return attend_finish(st, s, vslot, vbar, phase, next_v, lane, rows, mine, logit_scale_log2);
+    return attend_finish(st, s, vslot, vbar, phase, next_v, lane, rows, mine, kLog2e);
 }
 
 // output channel of O fragment (n-tile nt, column n)

@@ -25,7 +25,7 @@ DEV_BAD_SEQ_LEN = 2
 
 EXPORTS = ["ffd_status_string", "ffd_workspace_bytes", "ffd_workspace_init", "ffd_quantize_keys", "ffd_decode",
            "ffd_decode_dense", "ffd_unpack_codes", "ffd_read_device_status", "ffd_profile_events", "ffd_decode_static",
-           "ffd_append_kv", "ffd_append_decode", "ffd_quantize_residual", "ffd_decode_residual"]
+           "ffd_append_kv", "ffd_append_decode", "ffd_quantize_residual", "ffd_decode_residual", "ffd_workspace_bytes_residual"]
 
 
 class FfdError(RuntimeError):
@@ -74,6 +74,7 @@ def load_library() -> ctypes.CDLL:
         lib.ffd_status_string.restype = ctypes.c_char_p
         lib.ffd_status_string.argtypes = [ctypes.c_int]
         lib.ffd_workspace_bytes.argtypes = [cfgp, i32, i32, ctypes.POINTER(ctypes.c_size_t)]
+        lib.ffd_workspace_bytes_residual.argtypes = [cfgp, i32, i32, ctypes.POINTER(ctypes.c_size_t)]
         lib.ffd_workspace_init.argtypes = [_vp, ctypes.c_size_t, _vp]
         lib.ffd_quantize_keys.argtypes = [cfgp, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, _vp]
         lib.ffd_decode.argtypes = [cfgp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, ctypes.c_float, _vp, _vp,
@@ -123,9 +124,19 @@ def ffd_workspace_bytes(cfg: Config, batch: int, max_blocks_per_seq: int) -> int
     return int(n.value)
 
 
-def new_workspace(cfg: Config, batch: int, max_blocks_per_seq: int, device="cuda", stream=None) -> torch.Tensor:
-    """Allocate (with torch) and initialise a workspace for this geometry."""
-    ws = torch.empty(ffd_workspace_bytes(cfg, batch, max_blocks_per_seq), dtype=torch.uint8, device=device)
+def ffd_workspace_bytes_residual(cfg: Config, batch: int, max_blocks_per_seq: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(load_library().ffd_workspace_bytes_residual(ctypes.byref(cfg.c()), batch, max_blocks_per_seq,
+                                                       ctypes.byref(n)), "ffd_workspace_bytes_residual")
+    return int(n.value)
+
+
+def new_workspace(cfg: Config, batch: int, max_blocks_per_seq: int, device="cuda", stream=None, *,
+                  residual: bool = False) -> torch.Tensor:
+    """Allocate (with torch) and initialise a workspace for this geometry (``residual``: one that also serves
+    ``ffd_decode_residual``)."""
+    size = (ffd_workspace_bytes_residual if residual else ffd_workspace_bytes)(cfg, batch, max_blocks_per_seq)
+    ws = torch.empty(size, dtype=torch.uint8, device=device)
     _check(load_library().ffd_workspace_init(_p(ws), ws.numel(), _stream(stream)), "ffd_workspace_init")
     return ws
 
@@ -257,9 +268,11 @@ class DeviceCache:
                           first_token, max_blocks_per_seq=self.w.max_blocks)
 
     def quantize_residual(self, first_token=None):
-        """The 8-bit residuals of the keys (after ``quantize``); allocates ``k_res`` on first use."""
+        """The 8-bit residuals of the keys (after ``quantize``); on first use allocates ``k_res`` and swaps the
+        workspace for one that also holds the residual decode's score tiles."""
         if getattr(self, "k_res", None) is None:
             self.k_res = torch.zeros(self.w.num_pages, self.w.Hkv, 64, 128, dtype=torch.int8, device=self.device)
+            self.workspace = new_workspace(self.cfg, self.w.B, self.w.max_blocks, self.device, residual=True)
         ffd_quantize_residual(self.cfg, self.k_cache, self.k_scales, self.k_res, self.block_table, self.seq_lens,
                               first_token, max_blocks_per_seq=self.w.max_blocks)
 
