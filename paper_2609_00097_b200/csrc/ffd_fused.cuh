@@ -726,7 +726,7 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
     int issued_bi = -1, issued_lb = -1;   // block whose K/V copies are already in flight
     bool ok = true;
     AttendState st;
-    uint32_t qb[RES ? 16 : 1];
+    uint32_t qb[RES ? 8 : 1];
     FFD_ACC_DECL;
     for (int bi = 0; ok; ++bi) {
         const int slot = bi & (kNB - 1), use = bi / kNB;

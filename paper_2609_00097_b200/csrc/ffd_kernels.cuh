@@ -671,15 +671,16 @@ __device__ __forceinline__ void res_copy_async(uint32_t slot, const DecodeParams
 }
 static_assert(kScoreTileFloats / 4 - 64 <= 16, "score tile: at most 80 chunks");
 
-// Per batch: qb = bf16 q of head r % 4 for this lane's 32 residual channels.
-__device__ __forceinline__ void attend_setup_res(AttendState& st, uint32_t (&qb)[16], const DecodeParams& p, int b, int g,
+// Per batch: qb = bf16 q of head r % 4 for the 16 residual channels whose digits this lane works out
+// (16j..16j+15 in rows r < 4, 64+16j..64+16j+15 in rows r + 4).
+__device__ __forceinline__ void attend_setup_res(AttendState& st, uint32_t (&qb)[8], const DecodeParams& p, int b, int g,
                                                  int lane) {
     const int r = lane >> 2, j = lane & 3, head = r & 3;
-    const __nv_bfloat16* qh = p.q + ((size_t)b * p.Hq + (size_t)g * p.G + head) * kD;
+    const __nv_bfloat16* qh = p.q + ((size_t)b * p.Hq + (size_t)g * p.G + head) * kD + 64 * (r >> 2) + 16 * j;
 #pragma unroll
-    for (int x = 0; x < 4; ++x) {
+    for (int x = 0; x < 2; ++x) {
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (head < p.G) v = *reinterpret_cast<const uint4*>(qh + 64 * (x >> 1) + 16 * j + 8 * (x & 1));
+        if (head < p.G) v = *reinterpret_cast<const uint4*>(qh + 8 * x);
         qb[4 * x + 0] = v.x; qb[4 * x + 1] = v.y; qb[4 * x + 2] = v.z; qb[4 * x + 3] = v.w;
     }
     attend_reset(st);
@@ -691,7 +692,7 @@ __device__ __forceinline__ float2 res_qs(uint32_t q2, uint32_t s2) {
     return make_float2(__uint_as_float(q2 << 16) * sf.x, __uint_as_float(q2 & 0xffff0000u) * sf.y);
 }
 
-__device__ __forceinline__ bool attend_block_res(AttendState& st, const uint32_t (&qb)[16], const DecodeParams& p,
+__device__ __forceinline__ bool attend_block_res(AttendState& st, const uint32_t (&qb)[8], const DecodeParams& p,
                                                  uint32_t kslot, uint32_t vslot, uint32_t kbar, uint32_t vbar,
                                                  uint32_t& phase, int next_tile, const float* next_scores,
                                                  const uint4* next_v, int lane, int rows, unsigned keep4) {
@@ -701,36 +702,45 @@ __device__ __forceinline__ bool attend_block_res(AttendState& st, const uint32_t
     if (!mbar_wait(kbar, phase & 1u)) return false;
     float s[8][2];
     {
-        // this lane's 32 scales: channels 16j..16j+15 and 64+16j..64+16j+15
-        uint4 sv[4];
-#pragma unroll
-        for (int x = 0; x < 4; ++x) sv[x] = lds128(kslot + kResOffScales + (8 * (x >> 1) + 2 * j + (x & 1)) * 16);
-        const uint32_t* s2 = reinterpret_cast<const uint32_t*>(sv);
+        // The lanes of rows r and r + 4 need the digits of the same 32 channels of the same head (one the first, the
+        // other the second digit): each works out both digits of 16 of them and they swap.  This lane's half:
+        // channels 16j..16j+15 (piece 0) or 64+16j..64+16j+15 (piece 1) = registers 4 piece .. 4 piece + 3.
+        const uint4 sa = lds128(kslot + kResOffScales + (8 * piece + 2 * j) * 16);
+        const uint4 sb = lds128(kslot + kResOffScales + (8 * piece + 2 * j + 1) * 16);
+        const uint32_t s2[8] = {sa.x, sa.y, sa.z, sa.w, sb.x, sb.y, sb.z, sb.w};
+        float2 v[8];
         float vmax = 0.f;
 #pragma unroll
-        for (int y = 0; y < 16; ++y) {
-            const float2 v = res_qs(qb[y], s2[y]);
-            vmax = fmaxf(vmax, fmaxf(fabsf(v.x), fabsf(v.y)));
+        for (int y = 0; y < 8; ++y) {
+            v[y] = res_qs(qb[y], s2[y]);
+            vmax = fmaxf(vmax, fmaxf(fabsf(v[y].x), fabsf(v[y].y)));
         }
         vmax = fmaxf(vmax, __shfl_xor_sync(kFull, vmax, 1));
         vmax = fmaxf(vmax, __shfl_xor_sync(kFull, vmax, 2));
+        vmax = fmaxf(vmax, __shfl_xor_sync(kFull, vmax, 16));
         const float inv = vmax > 0.f ? 127.f / vmax : 0.f, step = vmax * (1.f / 127.f);
         const float inv1 = inv * 254.f;
         constexpr float kMagic = 12582912.f;   // 1.5 * 2^23: adding it leaves rint(x) in the low mantissa bits
-        uint32_t adig[8];   // register rho: channels 4 rho .. 4 rho + 3 of the lane's 32, one digit per byte
+        uint32_t adig[8];   // register rho: channels 4 rho .. 4 rho + 3 of the 32, this row's digit in every byte
 #pragma unroll
-        for (int rho = 0; rho < 8; ++rho) {
-            uint32_t bits[4];
+        for (int x = 0; x < 4; ++x) {
+            uint32_t b0[4], b1[4];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                const float2 v = res_qs(qb[2 * rho + h], s2[2 * rho + h]);
-                const float t0x = fmaf(v.x, inv, kMagic), t0y = fmaf(v.y, inv, kMagic);
-                const float t1x = fmaf(fmaf(-(t0x - kMagic), step, v.x), inv1, kMagic);
-                const float t1y = fmaf(fmaf(-(t0y - kMagic), step, v.y), inv1, kMagic);
-                bits[2 * h] = __float_as_uint(piece ? t1x : t0x);
-                bits[2 * h + 1] = __float_as_uint(piece ? t1y : t0y);
+                const float2 vv = v[2 * x + h];
+                const float t0x = fmaf(vv.x, inv, kMagic), t0y = fmaf(vv.y, inv, kMagic);
+                b0[2 * h] = __float_as_uint(t0x);
+                b0[2 * h + 1] = __float_as_uint(t0y);
+                b1[2 * h] = __float_as_uint(fmaf(fmaf(-(t0x - kMagic), step, vv.x), inv1, kMagic));
+                b1[2 * h + 1] = __float_as_uint(fmaf(fmaf(-(t0y - kMagic), step, vv.y), inv1, kMagic));
             }
-            adig[rho] = __byte_perm(__byte_perm(bits[0], bits[1], 0x0040), __byte_perm(bits[2], bits[3], 0x0040), 0x5410);
+            const uint32_t d0 = __byte_perm(__byte_perm(b0[0], b0[1], 0x0040), __byte_perm(b0[2], b0[3], 0x0040), 0x5410);
+            const uint32_t d1 = __byte_perm(__byte_perm(b1[0], b1[1], 0x0040), __byte_perm(b1[2], b1[3], 0x0040), 0x5410);
+            // keep this row's digit of the own half, hand the other digit to the partner and take its half
+            const uint32_t got = __shfl_xor_sync(kFull, piece ? d0 : d1, 16);
+            const uint32_t own = piece ? d1 : d0;
+            adig[x] = piece ? got : own;
+            adig[4 + x] = piece ? own : got;
         }
         // digits -> logits: v ~ step * (d0 + d1 / 254); a residual step is s / 254 (s is inside v)
         const float unit = p.sm_scale * step * (1.f / 254.f) * (piece ? 1.f / 254.f : 1.f);
