@@ -42,6 +42,9 @@ def test_workspace_bytes_grows_with_geometry():
     b = ffd.ffd_workspace_bytes(cfg, 4, 2048)
     assert 0 < a < b
     assert a % 256 == 0
+    # the residual decode's workspace: the same plus the score tiles, whose size does not depend on the geometry
+    ra, rb = ffd.ffd_workspace_bytes_residual(cfg, 1, 512), ffd.ffd_workspace_bytes_residual(cfg, 4, 2048)
+    assert ra - a == rb - b == 192 * 8 * 32 * 4 * 72 * 4
 
 
 @pytest.mark.parametrize("field,value,status", [
@@ -91,6 +94,19 @@ def test_null_and_range_arguments_are_rejected_before_any_launch(lib):
                                  ctypes.c_float(6.0), fake, None, None, None, fake, 1 << 30, None) == 1
     assert lib.ffd_append_decode(ctypes.byref(cfg), fake, fake, fake, fake, fake, fake, fake, None, fake, 1, 16, 16,
                                  ctypes.c_float(-1.0), fake, None, None, None, fake, 1 << 30, None) == 6
+    # 2 + 8 bit key format: NULL residuals, misaligned residuals, a workspace that only fits the 16-bit decode
+    assert lib.ffd_quantize_residual(ctypes.byref(cfg), fake, fake, None, None, fake, None, 1, 16, 16, None) == 1
+    assert lib.ffd_quantize_residual(ctypes.byref(cfg), fake, fake, odd, None, fake, None, 1, 16, 16, None) == 4
+    assert lib.ffd_quantize_residual(ctypes.byref(cfg), fake, fake, fake, None, fake, None, 1, 16, 0, None) == 2
+    assert lib.ffd_decode_residual(ctypes.byref(cfg), fake, None, fake, fake, fake, None, fake, 1, 16, 16,
+                                   ctypes.c_float(6.0), fake, None, None, None, fake, 1 << 30, None) == 1
+    assert lib.ffd_decode_residual(ctypes.byref(cfg), fake, odd, fake, fake, fake, None, fake, 1, 16, 16,
+                                   ctypes.c_float(6.0), fake, None, None, None, fake, 1 << 30, None) == 4
+    plain = ffd.ffd_workspace_bytes(ffd.Config(32, 8), 1, 16)
+    assert lib.ffd_decode_residual(ctypes.byref(cfg), fake, fake, fake, fake, fake, None, fake, 1, 16, 16,
+                                   ctypes.c_float(6.0), fake, None, None, None, fake, plain, None) == 5
+    assert lib.ffd_decode_residual(ctypes.byref(cfg), fake, fake, fake, fake, fake, None, fake, 1, 16, 16,
+                                   ctypes.c_float(float("nan")), fake, None, None, None, fake, 1 << 30, None) == 6
     assert lib.ffd_read_device_status(None, None, None) == 1
 
 

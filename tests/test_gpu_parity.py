@@ -89,8 +89,10 @@ def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None, k_res=Non
     for b, h in rows:
         nb = w.num_blocks(b)
         assert np.all(kept[b, h, nb:] == 255), "mask written past the sequence's blocks"
-        # debug output: fast-scan values carry the tensor-core accumulation error (~2e-6 of the accumulator size)
-        assert np.all(np.abs(bm[b, h, :nb] - r.block_max[b, h, :nb]) < 1e-4 + 6e-6 * np.abs(r.block_max[b, h, :nb]))
+        # debug output: fast-scan values carry the tensor-core accumulation error, a few 1e-6 of the accumulator's
+        # size, which can be several times the result's (the level offset is subtracted afterwards); decisions near
+        # the threshold do not rest on these values (the kernel redoes them precisely), see the mask check below
+        assert np.all(np.abs(bm[b, h, :nb] - r.block_max[b, h, :nb]) < 1e-4 + 2e-5 * np.abs(r.block_max[b, h, :nb]))
         diff = kept[b, h, :nb] != r.kept[b, h, :nb]
         if diff.any():
             differs = True
@@ -214,6 +216,70 @@ def test_tail_requantize_only_touches_the_last_block(ffd, oracle):
         assert torch.equal(dc.k_quant[last], q0[last]) and torch.equal(dc.k_scales[last], s0[last])
         if nb > 1:
             assert torch.all(dc.k_quant[w.page(b, 0)] == 0x55)
+
+
+def test_residual_tail_requantize_only_touches_the_last_block(ffd, oracle):
+    """With first_token the residuals of the block the newest token fell into are redone, nothing else."""
+    w = make_workload("C5", B=3, lens=(700, 2000))
+    dc = ffd.DeviceCache(w)
+    dc.quantize()
+    dc.quantize_residual()
+    r0 = dc.k_res.clone()
+    dc.k_res.fill_(0x55)
+    first = torch.from_numpy(w.seq_lens - 1).to("cuda")
+    dc.quantize(first_token=first)
+    dc.quantize_residual(first_token=first)
+    torch.cuda.synchronize()
+    for b in range(w.B):
+        nb = w.num_blocks(b)
+        assert torch.equal(dc.k_res[w.page(b, nb - 1)], r0[w.page(b, nb - 1)])
+        if nb > 1:
+            assert torch.all(dc.k_res[w.page(b, 0)] == 0x55)
+
+
+def test_residual_decode_edge_cases(ffd, oracle):
+    """Empty and one-token sequences, G = 1 and G = 2 groups, no sink, more local blocks than the pseudo-max kernel
+    has warps, a bad page (skipped and reported), bf16 output = rounding of the fp32 output."""
+    import paper_2609_00097_b200.workloads as W
+    w = make_workload("C5", B=3, lens=(100, 400))
+    w.seq_lens[:] = np.array([0, 1, int(w.seq_lens[2])], dtype=np.int32)
+    dc = ffd.DeviceCache(w)
+    codes, scales = check_quantize(ffd, oracle, w, dc)
+    k_res = check_residual(ffd, oracle, w, dc, codes, scales)
+    dc.out.fill_(7.0)
+    dc.decode_residual(6.0)
+    assert torch.all(dc.out[0] == 0) and torch.all(torch.isneginf(dc.lse[0]))
+    want = w.v_cache[w.page(1, 0)][:, 0].float().repeat_interleave(w.G, dim=0)   # the single token's value rows
+    assert (dc.out[1].cpu() - want).abs().max().item() < 1e-6
+    check_decode(ffd, oracle, w, dc, codes, scales, 6.0, k_res=k_res, units=[(b, h) for b in (1, 2) for h in range(w.Hq)])
+    try:
+        for G, Hkv, n_sink, n_local in [(1, 3, 1, 16), (2, 2, 0, 40), (4, 1, 2, 1)]:
+            W.CONFIGS["res_edge"] = dict(seed=5 + G, B=3, Hq=G * Hkv, Hkv=Hkv, lens=(65, 4000), frac=0.02, amp=3.0,
+                                         sink=bool(n_sink), deltas=(6.0,), paged=True, spare_pages=2)
+            w = make_workload("res_edge")
+            for out_dtype in (1, 0):
+                cfg = ffd.Config(G * Hkv, Hkv, n_sink_blocks=n_sink, n_local_blocks=n_local, out_dtype=out_dtype)
+                dc = ffd.DeviceCache(w, cfg)
+                codes, scales = check_quantize(ffd, oracle, w, dc)
+                k_res = check_residual(ffd, oracle, w, dc, codes, scales)
+                if out_dtype == 1:
+                    for delta in (0.0, 6.0, INF):
+                        check_decode(ffd, oracle, w, dc, codes, scales, delta, k_res=k_res)
+                    out32 = dc.out.clone()
+                else:
+                    dc.decode_residual(INF)
+                    assert torch.equal(dc.out, out32.to(torch.bfloat16))
+    finally:
+        W.CONFIGS.pop("res_edge", None)
+    # a page-table entry out of range: that block is skipped and the status word says so; nothing faults
+    w = make_workload("C5", B=2, lens=(500, 900))
+    dc = ffd.DeviceCache(w)
+    dc.quantize()
+    dc.quantize_residual()
+    dc.block_table[1, 2] = w.num_pages + 7
+    dc.decode_residual(6.0)
+    assert ffd.ffd_read_device_status(dc.workspace) & ffd.DEV_BAD_PAGE
+    assert torch.isfinite(dc.out.float()).all()
 
 
 def test_empty_and_single_token_sequences(ffd, oracle):
@@ -537,6 +603,23 @@ def test_very_long_contexts_on_sampled_heads(ffd, oracle, lens, short):
     assert ffd.ffd_read_device_status(dc.workspace) == 0
 
 
+def test_residual_with_many_short_sequences(ffd, oracle):
+    """The serving-size batch of short sequences on the 2 + 8 bit format: the score tiles of items that only some
+    scan warps take part in."""
+    import paper_2609_00097_b200.workloads as W
+    try:
+        W.CONFIGS["many_short"] = dict(seed=78, B=600, Hq=4, Hkv=2, lens=(1, 300), frac=0.02, amp=3.0, sink=True,
+                                       deltas=(6.0,), paged=True, spare_pages=5)
+        w = make_workload("many_short")
+    finally:
+        W.CONFIGS.pop("many_short", None)
+    dc = ffd.DeviceCache(w, ffd.Config(4, 2))
+    codes, scales = check_quantize(ffd, oracle, w, dc)
+    k_res = check_residual(ffd, oracle, w, dc, codes, scales)
+    for delta in (6.0, INF):
+        check_decode(ffd, oracle, w, dc, codes, scales, delta, k_res=k_res)
+
+
 # full-size configurations: the oracle checks a sample of (sequence, head) rows one by one
 FULL = [
     ("C2", dict(), 8),
@@ -570,3 +653,10 @@ def test_full_size_configs_on_sampled_heads(ffd, oracle, name, kw, n_units):
     for delta in w.deltas:
         check_decode(ffd, oracle, w, dc, codes, scales, delta, units=units)
     check_dense(ffd, oracle, w, dc, units=units[:2])
+    if name in ("C3", "C5"):   # the 2 + 8 bit key format at full size: residuals of sampled pages, sampled heads
+        dc.quantize_residual()
+        k_res = oracle.quantize_residual(w.bits("k_cache"), codes, scales, w.block_table, w.seq_lens, w.max_blocks)
+        for page in rng.choice(np.where(mapped)[0], size=64, replace=False):
+            assert np.array_equal(dc.k_res[int(page)].cpu().numpy(), k_res[page])
+        dc.k_cache = None
+        check_decode(ffd, oracle, w, dc, codes, scales, w.deltas[0], units=units, k_res=k_res)
