@@ -120,6 +120,16 @@ ffd_status ffd_quantize_residual(const ffd_config* cfg, const void* k_cache, con
                                  int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages, void* stream);
 
 /*
+ * ffd_quantize_keys and ffd_quantize_residual in one call.  With first_token (a decode step: only the block the
+ * newest token fell into is redone) both are written by a single kernel launch; without it the two whole-cache
+ * kernels run one after the other.  Results equal those of the two separate calls.
+ */
+ffd_status ffd_quantize_keys_residual(const ffd_config* cfg, const void* k_cache, void* k_quant, void* k_scales,
+                                      void* k_res, const int32_t* block_table, const int32_t* seq_lens,
+                                      const int32_t* first_token, int32_t batch, int32_t max_blocks_per_seq,
+                                      int32_t num_pages, void* stream);
+
+/*
  * Cache append for one decode step, all indices on the device (Sec. 3.3: a cache that a captured graph can replay
  * needs tensor indices instead of host-side lengths; App. A.1 for the quantizer).  For every sequence b with
  * pos = seq_lens[b] < max_blocks_per_seq*64: the rows k_new[b, g, :] and v_new[b, g, :] (bf16 [B, Hkv, 128], device)

@@ -68,7 +68,11 @@ __device__ __forceinline__ void quantize_tile(const __nv_bfloat16* sk, float* ss
     reinterpret_cast<uint4*>(codes_out)[mt * 32 + lane] = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-__global__ void __launch_bounds__(128) quantize_kernel(QuantParams p) {
+__device__ __forceinline__ void residual_rows(const __nv_bfloat16* sk, const float* ss, const float* sinv, int rows,
+                                              int8_t* res_out, int tid);
+
+// k_res != nullptr: also writes the tile's 8-bit residuals (see residual_kernel)
+__global__ void __launch_bounds__(128) quantize_kernel(QuantParams p, int8_t* k_res) {
     const int g = blockIdx.y, b = blockIdx.z;
     pdl_launch_dependents();
     pdl_wait();
@@ -78,7 +82,7 @@ __global__ void __launch_bounds__(128) quantize_kernel(QuantParams p) {
     const int nb = (n + kBlk - 1) / kBlk;
     const int first = p.first_token ? max(p.first_token[b], 0) / kBlk : 0;
     __shared__ __align__(16) __nv_bfloat16 sk[kBlk * kD];
-    __shared__ float ss[kD];
+    __shared__ float ss[kD], sinv[kD];
     const int tid = threadIdx.x;
     // the grid's x extent is bounded; every CTA walks its share of the blocks that need (re)quantizing
     for (int blk = first + blockIdx.x; blk < nb; blk += gridDim.x) {
@@ -93,6 +97,11 @@ __global__ void __launch_bounds__(128) quantize_kernel(QuantParams p) {
         for (int x = 0; x < 8; ++x) dst[tid + 128 * x] = ldg_stream(src + tid + 128 * x);
         __syncthreads();
         quantize_tile(sk, ss, rows, p.k_scales + tile * kD, p.k_quant + tile * kCodeBytes, tid);
+        if (k_res) {   // (uniform over the CTA)
+            sinv[tid] = __fdiv_rn(254.f, ss[tid]);
+            __syncthreads();
+            residual_rows(sk, ss, sinv, rows, k_res + tile * kBlk * kD, tid);
+        }
     }
 }
 
@@ -141,27 +150,31 @@ __global__ void __launch_bounds__(128) residual_kernel(ResidualParams p) {
         __syncthreads();   // the previous block's tile is no longer needed
 #pragma unroll
         for (int x = 0; x < 8; ++x) dst[tid + 128 * x] = ldg_stream(src + tid + 128 * x);
-        {
-            const float s = __half2float(p.k_scales[tile * kD + tid]);
-            ss[tid] = s;
-            sinv[tid] = __fdiv_rn(254.f, s);
-        }
+        ss[tid] = __half2float(p.k_scales[tile * kD + tid]);
+        sinv[tid] = __fdiv_rn(254.f, ss[tid]);
         __syncthreads();
-        uint4* out = reinterpret_cast<uint4*>(p.k_res + tile * kBlk * kD);
+        residual_rows(sk, ss, sinv, rows, p.k_res + tile * kBlk * kD, tid);
+    }
+}
+
+// the residual codes of a staged tile (sk) given its scales (ss) and 254 / scale (sinv), by 128 threads: 16 consecutive
+// channels of one token per thread and pass; rows past the sequence end get 0
+__device__ __forceinline__ void residual_rows(const __nv_bfloat16* sk, const float* ss, const float* sinv, int rows,
+                                              int8_t* res_out, int tid) {
+    uint4* out = reinterpret_cast<uint4*>(res_out);
 #pragma unroll
-        for (int x = 0; x < 4; ++x) {   // 16 consecutive channels of one token per thread and pass
-            const int chunk = tid + 128 * x, row = chunk >> 3, c0 = (chunk & 7) * 16;
-            uint32_t w[4] = {0u, 0u, 0u, 0u};
-            if (row < rows) {
+    for (int x = 0; x < 4; ++x) {
+        const int chunk = tid + 128 * x, row = chunk >> 3, c0 = (chunk & 7) * 16;
+        uint32_t w[4] = {0u, 0u, 0u, 0u};
+        if (row < rows) {
 #pragma unroll
-                for (int u = 0; u < 16; ++u) {
-                    const int c = c0 + u;
-                    const int code = residual_code(__bfloat162float(sk[row * kD + c]), ss[c], sinv[c]);
-                    w[u >> 2] |= (uint32_t)(code & 0xff) << (8 * (u & 3));
-                }
+            for (int u = 0; u < 16; ++u) {
+                const int c = c0 + u;
+                const int code = residual_code(__bfloat162float(sk[row * kD + c]), ss[c], sinv[c]);
+                w[u >> 2] |= (uint32_t)(code & 0xff) << (8 * (u & 3));
             }
-            out[chunk] = make_uint4(w[0], w[1], w[2], w[3]);
         }
+        out[chunk] = make_uint4(w[0], w[1], w[2], w[3]);
     }
 }
 
@@ -924,6 +937,10 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
 
 using namespace ffd;
 
+static ffd_status quantize_impl(const ffd_config* cfg, const void* k_cache, void* k_quant, void* k_scales, void* k_res,
+                                const int32_t* block_table, const int32_t* seq_lens, const int32_t* first_token,
+                                int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages, void* stream);
+
 extern "C" {
 
 const char* ffd_status_string(ffd_status status) {
@@ -974,6 +991,27 @@ ffd_status ffd_workspace_init(void* workspace, size_t workspace_bytes, void* str
 ffd_status ffd_quantize_keys(const ffd_config* cfg, const void* k_cache, void* k_quant, void* k_scales,
                              const int32_t* block_table, const int32_t* seq_lens, const int32_t* first_token,
                              int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages, void* stream) {
+    return quantize_impl(cfg, k_cache, k_quant, k_scales, nullptr, block_table, seq_lens, first_token, batch,
+                         max_blocks_per_seq, num_pages, stream);
+}
+
+ffd_status ffd_quantize_keys_residual(const ffd_config* cfg, const void* k_cache, void* k_quant, void* k_scales,
+                                      void* k_res, const int32_t* block_table, const int32_t* seq_lens,
+                                      const int32_t* first_token, int32_t batch, int32_t max_blocks_per_seq,
+                                      int32_t num_pages, void* stream) {
+    if (!k_res) return FFD_ERR_NULL;
+    if (misaligned(k_res)) return FFD_ERR_ALIGN;
+    return quantize_impl(cfg, k_cache, k_quant, k_scales, k_res, block_table, seq_lens, first_token, batch,
+                         max_blocks_per_seq, num_pages, stream);
+}
+
+}   // extern "C"
+
+// thumbnails, and with k_res also the residuals: in the same launch when only tail blocks are redone, else by the
+// streaming kernel followed by the residual kernel
+static ffd_status quantize_impl(const ffd_config* cfg, const void* k_cache, void* k_quant, void* k_scales, void* k_res,
+                                const int32_t* block_table, const int32_t* seq_lens, const int32_t* first_token,
+                                int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages, void* stream) {
     ffd_status st = check_config(cfg);
     if (st) return st;
     if (!k_cache || !k_quant || !k_scales || !seq_lens) return FFD_ERR_NULL;
@@ -992,7 +1030,7 @@ ffd_status ffd_quantize_keys(const ffd_config* cfg, const void* k_cache, void* k
     const int wide = max_blocks_per_seq < 64 ? max_blocks_per_seq : 64;
     if (first_token) {
         launch_pdl(quantize_kernel, dim3(wide < 2 ? wide : 2, cfg->num_kv_heads, batch), dim3(128), 0,
-                   static_cast<cudaStream_t>(stream), p);
+                   static_cast<cudaStream_t>(stream), p, static_cast<int8_t*>(k_res));
     } else {   // a whole cache: the streaming kernel; twelve CTAs fit an SM, and four times as many as fit at once are
                // launched so that sequences of different lengths even out
         if (cudaFuncSetAttribute(quantize_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kQbSmem) != cudaSuccess)
@@ -1002,9 +1040,17 @@ ffd_status ffd_quantize_keys(const ffd_config* cfg, const void* k_cache, void* k
         if (x > tiles) x = tiles;
         launch_pdl(quantize_bulk_kernel, dim3((unsigned)x, batch), dim3(kQbThreads), kQbSmem,
                    static_cast<cudaStream_t>(stream), p);
+        if (k_res) {
+            st = launch_status();
+            if (st) return st;
+            return ffd_quantize_residual(cfg, k_cache, k_scales, k_res, block_table, seq_lens, nullptr, batch,
+                                         max_blocks_per_seq, num_pages, stream);
+        }
     }
     return launch_status();
 }
+
+extern "C" {
 
 ffd_status ffd_quantize_residual(const ffd_config* cfg, const void* k_cache, const void* k_scales, void* k_res,
                                  const int32_t* block_table, const int32_t* seq_lens, const int32_t* first_token,

@@ -25,7 +25,8 @@ DEV_BAD_SEQ_LEN = 2
 
 EXPORTS = ["ffd_status_string", "ffd_workspace_bytes", "ffd_workspace_init", "ffd_quantize_keys", "ffd_decode",
            "ffd_decode_dense", "ffd_unpack_codes", "ffd_read_device_status", "ffd_profile_events", "ffd_decode_static",
-           "ffd_append_kv", "ffd_append_decode", "ffd_quantize_residual", "ffd_decode_residual", "ffd_workspace_bytes_residual"]
+           "ffd_append_kv", "ffd_append_decode", "ffd_quantize_residual", "ffd_decode_residual", "ffd_workspace_bytes_residual",
+           "ffd_quantize_keys_residual"]
 
 
 class FfdError(RuntimeError):
@@ -92,6 +93,7 @@ def load_library() -> ctypes.CDLL:
                                           ctypes.c_float, _vp, _vp, _vp, _vp, _vp, ctypes.c_size_t, _vp]
         lib.ffd_quantize_residual.argtypes = [cfgp, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, _vp]
         lib.ffd_decode_residual.argtypes = lib.ffd_decode.argtypes
+        lib.ffd_quantize_keys_residual.argtypes = [cfgp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, _vp]
         for name in EXPORTS:
             if name != "ffd_status_string":
                 getattr(lib, name).restype = ctypes.c_int
@@ -155,6 +157,14 @@ def ffd_quantize_residual(cfg: Config, k_cache, k_scales, k_res, block_table, se
                                                 _p(block_table), _p(seq_lens), _p(first_token), seq_lens.numel(),
                                                 max_blocks_per_seq, k_cache.shape[0], _stream(stream)),
            "ffd_quantize_residual")
+
+
+def ffd_quantize_keys_residual(cfg: Config, k_cache, k_quant, k_scales, k_res, block_table, seq_lens, first_token=None,
+                               *, max_blocks_per_seq: int, stream=None):
+    _check(load_library().ffd_quantize_keys_residual(ctypes.byref(cfg.c()), _p(k_cache), _p(k_quant), _p(k_scales),
+                                                     _p(k_res), _p(block_table), _p(seq_lens), _p(first_token),
+                                                     seq_lens.numel(), max_blocks_per_seq, k_cache.shape[0],
+                                                     _stream(stream)), "ffd_quantize_keys_residual")
 
 
 def ffd_decode_residual(cfg: Config, q, k_res, v_cache, k_quant, k_scales, block_table, seq_lens, delta: float, out, *,
@@ -275,6 +285,13 @@ class DeviceCache:
             self.workspace = new_workspace(self.cfg, self.w.B, self.w.max_blocks, self.device, residual=True)
         ffd_quantize_residual(self.cfg, self.k_cache, self.k_scales, self.k_res, self.block_table, self.seq_lens,
                               first_token, max_blocks_per_seq=self.w.max_blocks)
+
+    def quantize_both(self, first_token=None):
+        """Thumbnails and residuals in one call (one launch when ``first_token`` is given)."""
+        if getattr(self, "k_res", None) is None:
+            self.quantize_residual()
+        ffd_quantize_keys_residual(self.cfg, self.k_cache, self.k_quant, self.k_scales, self.k_res, self.block_table,
+                                   self.seq_lens, first_token, max_blocks_per_seq=self.w.max_blocks)
 
     def decode_residual(self, delta, kept_mask=None, block_max=None):
         ffd_decode_residual(self.cfg, self.q, self.k_res, self.v_cache, self.k_quant, self.k_scales, self.block_table,

@@ -98,6 +98,9 @@ def test_null_and_range_arguments_are_rejected_before_any_launch(lib):
     assert lib.ffd_quantize_residual(ctypes.byref(cfg), fake, fake, None, None, fake, None, 1, 16, 16, None) == 1
     assert lib.ffd_quantize_residual(ctypes.byref(cfg), fake, fake, odd, None, fake, None, 1, 16, 16, None) == 4
     assert lib.ffd_quantize_residual(ctypes.byref(cfg), fake, fake, fake, None, fake, None, 1, 16, 0, None) == 2
+    assert lib.ffd_quantize_keys_residual(ctypes.byref(cfg), fake, fake, fake, None, None, fake, None, 1, 16, 16, None) == 1
+    assert lib.ffd_quantize_keys_residual(ctypes.byref(cfg), fake, fake, fake, odd, None, fake, None, 1, 16, 16, None) == 4
+    assert lib.ffd_quantize_keys_residual(ctypes.byref(cfg), None, fake, fake, fake, None, fake, None, 1, 16, 16, None) == 1
     assert lib.ffd_decode_residual(ctypes.byref(cfg), fake, None, fake, fake, fake, None, fake, 1, 16, 16,
                                    ctypes.c_float(6.0), fake, None, None, None, fake, 1 << 30, None) == 1
     assert lib.ffd_decode_residual(ctypes.byref(cfg), fake, odd, fake, fake, fake, None, fake, 1, 16, 16,

@@ -235,6 +235,18 @@ def test_residual_tail_requantize_only_touches_the_last_block(ffd, oracle):
         assert torch.equal(dc.k_res[w.page(b, nb - 1)], r0[w.page(b, nb - 1)])
         if nb > 1:
             assert torch.all(dc.k_res[w.page(b, 0)] == 0x55)
+    # the combined call: one launch for the tail, two kernels for a whole cache; same bytes either way
+    q0, s0 = dc.k_quant.clone(), dc.k_scales.clone()
+    for ft in (first, None):
+        dc.k_res.fill_(0x55)
+        dc.k_quant.fill_(0x55)
+        dc.quantize_both(first_token=ft)
+        torch.cuda.synchronize()
+        for b in range(w.B):
+            pages = [w.page(b, w.num_blocks(b) - 1)] if ft is not None else [w.page(b, k) for k in range(w.num_blocks(b))]
+            for pg in pages:
+                assert torch.equal(dc.k_res[pg], r0[pg]) and torch.equal(dc.k_quant[pg], q0[pg])
+                assert torch.equal(dc.k_scales[pg], s0[pg])
 
 
 def test_residual_decode_edge_cases(ffd, oracle):
