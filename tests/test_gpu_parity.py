@@ -218,6 +218,67 @@ def test_tail_requantize_only_touches_the_last_block(ffd, oracle):
             assert torch.all(dc.k_quant[w.page(b, 0)] == 0x55)
 
 
+def test_residual_serving_loop_from_one_graph(ffd, oracle):
+    """The 2 + 8 bit format's serving step -- append a token, redo thumbnails and residuals of its block, decode from
+    the residuals -- captured once and replayed token after token; after every replay the cache tiles, the lengths and
+    the output equal those of the same steps run eagerly on a second copy, and the last output matches the oracle's
+    Dequant refinement of the lengthened sequences."""
+    w = make_workload("C5", B=3, lens=(700, 2000))
+    full = w.seq_lens.copy()
+    steps = 70                                  # crosses a block boundary in every sequence
+    w.seq_lens[:] = full - steps
+    a, b = ffd.DeviceCache(w), ffd.DeviceCache(w)
+    for dc in (a, b):
+        dc.quantize()
+        dc.quantize_residual()
+    k_new = torch.zeros(w.B, w.Hkv, 128, dtype=torch.bfloat16, device="cuda")
+    v_new = torch.zeros_like(k_new)
+    first = torch.zeros(w.B, dtype=torch.int32, device="cuda")
+
+    def step(dc):
+        first.copy_(dc.seq_lens)                # the position the new token goes to = start of the redone range
+        dc.append(k_new, v_new)
+        dc.quantize_both(first_token=first)
+        dc.decode_residual(6.0)
+
+    def rows(t):
+        for i in range(w.B):
+            pos = full[i] - steps + t
+            pg = w.page(i, pos // 64)
+            k_new[i].copy_(w.k_cache[pg, :, pos % 64])
+            v_new[i].copy_(w.v_cache[pg, :, pos % 64])
+
+    rows(0)
+    graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    lens0 = a.seq_lens.clone()
+    with torch.cuda.stream(side):
+        step(a)                                 # warm-up outside the capture ...
+        torch.cuda.synchronize()
+        a.seq_lens.copy_(lens0)                 # ... undone: the token is appended again by the first replay
+        with torch.cuda.graph(graph, stream=side):
+            step(a)
+    torch.cuda.synchronize()
+    a.seq_lens.copy_(lens0)
+    for t in range(steps):
+        rows(t)
+        graph.replay()
+        step(b)
+        torch.cuda.synchronize()
+        assert torch.equal(a.seq_lens, b.seq_lens)
+        assert (a.out - b.out).abs().max().item() <= 1e-6
+    assert ffd.ffd_read_device_status(a.workspace) == 0
+    w.seq_lens[:] = full
+    assert np.array_equal(a.seq_lens.cpu().numpy(), full)
+    codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
+    k_res = oracle.quantize_residual(w.bits("k_cache"), codes, scales, w.block_table, w.seq_lens, w.max_blocks)
+    _, mapped = valid_row_mask(w)
+    assert np.array_equal(a.k_res.cpu().numpy()[mapped], k_res[mapped])
+    r = oracle.decode(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), codes, scales, w.block_table, w.seq_lens,
+                      w.max_blocks, 6.0, k_res=k_res)
+    err = np.abs(a.out.cpu().numpy().astype(np.float64) - r.out)
+    assert err.max() < OUT_MAX_EXPECTED and np.abs(a.lse.cpu().numpy() - r.lse).max() < 1e-3
+
+
 def test_residual_tail_requantize_only_touches_the_last_block(ffd, oracle):
     """With first_token the residuals of the block the newest token fell into are redone, nothing else."""
     w = make_workload("C5", B=3, lens=(700, 2000))
