@@ -676,6 +676,30 @@ def test_very_long_contexts_on_sampled_heads(ffd, oracle, lens, short):
     assert ffd.ffd_read_device_status(dc.workspace) == 0
 
 
+def test_global_approximate_max_rule_through_the_configuration(ffd, oracle):
+    """Sec. 5.2 compares the pseudo-max with the two-phase rule that thresholds against the global approximate
+    maximum.  That rule is the library's own with an empty sink set and a local set that covers the whole sequence
+    (the pseudo-max kernel then scans every block first): the kept set must be exactly {bm >= max bm - delta}, a
+    subset of what the default sets keep, and the no-sink workload -- where the default rule falls back to keeping
+    everything -- becomes sparse again."""
+    for name, kw in (("C2", dict(N=8192, tail=5)), ("C2", dict(N=6000, sink=False)), ("C5", dict(B=3, lens=(700, 3000)))):
+        w = make_workload(name, **kw)
+        cfg = ffd.Config(w.Hq, w.Hkv, n_sink_blocks=0, n_local_blocks=w.max_blocks)
+        dc = ffd.DeviceCache(w, cfg)
+        codes, scales = check_quantize(ffd, oracle, w, dc)
+        for delta in (4.0, 6.0):
+            r = check_decode(ffd, oracle, w, dc, codes, scales, delta)
+            default = oracle.decode(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), codes, scales, w.block_table,
+                                    w.seq_lens, w.max_blocks, delta)
+            for b in range(w.B):
+                nb = w.num_blocks(b)
+                bm = r.block_max[b, :, :nb]
+                assert np.array_equal(r.kept[b, :, :nb].astype(bool), bm >= bm.max(-1, keepdims=True) - delta)
+                assert np.all(default.kept[b, :, :nb] >= r.kept[b, :, :nb])
+        if kw.get("sink") is False:
+            assert default.kept[0, :, : w.num_blocks(0)].mean() > 0.9 and r.kept[0, :, : w.num_blocks(0)].mean() < 0.2
+
+
 def test_residual_with_many_short_sequences(ffd, oracle):
     """The serving-size batch of short sequences on the 2 + 8 bit format: the score tiles of items that only some
     scan warps take part in."""
