@@ -520,7 +520,9 @@ __device__ __noinline__ float scan_block_precise(const uint4* codes_tile, const 
 
 // RES (2 + 8 bit key format): the per-token approximate logits of every block that may be kept are left in the
 // CTA's ring of score tiles in global memory (tile (batch slot, block) -- free again when the attend warps have
-// released the batch slot, which the scheduler waits for before it publishes into it).
+// released the batch slot, which the scheduler waits for before it publishes into it).  Writer and reader are threads
+// of this CTA: the release of the full barrier's arrive and the acquire of the attend warp's wait order the stores
+// before the reader's copies (a device-scope fence in between measured 1 - 3 us per step and buys nothing).
 template <bool RES>
 __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* smem, int w, int lane) {
     const int r = lane >> 2, j = lane & 3;
