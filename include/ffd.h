@@ -148,6 +148,15 @@ ffd_status ffd_append_kv(const ffd_config* cfg, const void* k_new, const void* v
                          void* stream);
 
 /*
+ * ffd_append_kv for the 2 + 8 bit key format: the residuals (k_res) of the block the new token falls into are redone
+ * together with its thumbnails, in the same two launches.  Everything else as for ffd_append_kv.
+ */
+ffd_status ffd_append_kv_residual(const ffd_config* cfg, const void* k_new, const void* v_new, void* k_cache,
+                                  void* v_cache, void* k_quant, void* k_scales, void* k_res, const int32_t* block_table,
+                                  int32_t* seq_lens, int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages,
+                                  void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * One sparse decode step (Alg. 1; Sec. 3.2 Eq. 1 and the pseudo-max equation; Sec. 3.3 kernel steps).
  * Per query head h of sequence b, with sm = sm_scale and khat = (code - 1.5) * scale:
  *   approx[t]  = sm * sum_c q[c] * khat[t,c]                      every valid token t

@@ -335,6 +335,7 @@ struct AppendParams {
     int32_t* seq_lens;
     uint32_t* status;
     int Hkv, max_blocks, num_pages;
+    int8_t* k_res;                // nullable: 2 + 8 bit key format, the block's residuals are redone too
 };
 
 // One CTA of 128 threads (one per channel) per (KV head, sequence): the new token's K and V rows go to position
@@ -368,6 +369,12 @@ __global__ void __launch_bounds__(128) append_kernel(AppendParams p) {
     sk[row * kD + tid] = kn;
     __syncthreads();
     quantize_tile(sk, ss, row + 1, p.k_scales + tile * kD, p.k_quant + tile * kCodeBytes, tid);
+    if (p.k_res) {   // (uniform over the CTA)
+        __shared__ float sinv[kD];
+        sinv[tid] = __fdiv_rn(254.f, ss[tid]);
+        __syncthreads();
+        residual_rows(sk, ss, sinv, row + 1, p.k_res + tile * kBlk * kD, tid);
+    }
 }
 
 // after every CTA of append_kernel has read the lengths: one more token per sequence that had room
@@ -1077,10 +1084,10 @@ ffd_status ffd_quantize_residual(const ffd_config* cfg, const void* k_cache, con
     return launch_status();
 }
 
-ffd_status ffd_append_kv(const ffd_config* cfg, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
-                         void* k_quant, void* k_scales, const int32_t* block_table, int32_t* seq_lens, int32_t batch,
-                         int32_t max_blocks_per_seq, int32_t num_pages, void* workspace, size_t workspace_bytes,
-                         void* stream) {
+static ffd_status append_impl(const ffd_config* cfg, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                              void* k_quant, void* k_scales, void* k_res, const int32_t* block_table, int32_t* seq_lens,
+                              int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages, void* workspace,
+                              size_t workspace_bytes, void* stream) {
     ffd_status st = check_config(cfg);
     if (st) return st;
     if (!k_new || !v_new || !k_cache || !v_cache || !k_quant || !k_scales || !seq_lens || !workspace) return FFD_ERR_NULL;
@@ -1088,18 +1095,36 @@ ffd_status ffd_append_kv(const ffd_config* cfg, const void* k_new, const void* v
     if (st) return st;
     if (cfg->num_kv_heads > 65535) return FFD_ERR_SHAPE;
     if (workspace_bytes < 256) return FFD_ERR_WORKSPACE;
-    const void* ptrs[] = {k_new, v_new, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, workspace};
+    const void* ptrs[] = {k_new, v_new, k_cache, v_cache, k_quant, k_scales, k_res, block_table, seq_lens, workspace};
     for (const void* ptr : ptrs)
         if (ptr && misaligned(ptr)) return FFD_ERR_ALIGN;
     AppendParams p{static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
                    static_cast<__nv_bfloat16*>(k_cache), static_cast<__nv_bfloat16*>(v_cache),
                    static_cast<uint8_t*>(k_quant), static_cast<__half*>(k_scales), block_table, seq_lens,
-                   static_cast<uint32_t*>(workspace), cfg->num_kv_heads, max_blocks_per_seq, num_pages};
+                   static_cast<uint32_t*>(workspace), cfg->num_kv_heads, max_blocks_per_seq, num_pages,
+                   static_cast<int8_t*>(k_res)};
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     launch_pdl(append_kernel, dim3(cfg->num_kv_heads, batch), dim3(128), 0, s, p);
     launch_pdl(bump_lengths_kernel, dim3((batch + 255) / 256), dim3(256), 0, s, seq_lens, (int)batch,
                (int)(max_blocks_per_seq * kBlk));
     return launch_status();
+}
+
+ffd_status ffd_append_kv(const ffd_config* cfg, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                         void* k_quant, void* k_scales, const int32_t* block_table, int32_t* seq_lens, int32_t batch,
+                         int32_t max_blocks_per_seq, int32_t num_pages, void* workspace, size_t workspace_bytes,
+                         void* stream) {
+    return append_impl(cfg, k_new, v_new, k_cache, v_cache, k_quant, k_scales, nullptr, block_table, seq_lens, batch,
+                       max_blocks_per_seq, num_pages, workspace, workspace_bytes, stream);
+}
+
+ffd_status ffd_append_kv_residual(const ffd_config* cfg, const void* k_new, const void* v_new, void* k_cache,
+                                  void* v_cache, void* k_quant, void* k_scales, void* k_res, const int32_t* block_table,
+                                  int32_t* seq_lens, int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages,
+                                  void* workspace, size_t workspace_bytes, void* stream) {
+    if (!k_res) return FFD_ERR_NULL;
+    return append_impl(cfg, k_new, v_new, k_cache, v_cache, k_quant, k_scales, k_res, block_table, seq_lens, batch,
+                       max_blocks_per_seq, num_pages, workspace, workspace_bytes, stream);
 }
 
 ffd_status ffd_decode(const ffd_config* cfg, const void* q, const void* k_cache, const void* v_cache,

@@ -26,7 +26,7 @@ DEV_BAD_SEQ_LEN = 2
 EXPORTS = ["ffd_status_string", "ffd_workspace_bytes", "ffd_workspace_init", "ffd_quantize_keys", "ffd_decode",
            "ffd_decode_dense", "ffd_unpack_codes", "ffd_read_device_status", "ffd_profile_events", "ffd_decode_static",
            "ffd_append_kv", "ffd_append_decode", "ffd_quantize_residual", "ffd_decode_residual", "ffd_workspace_bytes_residual",
-           "ffd_quantize_keys_residual"]
+           "ffd_quantize_keys_residual", "ffd_append_kv_residual"]
 
 
 class FfdError(RuntimeError):
@@ -93,6 +93,8 @@ def load_library() -> ctypes.CDLL:
                                           ctypes.c_float, _vp, _vp, _vp, _vp, _vp, ctypes.c_size_t, _vp]
         lib.ffd_quantize_residual.argtypes = [cfgp, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, _vp]
         lib.ffd_decode_residual.argtypes = lib.ffd_decode.argtypes
+        lib.ffd_append_kv_residual.argtypes = [cfgp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, _vp,
+                                               ctypes.c_size_t, _vp]
         lib.ffd_quantize_keys_residual.argtypes = [cfgp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, _vp]
         for name in EXPORTS:
             if name != "ffd_status_string":
@@ -184,6 +186,15 @@ def ffd_append_kv(cfg: Config, k_new, v_new, k_cache, v_cache, k_quant, k_scales
                                         max_blocks_per_seq, num_pages, _p(workspace),
                                         ctypes.c_size_t(workspace.numel() * workspace.element_size()),
                                         _stream(stream)), "ffd_append_kv")
+
+
+def ffd_append_kv_residual(cfg: Config, k_new, v_new, k_cache, v_cache, k_quant, k_scales, k_res, block_table, seq_lens,
+                           *, max_blocks_per_seq: int, workspace, stream=None):
+    _check(load_library().ffd_append_kv_residual(ctypes.byref(cfg.c()), _p(k_new), _p(v_new), _p(k_cache), _p(v_cache),
+                                                 _p(k_quant), _p(k_scales), _p(k_res), _p(block_table), _p(seq_lens),
+                                                 seq_lens.numel(), max_blocks_per_seq, k_cache.shape[0], _p(workspace),
+                                                 ctypes.c_size_t(workspace.numel() * workspace.element_size()),
+                                                 _stream(stream)), "ffd_append_kv_residual")
 
 
 def ffd_decode(cfg: Config, q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, delta: float, out, *,
@@ -301,6 +312,12 @@ class DeviceCache:
     def append(self, k_new, v_new):
         ffd_append_kv(self.cfg, k_new, v_new, self.k_cache, self.v_cache, self.k_quant, self.k_scales,
                       self.block_table, self.seq_lens, max_blocks_per_seq=self.w.max_blocks, workspace=self.workspace)
+
+    def append_residual(self, k_new, v_new):
+        """Append one token per sequence on the 2 + 8 bit format (thumbnails and residuals of its block redone)."""
+        ffd_append_kv_residual(self.cfg, k_new, v_new, self.k_cache, self.v_cache, self.k_quant, self.k_scales,
+                               self.k_res, self.block_table, self.seq_lens, max_blocks_per_seq=self.w.max_blocks,
+                               workspace=self.workspace)
 
     def append_decode(self, k_new, v_new, delta, kept_mask=None, block_max=None):
         ffd_append_decode(self.cfg, k_new, v_new, self.q, self.k_cache, self.v_cache, self.k_quant, self.k_scales,

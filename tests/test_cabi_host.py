@@ -89,6 +89,10 @@ def test_null_and_range_arguments_are_rejected_before_any_launch(lib):
                              None) == 5
     assert lib.ffd_append_kv(ctypes.byref(cfg), fake, fake, fake, fake, fake, fake, None, odd, 1, 16, 16, fake, 256,
                              None) == 4
+    assert lib.ffd_append_kv_residual(ctypes.byref(cfg), fake, fake, fake, fake, fake, fake, None, None, fake, 1, 16, 16,
+                                      fake, 256, None) == 1
+    assert lib.ffd_append_kv_residual(ctypes.byref(cfg), fake, fake, fake, fake, fake, fake, odd, None, fake, 1, 16, 16,
+                                      fake, 256, None) == 4
     # append + decode: NULL new rows; the decode's own checks behind them
     assert lib.ffd_append_decode(ctypes.byref(cfg), None, fake, fake, fake, fake, fake, fake, None, fake, 1, 16, 16,
                                  ctypes.c_float(6.0), fake, None, None, None, fake, 1 << 30, None) == 1

@@ -219,10 +219,11 @@ def test_tail_requantize_only_touches_the_last_block(ffd, oracle):
 
 
 def test_residual_serving_loop_from_one_graph(ffd, oracle):
-    """The 2 + 8 bit format's serving step -- append a token, redo thumbnails and residuals of its block, decode from
-    the residuals -- captured once and replayed token after token; after every replay the cache tiles, the lengths and
-    the output equal those of the same steps run eagerly on a second copy, and the last output matches the oracle's
-    Dequant refinement of the lengthened sequences."""
+    """The 2 + 8 bit format's serving step -- append a token, redo thumbnails and residuals of its block
+    (ffd_append_kv_residual), decode from the residuals -- captured once and replayed token after token; after every
+    replay the lengths and the output equal those of a second copy on which the same step is made of the separate calls
+    (append, ffd_quantize_keys_residual with first_token), run eagerly; at the end the residuals equal the oracle's
+    and the output matches its Dequant refinement of the lengthened sequences."""
     w = make_workload("C5", B=3, lens=(700, 2000))
     full = w.seq_lens.copy()
     steps = 70                                  # crosses a block boundary in every sequence
@@ -236,9 +237,12 @@ def test_residual_serving_loop_from_one_graph(ffd, oracle):
     first = torch.zeros(w.B, dtype=torch.int32, device="cuda")
 
     def step(dc):
-        first.copy_(dc.seq_lens)                # the position the new token goes to = start of the redone range
-        dc.append(k_new, v_new)
-        dc.quantize_both(first_token=first)
+        if dc is a:                             # one call that appends and redoes thumbnails + residuals ...
+            dc.append_residual(k_new, v_new)
+        else:                                   # ... against the separate calls
+            first.copy_(dc.seq_lens)            # the position the new token goes to = start of the redone range
+            dc.append(k_new, v_new)
+            dc.quantize_both(first_token=first)
         dc.decode_residual(6.0)
 
     def rows(t):
