@@ -40,7 +40,6 @@ KV_BYTES_PER_TILE = 2 * 64 * 128 * 2      # K tile + V tile of one kept (block, 
 # the ncu capture summarised in profiles/fused_sparse_kernel_C3_ctx32768.md (same kernel, same workload recipe at
 # context 32768; traffic grows in proportion to the blocks processed): (308.47 + 5.65) MB / 308.28 MB.
 NCU_TRAFFIC_RATIO = 1.018
-KERNEL_EVENT_EVERY = 4      # steps between two steps that carry the CUDA-event pair around the fused kernel
 
 
 def measured_peaks():
@@ -134,22 +133,25 @@ def algorithmic_bytes(w, kept_tiles: int, dense: bool = False) -> int:
     return tiles * CODE_BYTES_PER_TILE + kept_tiles * KV_BYTES_PER_TILE
 
 
-def cpu_baseline(w, delta, threads=None, seconds_target=15.0):
-    """Time the oracle, as it stands, on a bounded sample of (sequence, head) rows of the same workload and scale
-    to a whole step.  Reported context, not a target."""
+def cpu_baseline(w, delta, threads=None, rows_per_thread=None):
+    """Time the oracle, as it stands, on the same workload.  With ``rows_per_thread`` None every (sequence, query
+    head) row is computed (the measured time is the step); otherwise a bounded sample with the workload's own mix of
+    head kinds, and the measured and the scaled time are reported side by side.  Reported context, not a target."""
     from oracle import ffd_oracle as O
     cores = threads or O.max_threads()
     O.set_threads(cores)
-    # sample: one query head per KV-head kind (peaked / flat) per thread, so every core has work
-    flat = set(w.flat_heads)
-    kinds = {"peaked": [g for g in range(w.Hkv) if g not in flat], "flat": list(flat)}
-    units = []
-    for kind, gs in kinds.items():
-        for i in range(cores):
-            if gs:
-                g = gs[i % len(gs)]
-                units.append((i % w.B, g * w.G + (i // len(gs)) % w.G))
-    units = sorted(set(units))
+    total_rows = w.B * w.Hq
+    units = None
+    if rows_per_thread is not None:
+        flat = set(w.flat_heads)
+        kinds = [[g for g in range(w.Hkv) if g not in flat], sorted(flat)]
+        units = []
+        for gs in kinds:
+            for i in range(cores * rows_per_thread):
+                if gs:
+                    g = gs[i % len(gs)]
+                    units.append((i % w.B, g * w.G + (i // len(gs)) % w.G))
+        units = sorted(set(units))
     # the oracle quantizer output is an input of the timed stage (quantization is the append path)
     t0 = time.perf_counter()
     codes, scales = O.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
@@ -158,20 +160,19 @@ def cpu_baseline(w, delta, threads=None, seconds_target=15.0):
     O.decode(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), codes, scales, w.block_table, w.seq_lens,
              w.max_blocks, delta, units=units)
     t = time.perf_counter() - t0
-    n_flat = sum(1 for (_, h) in units if (h // w.G) in flat)
-    n_peak = len(units) - n_flat
-    total_rows = w.B * w.Hq
-    # the sample holds the two head kinds in the workload's own proportion, so one factor scales it to a step
-    scale = total_rows / len(units)
-    step_seconds = t * scale
-    return {"value": step_seconds * 1e6, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"{len(units)} of {total_rows} (sequence, query head) rows ({n_peak} peaked, {n_flat} flat), "
-                      f"scan+select+attend in {t:.2f} s scaled by {scale:.1f}; full-cache quantizer {t_quant:.1f} s "
-                      "not included"}
+    n_rows = total_rows if units is None else len(units)
+    scale = total_rows / n_rows
+    sample = (f"all {total_rows} (sequence, query head) rows, scan+select+attend, nothing scaled" if units is None else
+              f"{n_rows} of {total_rows} (sequence, query head) rows in the workload's own mix of head kinds, measured "
+              f"time scaled by {scale:.1f}")
+    return {"value": t * scale * 1e6, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "measured_seconds": t, "scaled_by": scale,
+            "sample": sample + f"; full-cache quantizer {t_quant:.1f} s not included"}
 
 
 def run_reference(args, rank, world):
-    """The reference arm of this build is the CPU oracle (there is no reference implementation to install)."""
+    """The reference arm of this build is the CPU oracle (there is no reference implementation to install): every
+    step computes every (sequence, query head) row of the workload, nothing is scaled."""
     if rank != 0:
         return
     from oracle import ffd_oracle as O
@@ -180,23 +181,15 @@ def run_reference(args, rank, world):
     cores = O.max_threads()
     O.set_threads(cores)
     codes, scales = O.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
-    flat = set(w.flat_heads)
-    units = []
-    for i in range(cores):
-        g = i % w.Hkv
-        units.append((i % w.B, g * w.G + (i // w.Hkv) % w.G))
-    units = sorted(set(units))
-    scale = w.B * w.Hq / len(units)
     times = []
     for it in range(args.warmup + args.steps):
         t0 = time.perf_counter()
         O.decode(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), codes, scales, w.block_table, w.seq_lens,
-                 w.max_blocks, delta, units=units)
+                 w.max_blocks, delta)
         if it >= args.warmup:
             times.append(time.perf_counter() - t0)
-    us = statistics.mean(times) * scale * 1e6
-    sample = (f"{len(units)} of {w.B * w.Hq} (sequence, query head) rows per step over all KV-head kinds, "
-              f"time scaled by {scale:.1f}")
+    us = statistics.mean(times) * 1e6
+    sample = f"all {w.B * w.Hq} (sequence, query head) rows every step, nothing scaled"
     line = {"impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
@@ -222,9 +215,98 @@ def workload_config(w, delta, args):
             "l2": "L2 flushed before every step (256 MiB written, then 256 MiB of another buffer read so that the "
                   "flush's own write-back drains before the timed region); inputs also larger than L2",
             "step": "tail-block re-quantize + pseudo-max + fused scan/select/attend + combine",
-            "kernel_events": f"every {KERNEL_EVENT_EVERY}th timed step carries the CUDA-event pair around the fused kernel "
-                             "(roofline.kernel_us is their mean); see step_us_without_kernel_events",
+            "kernel_events": "roofline.kernel_us comes from a separate loop of the same step in which every step carries "
+                             "a CUDA-event pair around the fused kernel; the steps behind `value` carry none",
             "aggregate": "value = max-over-ranks step time / n_gpus (each rank decodes its own batch)"}
+
+
+def stats(xs):
+    return {"mean": statistics.mean(xs), "median": statistics.median(xs), "min": min(xs), "samples": len(xs)}
+
+
+class Bench:
+    """One workload resident on the device and the timing loops over it."""
+
+    def __init__(self, ffd, w, delta, shared=None):
+        from tests.device_cache import DeviceCache
+        self.ffd, self.w, self.delta = ffd, w, delta
+        self.dc = DeviceCache(w, ffd.Config(w.Hq, w.Hkv, out_dtype=1))
+        self.dc.quantize()
+        self.first_token = torch.from_numpy(np.maximum(w.seq_lens - 1, 0)).to("cuda")
+        if shared is None:
+            shared = {"flush": torch.empty(256 << 20, dtype=torch.uint8, device="cuda"),
+                      "drain": torch.zeros(32 << 20, dtype=torch.int64, device="cuda"),      # 256 MiB, only ever read
+                      "k_start": torch.cuda.Event(enable_timing=True), "k_stop": torch.cuda.Event(enable_timing=True)}
+            shared["k_start"].record(), shared["k_stop"].record()   # materialise the CUDA events for the library
+        self.shared = shared
+        self.stream = torch.cuda.current_stream()
+        kept = torch.zeros(w.B, w.Hq, w.max_blocks, dtype=torch.uint8, device="cuda")
+        self.dc.decode(delta, kept_mask=kept)
+        assert ffd.ffd_read_device_status(self.dc.workspace) == 0
+        kept_np = kept.cpu().numpy()
+        self.kept_tiles = union_kept_tiles(kept_np, w)
+        self.total_tiles = sum(w.num_blocks(b) for b in range(w.B)) * w.Hkv
+        self.head_blocks = sum(w.num_blocks(b) for b in range(w.B)) * w.Hq
+        self.kept_head_blocks = sum(int(kept_np[b, :, : w.num_blocks(b)].sum()) for b in range(w.B))
+        self.sparse_bytes = algorithmic_bytes(w, self.kept_tiles)
+        self.dense_bytes = algorithmic_bytes(w, 0, dense=True)
+
+    def step(self):
+        self.dc.quantize(first_token=self.first_token)
+        self.dc.decode(self.delta)
+
+    def timed_loop(self, fn, n, profile_kernel=False, cold=True):
+        """n steps, each bracketed by CUDA events on the launching stream, L2 flushed (untimed) before each.
+        profile_kernel: every step also carries the library's event pair around its fused kernel."""
+        sh = self.shared
+        self.ffd.ffd_profile_events(sh["k_start"] if profile_kernel else None, sh["k_stop"] if profile_kernel else None)
+        total, kernel = [], []
+        for _ in range(n):
+            if cold:
+                sh["flush"].fill_(1)   # evicts every input line from L2 ...
+                sh["drain"].sum()      # ... and this read sweep pushes the fill's dirty lines out to HBM, so that their
+                                       # write-back (an artefact of the flush, not of the workload) ends before the timing starts
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(self.stream)
+            fn()
+            b.record(self.stream)
+            b.synchronize()
+            total.append(a.elapsed_time(b) * 1e3)
+            if profile_kernel:
+                kernel.append(sh["k_start"].elapsed_time(sh["k_stop"]) * 1e3)
+        self.ffd.ffd_profile_events(None, None)
+        return total, kernel
+
+    def fidelity(self):
+        """Sec. 5 "Retrieval Fidelity Analysis" on the GPU's own two paths: the sparse output against the dense one."""
+        dc = self.dc
+        dc.decode(self.delta)
+        torch.cuda.synchronize()
+        o_s, l_s = dc.out.double().clone(), dc.lse.double().clone()
+        dc.dense()
+        torch.cuda.synchronize()
+        o_d, l_d = dc.out.double(), dc.lse.double()
+        live = torch.from_numpy(self.w.seq_lens > 0).to("cuda")
+        cos = torch.nn.functional.cosine_similarity(o_s, o_d, dim=-1)[live]
+        return {"min_cosine_sparse_vs_dense": float(cos.min()), "mean_cosine_sparse_vs_dense": float(cos.mean()),
+                "max_abs_lse_error": float((l_s - l_d)[live].abs().max())}
+
+    def brief(self, steps, peak):
+        """The figures of a secondary workload: step, fused kernel, bytes and roofline fraction, dense step."""
+        self.timed_loop(self.step, 3)
+        step_us, _ = self.timed_loop(self.step, steps)
+        _, kernel_us = self.timed_loop(self.step, max(steps, 20), profile_kernel=True)
+        self.timed_loop(self.dc.dense, 3)
+        dense_us, _ = self.timed_loop(self.dc.dense, max(5, steps // 2))
+        t_k = statistics.mean(kernel_us)
+        gbs = self.sparse_bytes / (t_k * 1e-6) / 1e9
+        return {"workload": workload_config(self.w, self.delta, None)["workload"], "us_per_step": statistics.mean(step_us),
+                "us_per_step_median": statistics.median(step_us), "kernel_us": stats(kernel_us),
+                "algorithmic_bytes": self.sparse_bytes, "achieved_gbs": gbs, "frac": gbs / peak,
+                "dense_us_per_step": statistics.mean(dense_us),
+                "speedup_vs_dense": statistics.mean(dense_us) / statistics.mean(step_us),
+                "skipped_fraction_per_loaded_block": 1.0 - self.kept_tiles / self.total_tiles,
+                "fidelity": self.fidelity()}
 
 
 def main():
@@ -238,6 +320,7 @@ def main():
     ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--delta", type=float, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the secondary workloads (C4, C5) of the bench line")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -259,77 +342,31 @@ def main():
 
     w = make_workload(args.workload, **workload_overrides(args))
     delta = args.delta if args.delta is not None else w.deltas[0]
-    cfg = ffd.Config(w.Hq, w.Hkv, out_dtype=1)
-    dc = ffd.DeviceCache(w, cfg)
-    dc.quantize()
-    first_token = torch.from_numpy(np.maximum(w.seq_lens - 1, 0)).to("cuda")
-    kept = torch.zeros(w.B, w.Hq, w.max_blocks, dtype=torch.uint8, device="cuda")
-    dc.decode(delta, kept_mask=kept)
-    assert ffd.ffd_read_device_status(dc.workspace) == 0
-    kept_np = kept.cpu().numpy()
-    kept_tiles = union_kept_tiles(kept_np, w)
-    total_tiles = sum(w.num_blocks(b) for b in range(w.B)) * w.Hkv
-    head_blocks = sum(w.num_blocks(b) for b in range(w.B)) * w.Hq
-    kept_head_blocks = sum(int(kept_np[b, :, : w.num_blocks(b)].sum()) for b in range(w.B))
-    sparse_bytes = algorithmic_bytes(w, kept_tiles)
-    dense_bytes = algorithmic_bytes(w, 0, dense=True)
-
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    drain = torch.zeros(32 << 20, dtype=torch.int64, device="cuda")      # 256 MiB, only ever read
-    stream = torch.cuda.current_stream()
-    k_start, k_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    k_start.record(), k_stop.record()      # materialise the CUDA events before handing them to the library
-
-    def step():
-        dc.quantize(first_token=first_token)
-        dc.decode(delta)
-
-    def timed_loop(fn, n, profile_kernel, cold=True):
-        """n steps, each bracketed by CUDA events on the launching stream, L2 flushed (untimed) before each."""
-        total, kernel = [], []
-        for i in range(n):
-            if profile_kernel:
-                # The event pair around the fused kernel sits between the step's kernels and costs their
-                # programmatic-launch overlap (~10 us): it is recorded on every KERNEL_EVENT_EVERY-th step only.
-                probe = i % KERNEL_EVENT_EVERY == 0
-                ffd.ffd_profile_events(k_start if probe else None, k_stop if probe else None)
-            if cold:
-                flush.fill_(1)      # evicts every input line from L2 ...
-                drain.sum()         # ... and this read sweep pushes the fill's dirty lines out to HBM, so that their
-                                    # write-back (an artefact of the flush, not of the workload) ends before the timing starts
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            fn()
-            b.record(stream)
-            b.synchronize()
-            total.append(a.elapsed_time(b) * 1e3)
-            if profile_kernel and probe:
-                kernel.append(k_start.elapsed_time(k_stop) * 1e3)
-        return total, kernel
+    bench = Bench(ffd, w, delta)
+    dc, step, timed_loop = bench.dc, bench.step, bench.timed_loop
 
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    ffd.ffd_profile_events(k_start, k_stop)
     sampler = ClockSampler(local_rank)
     sampler.start()
-    timed_loop(step, args.warmup, False)
+    timed_loop(step, args.warmup)
     barrier()
     t_begin = time.perf_counter()
-    step_us, kernel_us = timed_loop(step, args.steps, True)
+    step_us, _ = timed_loop(step, args.steps)
     barrier()
     clocks = sampler.stop(t_begin, time.perf_counter())
+    # the fused kernel alone: the same step, every one with the library's event pair around that kernel (the records sit
+    # between the step's kernels and cost their programmatic-launch overlap, so these steps are not the ones behind `value`)
+    _, kernel_us = timed_loop(step, max(args.steps, 20), profile_kernel=True)
     # the dense path of the same library, same protocol (context for the speedup figure)
-    timed_loop(dc.dense, 3, False)
-    dense_us, dense_kernel_us = timed_loop(dc.dense, min(max(5, args.steps // 2), 100), True)
-    ffd.ffd_profile_events(None, None)
-    # the same step without the event pair around the fused kernel (the records sit between the step's kernels and
-    # cost their programmatic-launch overlap): what a caller who does not profile sees
-    plain_us, _ = timed_loop(step, min(args.steps, 200), False)
-    # the same without the flush (whatever of the previous step is still in L2 stays there) ...
-    warm_us, _ = timed_loop(step, min(args.steps, 200), False, cold=False)
+    timed_loop(dc.dense, 3)
+    dense_us, _ = timed_loop(dc.dense, min(max(5, args.steps // 2), 100))
+    _, dense_kernel_us = timed_loop(dc.dense, 20, profile_kernel=True)
+    # the same step without the flush (whatever of the previous step is still in L2 stays there) ...
+    warm_us, _ = timed_loop(step, min(args.steps, 200), cold=False)
     # ... submitted as one CUDA graph (cold L2) ...
     graph_us = None
     try:
@@ -341,13 +378,13 @@ def main():
             with torch.cuda.graph(graph, stream=side):
                 step()
         torch.cuda.synchronize()
-        graph_us, _ = timed_loop(graph.replay, min(args.steps, 200), False)
+        graph_us, _ = timed_loop(graph.replay, min(args.steps, 200))
     except Exception as exc:   # reported, not fatal: the graph number is an extra
         graph_us = None
         print(f"bench: CUDA graph capture failed: {exc}", file=sys.stderr)
     # ... and a pure-read calibration: a sum over 1 GiB (torch's reduction kernel), cold
     calib = torch.zeros(128 << 20, dtype=torch.int64, device="cuda")
-    calib_us, _ = timed_loop(calib.sum, 13, False)
+    calib_us, _ = timed_loop(calib.sum, 13)
     read_gbs = calib.numel() * 8 / (statistics.median(calib_us[3:]) * 1e-6) / 1e9
     del calib
 
@@ -362,10 +399,11 @@ def main():
         step()
         out_host.copy_(dc.out, non_blocking=True)
 
-    timed_loop(e2e_step, 3, False)
-    e2e_us, _ = timed_loop(e2e_step, min(args.steps, 200), False)
+    timed_loop(e2e_step, 3)
+    e2e_us, _ = timed_loop(e2e_step, min(args.steps, 200))
     h2d = in_host.numel()
     d2h = out_host.numel() * 4
+    fidelity = bench.fidelity()
 
     # the same step on the 2 + 8 bit key format (kept blocks refined from 8-bit residuals instead of 16-bit keys):
     # tail re-quantize of thumbnails and residuals + pseudo-max + fused kernel + combine, same protocol.  Measured
@@ -373,14 +411,13 @@ def main():
     dc.quantize_residual()
 
     def residual_step():
-        dc.quantize_both(first_token=first_token)
+        dc.quantize_both(first_token=bench.first_token)
         dc.decode_residual(delta)
 
-    ffd.ffd_profile_events(k_start, k_stop)
-    timed_loop(residual_step, 3, False)
-    res_us, res_kernel_us = timed_loop(residual_step, min(max(5, args.steps // 2), 100), True)
-    ffd.ffd_profile_events(None, None)
-    res_bytes = total_tiles * CODE_BYTES_PER_TILE + kept_tiles * (KV_BYTES_PER_TILE // 2 + KV_BYTES_PER_TILE // 4)
+    timed_loop(residual_step, 3)
+    res_us, _ = timed_loop(residual_step, min(max(5, args.steps // 2), 100))
+    _, res_kernel_us = timed_loop(residual_step, 20, profile_kernel=True)
+    res_bytes = bench.total_tiles * CODE_BYTES_PER_TILE + bench.kept_tiles * (KV_BYTES_PER_TILE // 2 + KV_BYTES_PER_TILE // 4)
 
     t_step = statistics.mean(step_us)
     t_e2e = statistics.mean(e2e_us)
@@ -391,9 +428,12 @@ def main():
         return
 
     peak, peak_kind = measured_peaks()
+    sparse_bytes = bench.sparse_bytes
     t_kernel = statistics.mean(kernel_us)
     achieved = sparse_bytes / (t_kernel * 1e-6) / 1e9
     t_dense = statistics.mean(dense_us)
+    t_dense_kernel = statistics.mean(dense_kernel_us)
+    t_res_kernel = statistics.mean(res_kernel_us)
     line = {
         "metric": METRIC, "value": t_step / world, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": t_step / 1e3, "higher_is_better": False, "scaling": "weak",
@@ -405,32 +445,48 @@ def main():
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": (None if NCU_TRAFFIC_RATIO is None else sparse_bytes * NCU_TRAFFIC_RATIO),
                      "peak_source": f"{peak_kind} copy bandwidth (of {peak_kind})", "kernel": "fused_sparse_kernel",
-                     "kernel_us": t_kernel, "algorithmic_bytes": sparse_bytes,
-                     "frac_of_nominal_8TBs": achieved / 8000.0},
+                     "kernel_us": t_kernel, "kernel_us_median": statistics.median(kernel_us),
+                     "kernel_us_min": min(kernel_us), "kernel_us_samples": len(kernel_us),
+                     "algorithmic_bytes": sparse_bytes, "frac_of_nominal_8TBs": achieved / 8000.0},
         "step_us_median": statistics.median(step_us), "step_us_min": min(step_us),
-        "step_us_without_kernel_events": statistics.mean(plain_us),
         "step_us_warm_l2": statistics.mean(warm_us),
         "step_us_cuda_graph": None if graph_us is None else statistics.mean(graph_us),
         "read_calibration_gbs": read_gbs,
         "effective_hbm_gbs_step": sparse_bytes / (t_step * 1e-6) / 1e9,
-        "sparsity": {"skipped_fraction_per_head": 1.0 - kept_head_blocks / head_blocks,
-                     "skipped_fraction_per_loaded_block": 1.0 - kept_tiles / total_tiles,
-                     "kept_tiles": kept_tiles, "total_tiles": total_tiles},
-        "dense": {"us_per_step": t_dense, "kernel_us": statistics.mean(dense_kernel_us), "bytes": dense_bytes,
-                  "effective_hbm_gbs": dense_bytes / (statistics.mean(dense_kernel_us) * 1e-6) / 1e9},
+        "sparsity": {"skipped_fraction_per_head": 1.0 - bench.kept_head_blocks / bench.head_blocks,
+                     "skipped_fraction_per_loaded_block": 1.0 - bench.kept_tiles / bench.total_tiles,
+                     "kept_tiles": bench.kept_tiles, "total_tiles": bench.total_tiles},
+        "fidelity": fidelity,
+        "dense": {"us_per_step": t_dense, "kernel_us": t_dense_kernel, "bytes": bench.dense_bytes,
+                  "effective_hbm_gbs": bench.dense_bytes / (t_dense_kernel * 1e-6) / 1e9},
         "speedup_vs_dense": t_dense / t_step,
-        "residual_format": {"us_per_step": statistics.mean(res_us), "kernel_us": statistics.mean(res_kernel_us),
+        "residual_format": {"us_per_step": statistics.mean(res_us), "kernel_us": t_res_kernel,
                             "algorithmic_bytes": res_bytes,
-                            "effective_hbm_gbs": res_bytes / (statistics.mean(res_kernel_us) * 1e-6) / 1e9,
-                            "frac": res_bytes / (statistics.mean(res_kernel_us) * 1e-6) / 1e9 / peak,
+                            "effective_hbm_gbs": res_bytes / (t_res_kernel * 1e-6) / 1e9,
+                            "frac": res_bytes / (t_res_kernel * 1e-6) / 1e9 / peak,
                             "note": "2-bit thumbnails + 8-bit residual keys: a kept block reads 8 KB + 16 KB "
                                     "instead of 32 KB; same selection, same protocol as the headline step"},
     }
+    if not args.no_extras and world == 1:
+        # the scan-bound configurations, same protocol, fewer steps: C4 (one 256K sequence) and C5 (paged batch of 16)
+        del bench, dc, step, timed_loop, in_host, out_host
+        torch.cuda.empty_cache()
+        extra = {}
+        for name in ("C4", "C5"):
+            if name == args.workload:
+                continue
+            wx = make_workload(name)
+            bx = Bench(ffd, wx, wx.deltas[1] if name == "C4" else wx.deltas[0])
+            extra[name.lower()] = bx.brief(min(args.steps, 50), peak)
+            del bx, wx
+            torch.cuda.empty_cache()
+        line["extra"] = extra
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(w, delta)
-        one = cpu_baseline(w, delta, threads=1, seconds_target=5.0)
+        one = cpu_baseline(w, delta, threads=1, rows_per_thread=8)
         line["cpu_baseline"]["value_1_thread"] = one["value"]
         line["cpu_baseline"]["sample_1_thread"] = one["sample"]
+        line["cpu_baseline"]["measured_seconds_1_thread"] = one["measured_seconds"]
     else:
         line["cpu_baseline"] = None
     print(json.dumps(line), flush=True)

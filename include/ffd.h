@@ -1,7 +1,7 @@
 /*
  * ffd.h - C ABI of the B200 (sm_100a) FFD sparse decode-attention library.
  *
- * The library implements one decode step of "Faster Flash Decoding" (FFD) for one attention layer:
+ * The library implements one decode step of "Faster Than Flash" (FFD) for one attention layer:
  * keys are kept twice, as 16-bit K and as a 2-bit mid-rise "thumbnail" with per-channel scales; a step
  * scans the thumbnails of every 64-token block, skips blocks whose best approximate score lies more than
  * delta below a pseudo-max taken from the sink and local blocks, and runs exact softmax attention over the
@@ -9,7 +9,10 @@
  *
  * Conventions for every entry point
  *   - All data pointers are DEVICE pointers, 16-byte aligned, owned by the caller; `cfg` and output
- *     size pointers are HOST pointers.  The library allocates no device memory and keeps no state.
+ *     size pointers are HOST pointers.  The library allocates no device memory.  It keeps no state between calls
+ *     apart from two things that are documented where they are declared: the event pair of ffd_profile_events and the
+ *     per-device address of the scratch array of ffd_decode_static.  Everything else a call needs from an earlier
+ *     one (zeroed work counters) lives in the caller's workspace.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only enqueue work;
  *     nothing synchronizes except ffd_read_device_status.
  *   - Host-detectable problems return a non-zero ffd_status and launch nothing.
@@ -56,6 +59,9 @@ typedef enum {
 #define FFD_DEV_BAD_PAGE 1u     /* a block_table entry was outside [0, num_pages); that block was skipped */
 #define FFD_DEV_BAD_SEQ_LEN 2u  /* a seq_len was negative or above max_blocks_per_seq*64; clamped */
 #define FFD_DEV_TIMEOUT 4u      /* a bounded wait for an asynchronous copy ran out; that split's result is incomplete */
+#define FFD_DEV_RANGE 8u        /* an approximate score left the binary32 range (non-finite); that block was kept */
+#define FFD_DEV_BAD_WORKSPACE 16u /* the workspace header was never initialised (ffd_workspace_init), or an interrupted
+                                     call left its work counters behind: no work was handed out, `out` is undefined */
 
 typedef struct {
     int32_t num_q_heads;
@@ -72,7 +78,9 @@ typedef struct {
 
 const char* ffd_status_string(ffd_status status);
 
-/* Bytes of device workspace ffd_decode / ffd_decode_dense need for this geometry (host call, no CUDA). */
+/* Bytes of device workspace ffd_decode / ffd_decode_dense need for this geometry.  A host computation; the split
+ * geometry follows the SM count of the current CUDA device (148, a B200's, when no device can be asked), so ask
+ * with the device current on which the workspace will be used. */
 ffd_status ffd_workspace_bytes(const ffd_config* cfg, int32_t batch, int32_t max_blocks_per_seq, size_t* bytes);
 
 /* The same for ffd_decode_residual: the workspace of ffd_decode for this geometry followed by the tiles in which the
@@ -81,10 +89,12 @@ ffd_status ffd_workspace_bytes(const ffd_config* cfg, int32_t batch, int32_t max
 ffd_status ffd_workspace_bytes_residual(const ffd_config* cfg, int32_t batch, int32_t max_blocks_per_seq,
                                         size_t* bytes);
 
-/* Zeroes the header of a freshly allocated workspace (status word, work counters).  Call once before the first
- * decode with that workspace.  The status word is sticky across calls until ffd_read_device_status clears it; the
- * work counters are left at zero by every completed ffd_decode.  If a decode call was interrupted (a CUDA error),
- * call this again before reusing the workspace. */
+/* Zeroes the header of a freshly allocated workspace (status word, work counters) and marks it as initialised.  Call
+ * once before the first decode with that workspace.  The status word is sticky across calls until
+ * ffd_read_device_status clears it; the work counters are put back to zero by the last kernel of every completed
+ * ffd_decode, for the next call.  If a decode call was interrupted (a CUDA error), call this again before reusing the
+ * workspace.  A decode on a workspace that was never initialised, or whose counters an interrupted call left behind,
+ * is detected on the device: it hands out no work, stores nothing out of range and reports FFD_DEV_BAD_WORKSPACE. */
 ffd_status ffd_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 
 /*
@@ -170,8 +180,13 @@ ffd_status ffd_append_kv_residual(const ffd_config* cfg, const void* k_new, cons
  *   lse       nullable fp32 [batch, num_q_heads]
  *   kept_mask nullable u8 [batch, num_q_heads, max_blocks_per_seq]: 0/1 for blk < nb, others untouched
  *   block_max nullable fp32 [batch, num_q_heads, max_blocks_per_seq]: bm (same validity)
- * delta must be >= 0 or +inf.  Arithmetic: approximate scores are fp32-accurate (tensor-core products of
- * exact operands, fp32 accumulation); exact scores bf16 x bf16 -> fp32; P.V with P split in two bf16 pieces.
+ * delta must be >= 0 or +inf.  Arithmetic: approximate scores are binary32-accurate (tensor-core products of
+ * exact fp16 operands, binary32 accumulation: error of a few 2^-24 of sm * sum_c |q[c]| * scale[c], the precise
+ * re-scan of blocks near the threshold included); exact scores bf16 x bf16 -> fp32; P.V with P split in two bf16
+ * pieces.  Input range: q, K and V must be finite.  Every magnitude of q is handled (each head's query is scaled by
+ * an exact power of two before it becomes an fp16 operand, undone afterwards); blocks with a scale above ~2000 (keys
+ * beyond +-3000) leave the tensor-core path and are scored in binary32 on the ordinary lanes, same result, slower.
+ * If an approximate score leaves the binary32 range altogether the block is kept and FFD_DEV_RANGE is reported.
  * Device-detected problems (bad page index, seq_len beyond max_blocks_per_seq*64) skip / clamp the
  * offending work and set bits in the workspace status word; nothing traps.
  */
@@ -253,15 +268,16 @@ ffd_status ffd_read_device_status(void* workspace, void* stream, uint32_t* statu
  *
  * Limits and rules
  *   - Geometry: ffd_workspace_bytes(cfg, batch, max_blocks_per_seq) must not exceed FFD_STATIC_SCRATCH_BYTES,
- *     otherwise FFD_ERR_STATIC_LIMIT is returned and nothing is launched.  With 32 query / 8 KV heads the 8 MiB
- *     hold batch 1 up to about 160 K tokens of context, batch 4 up to about 36 K, batch 16 up to about 9 K.
+ *     otherwise FFD_ERR_STATIC_LIMIT is returned and nothing is launched.  With 32 query / 8 KV heads on a 148-SM
+ *     GPU the 8 MiB hold batch 1 up to about 117 K tokens of context, batch 4 up to about 28 K, batch 16 up to about
+ *     6 K (ask ffd_workspace_bytes for the exact figure of a geometry).
  *   - First use on a device: the first call made while a given device is current looks up the device address of
  *     the array (cudaGetSymbolAddress) and remembers it.  Make that first call during start-up, outside of any
  *     stream capture.
  *   - One array for everybody: all calls on a device share the scratch, and it keeps whatever the previous call
- *     left in it.  The function clears the parts that must start at zero itself (the status word; the work counter
- *     is reset by its first kernel), but two calls whose kernels overlap on the GPU (different streams, or different
- *     host threads) overwrite each other's partial results.  Issue calls that can overlap through ffd_decode with
+ *     left in it.  The function rewrites the parts that must start at zero itself (a small kernel at the start of
+ *     every call clears the status word and the work counters), but two calls whose kernels overlap on the GPU
+ *     (different streams, or different host threads) overwrite each other's partial results.  Issue calls that can overlap through ffd_decode with
  *     separate workspaces instead.
  *   - Device-detected problems (bad page index, seq_len out of range) are skipped exactly as in ffd_decode, but the
  *     status word lives in the private scratch and cannot be read back: validate such inputs on the caller's side.
@@ -273,7 +289,7 @@ ffd_status ffd_decode_static(const ffd_config* cfg, const void* q, const void* k
                              float delta, void* out, float* lse, void* stream);
 
 /*
- * Measurement hook (process-wide, not thread-safe; the only state the library keeps): while both events are
+ * Measurement hook (process-wide, not thread-safe): while both events are
  * non-NULL, ffd_decode and ffd_decode_dense record `start` right before and `stop` right after their fused
  * scan-select-attend kernel on the call's stream, so a benchmark can time that kernel alone.  Both are
  * cudaEvent_t passed as void*; pass NULL, NULL to switch the hook off.  No counterpart in the paper.

@@ -469,7 +469,8 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
     for (int x = threadIdx.x; x < kPmHintBlocks * kMaxG; x += kPmWarps * 32) (&sbm[0][0])[x] = -INFINITY;
     __syncthreads();
     ScanQuery sq;
-    scan_setup(sq, p.q + ((size_t)b * p.Hq + (size_t)g * p.G) * kD, p.G, lane);
+    const __nv_bfloat16* q_group = p.q + ((size_t)b * p.Hq + (size_t)g * p.G) * kD;
+    scan_setup(sq, q_group, p.G, lane, p.sm_scale);
     unsigned char* rec = p.qrec + (size_t)(b * p.Hkv + g) * kQrecBytes;
     if (warp == 0) {   // query record of this (sequence, KV head): the fused kernel stages it per work item
         uint4* dst = reinterpret_cast<uint4*>(rec);
@@ -523,7 +524,12 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
         else
             scan_load(sr, reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes),
                       reinterpret_cast<const uint4*>(p.k_scales + tile * kD), lane);
-        const float bm = scan_compute<true>(sr, sq, lane, rows, p.sm_scale, band);
+        float bm = scan_compute<true>(sr, sq, lane, rows, band);
+        if (bm != bm) {   // (uniform) a scale too large for the fp16 operand: binary32 on the ordinary lanes
+            bm = scan_block_wide(reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes), p.k_scales + tile * kD,
+                                 q_group, p.G, lane, rows, p.sm_scale, nullptr, 0);
+            if (!(fabsf(bm) < INFINITY) && lane < p.G) atomicOr(p.status, kDevRange);
+        }
         if (lane < kMaxG && s < kPmHintBlocks) sbm[s][lane] = bm;
         if (!sample) best = fmaxf(best, bm);
     }
@@ -538,8 +544,15 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
             p.mtilde[(size_t)b * p.Hq + g * p.G + threadIdx.x] = m;
             thr = m - p.delta;
         }
-        reinterpret_cast<float*>(rec + kQrecThr)[threadIdx.x] = thr;
-        if (threadIdx.x < kMaxG) sthr[threadIdx.x] = thr;
+        if (threadIdx.x < kMaxG) {   // (lane h of warp 0 holds the unit of head h)
+            float* consts = reinterpret_cast<float*>(rec + kQrecThr);
+            const float bmul = 1.5f * 1.02f * sq.unit * (1.0f / 1048576.0f);
+            consts[threadIdx.x] = thr;
+            consts[4 + threadIdx.x] = sq.unit;
+            consts[8 + threadIdx.x] = bmul;
+            consts[12 + threadIdx.x] = 1e-3f + bmul * (1.0f / 131072.0f);
+            sthr[threadIdx.x] = thr;
+        }
     }
     __syncthreads();
     // Scheduling hint for the fused kernel: a (sequence, KV head) that keeps at least half of the sampled middle
@@ -558,21 +571,27 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
         atomicMax(&p.len_stats[0], (unsigned)nb);
         atomicMax(&p.len_stats[1], (unsigned)(p.max_blocks - nb));
         atomicAdd(&p.len_stats[2], (unsigned)item_count(p, nb));   // work items that exist
-        if (hinted > 0 && 2 * kept >= hinted) p.unit_list[atomicAdd(&p.class_counts[0], 1u)] = make_int2(bg, n);
-        else p.unit_list[p.units - 1 - (int)atomicAdd(&p.class_counts[1], 1u)] = make_int2(bg, n);
-        FFD_TL(14, blockIdx.y == 0);
+        // The list is filled from both ends with counters that every completed call leaves at zero.  A header that was
+        // never initialised, or counters left behind by an interrupted call, must not become store indices.
+        if (p.status[kHeaderCookieWord] != kHeaderCookie) {
+            atomicOr(p.status, kDevBadWorkspace);
+        } else {
+            const bool heavy = hinted > 0 && 2 * kept >= hinted;
+            const unsigned idx = atomicAdd(&p.class_counts[heavy ? 0 : 1], 1u);
+            if (idx < (unsigned)p.units) p.unit_list[heavy ? (int)idx : p.units - 1 - (int)idx] = make_int2(bg, n);
+            else atomicOr(p.status, kDevBadWorkspace);
+        }
     }
 }
 
-// ---- fused scan -> select -> attend over one split of one (sequence, KV head) ---------------------------
+// ---- dense decode attention over one split of one (sequence, KV head) (Sec. 4.2 baseline) ------------------
 struct BlockRef {
     int blk;        // logical block, -1 = none
     int rows;       // valid tokens
     size_t tile;    // (page, KV head) tile index
 };
 
-template <bool SPARSE>
-__global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(DecodeParams p) {
+__global__ void __launch_bounds__(kWarps * 32, 1) dense_kernel(DecodeParams p) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const int split = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -602,12 +621,6 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(DecodeParams p) 
     const size_t head0 = (size_t)b * p.Hq + (size_t)g * p.G;
     AttendState st;
     attend_setup(st, q_group, p.G, lane);
-    ScanQuery sq;
-    float thr = -INFINITY;
-    if (SPARSE) {
-        scan_setup(sq, q_group, p.G, lane);
-        if (j < p.G) thr = p.mtilde[head0 + j] - p.delta;   // delta = +inf -> -inf: everything passes
-    }
     const unsigned group_mask = (1u << p.G) - 1u;
     const float logit_scale_log2 = p.sm_scale * kLog2e;
     const uint4* kbase = reinterpret_cast<const uint4*>(p.k_cache);
@@ -630,58 +643,27 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(DecodeParams p) 
             return ref;
         }
     };
-    auto load_codes = [&](ScanRegs& sr, const BlockRef& ref) {
-        scan_load(sr, reinterpret_cast<const uint4*>(p.k_quant + ref.tile * kCodeBytes),
-                  reinterpret_cast<const uint4*>(p.k_scales + ref.tile * kD), lane);
-    };
 
     BlockRef cur = fetch();
-    ScanRegs cur_regs;
-    if (SPARSE && cur.blk >= 0) load_codes(cur_regs, cur);
-    BlockRef pending{-1, 0, 0};     // kept block whose K/V copies are in flight
-    unsigned pending_keep = 0;
+    BlockRef pending{-1, 0, 0};     // block whose K/V copies are in flight
     uint32_t phase = 0;
     bool ok = true;
-
     while (cur.blk >= 0 && ok) {
-        // prefetch the next block's codes into registers before working on this one
         const BlockRef nxt = fetch();
-        ScanRegs nxt_regs;
-        if (SPARSE && nxt.blk >= 0) load_codes(nxt_regs, nxt);
-
-        unsigned keep4 = group_mask;
-        if (SPARSE) {
-            float band;
-            float bm = scan_compute<false>(cur_regs, sq, lane, cur.rows, p.sm_scale, band);
-            // too close to call with the fast accumulation: redo the block with the arithmetic m_tilde used
-            if (__any_sync(kFull, (j < p.G) && fabsf(bm - thr) <= band))
-                bm = scan_compute<true>(cur_regs, sq, lane, cur.rows, p.sm_scale, band);
-            const bool keep = (j < p.G) && (bm >= thr);
-            keep4 = __ballot_sync(kFull, keep) & 0xFu;
-            if (r == 0 && j < p.G) {
-                const size_t o = (head0 + j) * p.max_blocks + cur.blk;
-                if (p.kept_mask) p.kept_mask[o] = keep ? 1 : 0;
-                if (p.block_max) p.block_max[o] = bm;
-            }
+        const uint4* ksrc = kbase + cur.tile * kTileVec;
+        const uint4* vsrc = vbase + cur.tile * kTileVec;
+        if (pending.blk >= 0) {
+            ok = attend_block(st, kslot, vslot, kbar, vbar, phase, ksrc, vsrc, lane, pending.rows, group_mask,
+                              logit_scale_log2);
+        } else {
+            tile_copy_async(kslot, ksrc, lane, kbar);
+            tile_copy_async(vslot, vsrc, lane, vbar);
         }
-        if (keep4) {
-            const uint4* ksrc = kbase + cur.tile * kTileVec;
-            const uint4* vsrc = vbase + cur.tile * kTileVec;
-            if (pending.blk >= 0) {
-                ok = attend_block(st, kslot, vslot, kbar, vbar, phase, ksrc, vsrc, lane, pending.rows, pending_keep,
-                                  logit_scale_log2);
-            } else {
-                tile_copy_async(kslot, ksrc, lane, kbar);
-                tile_copy_async(vslot, vsrc, lane, vbar);
-            }
-            pending = cur;
-            pending_keep = keep4;
-        }
+        pending = cur;
         cur = nxt;
-        if (SPARSE) cur_regs = nxt_regs;
     }
     if (ok && pending.blk >= 0)
-        ok = attend_block(st, kslot, vslot, kbar, vbar, phase, nullptr, nullptr, lane, pending.rows, pending_keep,
+        ok = attend_block(st, kslot, vslot, kbar, vbar, phase, nullptr, nullptr, lane, pending.rows, group_mask,
                           logit_scale_log2);
     cp_async_drain();
     if (!ok && lane == 0) atomicOr(p.status, kDevTimeout);
@@ -731,8 +713,12 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(DecodeParams p) 
 
 __global__ void clear_status_kernel(uint32_t* status) { *status = 0u; }
 
-// status word, work counters and class counts: the first 256 bytes of a workspace
-__global__ void clear_header_kernel(uint32_t* header) { header[threadIdx.x] = 0u; }
+// status word, work counters and class counts: the first 256 bytes of a workspace (64 threads), then the cookie
+__global__ void init_header_kernel(uint32_t* header) {
+    pdl_launch_dependents();
+    pdl_wait();
+    header[threadIdx.x] = threadIdx.x == kHeaderCookieWord ? kHeaderCookie : 0u;
+}
 
 // ---- host side --------------------------------------------------------------------------------------------
 
@@ -749,17 +735,30 @@ constexpr int kResMaxCtas = 192;
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-// Split geometry is a pure function of (batch, KV heads, max blocks) so that ffd_workspace_bytes and the
+// SM count of the current device; 148 (B200) when no device can be asked, so that the host-only entry points still
+// answer.  Asked on every call: the library caches nothing, and the answer must follow cudaSetDevice.
+constexpr int kDefaultSms = 148;
+static int device_sms() {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) {
+        (void)cudaGetLastError();
+        return kDefaultSms;
+    }
+    return sms;
+}
+
+// Split geometry is a pure function of (batch, KV heads, max blocks, SM count) so that ffd_workspace_bytes and the
 // launch agree.  Aim for at least two CTAs per SM before making splits longer than 8 blocks.
-static Plan make_plan(const ffd_config* cfg, int batch, int max_blocks) {
+static Plan make_plan(const ffd_config* cfg, int batch, int max_blocks, int sms) {
     Plan pl;
     int bps = 32;
     const long units = (long)batch * cfg->num_kv_heads;
-    while (bps > 8 && units * ((max_blocks + bps - 1) / bps) < 2 * 148) bps /= 2;
+    while (bps > 8 && units * ((max_blocks + bps - 1) / bps) < 2 * sms) bps /= 2;
     pl.blocks_per_split = bps;
     pl.splits = max_blocks > 0 ? (max_blocks + bps - 1) / bps : 1;
     const size_t heads = (size_t)batch * cfg->num_q_heads;
-    pl.total_items = item_geometry(units, max_blocks).item_rows * batch * cfg->num_kv_heads;
+    pl.total_items = item_geometry(units, max_blocks, sms).item_rows * batch * cfg->num_kv_heads;
     const size_t fslots = (size_t)pl.total_items * kNA * kMaxG;
     pl.off_mtilde = 256;
     pl.off_lens = align_up(pl.off_mtilde + heads * sizeof(float), 256);
@@ -796,13 +795,13 @@ static ffd_status check_geometry(int batch, int max_blocks, int num_pages) {
 }
 
 // Threads per combine CTA (one CTA per head): as many as still let all CTAs be resident at once.
-static int combine_threads(long heads) { return heads <= 2 * 148 ? 1024 : heads <= 4 * 148 ? 512 : 256; }
+static int combine_threads(long heads, int sms) { return heads <= 2 * sms ? 1024 : heads <= 4 * sms ? 512 : 256; }
 // CTAs per head (each takes a share of the channels): more when there are few heads with many partials each, so
 // that a long sequence's partials are not summed by a handful of SMs; never so many that a CTA is left with fewer
 // than 128 partials (its fixed cost would dominate) or that the grid exceeds two CTAs per SM.
-static int combine_split(long heads, long max_partials) {
+static int combine_split(long heads, long max_partials, int sms) {
     for (int z = 4; z > 1; z >>= 1)
-        if (heads * z <= 2 * 148 + 32 && max_partials / z >= 128) return z;
+        if (heads * z <= 2 * sms + 32 && max_partials / z >= 128) return z;
     return 1;
 }
 
@@ -827,12 +826,12 @@ static void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
 
 static ffd_status launch_status() { return cudaGetLastError() == cudaSuccess ? FFD_OK : FFD_ERR_CUDA; }
 
-static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, const void* k_cache,
-                             const void* v_cache, const void* k_quant, const void* k_scales,
-                             const int32_t* block_table, const int32_t* seq_lens, int batch, int max_blocks,
-                             int num_pages, float delta, void* out, float* lse, uint8_t* kept_mask,
-                             float* block_max, void* workspace, size_t workspace_bytes, void* stream,
-                             const AppendParams* append = nullptr, const void* k_res = nullptr) {
+// Everything about a decode call that can be refused on the host (nothing is launched when this fails).
+static ffd_status check_decode_args(bool sparse, const ffd_config* cfg, const void* q, const void* k_cache,
+                                    const void* v_cache, const void* k_quant, const void* k_scales,
+                                    const int32_t* block_table, const int32_t* seq_lens, int batch, int max_blocks,
+                                    int num_pages, float delta, const void* out, const float* lse,
+                                    const float* block_max, const void* workspace, const void* k_res) {
     ffd_status st = check_config(cfg);
     if (st) return st;
     if (!q || (!k_cache && !k_res) || !v_cache || !seq_lens || !out || !workspace) return FFD_ERR_NULL;
@@ -847,7 +846,20 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
                           workspace};
     for (const void* ptr : ptrs)
         if (ptr && misaligned(ptr)) return FFD_ERR_ALIGN;
-    const Plan pl = make_plan(cfg, batch, max_blocks);
+    return FFD_OK;
+}
+
+static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, const void* k_cache,
+                             const void* v_cache, const void* k_quant, const void* k_scales,
+                             const int32_t* block_table, const int32_t* seq_lens, int batch, int max_blocks,
+                             int num_pages, float delta, void* out, float* lse, uint8_t* kept_mask,
+                             float* block_max, void* workspace, size_t workspace_bytes, void* stream,
+                             const AppendParams* append = nullptr, const void* k_res = nullptr) {
+    const ffd_status st = check_decode_args(sparse, cfg, q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens,
+                                            batch, max_blocks, num_pages, delta, out, lse, block_max, workspace, k_res);
+    if (st) return st;
+    const int sms = device_sms();
+    const Plan pl = make_plan(cfg, batch, max_blocks, sms);
     if (workspace_bytes < (k_res ? pl.total_residual : pl.total)) return FFD_ERR_WORKSPACE;
 
     DecodeParams p;
@@ -888,9 +900,10 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
     p.unit_list = reinterpret_cast<int2*>(ws + pl.off_units);
     p.res_scores = reinterpret_cast<float*>(ws + pl.off_scores);
     p.units = batch * cfg->num_kv_heads;
-    p.item_rows = item_geometry(p.units, max_blocks).item_rows;
-    p.rows_small = item_geometry(p.units, max_blocks).rows_small;
-    p.item_blocks = item_geometry(p.units, max_blocks).item_blocks;
+    const ItemGeom geom = item_geometry(p.units, max_blocks, sms);
+    p.item_rows = geom.item_rows;
+    p.rows_small = geom.rows_small;
+    p.item_blocks = geom.item_blocks;
     p.units_magic = fast_div_magic((unsigned)p.units);
     p.hkv_magic = fast_div_magic((unsigned)cfg->num_kv_heads);
     p.kept_mask = kept_mask;
@@ -903,15 +916,12 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
     const dim3 grid(p.splits, p.Hkv, batch);
     const bool prof = g_prof_start && g_prof_stop;
     if (sparse) {
-        int dev = 0, sms = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-            cudaFuncSetAttribute(fused_sparse_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem) != cudaSuccess ||
+        if (cudaFuncSetAttribute(fused_sparse_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem) != cudaSuccess ||
             cudaFuncSetAttribute(fused_sparse_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem) != cudaSuccess)
             return FFD_ERR_CUDA;
         if (k_res && sms > kResMaxCtas) return FFD_ERR_UNSUPPORTED;
         // the work counters and class counts at ws + 64 are zero here: ffd_workspace_init zeroes them and the
-        // combine kernel of every call leaves them zeroed for the next one
+        // combine kernel of every call leaves them zeroed for the next one (the kernels check the header's cookie)
         if (append) {
             // the kernels after the first one read the lengths it leaves in the workspace
             int32_t* new_lens = reinterpret_cast<int32_t*>(ws + pl.off_lens);
@@ -926,16 +936,16 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
         launch_pdl(k_res ? fused_sparse_kernel<true> : fused_sparse_kernel<false>, dim3(min(p.total_items, sms)),
                    dim3(kFusedThreads), kFusedSmem, s, p);
         if (prof) cudaEventRecord(g_prof_stop, s);
-        launch_pdl(combine_kernel<true>, dim3(p.Hq, batch, combine_split(p.Hq * batch, (long)p.item_rows * kNA)),
-                   dim3(combine_threads(p.Hq * batch)), 0, s, p);
+        launch_pdl(combine_kernel<true>, dim3(p.Hq, batch, combine_split(p.Hq * batch, (long)p.item_rows * kNA, sms)),
+                   dim3(combine_threads(p.Hq * batch, sms)), 0, s, p);
     } else {
-        if (cudaFuncSetAttribute(decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem) != cudaSuccess)
+        if (cudaFuncSetAttribute(dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem) != cudaSuccess)
             return FFD_ERR_CUDA;
         if (prof) cudaEventRecord(g_prof_start, s);
-        launch_pdl(decode_kernel<false>, grid, dim3(kWarps * 32), kDecodeSmem, s, p);
+        launch_pdl(dense_kernel, grid, dim3(kWarps * 32), kDecodeSmem, s, p);
         if (prof) cudaEventRecord(g_prof_stop, s);
-        launch_pdl(combine_kernel<false>, dim3(p.Hq, batch, combine_split(p.Hq * batch, p.splits)),
-                   dim3(combine_threads(p.Hq * batch)), 0, s, p);
+        launch_pdl(combine_kernel<false>, dim3(p.Hq, batch, combine_split(p.Hq * batch, p.splits, sms)),
+                   dim3(combine_threads(p.Hq * batch, sms)), 0, s, p);
     }
     return launch_status();
 }
@@ -973,7 +983,7 @@ ffd_status ffd_workspace_bytes(const ffd_config* cfg, int32_t batch, int32_t max
     if (!bytes) return FFD_ERR_NULL;
     st = check_geometry(batch, max_blocks_per_seq, 1);
     if (st) return st;
-    *bytes = make_plan(cfg, batch, max_blocks_per_seq).total;
+    *bytes = make_plan(cfg, batch, max_blocks_per_seq, device_sms()).total;
     return FFD_OK;
 }
 
@@ -983,7 +993,7 @@ ffd_status ffd_workspace_bytes_residual(const ffd_config* cfg, int32_t batch, in
     if (!bytes) return FFD_ERR_NULL;
     st = check_geometry(batch, max_blocks_per_seq, 1);
     if (st) return st;
-    *bytes = make_plan(cfg, batch, max_blocks_per_seq).total_residual;
+    *bytes = make_plan(cfg, batch, max_blocks_per_seq, device_sms()).total_residual;
     return FFD_OK;
 }
 
@@ -991,7 +1001,8 @@ ffd_status ffd_workspace_init(void* workspace, size_t workspace_bytes, void* str
     if (!workspace) return FFD_ERR_NULL;
     if (workspace_bytes < 256) return FFD_ERR_WORKSPACE;
     if (misaligned(workspace)) return FFD_ERR_ALIGN;
-    clear_header_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<uint32_t*>(workspace));
+    launch_pdl(init_header_kernel, dim3(1), dim3(64), 0, static_cast<cudaStream_t>(stream),
+               static_cast<uint32_t*>(workspace));
     return launch_status();
 }
 
@@ -1043,7 +1054,7 @@ static ffd_status quantize_impl(const ffd_config* cfg, const void* k_cache, void
         if (cudaFuncSetAttribute(quantize_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kQbSmem) != cudaSuccess)
             return FFD_ERR_CUDA;
         const long tiles = (long)max_blocks_per_seq * cfg->num_kv_heads;
-        long x = (48 * 148 + batch - 1) / batch;
+        long x = (48L * device_sms() + batch - 1) / batch;
         if (x > tiles) x = tiles;
         launch_pdl(quantize_bulk_kernel, dim3((unsigned)x, batch), dim3(kQbThreads), kQbSmem,
                    static_cast<cudaStream_t>(stream), p);
@@ -1076,7 +1087,7 @@ ffd_status ffd_quantize_residual(const ffd_config* cfg, const void* k_cache, con
                      cfg->num_kv_heads, max_blocks_per_seq, num_pages};
     // as in ffd_quantize_keys: every CTA walks its share of the blocks; two per (sequence, KV head) when only the
     // tail block is redone, else enough to fill the GPU several times over
-    long x = first_token ? 2 : (16 * 148 + (long)batch * cfg->num_kv_heads - 1) / ((long)batch * cfg->num_kv_heads);
+    long x = first_token ? 2 : (16L * device_sms() + (long)batch * cfg->num_kv_heads - 1) / ((long)batch * cfg->num_kv_heads);
     if (x > max_blocks_per_seq) x = max_blocks_per_seq;
     if (x < 1) x = 1;
     launch_pdl(residual_kernel, dim3((unsigned)x, cfg->num_kv_heads, batch), dim3(128), 0,
@@ -1222,13 +1233,16 @@ ffd_status ffd_decode_static(const ffd_config* cfg, const void* q, const void* k
     if (st) return st;
     st = check_geometry(batch, max_blocks_per_seq, num_pages);
     if (st) return st;
-    if (make_plan(cfg, batch, max_blocks_per_seq).total > FFD_STATIC_SCRATCH_BYTES) return FFD_ERR_STATIC_LIMIT;
-    if (!q || !k_cache || !v_cache || !k_quant || !k_scales || !seq_lens || !out) return FFD_ERR_NULL;
+    if (make_plan(cfg, batch, max_blocks_per_seq, device_sms()).total > FFD_STATIC_SCRATCH_BYTES) return FFD_ERR_STATIC_LIMIT;
     void* scratch = nullptr;
     st = static_scratch_address(&scratch);
     if (st) return st;
-    // the array still holds the previous call's contents: the sticky status word has to start from zero
-    clear_status_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<uint32_t*>(scratch));
+    st = check_decode_args(true, cfg, q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, batch,
+                           max_blocks_per_seq, num_pages, delta, out, lse, nullptr, scratch, nullptr);
+    if (st) return st;
+    // The array still holds whatever the previous call left there, and nobody else can initialise it: the whole
+    // header (status word, work counters, cookie) is rewritten at the start of every call.
+    launch_pdl(init_header_kernel, dim3(1), dim3(64), 0, static_cast<cudaStream_t>(stream), static_cast<uint32_t*>(scratch));
     if (cudaGetLastError() != cudaSuccess) return FFD_ERR_CUDA;
     return run_decode(true, cfg, q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, batch,
                       max_blocks_per_seq, num_pages, delta, out, lse, nullptr, nullptr, scratch,
@@ -1257,17 +1271,3 @@ ffd_status ffd_read_device_status(void* workspace, void* stream, uint32_t* statu
 }
 
 }  // extern "C"
-
-// Diagnostic build only: copies the probe tables to the host ([160][16] first-hit timestamps in ns, then [160][8]
-// clock buckets of an attend warp, then [160][8] of a scan warp) and clears the timestamps.  Not part of the library's interface.
-#ifdef FFD_TIMELINE
-extern "C" int ffd_debug_timeline(unsigned long long* host) {
-    cudaDeviceSynchronize();
-    cudaMemcpyFromSymbol(host, g_tl, sizeof(unsigned long long) * 160 * 16);
-    static unsigned long long zeros[160 * 16];
-    cudaMemcpyToSymbol(g_tl, zeros, sizeof(zeros));
-    cudaMemcpyFromSymbol(host + 160 * 16, g_acc, sizeof(long long) * 160 * 8);
-    cudaMemcpyFromSymbol(host + 160 * 24, g_acc2, sizeof(long long) * 160 * 8);
-    return 0;
-}
-#endif

@@ -26,10 +26,7 @@
 namespace ffd {
 
 constexpr int kNS = 12;                // warps of the scheduling + scan roles (three warpgroups)
-#ifndef FFD_SCHED_WARP
-#define FFD_SCHED_WARP 1
-#endif
-constexpr int kSched = FFD_SCHED_WARP; // 1: warp 0 only draws and publishes items, warps 1..11 scan
+constexpr int kSched = 1;              // warp 0 only draws and publishes items, warps 1..11 scan
 constexpr int kScanners = kNS - kSched;
 static_assert(kSched == 1, "warp 0 schedules, warps 1 .. kNS - 1 scan");
 constexpr int kNA = 4;                 // attend warps (one warpgroup)
@@ -52,21 +49,17 @@ constexpr int kSmallBlocks = kScanners;
 
 struct ItemGeom { int rows_small, item_rows, item_blocks; };
 
-// pure function of the launch geometry (the workspace layout depends on it)
-__host__ __device__ inline ItemGeom item_geometry(long units, int max_blocks) {
+// pure function of the launch geometry and the GPU's SM count (the workspace layout depends on it)
+__host__ __device__ inline ItemGeom item_geometry(long units, int max_blocks, int sms) {
     ItemGeom g;
-#ifdef FFD_DBG_ITEM_BLOCKS
-    g.item_blocks = FFD_DBG_ITEM_BLOCKS;
-#else
-    g.item_blocks = units * ((max_blocks + kItemBlocksMax - 1) / kItemBlocksMax) >= 6 * 148 ? kItemBlocksMax : kItemBlocksMin;
-#endif
+    g.item_blocks = units * ((max_blocks + kItemBlocksMax - 1) / kItemBlocksMax) >= 6 * sms ? kItemBlocksMax : kItemBlocksMin;
     const int kItemBlocks = g.item_blocks;
     const int full_rows = (max_blocks + kItemBlocks - 1) / kItemBlocks;
     const int all_small = (max_blocks + kSmallBlocks - 1) / kSmallBlocks;
-    if (units * full_rows < 2 * 148) {
+    if (units * full_rows < 2 * sms) {
         g.rows_small = all_small;        // few items per SM: halve them all
     } else {
-        const long want = (6 * 148 + units - 1) / units;             // about three small heavy items per SM
+        const long want = (6 * sms + units - 1) / units;             // about three small heavy items per SM
         const long cap = all_small / 3;                              // at most a third of the blocks
         g.rows_small = (int)(want < cap ? want : cap);
     }
@@ -88,21 +81,16 @@ __device__ __forceinline__ int item_count(const DecodeParams& p, int nb) {
 }
 constexpr int kRing = 2;               // code-ring stages per scan warp (a third stage measured no faster)
 constexpr int kStageBytes = kCodeBytes + kD * 2;   // 2048 B codes + 256 B scales
-#ifndef FFD_NB
-#define FFD_NB 8
-#endif
-constexpr int kNB = FFD_NB;                 // batch descriptors: how far the scan warps may run ahead of the attend warps
-#ifndef FFD_HEAVY_AHEAD
-#define FFD_HEAVY_AHEAD 2
-#endif
-constexpr int kHeavyAhead = FFD_HEAVY_AHEAD;         // heavy batches outstanding at most once the attend warps are the bottleneck
+constexpr int kNB = 8;                 // batch descriptors: how far the scan warps may run ahead of the attend warps
+constexpr int kHeavyAhead = 2;         // heavy batches outstanding at most once the attend warps are the bottleneck
 constexpr int kUnitCache = 512;        // entries of each end of the unit list kept in shared memory
 constexpr int kRowCap = 512;           // item rows up to which the table of existing items is built (ragged batches)
 constexpr int kItemRing = 8;           // decoded items published ahead
 constexpr int kQrecRing = 4;           // query records staged ahead
 constexpr int kQrecAbs = 2048;         // query record: [4][32 lanes] uint4 of pre-scaled fp16 query fragments, ...
-constexpr int kQrecThr = 4096;         // ... the same fragments of |q| (not pre-scaled), then 4 thresholds (+ pad)
-constexpr int kQrecBytes = kQrecThr + 32;
+constexpr int kQrecThr = 4096;         // ... the same fragments of |q| (not pre-scaled), then per head (4 floats each): the
+                                       // threshold, the accumulator unit, the bound's multiplier and its slack
+constexpr int kQrecBytes = kQrecThr + 64;
 
 struct Item {
     int slot;                          // canonical number row * units + bg (names the partial slots); < 0: no more work
@@ -263,7 +251,10 @@ __device__ __forceinline__ Item decode_item(const DecodeParams& p, const ItemSch
         const int u = k - row * sc.n_light;
         un = u < kUnitCache ? unit_cache[kUnitCache + u] : p.unit_list[p.units - 1 - u];
     }
-    const int bg = un.x;
+    // (entries are written by the pseudo-max kernel of this call; the clamps only matter on a workspace whose
+    // counters an interrupted call left behind, where a stale entry of another geometry could be drawn)
+    const int bg = min(max(un.x, 0), p.units - 1);
+    un.y = min(max(un.y, 0), p.max_blocks * kBlk);
     row += sc.row_off;
     it.slot = row * p.units + bg;
     it.bg = bg;
@@ -343,8 +334,10 @@ __device__ __forceinline__ void sched_role(const DecodeParams& p, unsigned char*
     const volatile int* attend_done = reinterpret_cast<const volatile int*>(smem + kOffAttendDone);
     const int2* unit_cache = reinterpret_cast<const int2*>(smem + kOffUnits);
     ItemSched sc;
-    sc.n_heavy = min((int)p.class_counts[0], p.units);
-    sc.n_light = p.units - sc.n_heavy;
+    // (a workspace whose header was never initialised hands out no work: the pseudo-max kernel has reported it)
+    const bool header_ok = p.status[kHeaderCookieWord] == kHeaderCookie;
+    sc.n_heavy = header_ok ? min((int)p.class_counts[0], p.units) : 0;
+    sc.n_light = header_ok ? p.units - sc.n_heavy : 0;
     // Rows in use: up to the longest sequence of the batch (a cache sized for longer contexts than it holds would
     // otherwise spend most tickets on rows no sequence reaches).
     const int rows = item_count(p, min((int)p.len_stats[0], p.max_blocks));
@@ -365,7 +358,6 @@ __device__ __forceinline__ void sched_role(const DecodeParams& p, unsigned char*
     sc.released = 0;
     sc.heavy_queued = 0;
     sc.heavy_hist = 0ull;
-    FFD_TL(3, lane == 0);
 #pragma unroll 1
     for (int pub = 0;; ++pub) {
         bool ok = true;
@@ -430,7 +422,6 @@ __device__ __forceinline__ void sched_role(const DecodeParams& p, unsigned char*
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(item_bar(ibars, pub));
-        FFD_TL(4, lane == 0 && it.slot >= 0);
         if (it.slot < 0) break;
     }
     cp_async_drain();
@@ -504,7 +495,7 @@ __device__ __forceinline__ void qrec_issue(const DecodeParams& p, int seq, int b
 // The precise variant of the scan for one block, with the arithmetic m_tilde was computed in.  Kept out of line so
 // that its registers do not weigh on the fast path; it re-reads the block's codes and scales from global memory.
 __device__ __noinline__ float scan_block_precise(const uint4* codes_tile, const uint4* scales_tile, uint32_t qrec,
-                                                 int lane, int rows, float sm_scale) {
+                                                 int lane, int rows, float unit) {
     ScanRegs sr;
     scan_load(sr, codes_tile, scales_tile, lane);
     ScanQuery sq;
@@ -514,8 +505,9 @@ __device__ __noinline__ float scan_block_precise(const uint4* codes_tile, const 
         const uint4 v = lds128(qrec + (x * 32 + lane) * 16);
         sq.qh[4 * x] = v.x; sq.qh[4 * x + 1] = v.y; sq.qh[4 * x + 2] = v.z; sq.qh[4 * x + 3] = v.w;
     }
+    sq.unit = unit;
     float band;
-    return scan_compute<true>(sr, sq, lane, rows, sm_scale, band);
+    return scan_compute<true>(sr, sq, lane, rows, band);
 }
 
 // RES (2 + 8 bit key format): the per-token approximate logits of every block that may be kept are left in the
@@ -544,20 +536,15 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
     ic.pages = -1;
     int issued = 0, consumed = 0;   // this warp's blocks whose copies were started / whose data was taken
     int bound_state = 0;            // >= 0: failures of the scale-only bound in a row; < 0: blocks until it is tried again
-    FFD_ACC_DECL;
 
 #pragma unroll 1
     for (int seq = 0;; ++seq) {     // published item seq = batch seq
-        FFD_ACC(0);
         if (!item_wait(ibars, seq)) *abort_flag = 1;
-        FFD_ACC(5);
         const Item it = item_read(items, seq);
-        FFD_TL(5, w == 1 && lane == 0 && it.slot >= 0);
         // (the scheduling warp made sure, before it published the item, that the attend warps have released this
         // descriptor and wrote its header)
         const int slot = seq & (kNB - 1);
         BatchDesc& d = descs[slot];
-        FFD_ACC(6);
         if (it.slot < 0 || *abort_flag) {   // no more work: tell the attend warps
             if (lane == 0) {
                 if (w0 == 0) d.item = -1;
@@ -582,15 +569,17 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
             }
         if (!mbar_wait(qbars + (seq & (kQrecRing - 1)) * 8, (seq / kQrecRing) & 1)) *abort_flag = 1;
         const uint32_t qrec = qrecs + (seq & (kQrecRing - 1)) * kQrecBytes;
-        FFD_TL(6, w == 1 && lane == 0);
         const size_t head0 = (size_t)it.b * p.Hq + (size_t)it.g * p.G;
-        float thr, thr_col;   // threshold of head lane % 4 (block-max layout) and of head lane / 8 (B-column layout)
+        // threshold and accumulator unit of head lane % 4 (block-max layout); threshold, bound multiplier and bound
+        // slack of head lane / 8 (B-column layout)
+        float thr, unit, thr_col, bmul_col, badd_col;
         asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(thr) : "r"(qrec + kQrecThr + j * 4));
+        asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(unit) : "r"(qrec + kQrecThr + 16 + j * 4));
         asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(thr_col) : "r"(qrec + kQrecThr + (lane >> 3) * 4));
-        FFD_ACC(7);
+        asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(bmul_col) : "r"(qrec + kQrecThr + 32 + (lane >> 3) * 4));
+        asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(badd_col) : "r"(qrec + kQrecThr + 48 + (lane >> 3) * 4));
 #pragma unroll 1
         for (int lb = w0; lb < it.nblk; lb += kScanners) {
-            FFD_ACC(0);
             // keep the ring full: blocks consumed .. consumed + kRing - 1 of this warp's stream
             while (issued < consumed + kRing && cursor_next(p, ic, items, ibars, w0, lane)) {
                 ring_issue(p, ic, ring + (issued % kRing) * kStageBytes, stage_tile + issued % kRing, lane);
@@ -598,11 +587,8 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
             }
             const int st = consumed % kRing;
             const uint32_t stage = ring + st * kStageBytes;
-            FFD_TL(7, w == 1 && lane == 0);
             ring_wait(issued - consumed - 1);
             __syncwarp();
-            FFD_TL(8, w == 1 && lane == 0);
-            FFD_ACC(1);
             // No token of the block can score above 1.5 * sum |q s| (every level is at most 1.5 in magnitude).  If
             // that bound stays below the threshold for every head of the group, no head can keep the block: its
             // codes are not even read from shared memory, and the decision is the same as the full scan's.  (Not when
@@ -616,7 +602,7 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
                 __half2 sum_a = __floats2half2_rn(0.f, 0.f), sum_b = sum_a;
 #pragma unroll
                 for (int x = 0; x < 4; ++x) scan_abs_sum(lds128(qrec + kQrecAbs + (x * 32 + lane) * 16), sv[x], sum_a, sum_b);
-                cannot_keep = __all_sync(kFull, scan_bound(sum_a, sum_b, p.sm_scale) < thr_col);
+                cannot_keep = __all_sync(kFull, scan_bound(sum_a, sum_b, bmul_col, badd_col) < thr_col);
                 // a bound that fails 16 times in a row (a dense head) is left out for the next 48 blocks
                 bound_state = cannot_keep ? 0 : bound_state + 1;
                 if (bound_state == 16) bound_state = -48;
@@ -627,7 +613,6 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
             const int rows = min(kBlk, it.n - blk * kBlk);
             unsigned keep4 = 0;
             bool refilled = false;
-            FFD_ACC(2);
             if (tile >= 0 && !cannot_keep) {   // codes into registers; B operand from the staged scales and the record
                 uint4 wv[4];
                 uint32_t bfrag[16];
@@ -644,24 +629,38 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
                 refilled = true;
                 float band;
                 float tok[8];
-                float bm = scan_mma<false>(wv, bfrag, lane, rows, p.sm_scale, band, RES ? tok : nullptr);
-                if constexpr (RES) {
-                    if (__any_sync(kFull, (j < p.G) && bm >= thr - band)) {
-                        float* dst = p.res_scores + ((size_t)(blockIdx.x * kNB + slot) * kItemBlocksMax + lb) * kScoreTileFloats +
-                                     j * kScoreStride + r;
+                float bm = scan_mma<false>(wv, bfrag, lane, rows, unit, band, RES ? tok : nullptr);
+                bool force_keep = false;
+                if (bm != bm) {   // (uniform, rare) a scale too large for the fp16 operand: binary32 on the ordinary lanes
+                    float* scores = nullptr;
+                    if constexpr (RES)
+                        scores = p.res_scores + ((size_t)(blockIdx.x * kNB + slot) * kItemBlocksMax + lb) * kScoreTileFloats;
+                    bm = scan_block_wide(reinterpret_cast<const uint4*>(p.k_quant + (size_t)tile * kCodeBytes),
+                                         p.k_scales + (size_t)tile * kD, p.q + head0 * kD, p.G, lane, rows, p.sm_scale,
+                                         scores, kScoreStride);
+                    if (__any_sync(kFull, (j < p.G) && !(fabsf(bm) < INFINITY))) {   // beyond binary32 too: reported, kept
+                        if (lane == 0) atomicOr(p.status, kDevRange);
+                        force_keep = true;
+                    }
+                } else {
+                    if constexpr (RES) {
+                        if (__any_sync(kFull, (j < p.G) && bm >= thr - band)) {
+                            float* dst = p.res_scores + ((size_t)(blockIdx.x * kNB + slot) * kItemBlocksMax + lb) * kScoreTileFloats +
+                                         j * kScoreStride + r;
 #pragma unroll
-                        for (int mt = 0; mt < 4; ++mt) {
-                            dst[16 * mt] = tok[2 * mt];
-                            dst[16 * mt + 8] = tok[2 * mt + 1];
+                            for (int mt = 0; mt < 4; ++mt) {
+                                dst[16 * mt] = tok[2 * mt];
+                                dst[16 * mt + 8] = tok[2 * mt + 1];
+                            }
                         }
                     }
+                    // too close to call (rare): a separate, non-inlined routine re-reads the block and redoes it precisely
+                    if (__any_sync(kFull, (j < p.G) && fabsf(bm - thr) <= band))
+                        bm = scan_block_precise(reinterpret_cast<const uint4*>(p.k_quant + (size_t)tile * kCodeBytes),
+                                                reinterpret_cast<const uint4*>(p.k_scales + (size_t)tile * kD), qrec, lane,
+                                                rows, unit);
                 }
-                // too close to call (rare): a separate, non-inlined routine re-reads the block and redoes it precisely
-                if (__any_sync(kFull, (j < p.G) && fabsf(bm - thr) <= band))
-                    bm = scan_block_precise(reinterpret_cast<const uint4*>(p.k_quant + (size_t)tile * kCodeBytes),
-                                            reinterpret_cast<const uint4*>(p.k_scales + (size_t)tile * kD), qrec, lane,
-                                            rows, p.sm_scale);
-                const bool keep = (j < p.G) && (bm >= thr);
+                const bool keep = (j < p.G) && (force_keep || bm >= thr);
                 keep4 = __ballot_sync(kFull, keep) & 0xFu;
                 if (r == 0 && j < p.G) {
                     const size_t o = (head0 + j) * p.max_blocks + blk;
@@ -675,7 +674,6 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
                 ring_issue(p, ic, ring + (issued % kRing) * kStageBytes, stage_tile + issued % kRing, lane);
                 ++issued;
             }
-            FFD_ACC(3);
             if (cannot_keep && tile >= 0 && p.kept_mask && r == 0 && j < p.G)
                 p.kept_mask[(head0 + j) * p.max_blocks + blk] = 0;
             if (lane == 0) {
@@ -683,14 +681,11 @@ __device__ __forceinline__ void scan_role(const DecodeParams& p, unsigned char* 
                 d.keep4[lb] = (uint8_t)keep4;
                 d.rows[lb] = (uint8_t)rows;
             }
-            FFD_ACC(4);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(bars + slot * 8);   // this warp's share of the batch is published
-        FFD_TL(9, w == 1 && lane == 0);
     }
     cp_async_drain();
-    FFD_ACC_OUT2(w == 1 && lane == 0);
     if (*abort_flag && w0 == 0 && lane == 0) atomicOr(p.status, kDevTimeout);
 }
 
@@ -729,29 +724,22 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
     bool ok = true;
     AttendState st;
     uint32_t qb[RES ? 8 : 1];
-    FFD_ACC_DECL;
     for (int bi = 0; ok; ++bi) {
         const int slot = bi & (kNB - 1), use = bi / kNB;
-        FFD_ACC(0);
         if (!mbar_wait(bars + slot * 8, use & 1)) { ok = false; break; }
-        FFD_ACC(1);
         const BatchDesc& d = descs[slot];
         const int item = d.item;
         if (item < 0) break;
-        FFD_TL(10, a == 0 && lane == 0);
         Item it;
         it.slot = item; it.b = d.b; it.g = d.g; it.nblk = d.nblk;
         // the share rotates with the batch number: when the kept count is not a multiple of four, the extra blocks
         // go to a different warp each time
         unsigned mine = my_entries(d, it.nblk, (a + bi) & (kNA - 1), lane);
         const bool any = mine != 0;
-        FFD_ACC(6);
         if (any) {
             if constexpr (RES) attend_setup_res(st, qb, p, it.b, it.g, lane);
             else attend_setup(st, p.q + ((size_t)it.b * p.Hq + (size_t)it.g * p.G) * kD, p.G, lane);
         }
-        FFD_TL(11, a == 0 && lane == 0 && any);
-        FFD_ACC(2);
         while (mine && ok) {
             const int lb = __ffs(mine) - 1;
             mine &= mine - 1;
@@ -798,8 +786,6 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
                                   logit_scale_log2);
         }
         __syncwarp();
-        FFD_ACC(3);
-        FFD_TL(12, a == 0 && lane == 0 && any);
         if (lane == 0) {
             mbar_arrive(bars + (kNB + slot) * 8);   // done with this batch descriptor
             reinterpret_cast<volatile int*>(smem + kOffAttendDone)[a] = bi + 1;
@@ -835,8 +821,6 @@ __device__ __forceinline__ void attend_role(const DecodeParams& p, unsigned char
         }
     }
     cp_async_drain();
-    FFD_ACC_OUT(a == 0 && lane == 0);
-    FFD_TL(13, a == 0 && lane == 0);
     if (!ok && lane == 0) atomicOr(p.status, kDevTimeout);
 }
 
@@ -844,7 +828,6 @@ template <bool RES>
 __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodeParams p) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    FFD_TL(0, threadIdx.x == 0);
     if (threadIdx.x == 0) {
         const uint32_t bars = smem_u32(smem) + kOffBars;
         for (int s = 0; s < kNB; ++s) {
@@ -865,7 +848,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodePa
         pend_light = (int)atomicAdd(p.light_counter, 1u);
     }
     pdl_wait();   // the pseudo-max kernel's outputs (unit list, class counts, query records) are needed from here on
-    FFD_TL(1, threadIdx.x == 0);
     {   // shared-memory copy of both ends of the unit list (heavy units from the front, light units from the back)
         int2* cache = reinterpret_cast<int2*>(smem + kOffUnits);
         for (int u = threadIdx.x; u < min(p.units, kUnitCache); u += kFusedThreads) {
@@ -877,7 +859,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_sparse_kernel(DecodePa
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     __syncthreads();
-    FFD_TL(2, threadIdx.x == 0);
     if (warp < kNS) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kScanRegs));
         if (warp < kSched) sched_role(p, smem, lane, pend_heavy, pend_light);
@@ -917,7 +898,6 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
     const int chan0 = (int)blockIdx.z * 4 * cgn;
     pdl_launch_dependents();
     pdl_wait();
-    FFD_TL(15, FUSED && tid == 0 && blockIdx.y == 0 && blockIdx.z == 0);
     if (FUSED && h == 0 && b == 0 && blockIdx.z == 0 && tid == 0) {   // the next call's draws and class lists start from zero
         *p.item_counter = 0u;
         p.class_counts[0] = 0u;

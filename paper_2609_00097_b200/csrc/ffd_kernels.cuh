@@ -23,39 +23,13 @@ constexpr int kD = 128;            // head_dim
 constexpr int kBlk = 64;           // tokens per block
 constexpr int kTileBytes = kBlk * kD * 2;
 constexpr int kCodeBytes = kBlk * kD / 4;
-#ifndef FFD_DENSE_WARPS
-#define FFD_DENSE_WARPS 7
-#endif
-constexpr int kWarps = FFD_DENSE_WARPS;          // warps per decode CTA: 7 x (16 KB K slot + 16 KB V slot) of shared memory
+constexpr int kWarps = 7;          // warps per decode CTA: 7 x (16 KB K slot + 16 KB V slot) of shared memory
 constexpr int kSlotBytes = kTileBytes;
 constexpr int kDecodeSmem = kWarps * 2 * kSlotBytes + 128;   // + mbarriers
 constexpr uint32_t kSuspendHintNs = 200000u;       // upper bound of one hardware-suspended try_wait
 constexpr long long kSpinCycles = 2000000000LL;   // bounded mbarrier wait (~1 s of SM clocks); then report and stop
 constexpr int kMaxG = 4;           // query heads per KV head handled by one warp
 constexpr unsigned kFull = 0xffffffffu;
-
-// Diagnostic build only (-DFFD_TIMELINE): FFD_TL(i, cond) stores the global timer the first time CTA blockIdx.x
-// reaches probe i; FFD_ACC(i) adds the SM clocks since the previous FFD_ACC to bucket i of a per-thread table that
-// FFD_ACC_OUT writes out.  The normal build compiles all of them to nothing.
-#ifdef FFD_TIMELINE
-__device__ unsigned long long g_tl[160 * 16];
-#define FFD_TL(i, cond) do { if (cond) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); \
-    if (g_tl[blockIdx.x * 16 + (i)] == 0) g_tl[blockIdx.x * 16 + (i)] = t_; } } while (0)
-__device__ long long g_acc[160 * 8];
-#define FFD_ACC_DECL long long acc_t_[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long acc_c_ = clock64()
-#define FFD_ACC(i) do { const long long n_ = clock64(); acc_t_[i] += n_ - acc_c_; acc_c_ = n_; } while (0)
-#define FFD_ACC_OUT(cond) do { if (cond) for (int i_ = 0; i_ < 8; ++i_) g_acc[blockIdx.x * 8 + i_] = acc_t_[i_]; } while (0)
-__device__ long long g_acc2[160 * 8];
-#define FFD_ACC_OUT2(cond) do { if (cond) for (int i_ = 0; i_ < 8; ++i_) g_acc2[blockIdx.x * 8 + i_] = acc_t_[i_]; } while (0)
-#define FFD_CNT(i) (acc_t_[i] += 1)
-#else
-#define FFD_TL(i, cond)
-#define FFD_ACC_DECL
-#define FFD_ACC(i)
-#define FFD_ACC_OUT(cond)
-#define FFD_ACC_OUT2(cond)
-#define FFD_CNT(i)
-#endif
 
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -66,6 +40,14 @@ constexpr float kScanBandRel = 1.2e-5f;
 constexpr uint32_t kDevBadPage = 1u;
 constexpr uint32_t kDevBadSeqLen = 2u;
 constexpr uint32_t kDevTimeout = 4u;
+constexpr uint32_t kDevRange = 8u;          // an approximate score left the binary32 range; that block was kept
+constexpr uint32_t kDevBadWorkspace = 16u;  // the workspace header was not initialised (or a call was interrupted)
+
+// The workspace header (first 256 bytes): word 0 status, words 16 .. 22 work counters and batch statistics, word 24 a
+// cookie that ffd_workspace_init writes.  A kernel that finds another value there knows that the counters were never
+// zeroed: it reports kDevBadWorkspace and hands out no work instead of indexing with them.
+constexpr uint32_t kHeaderCookie = 0xFFD0B200u;
+constexpr int kHeaderCookieWord = 24;
 
 struct DecodeParams {
     const __nv_bfloat16* q;
@@ -279,6 +261,7 @@ __device__ __forceinline__ int clamped_seq_len(const DecodeParams& p, int b) {
 struct ScanQuery {
     uint32_t qh[16];  // half2: q of head (lane/8), channels 32j+4i+{0,1} (qh[2i]) and +{2,3} (qh[2i+1]), pre-scaled
     int piece;        // (lane/4) & 1
+    float unit;       // accumulator units -> logits for head lane % 4: 2^20 * sm_scale * 2^k of that head
 };
 
 __device__ __forceinline__ float scan_pos_scale(int i) {
@@ -286,24 +269,62 @@ __device__ __forceinline__ float scan_pos_scale(int i) {
     return e == 0 ? 16.f : e == 1 ? 4.f : e == 2 ? 1.f : e == 3 ? 0.25f : 0.0625f;
 }
 
-__device__ __forceinline__ void scan_setup(ScanQuery& sq, const __nv_bfloat16* q_group /* [G][128] */, int G,
-                                           int lane) {
-    const int n = lane >> 2, j = lane & 3;
-    const int head = n >> 1;
-    sq.piece = n & 1;
+// Range of the fp16 B operand.  The query of every head is brought into range by an exact power of two before it is
+// converted to fp16: k = the smallest integer >= 0 with 16 * max_c |q_c| * 2^-k <= 32, undone in `unit`.  The B operand
+// (16 q 2^-k) * s then overflows fp16 only for scales above 2047 (keys beyond +-3000); such a block shows up as a
+// non-finite level-offset sum and is redone by scan_block_wide in binary32.  Small products lose low bits to fp16
+// underflow, at most 2^-25 absolute per product, i.e. below 2^-30 of the head's largest |q_c| * s_c.
+// Returns 2^-k for the head lane / 8; all lanes of that head agree.
+__device__ __forceinline__ float scan_query_scale(const uint4 (&raw)[4]) {
+    float m = 0.f;
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        const uint32_t wds[4] = {raw[x].x, raw[x].y, raw[x].z, raw[x].w};
+#pragma unroll
+        for (int y = 0; y < 4; ++y)
+            m = fmaxf(m, fmaxf(fabsf(__uint_as_float(wds[y] << 16)), fabsf(__uint_as_float(wds[y] & 0xffff0000u))));
+    }
+    m = fmaxf(m, __shfl_xor_sync(kFull, m, 1));
+    m = fmaxf(m, __shfl_xor_sync(kFull, m, 2));
+    int e = 0;
+    (void)frexpf(m, &e);                 // m = f * 2^e, f in [0.5, 1): m * 2^-(e-1) < 2
+    const int k = min(max(e - 1, 0), 100);
+    return __uint_as_float((uint32_t)(127 - k) << 23);
+}
+
+// raw: this lane's 32 query values (bf16) of head lane / 8, channels 32j .. 32j + 31 (zero for heads >= G);
+// inv = 2^-k of that head
+__device__ __forceinline__ void scan_setup_scaled(ScanQuery& sq, const uint4 (&raw)[4], float inv, int lane) {
+    sq.piece = (lane >> 2) & 1;
 #pragma unroll
     for (int x = 0; x < 4; ++x) {   // 8 contiguous channels 32j + 8x .. + 7 = k-steps 2x and 2x + 1
-        uint4 raw = make_uint4(0u, 0u, 0u, 0u);
-        if (head < G) raw = *reinterpret_cast<const uint4*>(q_group + head * kD + 32 * j + 8 * x);
-        const uint32_t wds[4] = {raw.x, raw.y, raw.z, raw.w};
+        const uint32_t wds[4] = {raw[x].x, raw[x].y, raw[x].z, raw[x].w};
 #pragma unroll
         for (int y = 0; y < 4; ++y) {
-            const float sc = scan_pos_scale(2 * x + (y >> 1));
+            const float sc = scan_pos_scale(2 * x + (y >> 1)) * inv;
             const float lo = __uint_as_float(wds[y] << 16), hi = __uint_as_float(wds[y] & 0xffff0000u);
             const __half2 v = __floats2half2_rn(lo * sc, hi * sc);
             sq.qh[4 * x + y] = *reinterpret_cast<const uint32_t*>(&v);
         }
     }
+}
+
+// Loads the group's queries, picks the power of two per head and builds the fragments.  Returns 2^-k of head lane / 8.
+__device__ __forceinline__ float scan_setup(ScanQuery& sq, const __nv_bfloat16* q_group /* [G][128] */, int G,
+                                            int lane, float sm_scale) {
+    const int head = lane >> 3, j = lane & 3;
+    uint4 raw[4];
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        raw[x] = make_uint4(0u, 0u, 0u, 0u);
+        if (head < G) raw[x] = *reinterpret_cast<const uint4*>(q_group + head * kD + 32 * j + 8 * x);
+    }
+    const float inv = scan_query_scale(raw);
+    scan_setup_scaled(sq, raw, inv, lane);
+    // results come out for head lane % 4: its 2^k sits in the lanes of column head lane % 4, e.g. lane 8 * (lane % 4)
+    const float inv_res = __shfl_sync(kFull, inv, 8 * (lane & 3));
+    sq.unit = 1048576.0f * sm_scale / inv_res;
+    return inv;
 }
 
 // Returns, in every lane, the block maximum of the approximate logits (sm_scale applied) of head lane%4
@@ -391,34 +412,38 @@ __device__ __forceinline__ void scan_abs_sum(const uint4& qabs, const uint4& sv,
 // Upper bound (in logits) on the approximate score of every token of the block for the head this lane's column
 // belongs to: |sum_c q_c s_c level_c| <= 1.5 sum_c |q_c s_c|.  The factor 1.02 and the constant cover the fp16
 // roundings of the products and of the 16-term running sums (each below 2^-11 relative) and the lo pieces.
-__device__ __forceinline__ float scan_bound(__half2 sum_a, __half2 sum_b, float sm_scale) {
+// bmul = 1.5 * 1.02 * sm_scale * 2^k of the head, badd = 1e-3 + bmul * 2^-17 (the second term covers products that
+// underflowed in fp16: 128 of them, each rounded by at most 2^-25).
+__device__ __forceinline__ float scan_bound(__half2 sum_a, __half2 sum_b, float bmul, float badd) {
     const float2 a = __half22float2(sum_a), b = __half22float2(sum_b);
     float s = (a.x + a.y) + (b.x + b.y);
     s += __shfl_xor_sync(kFull, s, 1);
     s += __shfl_xor_sync(kFull, s, 2);
-    return 1.5f * 1.02f * sm_scale * s + 1e-3f;
+    return fmaf(bmul, s, badd);
 }
 
+// unit: accumulator units -> logits for head lane % 4 (ScanQuery::unit).  The result is NaN in every lane when the
+// fp16 B operand overflowed for any head of the group (the caller then redoes the block with scan_block_wide).
 template <bool PRECISE>
 __device__ __forceinline__ float scan_mma(const uint4 (&w)[4], const uint32_t (&bfrag)[16], int lane, int rows,
-                                          float sm_scale, float& band, float* tok = nullptr);
+                                          float unit, float& band, float* tok = nullptr);
 
 template <bool PRECISE>
 __device__ __forceinline__ float scan_compute(const ScanRegs& sr, const ScanQuery& sq, int lane, int rows,
-                                              float sm_scale, float& band) {
+                                              float& band) {
     uint32_t bfrag[16];
 #pragma unroll
     for (int x = 0; x < 4; ++x)
         scan_bfrag4(bfrag + 4 * x, make_uint4(sq.qh[4 * x], sq.qh[4 * x + 1], sq.qh[4 * x + 2], sq.qh[4 * x + 3]),
                     sr.s[x], sq.piece);
-    return scan_mma<PRECISE>(sr.w, bfrag, lane, rows, sm_scale, band);
+    return scan_mma<PRECISE>(sr.w, bfrag, lane, rows, sq.unit, band);
 }
 
 // tok (optional): the approximate logits themselves, tok[2 mt] for token 16 mt + lane/4 and tok[2 mt + 1] for the
 // token eight further on, head lane % 4 (rows past `rows` included: the caller masks them).
 template <bool PRECISE>
 __device__ __forceinline__ float scan_mma(const uint4 (&w)[4], const uint32_t (&bfrag)[16], int lane, int rows,
-                                          float sm_scale, float& band, float* tok) {
+                                          float unit, float& band, float* tok) {
     const int r = lane >> 2;
     float acc[4][4];
     float off[4] = {0.f, 0.f, 0.f, 0.f};
@@ -475,8 +500,9 @@ __device__ __forceinline__ float scan_mma(const uint4 (&w)[4], const uint32_t (&
     best = fmaxf(best, __shfl_xor_sync(kFull, best, 16));
     // sum_c (code - 1.5) q s = 2^20 * (acc - 1.5 * off)
     const float o = 1.5f * (off[0] + off[1]);
-    const float unit = 1048576.0f * sm_scale;
     band = kScanBandRel * (fabsf(best) + fabsf(o)) * unit;
+    // an overflowed B operand (+-inf) makes the level-offset sum of its head infinite or NaN
+    if (__any_sync(kFull, !(fabsf(o) < INFINITY))) return __int_as_float(0x7fc00000);
     if (tok) {
 #pragma unroll
         for (int mt = 0; mt < 4; ++mt) {
@@ -485,6 +511,60 @@ __device__ __forceinline__ float scan_mma(const uint4 (&w)[4], const uint32_t (&
         }
     }
     return (best - o) * unit;
+}
+
+// The scan of one block in plain binary32 on the ordinary lanes, for blocks whose fp16 B operand overflowed (scales
+// above ~2000): approx[h][t] = sm_scale * sum_c q[h][c] * s[c] * (code[t][c] - 1.5), fused multiply-adds in channel
+// order.  Lane L takes tokens 16 (L / 8) + L % 8 and eight further on.  Returns the block maximum of head lane % 4
+// over the first `rows` tokens (NaN or +-inf if binary32 overflowed as well); score_dst (optional): the per-token
+// logits, head h token t at score_dst[h * score_stride + t].  Rare by construction, so kept out of line and small.
+__device__ __noinline__ float scan_block_wide(const uint4* codes_tile, const __half* scales_tile,
+                                              const __nv_bfloat16* q_group, int G, int lane, int rows, float sm_scale,
+                                              float* score_dst, int score_stride) {
+    const int mt = lane >> 3, r = lane & 7;
+    float acc[kMaxG][2];
+#pragma unroll
+    for (int h = 0; h < kMaxG; ++h) acc[h][0] = acc[h][1] = 0.f;
+#pragma unroll 1
+    for (int j = 0; j < 4; ++j) {
+        const uint4 wv = ldg_plain(codes_tile + mt * 32 + 4 * r + j);
+        const uint32_t w[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll 1
+        for (int i = 0; i < 8; ++i) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int c = 32 * j + 4 * i + u, shift = 2 * i + 16 * (u & 1);
+                const float sc = __half2float(scales_tile[c]);
+                const float k0 = sc * ((float)((w[(u >> 1) * 2] >> shift) & 3u) - 1.5f);
+                const float k1 = sc * ((float)((w[(u >> 1) * 2 + 1] >> shift) & 3u) - 1.5f);
+#pragma unroll
+                for (int h = 0; h < kMaxG; ++h) {
+                    const float qv = h < G ? __bfloat162float(q_group[h * kD + c]) : 0.f;
+                    acc[h][0] = fmaf(qv, k0, acc[h][0]);
+                    acc[h][1] = fmaf(qv, k1, acc[h][1]);
+                }
+            }
+        }
+    }
+    const int t0 = 16 * mt + r, t1 = t0 + 8;
+    float mine = 0.f;
+#pragma unroll
+    for (int h = 0; h < kMaxG; ++h) {
+        const float a0 = acc[h][0] * sm_scale, a1 = acc[h][1] * sm_scale;
+        if (score_dst) {
+            score_dst[h * score_stride + t0] = a0;
+            score_dst[h * score_stride + t1] = a1;
+        }
+        float best = -INFINITY;
+        bool bad = false;
+        if (t0 < rows) { best = fmaxf(best, a0); bad |= !(fabsf(a0) < INFINITY); }
+        if (t1 < rows) { best = fmaxf(best, a1); bad |= !(fabsf(a1) < INFINITY); }
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) best = fmaxf(best, __shfl_xor_sync(kFull, best, o));
+        if (__any_sync(kFull, bad)) best = __int_as_float(0x7fc00000);   // fmaxf drops a NaN: say so explicitly
+        if ((lane & 3) == h) mine = best;
+    }
+    return mine;
 }
 
 // ---- attend: exact attention of one block, online softmax state in registers ------------------------------

@@ -15,6 +15,11 @@ becomes ``amp * q_dir[g*G + r % G] + N(0, 0.3)``, so every query head of the gro
 Needle blocks per (sequence, KV head): ``round(frac * nb)`` distinct blocks from the middle ``[1, nb-16)``,
 plus block 0 as an attention sink where the config says so.  Rows past ``seq_len`` in the tail block and
 all unused pages hold the finite poison value 1e4 in K and V: reading them shows up at once.
+
+Magnitude knobs (tests of the input range; the five configurations leave them at 1): ``q_gain`` / ``k_gain``
+multiply every query / key value; ``k_outliers = (count, gain)`` multiplies ``count`` seeded key channels per KV
+head by ``gain`` and ``q_outliers`` does the same to the queries of those channels, as the key and query caches of
+some model families show (a few channels hundreds of times larger than the rest).
 """
 from __future__ import annotations
 
@@ -76,10 +81,12 @@ class Workload:
 
 
 def make_workload(name: str, *, variant: int = 0, N: int | None = None, B: int | None = None,
-                  lens: tuple | None = None, sink: bool | None = None, tail: int = 0) -> Workload:
+                  lens: tuple | None = None, sink: bool | None = None, tail: int = 0, q_gain: float = 1.0,
+                  k_gain: float = 1.0, k_outliers: tuple | None = None, q_outliers: tuple | None = None) -> Workload:
     """Build config ``name`` (C1..C5).  ``N`` / ``B`` / ``lens`` shrink or reshape it for tests; ``tail`` subtracts
     that many tokens from every sequence (ragged last block); ``variant`` k adds 10*k to the seed;
-    ``sink=False`` gives the "no-sink" correctness variant."""
+    ``sink=False`` gives the "no-sink" correctness variant; the gains and outlier channels are described in the
+    module's header."""
     cfg = dict(CONFIGS[name])
     seed = cfg["seed"] + 10 * variant
     gen = torch.Generator().manual_seed(seed)
@@ -110,8 +117,22 @@ def make_workload(name: str, *, variant: int = 0, N: int | None = None, B: int |
         block_table = None
 
     q32 = torch.randn(Bn, Hq, HEAD_DIM, generator=gen)
-    q = q32.to(torch.bfloat16)
     q_dir = q32 / q32.pow(2).mean(dim=-1, keepdim=True).sqrt()
+    # per-channel multipliers of the magnitude knobs, drawn from a generator of their own (the five configurations'
+    # streams are the same with and without them)
+    k_mult = torch.full((Hkv, HEAD_DIM), float(k_gain))
+    q_mult = torch.full((Hq, HEAD_DIM), float(q_gain))
+    side = torch.Generator().manual_seed(seed + 7777)
+    for spec, which in ((k_outliers, "k"), (q_outliers, "q")):
+        if spec:
+            count, gain = spec
+            for g in range(Hkv):
+                chans = torch.randperm(HEAD_DIM, generator=side)[:count]
+                if which == "k":
+                    k_mult[g, chans] *= gain
+                else:
+                    q_mult[g * G:(g + 1) * G, chans] *= gain
+    q = (q32 * q_mult.unsqueeze(0)).to(torch.bfloat16)
 
     k_cache = torch.full((num_pages, Hkv, BLOCK_TOKENS, HEAD_DIM), POISON, dtype=torch.bfloat16)
     v_cache = torch.full((num_pages, Hkv, BLOCK_TOKENS, HEAD_DIM), POISON, dtype=torch.bfloat16)
@@ -152,6 +173,7 @@ def make_workload(name: str, *, variant: int = 0, N: int | None = None, B: int |
                     rec = sorted(set([0] + list(range(max(nb - n_rec, 0), nb))))
                     K[rec, g] = aligned_rows(b, g, cfg["recency_amp"], len(rec))
             needles[(b, g)] = planted
+        K *= k_mult.view(1, Hkv, 1, HEAD_DIM)
         valid_last = int(seq[b]) - (nb - 1) * BLOCK_TOKENS
         if valid_last < BLOCK_TOKENS:
             K[nb - 1, :, valid_last:] = POISON

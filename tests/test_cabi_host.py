@@ -47,6 +47,28 @@ def test_workspace_bytes_grows_with_geometry():
     assert ra - a == rb - b == 192 * 8 * 32 * 4 * 72 * 4
 
 
+def test_documented_limits_of_the_static_entry_point_are_the_computed_ones():
+    """include/ffd.h quotes, for 32 query / 8 KV heads on a 148-SM GPU, the longest contexts whose workspace fits the
+    built-in scratch array of ffd_decode_static; the figures must be the ones ffd_workspace_bytes gives."""
+    cfg = ffd.Config(32, 8)
+
+    def longest(batch):
+        lo, hi = 1, 1 << 16
+        while lo < hi:    # the workspace size is monotone in the block count
+            mid = (lo + hi + 1) // 2
+            if ffd.ffd_workspace_bytes(cfg, batch, mid) <= ffd.STATIC_SCRATCH_BYTES:
+                lo = mid
+            else:
+                hi = mid - 1
+        return lo * 64
+
+    text = " ".join(open(os.path.join(ROOT, "include", "ffd.h")).read().split())
+    m = re.search(r"batch 1 up to about (\d+) K tokens of context, batch 4 up to about (\d+) K, batch 16 up to about "
+                  r"\* (\d+) K", text)
+    assert m, "the limits sentence of ffd_decode_static has changed its wording"
+    assert [int(x) for x in m.groups()] == [longest(b) // 1000 for b in (1, 4, 16)]
+
+
 @pytest.mark.parametrize("field,value,status", [
     ("head_dim", 64, 3), ("block_tokens", 32, 3), ("quant_bits", 4, 3), ("num_kv_heads", 5, 2),
     ("num_q_heads", 64, 3), ("n_local_blocks", -1, 2), ("out_dtype", 7, 3), ("sm_scale", -1.0, 2),

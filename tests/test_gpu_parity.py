@@ -3,6 +3,11 @@
 Bars (from the benchmark spec): codes and scales bit-exact; kept-block mask bit-exact except blocks whose oracle
 block maximum lies within 1e-4 of the threshold; outputs (fp32) within 1e-2 max-abs and 1e-3 mean-abs; the bf16
 output is the rounding of the fp32 output.
+
+The 1e-4 band and the tighter regression bars are stated for the O(1) inputs of the five configurations, whose logits
+stay below ~50.  The approximate scores are binary32 sums, so their error grows with the size of the logits: on the
+large-magnitude cases every band is multiplied by max(1, L / 32), L = the largest approximate block maximum of the
+workload in the oracle (4 units of binary32 rounding at |logit| = 32 are 1.5e-5; the bars keep their 6x margin).
 """
 import math
 
@@ -11,6 +16,7 @@ import pytest
 import torch
 
 from paper_2609_00097_b200.workloads import make_workload, repage
+from tests.device_cache import DeviceCache
 
 pytestmark = pytest.mark.gpu
 
@@ -62,7 +68,13 @@ def check_residual(ffd, oracle, w, dc, codes, scales):
     return k_res
 
 
-def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None, k_res=None):
+def magnitude(r, w):
+    """max(1, L / 32) for the oracle result r: the factor by which the bands grow on large-magnitude inputs."""
+    finite = r.block_max[np.isfinite(r.block_max)]
+    return max(1.0, float(np.abs(finite).max()) / 32.0) if finite.size else 1.0
+
+
+def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None, k_res=None, expect_status=0):
     """k_res (the oracle's residuals): check the 2 + 8 bit format's decode against the oracle's Dequant refinement."""
     B, Hq, mb = w.B, w.Hq, w.max_blocks
     gpu_decode = dc.decode if k_res is None else dc.decode_residual
@@ -72,32 +84,39 @@ def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None, k_res=Non
     # bound already rules them out: the decisions and the output must not change
     kept_fast = torch.full((B, Hq, mb), 255, dtype=torch.uint8, device="cuda")
     gpu_decode(delta, kept_mask=kept_fast)
-    assert ffd.ffd_read_device_status(dc.workspace) == 0
+    assert ffd.ffd_read_device_status(dc.workspace) == expect_status
     out_fast = dc.out.clone()
     gpu_decode(delta, kept_mask=kept, block_max=bm)
-    assert ffd.ffd_read_device_status(dc.workspace) == 0
+    assert ffd.ffd_read_device_status(dc.workspace) == expect_status
     assert torch.equal(kept, kept_fast)
     assert (dc.out - out_fast).abs().max().item() <= 1e-6
     out = dc.out.cpu().numpy().astype(np.float64)
     lse = dc.lse.cpu().numpy().astype(np.float64)
     kept = kept.cpu().numpy()
-    bm = bm.cpu().numpy()
+    bm = bm.cpu().numpy().astype(np.float64)
     r = oracle.decode(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), codes, scales, w.block_table, w.seq_lens,
                       mb, delta, n_sink=dc.cfg.n_sink_blocks, n_local=dc.cfg.n_local_blocks, units=units, k_res=k_res)
     rows = units if units is not None else [(b, h) for b in range(B) for h in range(Hq)]
+    mag = magnitude(r, w)
     differs = False
-    for b, h in rows:
+    wanted = np.zeros((B, Hq), dtype=bool)
+    wanted[tuple(np.array(rows).T)] = True
+    for b in range(B):
+        hs = np.where(wanted[b])[0]
+        if hs.size == 0:
+            continue
         nb = w.num_blocks(b)
-        assert np.all(kept[b, h, nb:] == 255), "mask written past the sequence's blocks"
+        assert np.all(kept[b, hs, nb:] == 255), "mask written past the sequence's blocks"
         # debug output: fast-scan values carry the tensor-core accumulation error, a few 1e-6 of the accumulator's
         # size, which can be several times the result's (the level offset is subtracted afterwards); decisions near
         # the threshold do not rest on these values (the kernel redoes them precisely), see the mask check below
-        assert np.all(np.abs(bm[b, h, :nb] - r.block_max[b, h, :nb]) < 1e-4 + 2e-5 * np.abs(r.block_max[b, h, :nb]))
-        diff = kept[b, h, :nb] != r.kept[b, h, :nb]
+        want_bm = r.block_max[b, hs, :nb]
+        assert np.all(np.abs(bm[b, hs, :nb] - want_bm) < 1e-4 * mag + 2e-5 * np.abs(want_bm))
+        diff = kept[b, hs, :nb] != r.kept[b, hs, :nb]
         if diff.any():
             differs = True
-            margin = np.abs(r.block_max[b, h, :nb] - (r.mtilde[b, h] - delta))
-            assert np.all(margin[diff] < MASK_BAND), (b, h, np.where(diff)[0], margin[diff])
+            margin = np.abs(want_bm - (r.mtilde[b, hs, None] - delta))
+            assert np.all(margin[diff] < MASK_BAND * mag), (b, np.where(diff), margin[diff])
     if differs:   # compare the output against the oracle's attention over the GPU's (equally valid) mask
         forced = np.where(kept == 255, 0, kept).astype(np.uint8)
         r = oracle.decode(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), codes, scales, w.block_table,
@@ -105,8 +124,8 @@ def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None, k_res=Non
     idx = tuple(np.array(rows).T)
     err = np.abs(out[idx] - r.out[idx])
     assert err.max() < OUT_MAX and err.mean() < OUT_MEAN
-    assert err.max() < OUT_MAX_EXPECTED, err.max()
-    assert np.abs(lse[idx] - r.lse[idx]).max() < 1e-3
+    assert err.max() < OUT_MAX_EXPECTED * mag, err.max()
+    assert np.abs(lse[idx] - r.lse[idx]).max() < 1e-3 * mag
     return r
 
 
@@ -143,7 +162,7 @@ SMALL = [
 @pytest.mark.parametrize("name,kw,_", SMALL)
 def test_small_configs_element_by_element(ffd, oracle, name, kw, _):
     w = make_workload(name, **kw)
-    dc = ffd.DeviceCache(w)
+    dc = DeviceCache(w)
     codes, scales = check_quantize(ffd, oracle, w, dc)
     for delta in w.deltas:
         check_decode(ffd, oracle, w, dc, codes, scales, delta)
@@ -156,7 +175,7 @@ def test_small_configs_residual_key_format(ffd, oracle, name, kw, _):
     """Sec. 3.1 / 3.3: the 2 + 8 bit key format.  Residual codes bit for bit; the decode that refines from
     k_quant + k_res (two-term score) against the oracle's Dequant refinement at the same bars as the 16-bit path."""
     w = make_workload(name, **kw)
-    dc = ffd.DeviceCache(w)
+    dc = DeviceCache(w)
     codes, scales = check_quantize(ffd, oracle, w, dc)
     k_res = check_residual(ffd, oracle, w, dc, codes, scales)
     dc.k_cache = None   # the residual decode must not need the 16-bit keys
@@ -166,10 +185,10 @@ def test_small_configs_residual_key_format(ffd, oracle, name, kw, _):
 
 def test_bf16_output_is_rounding_of_fp32_output(ffd, oracle):
     w = make_workload("C1")
-    dc32 = ffd.DeviceCache(w)
+    dc32 = DeviceCache(w)
     dc32.quantize()
     dc32.decode(6.0)
-    dc16 = ffd.DeviceCache(w, ffd.Config(w.Hq, w.Hkv, out_dtype=0))
+    dc16 = DeviceCache(w, ffd.Config(w.Hq, w.Hkv, out_dtype=0))
     dc16.quantize()
     dc16.decode(6.0)
     torch.cuda.synchronize()
@@ -179,7 +198,7 @@ def test_bf16_output_is_rounding_of_fp32_output(ffd, oracle):
 def test_paged_equals_contiguous_bitwise(ffd, oracle):
     w = make_workload("C2", N=5000)
     wp = repage(w)
-    a, b = ffd.DeviceCache(w), ffd.DeviceCache(wp)
+    a, b = DeviceCache(w), DeviceCache(wp)
     a.quantize(), b.quantize()
     ka = torch.zeros(w.B, w.Hq, w.max_blocks, dtype=torch.uint8, device="cuda")
     kb = torch.zeros_like(ka)
@@ -192,7 +211,7 @@ def test_paged_equals_contiguous_bitwise(ffd, oracle):
 
 def test_delta_inf_matches_dense_path_and_split_merge_is_stable(ffd, oracle):
     w = make_workload("C2", N=8192, tail=9)
-    dc = ffd.DeviceCache(w)
+    dc = DeviceCache(w)
     dc.quantize()
     dc.decode(INF)
     sparse = dc.out.clone()
@@ -203,7 +222,7 @@ def test_delta_inf_matches_dense_path_and_split_merge_is_stable(ffd, oracle):
 
 def test_tail_requantize_only_touches_the_last_block(ffd, oracle):
     w = make_workload("C5", B=3, lens=(700, 2000))
-    dc = ffd.DeviceCache(w)
+    dc = DeviceCache(w)
     dc.quantize()
     q0, s0 = dc.k_quant.clone(), dc.k_scales.clone()
     dc.k_quant.fill_(0x55)
@@ -228,7 +247,7 @@ def test_residual_serving_loop_from_one_graph(ffd, oracle):
     full = w.seq_lens.copy()
     steps = 70                                  # crosses a block boundary in every sequence
     w.seq_lens[:] = full - steps
-    a, b = ffd.DeviceCache(w), ffd.DeviceCache(w)
+    a, b = DeviceCache(w), DeviceCache(w)
     for dc in (a, b):
         dc.quantize()
         dc.quantize_residual()
@@ -286,7 +305,7 @@ def test_residual_serving_loop_from_one_graph(ffd, oracle):
 def test_residual_tail_requantize_only_touches_the_last_block(ffd, oracle):
     """With first_token the residuals of the block the newest token fell into are redone, nothing else."""
     w = make_workload("C5", B=3, lens=(700, 2000))
-    dc = ffd.DeviceCache(w)
+    dc = DeviceCache(w)
     dc.quantize()
     dc.quantize_residual()
     r0 = dc.k_res.clone()
@@ -320,7 +339,7 @@ def test_residual_decode_edge_cases(ffd, oracle):
     import paper_2609_00097_b200.workloads as W
     w = make_workload("C5", B=3, lens=(100, 400))
     w.seq_lens[:] = np.array([0, 1, int(w.seq_lens[2])], dtype=np.int32)
-    dc = ffd.DeviceCache(w)
+    dc = DeviceCache(w)
     codes, scales = check_quantize(ffd, oracle, w, dc)
     k_res = check_residual(ffd, oracle, w, dc, codes, scales)
     dc.out.fill_(7.0)
@@ -336,7 +355,7 @@ def test_residual_decode_edge_cases(ffd, oracle):
             w = make_workload("res_edge")
             for out_dtype in (1, 0):
                 cfg = ffd.Config(G * Hkv, Hkv, n_sink_blocks=n_sink, n_local_blocks=n_local, out_dtype=out_dtype)
-                dc = ffd.DeviceCache(w, cfg)
+                dc = DeviceCache(w, cfg)
                 codes, scales = check_quantize(ffd, oracle, w, dc)
                 k_res = check_residual(ffd, oracle, w, dc, codes, scales)
                 if out_dtype == 1:
@@ -350,7 +369,7 @@ def test_residual_decode_edge_cases(ffd, oracle):
         W.CONFIGS.pop("res_edge", None)
     # a page-table entry out of range: that block is skipped and the status word says so; nothing faults
     w = make_workload("C5", B=2, lens=(500, 900))
-    dc = ffd.DeviceCache(w)
+    dc = DeviceCache(w)
     dc.quantize()
     dc.quantize_residual()
     dc.block_table[1, 2] = w.num_pages + 7
@@ -363,7 +382,7 @@ def test_empty_and_single_token_sequences(ffd, oracle):
     w = make_workload("C5", B=3, lens=(100, 400))
     w.seq_lens[0] = 0
     w.seq_lens[1] = 1
-    dc = ffd.DeviceCache(w)
+    dc = DeviceCache(w)
     dc.quantize()
     dc.out.fill_(7.0)
     dc.decode(6.0)
@@ -379,7 +398,7 @@ def test_empty_and_single_token_sequences(ffd, oracle):
 def test_bad_page_index_sets_status_and_does_not_fault(ffd, oracle):
     """A block_table entry outside [0, num_pages) is skipped and reported; nothing is read through it."""
     w = make_workload("C5", B=2, lens=(600, 900))
-    dc = ffd.DeviceCache(w)
+    dc = DeviceCache(w)
     dc.quantize()
     dc.block_table[0, 1] = w.num_pages + 5
     dc.decode(6.0)
@@ -393,7 +412,7 @@ def test_cache_with_room_for_much_longer_sequences(ffd, oracle):
     give the same results, and the work items of the rows nobody reaches must not be handed out."""
     w = make_workload("C5", B=4, lens=(3000, 5000))
     w.seq_lens[:] = np.array([700, 64, 1, 333], dtype=np.int32)       # capacity stays ~79 blocks
-    dc = ffd.DeviceCache(w)
+    dc = DeviceCache(w)
     codes, scales = check_quantize(ffd, oracle, w, dc)
     check_decode(ffd, oracle, w, dc, codes, scales, 6.0)
     check_decode(ffd, oracle, w, dc, codes, scales, INF)
@@ -405,7 +424,7 @@ def test_one_long_sequence_among_short_ones(ffd, oracle):
     existing items.  Same results as ever."""
     w = make_workload("C5", B=6, lens=(4000, 5000))
     w.seq_lens[:] = np.array([int(w.seq_lens[0]), 200, 130, 64, 1, 2049], dtype=np.int32)
-    dc = ffd.DeviceCache(w)
+    dc = DeviceCache(w)
     codes, scales = check_quantize(ffd, oracle, w, dc)
     for delta in (6.0, 0.0, INF):
         check_decode(ffd, oracle, w, dc, codes, scales, delta)
@@ -415,7 +434,7 @@ def test_step_replays_from_a_cuda_graph(ffd, oracle):
     """A whole step (tail re-quantize + decode) captured once and replayed gives the eager step's result; every
     step-varying argument (q, seq_lens, first_token, block_table) lives on the device (Sec. 3.3)."""
     w = make_workload("C5", B=4, lens=(1000, 5000))
-    dc = ffd.DeviceCache(w)
+    dc = DeviceCache(w)
     dc.quantize()
     first = torch.from_numpy(np.maximum(w.seq_lens - 1, 0).astype(np.int32)).cuda()
 
@@ -458,7 +477,7 @@ def test_append_writes_the_token_requantizes_its_block_and_bumps_the_length(ffd,
     full = w.seq_lens.copy()
     full[0] = 64 * ((full[0] - 3) // 64) + 2            # sequence 0 crosses into a new block during the appends
     full[1] = 64 * ((full[1] - steps - 1) // 64) + steps    # sequence 1 starts its last block at row 0
-    dc = ffd.DeviceCache(w)
+    dc = DeviceCache(w)
     k_all, v_all = dc.k_cache.clone(), dc.v_cache.clone()
     start = (full - steps).astype(np.int32)
     dc.seq_lens.copy_(torch.from_numpy(start))
@@ -509,7 +528,7 @@ def test_serving_loop_append_and_decode_from_one_graph(ffd, oracle):
     calls give when issued eagerly on a second copy of the cache."""
     w = make_workload("C5", B=4, lens=(1000, 5000))
     w.seq_lens[:] = w.seq_lens - 8                      # room for the appended tokens inside the mapped blocks
-    a, b = ffd.DeviceCache(w), ffd.DeviceCache(w)
+    a, b = DeviceCache(w), DeviceCache(w)
     a.quantize(), b.quantize()
     gen = torch.Generator(device="cuda").manual_seed(5)
     k_new = torch.randn(w.B, w.Hkv, 128, device="cuda", generator=gen).to(torch.bfloat16)
@@ -551,7 +570,7 @@ def test_append_decode_equals_append_then_decode(ffd, oracle):
     w = make_workload("C5", B=4, lens=(1000, 5000))
     w.seq_lens[:] = w.seq_lens - 70                      # the appends below cross at least one block boundary
     w.seq_lens[1] = 64 * (int(w.seq_lens[1]) // 64)      # sequence 1 starts a block with its first append
-    a, b = ffd.DeviceCache(w), ffd.DeviceCache(w)
+    a, b = DeviceCache(w), DeviceCache(w)
     a.quantize(), b.quantize()
     gen = torch.Generator(device="cuda").manual_seed(9)
     kept_a = torch.zeros(w.B, w.Hq, w.max_blocks, dtype=torch.uint8, device="cuda")
@@ -618,7 +637,7 @@ def test_randomised_geometries(ffd, oracle):
             delta = float(rng.choice([0.0, 0.5, 3.0, 6.0, 12.0, np.inf]))
             W.CONFIGS["sweep"] = recipe
             w = make_workload("sweep")
-            dc = ffd.DeviceCache(w, ffd.Config(G * Hkv, Hkv, n_sink_blocks=n_sink, n_local_blocks=n_local))
+            dc = DeviceCache(w, ffd.Config(G * Hkv, Hkv, n_sink_blocks=n_sink, n_local_blocks=n_local))
             codes, scales = check_quantize(ffd, oracle, w, dc)
             check_decode(ffd, oracle, w, dc, codes, scales, delta)
             check_dense(ffd, oracle, w, dc)
@@ -642,7 +661,7 @@ def test_many_short_sequences(ffd, oracle, B, Hkv, G, lens, paged):
     try:
         W.CONFIGS["many_short"] = recipe
         w = make_workload("many_short")
-        dc = ffd.DeviceCache(w, ffd.Config(G * Hkv, Hkv))
+        dc = DeviceCache(w, ffd.Config(G * Hkv, Hkv))
         codes, scales = check_quantize(ffd, oracle, w, dc)
         for delta in (6.0, INF):
             check_decode(ffd, oracle, w, dc, codes, scales, delta)
@@ -668,7 +687,7 @@ def test_very_long_contexts_on_sampled_heads(ffd, oracle, lens, short):
         W.CONFIGS.pop("very_long", None)
     if short is not None:
         w.seq_lens[1] = short
-    dc = ffd.DeviceCache(w)
+    dc = DeviceCache(w)
     dc.quantize()
     codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
     _, mapped = valid_row_mask(w)
@@ -689,7 +708,7 @@ def test_global_approximate_max_rule_through_the_configuration(ffd, oracle):
     for name, kw in (("C2", dict(N=8192, tail=5)), ("C2", dict(N=6000, sink=False)), ("C5", dict(B=3, lens=(700, 3000)))):
         w = make_workload(name, **kw)
         cfg = ffd.Config(w.Hq, w.Hkv, n_sink_blocks=0, n_local_blocks=w.max_blocks)
-        dc = ffd.DeviceCache(w, cfg)
+        dc = DeviceCache(w, cfg)
         codes, scales = check_quantize(ffd, oracle, w, dc)
         for delta in (4.0, 6.0):
             r = check_decode(ffd, oracle, w, dc, codes, scales, delta)
@@ -714,50 +733,100 @@ def test_residual_with_many_short_sequences(ffd, oracle):
         w = make_workload("many_short")
     finally:
         W.CONFIGS.pop("many_short", None)
-    dc = ffd.DeviceCache(w, ffd.Config(4, 2))
+    dc = DeviceCache(w, ffd.Config(4, 2))
     codes, scales = check_quantize(ffd, oracle, w, dc)
     k_res = check_residual(ffd, oracle, w, dc, codes, scales)
     for delta in (6.0, INF):
         check_decode(ffd, oracle, w, dc, codes, scales, delta, k_res=k_res)
 
 
-# full-size configurations: the oracle checks a sample of (sequence, head) rows one by one
-FULL = [
-    ("C2", dict(), 8),
-    ("C3", dict(), 6),
-    ("C4", dict(), 4),
-    ("C5", dict(), 6),
+# full-size configurations: every (sequence, query head) row and every mapped page against the oracle
+FULL = ["C2", "C3", "C4", "C5"]
+
+
+@pytest.mark.parametrize("name", FULL)
+def test_full_size_configs_every_row(ffd, oracle, name):
+    """The configurations at the sizes the benchmark runs them, in the launch configuration it times: codes and
+    scales of every mapped tile, and mask, block maxima, output and log-sum-exp of every (sequence, query head) row at
+    every delta of the configuration; C3 and C5 also on the 2 + 8 bit key format."""
+    oracle.set_threads(oracle.max_threads())
+    try:
+        w = make_workload(name)
+        dc = DeviceCache(w)
+        codes, scales = check_quantize(ffd, oracle, w, dc)
+        for delta in w.deltas:
+            check_decode(ffd, oracle, w, dc, codes, scales, delta)
+        check_dense(ffd, oracle, w, dc)
+        if name in ("C3", "C5"):
+            k_res = check_residual(ffd, oracle, w, dc, codes, scales)
+            dc.k_cache = None
+            check_decode(ffd, oracle, w, dc, codes, scales, w.deltas[0], k_res=k_res)
+    finally:
+        oracle.set_threads(min(8, oracle.max_threads()))
+
+
+LARGE = [
+    dict(q_gain=8.0),
+    dict(k_gain=64.0),
+    dict(k_gain=512.0),
+    dict(q_gain=64.0, k_gain=8.0),
+    dict(k_outliers=(4, 100.0)),                          # a few key channels 100 times larger than the rest
+    dict(k_outliers=(3, 300.0), q_outliers=(3, 20.0)),    # ... and the matching query channels
+    dict(k_gain=8.0, k_outliers=(4, 100.0)),              # scales above 2047: blocks leave the tensor-core scan
+    dict(q_gain=3000.0, q_outliers=(1, 100.0)),           # |q| up to ~1e6: far beyond fp16 without the per-head scaling
+    dict(q_gain=1e-3, k_gain=1e-3),                       # everything tiny
 ]
 
 
-@pytest.mark.parametrize("name,kw,n_units", FULL)
-def test_full_size_configs_on_sampled_heads(ffd, oracle, name, kw, n_units):
-    w = make_workload(name, **kw)
-    dc = ffd.DeviceCache(w)
+@pytest.mark.parametrize("knobs", LARGE)
+def test_large_magnitude_inputs(ffd, oracle, knobs):
+    """The scan forms its tensor-core operand in fp16: queries and scales of any magnitude must give the oracle's
+    decisions (App. A.1 puts no bound on the scale), never a silently dropped head.  Gains of 8 .. 512, outlier
+    channels of x100 .. x300 as in the key caches of some model families, and scales beyond what the fp16 operand
+    holds (those blocks are scored in binary32 instead)."""
+    for name, kw in (("C2", dict(N=6144, tail=11)), ("C5", dict(B=3, lens=(700, 3000)))):
+        w = make_workload(name, **kw, **knobs)
+        dc = DeviceCache(w)
+        codes, scales = check_quantize(ffd, oracle, w, dc)
+        for delta in (6.0, 0.0, INF):
+            check_decode(ffd, oracle, w, dc, codes, scales, delta)
+        if name == "C5":
+            k_res = check_residual(ffd, oracle, w, dc, codes, scales)
+            check_decode(ffd, oracle, w, dc, codes, scales, 6.0, k_res=k_res)
+
+
+def test_scores_beyond_binary32_are_reported_not_dropped(ffd, oracle):
+    """Queries of ~1e34 against saturated scales: the approximate scores overflow binary32.  Nothing sensible can be
+    computed, but the library says so (FFD_DEV_RANGE) instead of returning a quietly empty selection."""
+    w = make_workload("C1", q_gain=1e34, k_gain=1e6)
+    dc = DeviceCache(w)
     dc.quantize()
-    rng = np.random.default_rng(11)
-    units = sorted({(int(rng.integers(w.B)), int(rng.integers(w.Hq))) for _ in range(4 * n_units)})[:n_units]
-    if w.flat_heads:   # make sure both head kinds are sampled
-        units = sorted(set(units[: n_units - 2] + [(0, w.flat_heads[0] * w.G), (w.B - 1, 0)]))
-    # oracle quantizer on the sampled KV heads only would need a sub-cache; the GPU codes were verified bit-exact
-    # on the small configs, and here the oracle runs its own quantizer over the whole cache
-    codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
-    g_scales = dc.k_scales.cpu().view(torch.int16).numpy().view(np.uint16)
-    _, mapped = valid_row_mask(w)
-    assert np.array_equal(g_scales[mapped], scales[mapped])
-    vm, _ = valid_row_mask(w)
-    g_codes = dc.canonical_codes().cpu().numpy()
-    for page in rng.choice(np.where(mapped)[0], size=64, replace=False):
-        sel = np.broadcast_to(vm[page], codes[page].shape)
-        assert np.array_equal(g_codes[page][sel], codes[page][sel])
-    del g_codes
-    for delta in w.deltas:
-        check_decode(ffd, oracle, w, dc, codes, scales, delta, units=units)
-    check_dense(ffd, oracle, w, dc, units=units[:2])
-    if name in ("C3", "C5"):   # the 2 + 8 bit key format at full size: residuals of sampled pages, sampled heads
-        dc.quantize_residual()
-        k_res = oracle.quantize_residual(w.bits("k_cache"), codes, scales, w.block_table, w.seq_lens, w.max_blocks)
-        for page in rng.choice(np.where(mapped)[0], size=64, replace=False):
-            assert np.array_equal(dc.k_res[int(page)].cpu().numpy(), k_res[page])
-        dc.k_cache = None
-        check_decode(ffd, oracle, w, dc, codes, scales, w.deltas[0], units=units, k_res=k_res)
+    kept = torch.zeros(w.B, w.Hq, w.max_blocks, dtype=torch.uint8, device="cuda")
+    dc.decode(6.0, kept_mask=kept)
+    assert ffd.ffd_read_device_status(dc.workspace) & ffd.DEV_RANGE
+    assert int(kept.sum()) > 0
+
+
+def test_uninitialised_workspace_is_detected(ffd, oracle):
+    """A workspace that never saw ffd_workspace_init (garbage work counters): the decode must not index with them;
+    it reports FFD_DEV_BAD_WORKSPACE.  After the init the same workspace works."""
+    w = make_workload("C1")
+    dc = DeviceCache(w)
+    dc.quantize()
+    dc.decode(6.0)
+    torch.cuda.synchronize()
+    want = dc.out.clone()
+    good = dc.workspace
+    dc.workspace = torch.full_like(good, 0xA5)
+    dc.decode(6.0)
+    assert ffd.ffd_read_device_status(dc.workspace) & ffd.DEV_BAD_WORKSPACE
+    # counters an interrupted call left behind, under a valid header: reported too, nothing stored out of range
+    dc.workspace = good
+    good.view(torch.int32)[17] = 12345          # the heavy-class count
+    good.view(torch.int32)[18] = 54321          # the light-class count
+    dc.decode(6.0)
+    assert ffd.ffd_read_device_status(dc.workspace) & ffd.DEV_BAD_WORKSPACE
+    ffd.ffd_workspace_init(dc.workspace)
+    dc.decode(6.0)
+    assert ffd.ffd_read_device_status(dc.workspace) == 0
+    assert torch.equal(dc.out, want)
