@@ -4,10 +4,12 @@ Bars (from the benchmark spec): codes and scales bit-exact; kept-block mask bit-
 block maximum lies within 1e-4 of the threshold; outputs (fp32) within 1e-2 max-abs and 1e-3 mean-abs; the bf16
 output is the rounding of the fp32 output.
 
-The 1e-4 band and the tighter regression bars are stated for the O(1) inputs of the five configurations, whose logits
-stay below ~50.  The approximate scores are binary32 sums, so their error grows with the size of the logits: on the
-large-magnitude cases every band is multiplied by max(1, L / 32), L = the largest approximate block maximum of the
-workload in the oracle (4 units of binary32 rounding at |logit| = 32 are 1.5e-5; the bars keep their 6x margin).
+The bars are stated for the O(1) inputs of the five configurations, whose logits stay below ~50.  Approximate and
+exact scores are binary32 sums (and the softmax exponent is a binary32 number of the logits' size), so their
+absolute error grows with the size of the logits: a logit of 20000 carries an error of several 1e-3 whatever the
+kernel does, and the softmax weights inherit it.  On the large-magnitude cases every bar is therefore multiplied by
+max(1, L / 64), L = the largest approximate block maximum of the workload in the oracle; on the five configurations
+(L < 64) the factor is exactly 1.
 """
 import math
 
@@ -69,9 +71,9 @@ def check_residual(ffd, oracle, w, dc, codes, scales):
 
 
 def magnitude(r, w):
-    """max(1, L / 32) for the oracle result r: the factor by which the bands grow on large-magnitude inputs."""
+    """max(1, L / 64) for the oracle result r: the factor by which the bars grow on large-magnitude inputs."""
     finite = r.block_max[np.isfinite(r.block_max)]
-    return max(1.0, float(np.abs(finite).max()) / 32.0) if finite.size else 1.0
+    return max(1.0, float(np.abs(finite).max()) / 64.0) if finite.size else 1.0
 
 
 def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None, k_res=None, expect_status=0):
@@ -123,8 +125,8 @@ def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None, k_res=Non
                           w.seq_lens, mb, delta, forced_mask=forced, units=units, k_res=k_res)
     idx = tuple(np.array(rows).T)
     err = np.abs(out[idx] - r.out[idx])
-    assert err.max() < OUT_MAX and err.mean() < OUT_MEAN
-    assert err.max() < OUT_MAX_EXPECTED * mag, err.max()
+    assert err.max() < OUT_MAX * mag and err.mean() < OUT_MEAN * mag, (err.max(), err.mean(), mag)
+    assert err.max() < OUT_MAX_EXPECTED * mag, (err.max(), mag)
     assert np.abs(lse[idx] - r.lse[idx]).max() < 1e-3 * mag
     return r
 
