@@ -126,7 +126,9 @@ def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None, k_res=Non
     idx = tuple(np.array(rows).T)
     err = np.abs(out[idx] - r.out[idx])
     assert err.max() < OUT_MAX * mag and err.mean() < OUT_MEAN * mag, (err.max(), err.mean(), mag)
-    assert err.max() < OUT_MAX_EXPECTED * mag, (err.max(), mag)
+    # the regression bar: 2e-4 on the five configurations; a relative error of ~1e-6 L in the softmax weights (the
+    # binary32 exponent) times the spread of V beyond that
+    assert err.max() < OUT_MAX_EXPECTED * max(1.0, 1.6 * mag), (err.max(), mag)
     assert np.abs(lse[idx] - r.lse[idx]).max() < 1e-3 * mag
     return r
 
