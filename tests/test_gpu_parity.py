@@ -113,7 +113,9 @@ def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None, k_res=Non
         # size, which can be several times the result's (the level offset is subtracted afterwards); decisions near
         # the threshold do not rest on these values (the kernel redoes them precisely), see the mask check below
         want_bm = r.block_max[b, hs, :nb]
-        assert np.all(np.abs(bm[b, hs, :nb] - want_bm) < 1e-4 * mag + 2e-5 * np.abs(want_bm))
+        # (on the large-magnitude cases the accumulator's size is that of the largest logits of the workload, not of the
+        # block's own maximum: outlier channels make small results out of large terms)
+        assert np.all(np.abs(bm[b, hs, :nb] - want_bm) < 1e-4 * mag + 2e-5 * np.maximum(np.abs(want_bm), 64.0 * (mag - 1.0)))
         diff = kept[b, hs, :nb] != r.kept[b, hs, :nb]
         if diff.any():
             differs = True
