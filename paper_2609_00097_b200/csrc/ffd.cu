@@ -711,13 +711,290 @@ __global__ void __launch_bounds__(kWarps * 32, 1) dense_kernel(DecodeParams p) {
     }
 }
 
-__global__ void clear_status_kernel(uint32_t* status) { *status = 0u; }
+// precise scan of one block straight from global memory, out of line (the rare re-check of a block whose fast result
+// is too close to the threshold): its registers must not weigh on the caller's hot loop
+__device__ __noinline__ float scan_precise_from_global(const uint4* codes_tile, const uint4* scales_tile,
+                                                       const __nv_bfloat16* q_group, int G, int lane, int rows,
+                                                       float sm_scale) {
+    ScanQuery sq;
+    scan_setup(sq, q_group, G, lane, sm_scale);
+    ScanRegs sr;
+    scan_load(sr, codes_tile, scales_tile, lane);
+    float band;
+    float bm = scan_compute<true>(sr, sq, lane, rows, band);
+    if (bm != bm)   // (a scale too large for the fp16 operand)
+        bm = scan_block_wide(codes_tile, reinterpret_cast<const __half*>(scales_tile), q_group, G, lane, rows, sm_scale, nullptr, 0);
+    return bm;
+}
 
-// status word, work counters and class counts: the first 256 bytes of a workspace (64 threads), then the cookie
-__global__ void init_header_kernel(uint32_t* header) {
+// ---- the whole sparse step in one launch, for launches with little work -----------------------------------------
+// With fewer than two 32-block work items per SM the persistent kernel and its two companions (pseudo-max before,
+// combine after) are three dependent launches of a few microseconds each around almost no work.  This kernel does the
+// step in one: a CTA per (split of the sequence, KV head, sequence), the grid of the dense kernel.  Every CTA first
+// scans the unit's sink and local blocks itself (precise arithmetic, the blocks come from the L2 after the first CTA)
+// and so has m_tilde without waiting for anybody (Sec. 3.2, Alg. 1 "Pseudo-max estimation"); then its warps take the
+// blocks of its split one by one: scan, top-delta test (Eq. 1), exact attention over the kept ones through the same
+// staged pipeline as the dense kernel (Alg. 1 "Fine-grained refinement").  The CTA's partial goes to the workspace; the
+// CTA that finds itself the last of its unit to arrive (a counter in the workspace, left at zero again) merges the
+// unit's partials (log-sum-exp) and writes the output.  No CTA waits for another.
+__global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodeParams p, uint32_t* arrive) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const int split = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r = lane >> 2, j = lane & 3;
     pdl_launch_dependents();
     pdl_wait();
-    header[threadIdx.x] = threadIdx.x == kHeaderCookieWord ? kHeaderCookie : 0u;
+    const int n = clamped_seq_len(p, b);
+    const int nb = (n + kBlk - 1) / kBlk;
+    const int blk_begin = split * p.blocks_per_split;
+    const int blk_end = min(nb, blk_begin + p.blocks_per_split);
+
+    __shared__ int is_last;
+    __shared__ float sm_m[kWarps][kMaxG], sm_l[kWarps][kMaxG];
+    __shared__ float smax[kWarps][kMaxG];
+    const uint32_t kslot = smem_u32(smem) + warp * 2 * kSlotBytes;
+    const uint32_t vslot = kslot + kSlotBytes;
+    const uint32_t kbar = smem_u32(smem) + kWarps * 2 * kSlotBytes + warp * 16;
+    const uint32_t vbar = kbar + 8;
+    if (lane == 0) {
+        mbar_init(kbar, 32);
+        mbar_init(vbar, 32);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    const __nv_bfloat16* q_group = p.q + ((size_t)b * p.Hq + (size_t)g * p.G) * kD;
+    const size_t head0 = (size_t)b * p.Hq + (size_t)g * p.G;
+    AttendState st;
+    bool ok = true;
+    if (blk_begin >= nb) attend_reset(st);
+    if (blk_begin < nb) {   // (uniform over the CTA; a split past the sequence's end only reports an empty partial)
+        ScanQuery sq;
+        scan_setup(sq, q_group, p.G, lane, p.sm_scale);
+        // scan of one block, precise or fast; falls back to binary32 when the fp16 operand overflowed
+        auto judge = [&](bool precise, const ScanRegs& sr, size_t tile, int rows, float& band) {
+            float bm = precise ? scan_compute<true>(sr, sq, lane, rows, band) : scan_compute<false>(sr, sq, lane, rows, band);
+            if (bm != bm) {
+                bm = scan_block_wide(reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes), p.k_scales + tile * kD,
+                                     q_group, p.G, lane, rows, p.sm_scale, nullptr, 0);
+                band = 0.f;
+                if (!(fabsf(bm) < INFINITY) && j < p.G) { atomicOr(p.status, kDevRange); bm = INFINITY; }   // reported, kept
+            }
+            return bm;
+        };
+        {   // m_tilde over the sink and local blocks: warp w takes every kWarps-th of them, the next one's codes on their
+            // way into registers while the current one is scanned
+            const int ns = min(p.n_sink, nb);
+            const int local_begin = max(nb - p.n_local, ns);
+            const int count = ns + (nb - local_begin);
+            auto ref_of = [&](int s) {
+                BlockRef ref{-1, 0, 0};
+                if (s < count) {
+                    const int blk = s < ns ? s : local_begin + (s - ns);
+                    const int page = page_of(p, b, blk);
+                    if (page >= 0) { ref.blk = blk; ref.rows = min(kBlk, n - blk * kBlk); ref.tile = (size_t)page * p.Hkv + g; }
+                }
+                return ref;
+            };
+            float best = -INFINITY;
+            BlockRef cur = ref_of(warp);
+            ScanRegs cur_regs;
+            if (cur.blk >= 0)
+                scan_load(cur_regs, reinterpret_cast<const uint4*>(p.k_quant + cur.tile * kCodeBytes),
+                          reinterpret_cast<const uint4*>(p.k_scales + cur.tile * kD), lane);
+            for (int s = warp; s < count; s += kWarps) {
+                const BlockRef nxt = ref_of(s + kWarps);
+                ScanRegs nxt_regs;
+                if (nxt.blk >= 0)
+                    scan_load(nxt_regs, reinterpret_cast<const uint4*>(p.k_quant + nxt.tile * kCodeBytes),
+                              reinterpret_cast<const uint4*>(p.k_scales + nxt.tile * kD), lane);
+                float band;
+                if (cur.blk >= 0) best = fmaxf(best, judge(true, cur_regs, cur.tile, cur.rows, band));
+                cur = nxt;
+                cur_regs = nxt_regs;
+            }
+            if (lane < kMaxG) smax[warp][lane] = best;
+        }
+        __syncthreads();
+        float thr = INFINITY;   // of head lane % 4
+        if (j < p.G) {
+            float m = -INFINITY;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) m = fmaxf(m, smax[w][j]);
+            thr = m - p.delta;   // delta = +inf -> -inf: everything passes
+            if (split == 0 && warp == 0 && r == 0) p.mtilde[head0 + j] = m;
+        }
+        attend_reset(st);
+        attend_load_q(st.qa, q_group, p.G, lane);
+        const float logit_scale_log2 = p.sm_scale * kLog2e;
+        const uint4* kbase = reinterpret_cast<const uint4*>(p.k_cache);
+        const uint4* vbase = reinterpret_cast<const uint4*>(p.v_cache);
+        constexpr size_t kTileVec = kTileBytes / 16;
+        // next block of this split for this warp: blocks blk_begin + warp, + kWarps, ... (a fixed assignment, so that
+        // the order of the sums does not change from run to run), skipping blocks whose page index is bad
+        int my_next = blk_begin + warp;
+        auto fetch = [&]() {
+            BlockRef ref{-1, 0, 0};
+            for (;;) {
+                const int blk = my_next;
+                my_next += kWarps;
+                if (blk >= blk_end) return ref;
+                const int page = page_of(p, b, blk);
+                if (page < 0) continue;
+                ref.blk = blk;
+                ref.rows = min(kBlk, n - blk * kBlk);
+                ref.tile = (size_t)page * p.Hkv + g;
+                return ref;
+            }
+        };
+        auto load_codes = [&](ScanRegs& sr, const BlockRef& ref) {
+            scan_load(sr, reinterpret_cast<const uint4*>(p.k_quant + ref.tile * kCodeBytes),
+                      reinterpret_cast<const uint4*>(p.k_scales + ref.tile * kD), lane);
+        };
+        BlockRef cur = fetch();
+        ScanRegs cur_regs;
+        if (cur.blk >= 0) load_codes(cur_regs, cur);
+        BlockRef pending{-1, 0, 0};     // kept block whose K/V copies are in flight
+        unsigned pending_keep = 0;
+        uint32_t phase = 0;
+        while (cur.blk >= 0 && ok) {
+            // the next block's codes on their way into registers before this one is judged
+            const BlockRef nxt = fetch();
+            ScanRegs nxt_regs;
+            if (nxt.blk >= 0) load_codes(nxt_regs, nxt);
+            float band;
+            float bm = judge(false, cur_regs, cur.tile, cur.rows, band);
+            // too close to call with the fast accumulation: redo the block with the arithmetic m_tilde used
+            if (__any_sync(kFull, (j < p.G) && fabsf(bm - thr) <= band))
+                bm = scan_precise_from_global(reinterpret_cast<const uint4*>(p.k_quant + cur.tile * kCodeBytes),
+                                              reinterpret_cast<const uint4*>(p.k_scales + cur.tile * kD), q_group, p.G, lane,
+                                              cur.rows, p.sm_scale);
+            const bool keep = (j < p.G) && (bm >= thr);
+            const unsigned keep4 = __ballot_sync(kFull, keep) & 0xFu;
+            if (r == 0 && j < p.G) {
+                const size_t o = (head0 + j) * p.max_blocks + cur.blk;
+                if (p.kept_mask) p.kept_mask[o] = keep ? 1 : 0;
+                if (p.block_max) p.block_max[o] = bm;
+            }
+            if (keep4) {
+                const uint4* ksrc = kbase + cur.tile * kTileVec;
+                const uint4* vsrc = vbase + cur.tile * kTileVec;
+                if (pending.blk >= 0) {
+                    ok = attend_block(st, kslot, vslot, kbar, vbar, phase, ksrc, vsrc, lane, pending.rows, pending_keep,
+                                      logit_scale_log2);
+                } else {
+                    tile_copy_async(kslot, ksrc, lane, kbar);
+                    tile_copy_async(vslot, vsrc, lane, vbar);
+                }
+                pending = cur;
+                pending_keep = keep4;
+            }
+            cur = nxt;
+            cur_regs = nxt_regs;
+        }
+        if (ok && pending.blk >= 0)
+            ok = attend_block(st, kslot, vslot, kbar, vbar, phase, nullptr, nullptr, lane, pending.rows, pending_keep,
+                              logit_scale_log2);
+        cp_async_drain();
+        if (!ok && lane == 0) atomicOr(p.status, kDevTimeout);
+    } else {
+        __syncthreads();   // (the barrier the other branch passes)
+    }
+
+    // fold the warp's state: row sums over the 4 lanes of a row, bf16 remainder rows onto the main rows
+    float l = st.l;
+    l += __shfl_xor_sync(kFull, l, 1);
+    l += __shfl_xor_sync(kFull, l, 2);
+#pragma unroll
+    for (int nt = 0; nt < 16; ++nt) {
+        st.acc[nt][0] += __shfl_xor_sync(kFull, st.acc[nt][0], 16);
+        st.acc[nt][1] += __shfl_xor_sync(kFull, st.acc[nt][1], 16);
+    }
+    // the warp's own K slot is free now: it holds the warp's [4][128] accumulators for the merge
+    float* my_acc = reinterpret_cast<float*>(smem + (size_t)warp * 2 * kSlotBytes);
+    if (r < kMaxG) {
+        if (j == 0) { sm_m[warp][r] = st.m; sm_l[warp][r] = l; }
+#pragma unroll
+        for (int nt = 0; nt < 16; ++nt) {
+            my_acc[r * kD + attend_channel(nt, 2 * j)] = st.acc[nt][0];
+            my_acc[r * kD + attend_channel(nt, 2 * j + 1)] = st.acc[nt][1];
+        }
+    }
+    __syncthreads();
+    // merge the warps; each work item is one head and a pair of channels
+    for (int item = threadIdx.x; item < p.G * (kD / 2); item += kWarps * 32) {
+        const int h = item / (kD / 2), c = (item % (kD / 2)) * 2;
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) M = fmaxf(M, sm_m[w][h]);
+        float L = 0.f, a0 = 0.f, a1 = 0.f;
+        if (M != -INFINITY) {
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) {
+                const float f = exp2f(sm_m[w][h] - M);
+                const float* wacc = reinterpret_cast<const float*>(smem + (size_t)w * 2 * kSlotBytes) + h * kD + c;
+                L += f * sm_l[w][h];
+                a0 += f * wacc[0];
+                a1 += f * wacc[1];
+            }
+        }
+        const size_t slot = (head0 + h) * p.splits + split;
+        if (c == 0) { p.part_ml[2 * slot] = M; p.part_ml[2 * slot + 1] = L; }
+        *reinterpret_cast<float2*>(p.part_acc + slot * kD + c) = make_float2(a0, a1);
+    }
+    // the last CTA of the unit to get here merges the unit's splits
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        is_last = 0;
+        if (p.status[kHeaderCookieWord] != kHeaderCookie) {   // counters that were never zeroed decide nothing
+            atomicOr(p.status, kDevBadWorkspace);
+        } else {
+            const unsigned old = atomicAdd(&arrive[b * p.Hkv + g], 1u);
+            is_last = old + 1u == gridDim.x;
+            if (is_last) arrive[b * p.Hkv + g] = 0u;   // for the next call
+        }
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    for (int item = threadIdx.x; item < p.G * (kD / 2); item += kWarps * 32) {
+        const int h = item / (kD / 2), c = (item % (kD / 2)) * 2;
+        const size_t base = (head0 + h) * p.splits;
+        float M = -INFINITY;
+        for (int sp = 0; sp < (int)gridDim.x; ++sp) {
+            const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + 2 * (base + sp)));
+            if (ml.y > 0.f) M = fmaxf(M, ml.x);
+        }
+        float L = 0.f, a0 = 0.f, a1 = 0.f;
+        if (M != -INFINITY) {
+            for (int sp = 0; sp < (int)gridDim.x; ++sp) {
+                const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + 2 * (base + sp)));
+                if (!(ml.y > 0.f)) continue;
+                const float f = exp2f(ml.x - M);
+                const float2 a = __ldcg(reinterpret_cast<const float2*>(p.part_acc + (base + sp) * kD + c));
+                L += f * ml.y;
+                a0 += f * a.x;
+                a1 += f * a.y;
+            }
+        }
+        const float inv = L > 0.f ? 1.f / L : 0.f;
+        if (p.out_fp32) {
+            *reinterpret_cast<float2*>(static_cast<float*>(p.out) + (head0 + h) * kD + c) = make_float2(a0 * inv, a1 * inv);
+        } else {
+            *reinterpret_cast<__nv_bfloat162*>(static_cast<__nv_bfloat16*>(p.out) + (head0 + h) * kD + c) =
+                __floats2bfloat162_rn(a0 * inv, a1 * inv);
+        }
+        if (p.lse && c == 0) p.lse[head0 + h] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
+    }
+}
+
+__global__ void clear_status_kernel(uint32_t* status) { *status = 0u; }
+
+// status word, work counters and class counts (the first 256 bytes of a workspace, with the cookie) and the arrival
+// counters of the single-launch kernel that follow them: `words` 32-bit words in all
+__global__ void init_header_kernel(uint32_t* header, int words) {
+    pdl_launch_dependents();
+    pdl_wait();
+    for (int i = threadIdx.x; i < words; i += blockDim.x) header[i] = i == kHeaderCookieWord ? kHeaderCookie : 0u;
 }
 
 // ---- host side --------------------------------------------------------------------------------------------
@@ -725,9 +1002,16 @@ __global__ void init_header_kernel(uint32_t* header) {
 struct Plan {
     int blocks_per_split, splits;     // dense path
     int total_items;                  // fused path
-    size_t off_mtilde, off_lens, off_units, off_qrec, off_ml, off_acc, off_fml, off_facc, total;
+    bool small;                       // the geometry is served by the single-launch kernel
+    int small_bps, small_splits;      // ... with these splits: at most one CTA per SM, never more splits than the dense path
+    size_t off_arrive, off_mtilde, off_lens, off_units, off_qrec, off_ml, off_acc, off_fml, off_facc, total;
     size_t off_scores, total_residual;   // 2 + 8 bit key format: the score tiles follow everything else
 };
+
+constexpr size_t kHeaderBytes = 256;
+// ffd_workspace_init does not know the geometry: it zeroes the header and as many arrival counters as any geometry can
+// have (one per (sequence, KV head), fewer than 65536 of them)
+constexpr size_t kInitBytes = kHeaderBytes + 65536 * sizeof(uint32_t);
 
 // score tiles of the 2 + 8 bit format: one ring of (batch descriptors x blocks per item) tiles per CTA of the fused
 // kernel, which runs one CTA per SM; sized for GPUs of up to this many SMs
@@ -760,7 +1044,13 @@ static Plan make_plan(const ffd_config* cfg, int batch, int max_blocks, int sms)
     const size_t heads = (size_t)batch * cfg->num_q_heads;
     pl.total_items = item_geometry(units, max_blocks, sms).item_rows * batch * cfg->num_kv_heads;
     const size_t fslots = (size_t)pl.total_items * kNA * kMaxG;
-    pl.off_mtilde = 256;
+    // fewer than two full work items per SM: the single-launch kernel (a pure function of the geometry, like the rest)
+    pl.small = units * ((max_blocks + kItemBlocksMax - 1) / kItemBlocksMax) < 2 * sms;
+    pl.small_bps = bps;               // (every CTA repeats the scan of the sink and local blocks: few, long splits)
+    while (pl.small_bps < max_blocks && units * ((max_blocks + pl.small_bps - 1) / pl.small_bps) > sms) pl.small_bps *= 2;
+    pl.small_splits = (max_blocks + pl.small_bps - 1) / pl.small_bps;
+    pl.off_arrive = kHeaderBytes;     // one arrival counter per (sequence, KV head), zeroed with the header
+    pl.off_mtilde = align_up(pl.off_arrive + (size_t)units * sizeof(uint32_t), 256);
     pl.off_lens = align_up(pl.off_mtilde + heads * sizeof(float), 256);
     pl.off_units = align_up(pl.off_lens + (size_t)batch * sizeof(int32_t), 256);
     pl.off_qrec = align_up(pl.off_units + (size_t)batch * cfg->num_kv_heads * sizeof(int2), 256);
@@ -922,6 +1212,17 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
         if (k_res && sms > kResMaxCtas) return FFD_ERR_UNSUPPORTED;
         // the work counters and class counts at ws + 64 are zero here: ffd_workspace_init zeroes them and the
         // combine kernel of every call leaves them zeroed for the next one (the kernels check the header's cookie)
+        if (pl.small && !append && !k_res) {   // little work: the whole step in one launch
+            if (cudaFuncSetAttribute(small_sparse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem) != cudaSuccess)
+                return FFD_ERR_CUDA;
+            p.blocks_per_split = pl.small_bps;
+            p.splits = pl.small_splits;
+            if (prof) cudaEventRecord(g_prof_start, s);
+            launch_pdl(small_sparse_kernel, dim3(p.splits, p.Hkv, batch), dim3(kWarps * 32), kDecodeSmem, s, p,
+                       reinterpret_cast<uint32_t*>(ws + pl.off_arrive));
+            if (prof) cudaEventRecord(g_prof_stop, s);
+            return launch_status();
+        }
         if (append) {
             // the kernels after the first one read the lengths it leaves in the workspace
             int32_t* new_lens = reinterpret_cast<int32_t*>(ws + pl.off_lens);
@@ -1001,8 +1302,9 @@ ffd_status ffd_workspace_init(void* workspace, size_t workspace_bytes, void* str
     if (!workspace) return FFD_ERR_NULL;
     if (workspace_bytes < 256) return FFD_ERR_WORKSPACE;
     if (misaligned(workspace)) return FFD_ERR_ALIGN;
-    launch_pdl(init_header_kernel, dim3(1), dim3(64), 0, static_cast<cudaStream_t>(stream),
-               static_cast<uint32_t*>(workspace));
+    const size_t bytes = workspace_bytes < kInitBytes ? workspace_bytes : kInitBytes;
+    launch_pdl(init_header_kernel, dim3(1), dim3(1024), 0, static_cast<cudaStream_t>(stream),
+               static_cast<uint32_t*>(workspace), (int)(bytes / sizeof(uint32_t)));
     return launch_status();
 }
 
@@ -1242,7 +1544,9 @@ ffd_status ffd_decode_static(const ffd_config* cfg, const void* q, const void* k
     if (st) return st;
     // The array still holds whatever the previous call left there, and nobody else can initialise it: the whole
     // header (status word, work counters, cookie) is rewritten at the start of every call.
-    launch_pdl(init_header_kernel, dim3(1), dim3(64), 0, static_cast<cudaStream_t>(stream), static_cast<uint32_t*>(scratch));
+    const Plan spl = make_plan(cfg, batch, max_blocks_per_seq, device_sms());
+    launch_pdl(init_header_kernel, dim3(1), dim3(1024), 0, static_cast<cudaStream_t>(stream), static_cast<uint32_t*>(scratch),
+               (int)(spl.off_mtilde / sizeof(uint32_t)));
     if (cudaGetLastError() != cudaSuccess) return FFD_ERR_CUDA;
     return run_decode(true, cfg, q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, batch,
                       max_blocks_per_seq, num_pages, delta, out, lse, nullptr, nullptr, scratch,

@@ -353,8 +353,9 @@ __device__ __forceinline__ void sched_role(const DecodeParams& p, unsigned char*
     }
     sc.magic_heavy = fast_div_magic((unsigned)max(sc.n_heavy, 1));
     sc.magic_light = fast_div_magic((unsigned)max(sc.n_light, 1));
-    sc.pend_heavy = pend_heavy;
-    sc.pend_light = pend_light;
+    // (draws from counters that were never zeroed are not draws: a negative one would pass for "work left")
+    sc.pend_heavy = header_ok && pend_heavy >= 0 ? pend_heavy : 0x7fffffff;
+    sc.pend_light = header_ok && pend_light >= 0 ? pend_light : 0x7fffffff;
     sc.released = 0;
     sc.heavy_queued = 0;
     sc.heavy_hist = 0ull;
@@ -390,8 +391,8 @@ __device__ __forceinline__ void sched_role(const DecodeParams& p, unsigned char*
                         if (clock64() - t0 > kSpinCycles) { *abort_flag = 1; break; }
                     }
                 }
-                if (kind == 1) { cand = sc.pend_heavy; sc.pend_heavy = (int)atomicAdd(p.item_counter, 1u); }
-                if (kind == 0) { cand = sc.pend_light; sc.pend_light = (int)atomicAdd(p.light_counter, 1u); }
+                if (kind == 1) { cand = sc.pend_heavy; sc.pend_heavy = (int)min(atomicAdd(p.item_counter, 1u), 0x7fffffffu); }
+                if (kind == 0) { cand = sc.pend_light; sc.pend_light = (int)min(atomicAdd(p.light_counter, 1u), 0x7fffffffu); }
             }
             kind = __shfl_sync(kFull, kind, 0);
             cand = __shfl_sync(kFull, cand, 0);
