@@ -956,24 +956,40 @@ __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodePara
     __syncthreads();
     if (!is_last) return;
     __threadfence();
+    // The (m, l) pairs of all splits first, side by side, into shared memory (the K/V slots are free now); then every
+    // thread sums its pair of channels over the splits with several loads in flight.
+    float2* s_ml = reinterpret_cast<float2*>(smem);   // [G][splits]
+    const int nsp = (int)gridDim.x;
+    for (int x = threadIdx.x; x < p.G * nsp; x += kWarps * 32) {
+        const int h = x / nsp, sp = x % nsp;
+        const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + 2 * ((head0 + h) * p.splits + sp)));
+        s_ml[x] = ml.y > 0.f ? ml : make_float2(-INFINITY, 0.f);
+    }
+    __syncthreads();
     for (int item = threadIdx.x; item < p.G * (kD / 2); item += kWarps * 32) {
         const int h = item / (kD / 2), c = (item % (kD / 2)) * 2;
         const size_t base = (head0 + h) * p.splits;
+        const float2* ml = s_ml + h * nsp;
         float M = -INFINITY;
-        for (int sp = 0; sp < (int)gridDim.x; ++sp) {
-            const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + 2 * (base + sp)));
-            if (ml.y > 0.f) M = fmaxf(M, ml.x);
-        }
+        for (int sp = 0; sp < nsp; ++sp) M = fmaxf(M, ml[sp].x);
         float L = 0.f, a0 = 0.f, a1 = 0.f;
         if (M != -INFINITY) {
-            for (int sp = 0; sp < (int)gridDim.x; ++sp) {
-                const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + 2 * (base + sp)));
-                if (!(ml.y > 0.f)) continue;
-                const float f = exp2f(ml.x - M);
-                const float2 a = __ldcg(reinterpret_cast<const float2*>(p.part_acc + (base + sp) * kD + c));
-                L += f * ml.y;
-                a0 += f * a.x;
-                a1 += f * a.y;
+            for (int sp0 = 0; sp0 < nsp; sp0 += 8) {
+                float2 a[8];
+                float f[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int sp = sp0 + u;
+                    f[u] = sp < nsp ? exp2f(ml[sp].x - M) : 0.f;   // exp2(-inf) = 0 for empty splits
+                    a[u] = make_float2(0.f, 0.f);
+                    if (f[u] != 0.f) a[u] = __ldcg(reinterpret_cast<const float2*>(p.part_acc + (base + sp) * kD + c));
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    if (sp0 + u < nsp) L += f[u] * ml[sp0 + u].y;
+                    a0 += f[u] * a[u].x;
+                    a1 += f[u] * a[u].y;
+                }
             }
         }
         const float inv = L > 0.f ? 1.f / L : 0.f;
