@@ -16,6 +16,10 @@
  * Readings of the paper that this file fixes (each is a reading, not something the paper prints; the
  * ones marked "parity unpinned" have no independent pin):
  *   - bit width 2, codebook {-1.5,-0.5,+0.5,+1.5}, scale = absmax/1.5            (App. A.1, printed)
+ *   - the deeper thumbnails of App. "Bandwidth Proportionality of Quantization Depth" (4 and 8 bits): the paper
+ *     prints no formulas for them; reading: the same symmetric mid-rise construction with 2^b levels
+ *     +-(k + 1/2), k = 0 .. 2^(b-1) - 1, scale = absmax / (2^(b-1) - 1/2), nearest level with ties outward
+ *     (for b = 2 this is the printed codebook and scale)                        (parity unpinned: a reading)
  *   - one scale per (64-token block, KV head, channel), absmax over the block's valid rows;
  *     stored as fp16 = RNE(fp32(absmax)/1.5f), saturated at 65504             (parity unpinned)
  *   - nearest level written as comparisons: |x| >= s -> outer level, x = 0 -> +0.5; this equals the
@@ -127,16 +131,20 @@ static int valid_rows(int seq_len, int blk, int BLK) {
 
 /* ---- App. A.1: the quantizer ----------------------------------------------------------------- */
 
-/* One (page, KV head) tile.  For every channel c: a = max over valid rows of |K[r,c]|;
- * s = fp16(fp32(a)/1.5f) saturated at 65504; code by comparisons against s. */
-static void quantize_tile(const uint16_t* k_tile, int rows, int BLK, int D, uint8_t* codes, uint16_t* scales) {
+/* One (page, KV head) tile with b-bit thumbnails.  For every channel c: a = max over valid rows of |K[r,c]|;
+ * s = fp16(fp32(a) / (2^(b-1) - 1/2)) saturated at 65504; the code of x is the index (0 .. 2^b - 1) of the nearest of
+ * the 2^b levels +-(k + 1/2) * s, found by counting the cell boundaries k * s that |x| reaches (k * s is exact in
+ * double): ties go outward, +-0 takes +1/2.  b = 2 is App. A.1 as printed. */
+static void quantize_tile(const uint16_t* k_tile, int rows, int BLK, int D, int bits, uint8_t* codes, uint16_t* scales) {
+    const int half_levels = 1 << (bits - 1);                 /* levels on each side of zero */
+    const float top = (float)half_levels - 0.5f;             /* 1.5, 7.5, 127.5 */
     for (int c = 0; c < D; ++c) {
         float a = 0.0f;
         for (int r = 0; r < rows; ++r) {
             float x = (float)fabs(bf16_value(k_tile[(int64_t)r * D + c]));
             if (x > a) a = x;
         }
-        float s32 = a / 1.5f;                     /* IEEE binary32 division, round to nearest */
+        float s32 = a / top;                      /* IEEE binary32 division, round to nearest */
         if (s32 > 65504.0f) s32 = 65504.0f;
         uint16_t sbits = fp16_round_nonneg(s32);
         scales[c] = sbits;
@@ -146,17 +154,20 @@ static void quantize_tile(const uint16_t* k_tile, int rows, int BLK, int D, uint
             if (r < rows) {
                 double x = bf16_value(k_tile[(int64_t)r * D + c]);
                 int neg = x < 0.0;                /* -0.0 is not negative */
-                int big = fabs(x) >= s;
-                code = neg ? (big ? 0 : 1) : (big ? 3 : 2);
+                int m = 0;                        /* cell of |x|: [m s, (m + 1) s), the last one open-ended */
+                for (int k = 1; k < half_levels; ++k)
+                    if (fabs(x) >= (double)k * s) m = k;
+                code = (uint8_t)(neg ? half_levels - 1 - m : half_levels + m);
             }
             codes[(int64_t)r * D + c] = code;
         }
     }
 }
 
-/* Quantize every logical block of every sequence that holds at least one valid token. */
+/* Quantize every logical block of every sequence that holds at least one valid token (bits = 2, 4 or 8). */
 int ffd_oracle_quantize(const uint16_t* k_cache, uint8_t* codes, uint16_t* scales, const int32_t* block_table,
-                        const int32_t* seq_lens, int B, int Hkv, int D, int BLK, int max_blocks, int num_pages) {
+                        const int32_t* seq_lens, int B, int Hkv, int D, int BLK, int max_blocks, int num_pages, int bits) {
+    if (bits != 2 && bits != 4 && bits != 8) return 5;
     for (int b = 0; b < B; ++b) {
         int nb = (seq_lens[b] + BLK - 1) / BLK;
         if (seq_lens[b] < 0 || nb > max_blocks) return 2;
@@ -173,7 +184,7 @@ int ffd_oracle_quantize(const uint16_t* k_cache, uint8_t* codes, uint16_t* scale
             int rows = valid_rows(seq_lens[b], blk, BLK);
             for (int g = 0; g < Hkv; ++g) {
                 int64_t tile = page * Hkv + g;
-                quantize_tile(k_cache + tile * BLK * D, rows, BLK, D, codes + tile * BLK * D, scales + tile * D);
+                quantize_tile(k_cache + tile * BLK * D, rows, BLK, D, bits, codes + tile * BLK * D, scales + tile * D);
             }
         }
     }
@@ -242,6 +253,7 @@ typedef struct {
     const int32_t *block_table, *seq_lens;
     int B, Hq, Hkv, D, BLK, max_blocks, num_pages, n_sink, n_local;
     double sm_scale, delta;
+    double level_offset;        /* level of code c = c - level_offset: (2^b - 1) / 2 = 1.5, 7.5, 127.5 */
     const uint8_t* forced_mask; /* nullable [B,Hq,max_blocks]: use these decisions instead of top-delta */
     double *out, *lse, *block_max, *mtilde;
     uint8_t* kept;
@@ -310,7 +322,7 @@ static void decode_one(const decode_args* a, int b, int h) {
         for (int r = 0; r < rows; ++r) {
             double dot = 0.0;
             for (int c = 0; c < D; ++c) {
-                double khat = ((double)a->codes[(tile * BLK + r) * D + c] - 1.5) * fp16_value(a->scales[tile * D + c]);
+                double khat = ((double)a->codes[(tile * BLK + r) * D + c] - a->level_offset) * fp16_value(a->scales[tile * D + c]);
                 dot += bf16_value(qv[c]) * khat;
             }
             double s_approx = a->sm_scale * dot;
@@ -353,10 +365,13 @@ int ffd_oracle_decode(const uint16_t* q, const uint16_t* k_cache, const uint16_t
                       const uint16_t* scales, const int32_t* block_table, const int32_t* seq_lens, int B, int Hq,
                       int Hkv, int D, int BLK, int max_blocks, int num_pages, int n_sink, int n_local,
                       double sm_scale, double delta, const uint8_t* forced_mask, const int32_t* units, int n_units,
-                      double* out, double* lse, uint8_t* kept, double* block_max, double* mtilde, const int8_t* k_res) {
+                      double* out, double* lse, uint8_t* kept, double* block_max, double* mtilde, const int8_t* k_res,
+                      int bits) {
+    if (bits != 2 && bits != 4 && bits != 8) return 5;
+    if (k_res && bits != 2) return 5;             /* the residual format is defined on the 2-bit thumbnails */
     decode_args a = {q, k_cache, v_cache, scales, codes, block_table, seq_lens, B, Hq, Hkv, D, BLK, max_blocks,
-                     num_pages, n_sink, n_local, sm_scale, delta, forced_mask, out, lse, block_max, mtilde, kept,
-                     k_res};
+                     num_pages, n_sink, n_local, sm_scale, delta, (double)((1 << bits) - 1) / 2.0, forced_mask, out, lse,
+                     block_max, mtilde, kept, k_res};
     int rc = check_geometry(&a);
     if (rc) return rc;
     if (isnan(delta) || delta < 0.0) return 4;
@@ -375,7 +390,7 @@ int ffd_oracle_dense(const uint16_t* q, const uint16_t* k_cache, const uint16_t*
                      const int32_t* seq_lens, int B, int Hq, int Hkv, int D, int BLK, int max_blocks, int num_pages,
                      double sm_scale, const int32_t* units, int n_units, double* out, double* lse) {
     decode_args a = {q, k_cache, v_cache, NULL, NULL, block_table, seq_lens, B, Hq, Hkv, D, BLK, max_blocks,
-                     num_pages, 0, 0, sm_scale, INFINITY, NULL, out, lse, NULL, NULL, NULL, NULL};
+                     num_pages, 0, 0, sm_scale, INFINITY, 1.5, NULL, out, lse, NULL, NULL, NULL, NULL};
     int rc = check_geometry(&a);
     if (rc) return rc;
     int total = units ? n_units : B * Hq;

@@ -79,11 +79,12 @@ def _i32(a):
     return None if a is None else np.ascontiguousarray(a, dtype=np.int32)
 
 
-def quantize(k_cache, block_table, seq_lens, max_blocks):
+def quantize(k_cache, block_table, seq_lens, max_blocks, bits: int = 2):
     """App. A.1 quantizer over every logical block with a valid token.
 
-    k_cache: uint16 (bf16 bits) [num_pages, Hkv, BLK, D].  Returns (codes u8 [pages,Hkv,BLK,D] with values 0..3,
-    level = code - 1.5; scales uint16 fp16 bits [pages,Hkv,D]).  Tiles that no sequence maps stay zero.
+    k_cache: uint16 (bf16 bits) [num_pages, Hkv, BLK, D].  Returns (codes u8 [pages,Hkv,BLK,D] with values
+    0 .. 2^bits - 1, level = code - (2^bits - 1) / 2; scales uint16 fp16 bits [pages,Hkv,D]).  Tiles that no sequence
+    maps stay zero.  bits = 2 is the paper's thumbnail; 4 and 8 are the deeper ones of its quantization-depth appendix.
     """
     k_cache = _u16(k_cache)
     P, Hkv, BLK, D = k_cache.shape
@@ -93,7 +94,7 @@ def quantize(k_cache, block_table, seq_lens, max_blocks):
     scales = np.zeros((P, Hkv, D), dtype=np.uint16)
     rc = lib().ffd_oracle_quantize(_ptr(k_cache, ctypes.c_uint16), _ptr(codes, ctypes.c_uint8),
                                    _ptr(scales, ctypes.c_uint16), _ptr(block_table, ctypes.c_int32),
-                                   _ptr(seq_lens, ctypes.c_int32), len(seq_lens), Hkv, D, BLK, int(max_blocks), P)
+                                   _ptr(seq_lens, ctypes.c_int32), len(seq_lens), Hkv, D, BLK, int(max_blocks), P, int(bits))
     if rc:
         raise ValueError(f"ffd_oracle_quantize: geometry error {rc}")
     return codes, scales
@@ -137,7 +138,7 @@ def _units(units):
 
 
 def decode(q, k_cache, v_cache, codes, scales, block_table, seq_lens, max_blocks, delta, *, n_sink=1, n_local=16,
-           sm_scale=None, forced_mask=None, units=None, k_res=None) -> DecodeResult:
+           sm_scale=None, forced_mask=None, units=None, k_res=None, bits: int = 2) -> DecodeResult:
     """Alg. 1: approximate scores -> pseudo-max -> top-delta -> exact attention over kept blocks.
 
     ``k_res`` (int8, from ``quantize_residual``): refine from Dequant(codes, k_res) instead of the 16-bit K.
@@ -171,7 +172,7 @@ def decode(q, k_cache, v_cache, codes, scales, block_table, seq_lens, max_blocks
         _ptr(seq_lens, ctypes.c_int32), B, Hq, Hkv, D, BLK, int(max_blocks), P, int(n_sink), int(n_local),
         ctypes.c_double(sm_scale), ctypes.c_double(delta), _ptr(fm, ctypes.c_uint8), _ptr(u, ctypes.c_int32), nu,
         _ptr(out, ctypes.c_double), _ptr(lse, ctypes.c_double), _ptr(kept, ctypes.c_uint8),
-        _ptr(bm, ctypes.c_double), _ptr(mt, ctypes.c_double), _ptr(kr, ctypes.c_int8))
+        _ptr(bm, ctypes.c_double), _ptr(mt, ctypes.c_double), _ptr(kr, ctypes.c_int8), int(bits))
     if rc:
         raise ValueError(f"ffd_oracle_decode: error {rc}")
     return DecodeResult(out, lse, kept, bm, mt)

@@ -379,7 +379,8 @@ def test_dense_and_delta_inf_equal_library_softmax_attention(oracle, name, kw):
 # Alg. 1 re-derived by brute force on small inputs (numpy matrices, written from the algorithm box)
 # ---------------------------------------------------------------------------------------------------------
 
-def _brute_force(w, codes, scales, delta, n_sink, n_local):
+def _brute_force(w, codes, scales, delta, n_sink, n_local, bits=2):
+    levels = np.arange(1 << bits) - ((1 << bits) - 1) / 2.0       # {-1.5 .. 1.5}, {-7.5 .. 7.5}, {-127.5 .. 127.5}
     B, Hq, G = w.B, w.Hq, w.G
     out = np.zeros((B, Hq, 128))
     kept = np.zeros((B, Hq, w.max_blocks), dtype=np.uint8)
@@ -394,7 +395,7 @@ def _brute_force(w, codes, scales, delta, n_sink, n_local):
         pages = [w.page(b, i) for i in range(nb)]
         for h in range(Hq):
             g = h // G
-            Khat = np.concatenate([CODEBOOK[codes[p, g]] * S[p, g][None, :] for p in pages])[:N]
+            Khat = np.concatenate([levels[codes[p, g]] * S[p, g][None, :] for p in pages])[:N]
             approx = Khat @ Q[b, h] / math.sqrt(128)
             token_block = np.arange(N) // 64
             bm = np.array([approx[token_block == i].max() for i in range(nb)])
@@ -422,6 +423,109 @@ def test_decode_equals_brute_force_on_small_inputs(oracle, delta):
     assert np.abs(r.mtilde - mt).max() < 1e-11
     assert np.array_equal(r.kept, kept)
     assert np.abs(r.out - out).max() < 1e-11
+
+
+# ---------------------------------------------------------------------------------------------------------
+# the deeper thumbnails of the quantization-depth appendix (4 and 8 bits): same construction, 2^b levels
+# ---------------------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("bits", [4, 8])
+@pytest.mark.parametrize("absmax", [7.5, 2.71875, 1000.0, 3.0e-4])
+def test_deeper_codes_equal_argmin_over_all_bf16_values(oracle, bits, absmax):
+    """The mid-rise construction of App. A.1 with 2^b levels +-(k + 1/2) and s = max|x| / (2^(b-1) - 1/2): every bf16
+    value below the maximum takes the nearest level (arg-min, in exact rational arithmetic where double cannot tell),
+    ties go outward; the scale is the stated quotient in the stated precisions."""
+    absmax = float(bits_to_f64(bf16_bits([absmax]))[0])          # (the nearest bf16 value)
+    allbits = np.arange(65536, dtype=np.uint16)
+    vals = bits_to_f64(allbits)
+    keep = np.isfinite(vals) & (np.abs(vals) <= absmax)
+    column = np.concatenate([allbits[keep][::3], bf16_bits([absmax, -absmax, 0.0])])
+    k, seq = _one_column(column)
+    codes, scales = oracle.quantize(k, None, seq, 1, bits=bits)
+    top = (1 << (bits - 1)) - 0.5
+    want_scale = (np.float32(absmax) / np.float32(top)).astype(np.float16)
+    assert scales[0, 0, 0] == want_scale.view(np.uint16)
+    s = float(want_scale)
+    levels = np.arange(1 << bits) - ((1 << bits) - 1) / 2.0
+    x = bits_to_f64(column)
+    got = codes[0, 0, :, 0].astype(np.int64)
+    assert got.min() >= 0 and got.max() <= (1 << bits) - 1
+    dist = np.abs(x[:, None] / s - levels[None, :])
+    order = np.sort(dist, axis=1)
+    clear = (order[:, 1] - order[:, 0]) > 1e-9
+    assert np.array_equal(got[clear], np.argmin(dist, axis=1)[clear])
+    fs = Fraction(s)
+    flevels = [Fraction(int(2 * l), 2) for l in levels]
+    ties = 0
+    for i in np.where(~clear)[0]:
+        d = [abs(Fraction(float(x[i])) / fs - c) for c in flevels]
+        best = min(d)
+        winners = [j for j in range(len(flevels)) if d[j] == best]
+        if len(winners) > 1:      # an exact tie |x| = k s: outward (the level of larger magnitude); +-0: +1/2
+            ties += 1
+            want = max(winners, key=lambda j: (abs(flevels[j]), flevels[j]))
+            assert got[i] == want, (x[i], got[i], winners)
+            continue
+        assert got[i] == winners[0], (x[i], got[i], winners)
+    assert ties >= 2                                              # +0 and -0 at least
+    assert got[-3] == (1 << bits) - 1 and got[-2] == 0            # the absmax element takes the outermost level, either sign
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_deeper_roundtrip_bound_and_worked_column(oracle, bits):
+    """Half a step: |x - level * s| <= s/2 up to the fp16 rounding of s, on a workload; and a column worked by hand."""
+    w = make_workload("C1", N=1024, tail=13)
+    codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks, bits=bits)
+    K = bits_to_f64(w.bits("k_cache"))
+    S = scales.view(np.float16).astype(np.float64)[:, :, None, :]
+    off = ((1 << bits) - 1) / 2.0
+    top = (1 << (bits - 1)) - 0.5
+    for blk in range(w.num_blocks(0)):
+        rows = min(64, int(w.seq_lens[0]) - 64 * blk)
+        k, c, s = K[blk, :, :rows], codes[blk, :, :rows].astype(np.float64), S[blk]
+        assert np.all(np.abs(k - (c - off) * s) <= s * (0.5 + top * 2.0 ** -10))
+        a = np.abs(k).max(axis=1, keepdims=True)
+        assert np.array_equal(scales[blk].view(np.float16), (a[:, 0].astype(np.float32) / np.float32(top)).astype(np.float16))
+    # by hand, 4 bits: absmax 15 -> s = 2; cells [0,2) -> +0.5, [2,4) -> +1.5, ..., [14, inf) -> +7.5
+    col = bf16_bits([15.0, 0.0, 1.99, 2.0, -2.0, -1.0, 13.9, 14.0, -15.0, 7.0, -7.0])
+    k, seq = _one_column(col)
+    c4, s4 = oracle.quantize(k, None, seq, 1, bits=4)
+    assert s4.view(np.float16)[0, 0, 0] == np.float16(2.0)
+    assert c4[0, 0, :, 0].tolist() == [15, 8, 8, 9, 6, 7, 14, 15, 0, 11, 4]
+    # 8 bits: absmax 255 -> s = 2; x = 3 lies in [2, 4): level +1.5 = code 129
+    col = bf16_bits([255.0, 3.0, -3.0, 0.5, -255.0])
+    k, seq = _one_column(col)
+    c8, s8 = oracle.quantize(k, None, seq, 1, bits=8)
+    assert s8.view(np.float16)[0, 0, 0] == np.float16(2.0)
+    assert c8[0, 0, :, 0].tolist() == [255, 129, 126, 128, 0]
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_deeper_decode_equals_brute_force_and_tightens_the_scan(oracle, bits):
+    """Alg. 1 with deeper thumbnails against the numpy matrix form; and what the appendix's premise needs: more bits
+    bring the approximate block maxima closer to the exact ones."""
+    w = make_workload("C5", B=3, lens=(700, 2600), variant=2)
+    codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks, bits=bits)
+    r = oracle.decode(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), codes, scales, w.block_table, w.seq_lens,
+                      w.max_blocks, 6.0, n_sink=1, n_local=4, bits=bits)
+    out, kept, mt = _brute_force(w, codes, scales, 6.0, 1, 4, bits=bits)
+    assert np.abs(r.mtilde - mt).max() < 1e-10
+    assert np.array_equal(r.kept, kept)
+    assert np.abs(r.out - out).max() < 1e-10
+    # exact block maxima (16-bit keys) against the approximate ones of 2 bits and of `bits` bits
+    Kc, Q = bits_to_f64(w.bits("k_cache")), bits_to_f64(w.bits("q"))
+    c2, s2 = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
+    r2 = oracle.decode(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), c2, s2, w.block_table, w.seq_lens,
+                       w.max_blocks, 6.0, n_sink=1, n_local=4)
+    err2 = errb = 0.0
+    for b in range(w.B):
+        for blk in range(w.num_blocks(b)):
+            rows = min(64, int(w.seq_lens[b]) - 64 * blk)
+            for h in range(0, w.Hq, 5):
+                exact = (Kc[w.page(b, blk), h // w.G, :rows] @ Q[b, h]).max() / math.sqrt(128)
+                err2 += abs(r2.block_max[b, h, blk] - exact)
+                errb += abs(r.block_max[b, h, blk] - exact)
+    assert errb < err2 / 3
 
 
 # ---------------------------------------------------------------------------------------------------------
