@@ -19,7 +19,8 @@
  *   - Layouts (row-major, innermost last), D = head_dim = 128, BLK = block_tokens = 64:
  *       q        bf16  [batch, num_q_heads, D]
  *       k_cache  bf16  [num_pages, num_kv_heads, BLK, D]     (v_cache the same)
- *       k_quant  u8    [num_pages, num_kv_heads, 2048]       packed 2-bit codes, physical order below
+ *       k_quant  u8    [num_pages, num_kv_heads, 1024 * quant_bits]  packed codes (2048 bytes per tile for the
+ *                                                            2-bit thumbnails), physical order below
  *       k_scales fp16  [num_pages, num_kv_heads, D]          one scale per (page, KV head, channel)
  *       block_table int32 [batch, max_blocks_per_seq]        logical block -> physical page;
  *                                                            NULL = page b*max_blocks_per_seq + blk
@@ -31,6 +32,21 @@
  *     and r+8 (W1, W3) of the group.  Bits [2i+1:2i] of the low / high half of W0 (W1) hold the codes of
  *     channels 32j+4i and 32j+4i+1; those of W2 (W3) hold channels 32j+4i+2 and 32j+4i+3 (i = 0..7).
  *     A code c in 0..3 stands for level c - 1.5.  ffd_unpack_codes returns the canonical form.
+ *   - Deeper thumbnails, quant_bits = 4 or 8 (the quantization-depth study of the appendix "Bandwidth Proportionality
+ *     of Quantization Depth").  The paper states no quantizer for them; the library continues the 2-bit construction:
+ *     2^b levels +-(k + 1/2) * s, k = 0 .. 2^(b-1) - 1, s = fp16_rne(min(fp32(absmax) / (2^(b-1) - 1/2), 65504)) (the
+ *     outermost level at the channel's absolute maximum, as 1.5 s is for 2 bits), nearest level with ties outward, +-0
+ *     to +1/2, an all-zero channel coded with the outermost positive level; a code c in 0 .. 2^b - 1 stands for level
+ *     c - (2^b - 1) / 2.  Physical order of a (page, head) tile: 4 groups of 16 tokens; inside a group lane = 4*r + j
+ *     owns 2*b 32-bit words.  Word n of the lane is at byte offset ((((mt*V + n/4)*32 + lane)*4 + n%4)*4 of the tile
+ *     (mt = group, V = b/2).  4 bits: word i (i = 0..7) holds, in nibble x of its low / high half, the codes of token
+ *     16*mt + r + 8*(x&1), channels 32j + 4i + 2*(x>>1) and that channel + 1.  8 bits: words 2i and 2i+1; byte n of the
+ *     low / high half of word 2i + h holds token 16*mt + r + 8*n, channels 32j + 4i + 2h and + 1.  Supported by
+ *     ffd_quantize_keys, ffd_unpack_codes, ffd_workspace_bytes, ffd_workspace_init, ffd_decode, ffd_decode_dense and
+ *     ffd_read_device_status; the entry points of the 2 + 8 bit key format, of the device-side append and
+ *     ffd_decode_static return FFD_ERR_UNSUPPORTED for them.  The scan forms q * s in fp16 after scaling each head's
+ *     query to below 2 in magnitude: blocks whose scales exceed about 30000 overflow it, are kept and reported with
+ *     FFD_DEV_RANGE (the 2-bit scan falls back to binary32 there instead).
  */
 #ifndef FFD_H_
 #define FFD_H_
@@ -46,7 +62,8 @@ typedef enum {
     FFD_OK = 0,
     FFD_ERR_NULL = 1,          /* a required pointer is NULL */
     FFD_ERR_SHAPE = 2,         /* batch / heads / block counts out of range */
-    FFD_ERR_UNSUPPORTED = 3,   /* head_dim != 128, block_tokens != 64, quant_bits != 2, group size not 1..4 ... */
+    FFD_ERR_UNSUPPORTED = 3,   /* head_dim != 128, block_tokens != 64, quant_bits not 2, 4 or 8 (or not 2 where the entry
+                                  point needs the 2-bit thumbnails), group size not 1..4 ... */
     FFD_ERR_ALIGN = 4,         /* a device pointer is not 16-byte aligned */
     FFD_ERR_WORKSPACE = 5,     /* workspace smaller than ffd_workspace_bytes reports */
     FFD_ERR_DELTA = 6,         /* delta is NaN or negative */
@@ -68,7 +85,7 @@ typedef struct {
     int32_t num_kv_heads;
     int32_t head_dim;        /* 128 */
     int32_t block_tokens;    /* 64 */
-    int32_t quant_bits;      /* 2 */
+    int32_t quant_bits;      /* 2 (the paper's thumbnails), 4 or 8 (deeper thumbnails, see above) */
     int32_t n_sink_blocks;   /* size of the sink set S_global in blocks (>= 0) */
     int32_t n_local_blocks;  /* size of the local set S_local in blocks, counted from the last block (>= 0);
                                 n_sink_blocks + n_local_blocks must be >= 1 */

@@ -178,6 +178,101 @@ __device__ __forceinline__ void residual_rows(const __nv_bfloat16* sk, const flo
     }
 }
 
+// ---- deeper thumbnails: 4 and 8 bits (App. "Bandwidth Proportionality of Quantization Depth") ----------------
+// s = fp16(fp32(absmax) / (2^(b-1) - 1/2)); the cell of |x| is found by exact comparisons with k * s (exact in
+// binary32: at most 7 x 11 significant bits), ties outward, +-0 on the positive side; an all-zero channel (s = 0)
+// takes the outermost positive level like the 2-bit quantizer.  Packed order: see WideScan.
+template <int BITS>
+__device__ __forceinline__ uint32_t wide_code(float x, float s) {
+    constexpr int kHalf = 1 << (BITS - 1);
+    const float ax = fabsf(x);
+    int m = kHalf - 1;
+    if (s > 0.f) {
+        m = (int)fminf(__fdiv_rn(ax, s), (float)(kHalf - 1));   // within one of the cell; settled by the exact comparisons below
+        while (m + 1 <= kHalf - 1 && ax >= __fmul_rn((float)(m + 1), s)) ++m;
+        while (m > 0 && ax < __fmul_rn((float)m, s)) --m;
+    }
+    return x < 0.f ? (uint32_t)(kHalf - 1 - m) : (uint32_t)(kHalf + m);
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(128) quantize_wide_kernel(QuantParams p) {
+    const int g = blockIdx.y, b = blockIdx.z;
+    pdl_launch_dependents();
+    pdl_wait();
+    int n = p.seq_lens[b];
+    const int cap = p.max_blocks * kBlk;
+    n = n < 0 ? 0 : (n > cap ? cap : n);
+    const int nb = (n + kBlk - 1) / kBlk;
+    const int first = p.first_token ? max(p.first_token[b], 0) / kBlk : 0;
+    __shared__ __align__(16) __nv_bfloat16 sk[kBlk * kD];
+    __shared__ float ss[kD];
+    const int tid = threadIdx.x;
+    constexpr float kTop = (float)(1 << (BITS - 1)) - 0.5f;
+    for (int blk = first + blockIdx.x; blk < nb; blk += gridDim.x) {
+        const int page = p.block_table ? p.block_table[(size_t)b * p.max_blocks + blk] : b * p.max_blocks + blk;
+        if (page < 0 || page >= p.num_pages) continue;
+        const int rows = min(kBlk, n - blk * kBlk);
+        const size_t tile = (size_t)page * p.Hkv + g;
+        const uint4* src = reinterpret_cast<const uint4*>(p.k_cache + tile * kBlk * kD);
+        uint4* dst = reinterpret_cast<uint4*>(sk);
+        __syncthreads();   // the previous block's tile is no longer needed
+#pragma unroll
+        for (int x = 0; x < 8; ++x) dst[tid + 128 * x] = ldg_stream(src + tid + 128 * x);
+        __syncthreads();
+        {
+            float a = 0.f;
+            for (int r = 0; r < kBlk; ++r)
+                if (r < rows) a = fmaxf(a, fabsf(__bfloat162float(sk[r * kD + tid])));
+            const __half s = __float2half_rn(fminf(__fdiv_rn(a, kTop), 65504.f));
+            p.k_scales[tile * kD + tid] = s;
+            ss[tid] = __half2float(s);
+        }
+        __syncthreads();
+        const int mt = tid >> 5, lane = tid & 31, r = lane >> 2, j = lane & 3;
+        uint32_t* out = reinterpret_cast<uint32_t*>(p.k_quant + tile * WideScan<BITS>::kTileBytes);
+        for (int i = 0; i < 8; ++i) {
+            uint32_t c[4][2];   // A register x, low / high element
+#pragma unroll
+            for (int x = 0; x < 4; ++x)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int tok = 16 * mt + r + 8 * (x & 1), ch = 32 * j + 4 * i + 2 * (x >> 1) + e;
+                    c[x][e] = wide_code<BITS>(__bfloat162float(sk[tok * kD + ch]), ss[ch]);
+                }
+            if (BITS == 4) {
+                uint32_t w = 0;
+#pragma unroll
+                for (int x = 0; x < 4; ++x) w |= (c[x][0] << (4 * x)) | (c[x][1] << (16 + 4 * x));
+                out[WideScan<BITS>::word(mt, lane, i)] = w;
+            } else {
+                out[WideScan<BITS>::word(mt, lane, 2 * i)] = c[0][0] | (c[1][0] << 8) | (c[0][1] << 16) | (c[1][1] << 24);
+                out[WideScan<BITS>::word(mt, lane, 2 * i + 1)] = c[2][0] | (c[3][0] << 8) | (c[2][1] << 16) | (c[3][1] << 24);
+            }
+        }
+    }
+}
+
+// canonical codes [pages, Hkv, 64, 128] (0 .. 2^b - 1) from the packed layout of the deeper thumbnails
+template <int BITS>
+__global__ void __launch_bounds__(128) unpack_wide_kernel(const uint8_t* k_quant, uint8_t* codes, size_t tiles) {
+    const size_t tile = blockIdx.x;
+    if (tile >= tiles) return;
+    const int tid = threadIdx.x;
+    const int mt = tid >> 5, lane = tid & 31, r = lane >> 2, j = lane & 3;
+    const uint32_t* w = reinterpret_cast<const uint32_t*>(k_quant + tile * WideScan<BITS>::kTileBytes);
+    uint8_t* dst = codes + tile * kBlk * kD;
+    for (int i = 0; i < 8; ++i)
+        for (int x = 0; x < 4; ++x)
+            for (int e = 0; e < 2; ++e) {
+                const int tok = 16 * mt + r + 8 * (x & 1), ch = 32 * j + 4 * i + 2 * (x >> 1) + e;
+                uint32_t c;
+                if (BITS == 4) c = (w[WideScan<BITS>::word(mt, lane, i)] >> (4 * x + 16 * e)) & 0xFu;
+                else c = (w[WideScan<BITS>::word(mt, lane, 2 * i + (x >> 1))] >> (8 * (x & 1) + 16 * e)) & 0xFFu;
+                dst[tok * kD + ch] = (uint8_t)c;
+            }
+}
+
 // ---- whole-cache quantizer ---------------------------------------------------------------------------------
 // The same arithmetic as quantize_tile, organised for bandwidth: per element the plain routine spends ~9
 // instructions (16-bit shared-memory reads, conversions, two compares, selects, shifts) and is instruction-bound at
@@ -727,6 +822,74 @@ __device__ __noinline__ float scan_precise_from_global(const uint4* codes_tile, 
     return bm;
 }
 
+// ---- the scan on its own: 4- and 8-bit thumbnails on large geometries -------------------------------------------
+// One warp per block, many warps per SM: the thumbnails of a long cache stream through at memory speed, which the decode
+// kernel's seven fat warps per SM cannot do for codes this wide.  Writes the block maxima of the approximate logits
+// (precise accumulation, the arithmetic of m_tilde) for the decode kernel that follows: p.bmax[b][head][block]; NaN for a
+// block whose page index is bad (never kept, ignored by every maximum).
+constexpr int kScanCtaBlocks = 64;   // blocks of one (sequence, KV head) per CTA: 8 per warp
+template <int BITS>
+__global__ void __launch_bounds__(256, 2) scan_blocks_kernel(DecodeParams p) {
+    const int g = blockIdx.y, b = blockIdx.z;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r = lane >> 2, j = lane & 3;
+    pdl_launch_dependents();
+    pdl_wait();
+    const int n = clamped_seq_len(p, b);
+    const int nb = (n + kBlk - 1) / kBlk;
+    const int first = blockIdx.x * kScanCtaBlocks;
+    if (first >= nb) return;
+    const int last = min(nb, first + kScanCtaBlocks);
+    const __nv_bfloat16* q_group = p.q + ((size_t)b * p.Hq + (size_t)g * p.G) * kD;
+    float* out = p.bmax + ((size_t)b * p.Hq + (size_t)g * p.G) * p.max_blocks;
+    auto raw_page = [&](int blk) {
+        return p.block_table ? p.block_table[(size_t)b * p.max_blocks + blk] : b * p.max_blocks + blk;
+    };
+    auto prefetch = [&](int page) {
+        if (page >= 0 && page < p.num_pages) {
+            const size_t tile = (size_t)page * p.Hkv + g;
+            wide_prefetch_l2<BITS>(p.k_quant + tile * WideScan<BITS>::kTileBytes, p.k_scales + tile * kD, lane);
+        }
+    };
+    // the warp's first two tiles are on their way while it prepares its query fragments
+    int blk = first + warp;
+    int page = blk < last ? raw_page(blk) : -1;
+    int next_page = blk + 8 < last ? raw_page(blk + 8) : -1;
+    prefetch(page);
+    prefetch(next_page);
+    ScanQuery sq;
+    scan_setup_wide(sq, q_group, p.G, lane, p.sm_scale);
+    for (; blk < last; blk += 8) {
+        const int after = blk + 16 < last ? raw_page(blk + 16) : -1;   // (read now, used for the hint one turn later)
+        float bm = __int_as_float(0x7fc00000);
+        if (page >= 0 && page < p.num_pages) {
+            const size_t tile = (size_t)page * p.Hkv + g;
+            float band;
+            bm = scan_wide<BITS, true>(p.k_quant + tile * WideScan<BITS>::kTileBytes, p.k_scales + tile * kD, sq, lane,
+                                       min(kBlk, n - blk * kBlk), band);
+            if (bm != bm) {   // scales beyond the fp16 operand's range: reported, the block kept
+                if (j < p.G) atomicOr(p.status, kDevRange);
+                bm = INFINITY;
+            }
+        } else if (lane == 0) {
+            atomicOr(p.status, kDevBadPage);
+        }
+        if (r == 0 && j < p.G) out[(size_t)j * p.max_blocks + blk] = bm;
+        page = next_page;
+        next_page = after;
+        prefetch(after);
+    }
+}
+
+// the deeper scans' precise pass, out of line: it runs for the sink and local blocks and for the rare block within
+// the fast pass's error band of the threshold, and inlining it twice costs the decode loop its registers
+template <int BITS>
+__device__ __noinline__ float scan_wide_precise(const unsigned char* codes_tile, const __half* scales_tile, const ScanQuery& sq,
+                                                int lane, int rows) {
+    float band;
+    return scan_wide<BITS, true>(codes_tile, scales_tile, sq, lane, rows, band);
+}
+
 // ---- the whole sparse step in one launch, for launches with little work -----------------------------------------
 // With fewer than two 32-block work items per SM the persistent kernel and its two companions (pseudo-max before,
 // combine after) are three dependent launches of a few microseconds each around almost no work.  This kernel does the
@@ -737,6 +900,7 @@ __device__ __noinline__ float scan_precise_from_global(const uint4* codes_tile, 
 // staged pipeline as the dense kernel (Alg. 1 "Fine-grained refinement").  The CTA's partial goes to the workspace; the
 // CTA that finds itself the last of its unit to arrive (a counter in the workspace, left at zero again) merges the
 // unit's partials (log-sum-exp) and writes the output.  No CTA waits for another.
+template <int BITS>
 __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodeParams p, uint32_t* arrive) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const int split = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
@@ -768,10 +932,32 @@ __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodePara
     if (blk_begin >= nb) attend_reset(st);
     if (blk_begin < nb) {   // (uniform over the CTA; a split past the sequence's end only reports an empty partial)
         ScanQuery sq;
-        scan_setup(sq, q_group, p.G, lane, p.sm_scale);
-        // scan of one block, precise or fast; falls back to binary32 when the fp16 operand overflowed
+        if constexpr (BITS == 2) scan_setup(sq, q_group, p.G, lane, p.sm_scale);
+        else if constexpr (BITS != 0) scan_setup_wide(sq, q_group, p.G, lane, p.sm_scale);
+        constexpr size_t kCodeTile = BITS == 2 ? (size_t)kCodeBytes : (size_t)WideScan<BITS>::kTileBytes;
+        // BITS == 0: the block maxima come from the scan kernel that ran before this one (p.bmax)
+        const float* bmx = p.bmax + head0 * p.max_blocks;
+        // scan of one block, precise or fast.  2 bits: from the codes in registers, with the binary32 fallback when the
+        // fp16 operand overflowed; deeper thumbnails: straight from global memory (an overflow there -- scales beyond
+        // 30000 -- is reported and the block kept)
         auto judge = [&](bool precise, const ScanRegs& sr, size_t tile, int rows, float& band) {
-            float bm = precise ? scan_compute<true>(sr, sq, lane, rows, band) : scan_compute<false>(sr, sq, lane, rows, band);
+            float bm;
+            if constexpr (BITS == 0) {
+                band = 0.f;
+                return 0.f;
+            } else if constexpr (BITS == 2) {
+                bm = precise ? scan_compute<true>(sr, sq, lane, rows, band) : scan_compute<false>(sr, sq, lane, rows, band);
+            } else {
+                band = 0.f;
+                bm = precise ? scan_wide_precise<BITS>(p.k_quant + tile * kCodeTile, p.k_scales + tile * kD, sq, lane, rows)
+                             : scan_wide<BITS, false>(p.k_quant + tile * kCodeTile, p.k_scales + tile * kD, sq, lane, rows, band);
+                if (bm != bm) {
+                    band = 0.f;
+                    if (j < p.G) atomicOr(p.status, kDevRange);
+                    bm = INFINITY;
+                }
+                return bm;
+            }
             if (bm != bm) {
                 bm = scan_block_wide(reinterpret_cast<const uint4*>(p.k_quant + tile * kCodeBytes), p.k_scales + tile * kD,
                                      q_group, p.G, lane, rows, p.sm_scale, nullptr, 0);
@@ -779,6 +965,20 @@ __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodePara
                 if (!(fabsf(bm) < INFINITY) && j < p.G) { atomicOr(p.status, kDevRange); bm = INFINITY; }   // reported, kept
             }
             return bm;
+        };
+        // deeper thumbnails: no codes wait in registers; instead every warp asks L2 for the tiles of its blocks two
+        // turns ahead (a hint: a bad page index is simply not prefetched; the scan itself reports it)
+        auto raw_page = [&](int blk) {
+            return p.block_table ? p.block_table[(size_t)b * p.max_blocks + blk] : b * p.max_blocks + blk;
+        };
+        auto prefetch_page = [&](int page) {
+            if (page >= 0 && page < p.num_pages) {
+                const size_t tile = (size_t)page * p.Hkv + g;
+                wide_prefetch_l2<BITS>(p.k_quant + tile * kCodeTile, p.k_scales + tile * kD, lane);
+            }
+        };
+        auto prefetch_block = [&](int blk) {
+            if (blk < blk_end) prefetch_page(raw_page(blk));
         };
         {   // m_tilde over the sink and local blocks: warp w takes every kWarps-th of them, the next one's codes on their
             // way into registers while the current one is scanned
@@ -795,15 +995,31 @@ __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodePara
                 return ref;
             };
             float best = -INFINITY;
-            BlockRef cur = ref_of(warp);
+            if constexpr (BITS == 0) {   // every warp for itself: lane 4 r + j takes every eighth of the blocks for head j
+                if (j < p.G)
+                    for (int s = r; s < count; s += 8)
+                        best = fmaxf(best, bmx[(size_t)j * p.max_blocks + (s < ns ? s : local_begin + (s - ns))]);
+                best = fmaxf(best, __shfl_xor_sync(kFull, best, 4));
+                best = fmaxf(best, __shfl_xor_sync(kFull, best, 8));
+                best = fmaxf(best, __shfl_xor_sync(kFull, best, 16));
+            }
+            BlockRef cur = ref_of(BITS == 0 ? count : warp);
+            if constexpr (BITS != 2 && BITS != 0) {   // this warp's sink / local blocks on their way into L2 before the first is scanned
+                for (int s = warp; s < count; s += kWarps) {
+                    const BlockRef ref = ref_of(s);
+                    if (ref.blk >= 0) wide_prefetch_l2<BITS>(p.k_quant + ref.tile * kCodeTile, p.k_scales + ref.tile * kD, lane);
+                }
+                prefetch_block(blk_begin + warp);
+                prefetch_block(blk_begin + warp + kWarps);
+            }
             ScanRegs cur_regs;
-            if (cur.blk >= 0)
+            if (BITS == 2 && cur.blk >= 0)
                 scan_load(cur_regs, reinterpret_cast<const uint4*>(p.k_quant + cur.tile * kCodeBytes),
                           reinterpret_cast<const uint4*>(p.k_scales + cur.tile * kD), lane);
-            for (int s = warp; s < count; s += kWarps) {
+            for (int s = BITS == 0 ? count : warp; s < count; s += kWarps) {
                 const BlockRef nxt = ref_of(s + kWarps);
                 ScanRegs nxt_regs;
-                if (nxt.blk >= 0)
+                if (BITS == 2 && nxt.blk >= 0)
                     scan_load(nxt_regs, reinterpret_cast<const uint4*>(p.k_quant + nxt.tile * kCodeBytes),
                               reinterpret_cast<const uint4*>(p.k_scales + nxt.tile * kD), lane);
                 float band;
@@ -846,16 +1062,72 @@ __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodePara
             }
         };
         auto load_codes = [&](ScanRegs& sr, const BlockRef& ref) {
-            scan_load(sr, reinterpret_cast<const uint4*>(p.k_quant + ref.tile * kCodeBytes),
-                      reinterpret_cast<const uint4*>(p.k_scales + ref.tile * kD), lane);
+            if constexpr (BITS == 2)
+                scan_load(sr, reinterpret_cast<const uint4*>(p.k_quant + ref.tile * kCodeBytes),
+                          reinterpret_cast<const uint4*>(p.k_scales + ref.tile * kD), lane);
         };
-        BlockRef cur = fetch();
-        ScanRegs cur_regs;
-        if (cur.blk >= 0) load_codes(cur_regs, cur);
         BlockRef pending{-1, 0, 0};     // kept block whose K/V copies are in flight
         unsigned pending_keep = 0;
         uint32_t phase = 0;
+        // a kept block: its K/V copies start now; the block kept before it is attended while they fly
+        auto consume = [&](const BlockRef& blk_ref, unsigned keep4) {
+            const uint4* ksrc = kbase + blk_ref.tile * kTileVec;
+            const uint4* vsrc = vbase + blk_ref.tile * kTileVec;
+            if (pending.blk >= 0) {
+                ok = attend_block(st, kslot, vslot, kbar, vbar, phase, ksrc, vsrc, lane, pending.rows, pending_keep,
+                                  logit_scale_log2);
+            } else {
+                tile_copy_async(kslot, ksrc, lane, kbar);
+                tile_copy_async(vslot, vsrc, lane, vbar);
+            }
+            pending = blk_ref;
+            pending_keep = keep4;
+        };
+        if constexpr (BITS == 0) {
+            // Decisions from the stored maxima, 32 of the warp's blocks at a time (lane L looks at the L-th of them); only
+            // the kept ones cost a page lookup and a turn of the pipeline.
+            float thr_h[kMaxG];
+#pragma unroll
+            for (int h = 0; h < kMaxG; ++h) thr_h[h] = __shfl_sync(kFull, thr, h);
+            for (int base = blk_begin + warp; base < blk_end && ok; base += 32 * kWarps) {
+                const int mine = base + lane * kWarps;
+                unsigned k4 = 0;
+                if (mine < blk_end) {
+#pragma unroll
+                    for (int h = 0; h < kMaxG; ++h)
+                        if (h < p.G) {
+                            const float bm = bmx[(size_t)h * p.max_blocks + mine];
+                            const bool keep = bm >= thr_h[h];
+                            k4 |= (keep ? 1u : 0u) << h;
+                            const size_t o = (head0 + h) * p.max_blocks + mine;
+                            if (p.kept_mask) p.kept_mask[o] = keep ? 1 : 0;
+                            if (p.block_max) p.block_max[o] = bm;
+                        }
+                }
+                unsigned any = __ballot_sync(kFull, k4 != 0);
+                while (any && ok) {
+                    const int src = __ffs(any) - 1;
+                    any &= any - 1;
+                    const unsigned keep4 = __shfl_sync(kFull, k4, src);
+                    const int blk = base + src * kWarps;
+                    const int page = page_of(p, b, blk);
+                    if (page < 0) continue;
+                    consume(BlockRef{blk, min(kBlk, n - blk * kBlk), (size_t)page * p.Hkv + g}, keep4);
+                }
+            }
+        }
+        BlockRef cur = fetch();
+        if (BITS == 0) cur.blk = -1;
+        ScanRegs cur_regs;
+        if (cur.blk >= 0) load_codes(cur_regs, cur);
+        int pf_blk = blk_begin + warp + 2 * kWarps, pf_page = -1;   // (the page index is read one turn before its use)
+        if (BITS != 2 && BITS != 0 && pf_blk < blk_end) pf_page = raw_page(pf_blk);
         while (cur.blk >= 0 && ok) {
+            if constexpr (BITS != 2) {
+                prefetch_page(pf_page);
+                pf_blk += kWarps;
+                pf_page = pf_blk < blk_end ? raw_page(pf_blk) : -1;
+            }
             // the next block's codes on their way into registers before this one is judged
             const BlockRef nxt = fetch();
             ScanRegs nxt_regs;
@@ -863,10 +1135,14 @@ __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodePara
             float band;
             float bm = judge(false, cur_regs, cur.tile, cur.rows, band);
             // too close to call with the fast accumulation: redo the block with the arithmetic m_tilde used
-            if (__any_sync(kFull, (j < p.G) && fabsf(bm - thr) <= band))
-                bm = scan_precise_from_global(reinterpret_cast<const uint4*>(p.k_quant + cur.tile * kCodeBytes),
-                                              reinterpret_cast<const uint4*>(p.k_scales + cur.tile * kD), q_group, p.G, lane,
-                                              cur.rows, p.sm_scale);
+            if (__any_sync(kFull, (j < p.G) && fabsf(bm - thr) <= band)) {
+                if constexpr (BITS == 2)
+                    bm = scan_precise_from_global(reinterpret_cast<const uint4*>(p.k_quant + cur.tile * kCodeBytes),
+                                                  reinterpret_cast<const uint4*>(p.k_scales + cur.tile * kD), q_group, p.G, lane,
+                                                  cur.rows, p.sm_scale);
+                else
+                    bm = judge(true, cur_regs, cur.tile, cur.rows, band);
+            }
             const bool keep = (j < p.G) && (bm >= thr);
             const unsigned keep4 = __ballot_sync(kFull, keep) & 0xFu;
             if (r == 0 && j < p.G) {
@@ -874,19 +1150,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodePara
                 if (p.kept_mask) p.kept_mask[o] = keep ? 1 : 0;
                 if (p.block_max) p.block_max[o] = bm;
             }
-            if (keep4) {
-                const uint4* ksrc = kbase + cur.tile * kTileVec;
-                const uint4* vsrc = vbase + cur.tile * kTileVec;
-                if (pending.blk >= 0) {
-                    ok = attend_block(st, kslot, vslot, kbar, vbar, phase, ksrc, vsrc, lane, pending.rows, pending_keep,
-                                      logit_scale_log2);
-                } else {
-                    tile_copy_async(kslot, ksrc, lane, kbar);
-                    tile_copy_async(vslot, vsrc, lane, vbar);
-                }
-                pending = cur;
-                pending_keep = keep4;
-            }
+            if (keep4) consume(cur, keep4);
             cur = nxt;
             cur_regs = nxt_regs;
         }
@@ -1020,7 +1284,9 @@ struct Plan {
     int total_items;                  // fused path
     bool small;                       // the geometry is served by the single-launch kernel
     int small_bps, small_splits;      // ... with these splits: at most one CTA per SM, never more splits than the dense path
+    int wide_bps, wide_splits;        // the single-launch kernel on large geometries (deeper thumbnails): a few waves
     size_t off_arrive, off_mtilde, off_lens, off_units, off_qrec, off_ml, off_acc, off_fml, off_facc, total;
+    size_t off_bmax;
     size_t off_scores, total_residual;   // 2 + 8 bit key format: the score tiles follow everything else
 };
 
@@ -1065,6 +1331,16 @@ static Plan make_plan(const ffd_config* cfg, int batch, int max_blocks, int sms)
     pl.small_bps = bps;               // (every CTA repeats the scan of the sink and local blocks: few, long splits)
     while (pl.small_bps < max_blocks && units * ((max_blocks + pl.small_bps - 1) / pl.small_bps) > sms) pl.small_bps *= 2;
     pl.small_splits = (max_blocks + pl.small_bps - 1) / pl.small_bps;
+    // The same kernel on large geometries (4- and 8-bit thumbnails; decisions from stored block maxima): a CTA's cost is
+    // its kept blocks, which no geometry can know, so about four CTAs per SM let the hardware even them out; never
+    // shorter splits than the dense path's
+    {
+        long per_unit = 4L * sms / units;
+        if (per_unit < 1) per_unit = 1;
+        pl.wide_bps = (int)((max_blocks + per_unit - 1) / per_unit);
+        if (pl.wide_bps < bps) pl.wide_bps = bps;
+        pl.wide_splits = max_blocks > 0 ? (max_blocks + pl.wide_bps - 1) / pl.wide_bps : 1;
+    }
     pl.off_arrive = kHeaderBytes;     // one arrival counter per (sequence, KV head), zeroed with the header
     pl.off_mtilde = align_up(pl.off_arrive + (size_t)units * sizeof(uint32_t), 256);
     pl.off_lens = align_up(pl.off_mtilde + heads * sizeof(float), 256);
@@ -1075,14 +1351,18 @@ static Plan make_plan(const ffd_config* cfg, int batch, int max_blocks, int sms)
     pl.off_fml = align_up(pl.off_acc + heads * pl.splits * kD * sizeof(float), 256);
     pl.off_facc = align_up(pl.off_fml + fslots * 2 * sizeof(float), 256);
     pl.total = align_up(pl.off_facc + fslots * kD * sizeof(float), 256);
+    pl.off_bmax = pl.total;   // deeper thumbnails only: the block maxima between the scan kernel and the decode kernel
+    if (cfg->quant_bits != 2) pl.total = align_up(pl.off_bmax + heads * (size_t)max_blocks * sizeof(float), 256);
     pl.off_scores = pl.total;
     pl.total_residual = pl.off_scores + (size_t)kResMaxCtas * kNB * kItemBlocksMax * kScoreTileFloats * sizeof(float);
     return pl;
 }
 
-static ffd_status check_config(const ffd_config* cfg) {
+// two_bit_only: the entry point exists for the 2-bit thumbnails only (the 2 + 8 bit format, the device-side append)
+static ffd_status check_config(const ffd_config* cfg, bool two_bit_only = false) {
     if (!cfg) return FFD_ERR_NULL;
-    if (cfg->head_dim != kD || cfg->block_tokens != kBlk || cfg->quant_bits != 2) return FFD_ERR_UNSUPPORTED;
+    if (cfg->head_dim != kD || cfg->block_tokens != kBlk) return FFD_ERR_UNSUPPORTED;
+    if (cfg->quant_bits != 2 && (two_bit_only || (cfg->quant_bits != 4 && cfg->quant_bits != 8))) return FFD_ERR_UNSUPPORTED;
     if (cfg->num_q_heads <= 0 || cfg->num_kv_heads <= 0 || cfg->num_q_heads % cfg->num_kv_heads) return FFD_ERR_SHAPE;
     if (cfg->num_q_heads / cfg->num_kv_heads > kMaxG) return FFD_ERR_UNSUPPORTED;
     if (cfg->n_sink_blocks < 0 || cfg->n_local_blocks < 0 || cfg->n_sink_blocks + cfg->n_local_blocks < 1)
@@ -1205,6 +1485,7 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
     p.len_stats = reinterpret_cast<uint32_t*>(ws + 80);
     p.unit_list = reinterpret_cast<int2*>(ws + pl.off_units);
     p.res_scores = reinterpret_cast<float*>(ws + pl.off_scores);
+    p.bmax = reinterpret_cast<float*>(ws + pl.off_bmax);
     p.units = batch * cfg->num_kv_heads;
     const ItemGeom geom = item_geometry(p.units, max_blocks, sms);
     p.item_rows = geom.item_rows;
@@ -1228,13 +1509,30 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
         if (k_res && sms > kResMaxCtas) return FFD_ERR_UNSUPPORTED;
         // the work counters and class counts at ws + 64 are zero here: ffd_workspace_init zeroes them and the
         // combine kernel of every call leaves them zeroed for the next one (the kernels check the header's cookie)
-        if (pl.small && !append && !k_res) {   // little work: the whole step in one launch
-            if (cudaFuncSetAttribute(small_sparse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem) != cudaSuccess)
+        // 4- / 8-bit thumbnails: the single-launch kernel on small geometries, a scan kernel followed by the same decode
+        // kernel on large ones
+        const bool deeper = cfg->quant_bits != 2;
+        if (deeper && (append || k_res)) return FFD_ERR_UNSUPPORTED;
+        if ((pl.small || deeper) && !append && !k_res) {   // little work: the whole step in one launch
+            // deeper thumbnails on a large geometry: the scan as a kernel of its own, then the same decode kernel taking
+            // its decisions from the stored block maxima
+            void (*kernel)(DecodeParams, uint32_t*) = !pl.small ? small_sparse_kernel<0>
+                                                      : cfg->quant_bits == 2 ? small_sparse_kernel<2>
+                                                      : cfg->quant_bits == 4 ? small_sparse_kernel<4> : small_sparse_kernel<8>;
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem) != cudaSuccess)
                 return FFD_ERR_CUDA;
-            p.blocks_per_split = pl.small_bps;
-            p.splits = pl.small_splits;
+            if (pl.small) {
+                p.blocks_per_split = pl.small_bps;
+                p.splits = pl.small_splits;
+            } else {
+                p.blocks_per_split = pl.wide_bps;
+                p.splits = pl.wide_splits;
+            }
             if (prof) cudaEventRecord(g_prof_start, s);
-            launch_pdl(small_sparse_kernel, dim3(p.splits, p.Hkv, batch), dim3(kWarps * 32), kDecodeSmem, s, p,
+            if (!pl.small)
+                launch_pdl(cfg->quant_bits == 4 ? scan_blocks_kernel<4> : scan_blocks_kernel<8>,
+                           dim3((p.max_blocks + kScanCtaBlocks - 1) / kScanCtaBlocks, p.Hkv, batch), dim3(256), 0, s, p);
+            launch_pdl(kernel, dim3(p.splits, p.Hkv, batch), dim3(kWarps * 32), kDecodeSmem, s, p,
                        reinterpret_cast<uint32_t*>(ws + pl.off_arrive));
             if (prof) cudaEventRecord(g_prof_stop, s);
             return launch_status();
@@ -1305,7 +1603,7 @@ ffd_status ffd_workspace_bytes(const ffd_config* cfg, int32_t batch, int32_t max
 }
 
 ffd_status ffd_workspace_bytes_residual(const ffd_config* cfg, int32_t batch, int32_t max_blocks_per_seq, size_t* bytes) {
-    ffd_status st = check_config(cfg);
+    ffd_status st = check_config(cfg, true);
     if (st) return st;
     if (!bytes) return FFD_ERR_NULL;
     st = check_geometry(batch, max_blocks_per_seq, 1);
@@ -1357,9 +1655,17 @@ static ffd_status quantize_impl(const ffd_config* cfg, const void* k_cache, void
     const void* ptrs[] = {k_cache, k_quant, k_scales, block_table, seq_lens, first_token};
     for (const void* ptr : ptrs)
         if (ptr && misaligned(ptr)) return FFD_ERR_ALIGN;
+    if (k_res && cfg->quant_bits != 2) return FFD_ERR_UNSUPPORTED;   // the residual format is defined on the 2-bit thumbnails
     QuantParams p{static_cast<const __nv_bfloat16*>(k_cache), static_cast<uint8_t*>(k_quant),
                   static_cast<__half*>(k_scales), block_table, seq_lens, first_token,
                   cfg->num_kv_heads, max_blocks_per_seq, num_pages};
+    if (cfg->quant_bits != 2) {   // 4 or 8 bits: the plain tile-at-a-time kernel for whole caches and tail blocks alike
+        long x = first_token ? 2 : (16L * device_sms() + (long)batch * cfg->num_kv_heads - 1) / ((long)batch * cfg->num_kv_heads);
+        x = x > max_blocks_per_seq ? max_blocks_per_seq : (x < 1 ? 1 : x);
+        launch_pdl(cfg->quant_bits == 4 ? quantize_wide_kernel<4> : quantize_wide_kernel<8>,
+                   dim3((unsigned)x, cfg->num_kv_heads, batch), dim3(128), 0, static_cast<cudaStream_t>(stream), p);
+        return launch_status();
+    }
     // CTAs per (sequence, KV head): every CTA walks its share of the blocks, so any number is correct.  With
     // first_token (decode steps re-quantize the block the new token fell into) two are plenty and a wide grid
     // would only launch thousands of CTAs that find nothing to do.
@@ -1391,7 +1697,7 @@ extern "C" {
 ffd_status ffd_quantize_residual(const ffd_config* cfg, const void* k_cache, const void* k_scales, void* k_res,
                                  const int32_t* block_table, const int32_t* seq_lens, const int32_t* first_token,
                                  int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages, void* stream) {
-    ffd_status st = check_config(cfg);
+    ffd_status st = check_config(cfg, true);
     if (st) return st;
     if (!k_cache || !k_scales || !k_res || !seq_lens) return FFD_ERR_NULL;
     st = check_geometry(batch, max_blocks_per_seq, num_pages);
@@ -1417,7 +1723,7 @@ static ffd_status append_impl(const ffd_config* cfg, const void* k_new, const vo
                               void* k_quant, void* k_scales, void* k_res, const int32_t* block_table, int32_t* seq_lens,
                               int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages, void* workspace,
                               size_t workspace_bytes, void* stream) {
-    ffd_status st = check_config(cfg);
+    ffd_status st = check_config(cfg, true);
     if (st) return st;
     if (!k_new || !v_new || !k_cache || !v_cache || !k_quant || !k_scales || !seq_lens || !workspace) return FFD_ERR_NULL;
     st = check_geometry(batch, max_blocks_per_seq, num_pages);
@@ -1511,8 +1817,10 @@ ffd_status ffd_unpack_codes(const ffd_config* cfg, const void* k_quant, uint8_t*
     if (misaligned(k_quant) || misaligned(codes)) return FFD_ERR_ALIGN;
     const size_t tiles = (size_t)num_pages * cfg->num_kv_heads;
     if (tiles > 0x7fffffffu) return FFD_ERR_SHAPE;
-    unpack_kernel<<<(unsigned)tiles, 128, 0, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const uint8_t*>(k_quant), codes, tiles);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cfg->quant_bits == 2) unpack_kernel<<<(unsigned)tiles, 128, 0, s>>>(static_cast<const uint8_t*>(k_quant), codes, tiles);
+    else if (cfg->quant_bits == 4) unpack_wide_kernel<4><<<(unsigned)tiles, 128, 0, s>>>(static_cast<const uint8_t*>(k_quant), codes, tiles);
+    else unpack_wide_kernel<8><<<(unsigned)tiles, 128, 0, s>>>(static_cast<const uint8_t*>(k_quant), codes, tiles);
     return launch_status();
 }
 
@@ -1547,7 +1855,7 @@ ffd_status ffd_decode_static(const ffd_config* cfg, const void* q, const void* k
                              const int32_t* seq_lens, int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages,
                              float delta, void* out, float* lse, void* stream) {
     // everything that can be refused on the host is refused before the device is touched
-    ffd_status st = check_config(cfg);
+    ffd_status st = check_config(cfg, true);   // (the built-in scratch is sized for the 2-bit path)
     if (st) return st;
     st = check_geometry(batch, max_blocks_per_seq, num_pages);
     if (st) return st;

@@ -86,6 +86,7 @@ struct DecodeParams {
     unsigned long long units_magic, hkv_magic;   // reciprocals for fast_div
     uint8_t* kept_mask;      // nullable [B, Hq, max_blocks]
     float* block_max;        // nullable [B, Hq, max_blocks]
+    float* bmax;             // deeper thumbnails on large geometries: [B, Hq, max_blocks] block maxima, scan kernel -> decode kernel (workspace)
     void* out;               // [B, Hq, 128] bf16 or fp32
     float* lse;              // nullable [B, Hq]
     int out_fp32;
@@ -511,6 +512,164 @@ __device__ __forceinline__ float scan_mma(const uint4 (&w)[4], const uint32_t (&
         }
     }
     return (best - o) * unit;
+}
+
+// ---- deeper thumbnails (4 and 8 bits; App. "Bandwidth Proportionality of Quantization Depth") -------------------
+// The same mid-rise construction with 2^b levels +-(k + 1/2).  Physical order of a (page, head) tile: 4 groups of 16
+// tokens; inside a group lane = 4 r + j owns 2 b words of 32 bits, k-step after k-step (i = 0 .. 7) the eight codes of its
+// MMA A fragment.  The k index of the contraction is a permutation of the channels chosen so that lane j's B operand
+// covers the 32 consecutive channels 32 j .. 32 j + 31: k-step i, A register x (x & 1: token r or r + 8; x >> 1: lower or
+// upper half of the k-step), element e  <->  token 16 mt + r + 8 (x & 1), channel 32 j + 4 i + 2 (x >> 1) + e.
+//   4 bits: one word per k-step; nibble x of the low / high half-word = A register x, element 0 / 1
+//   8 bits: two words per k-step; byte n of the low / high half-word of word h = A register 2 h + n, element 0 / 1
+// Word n of a lane sits in 16-byte vector n / 4 of the group, the vectors of the 32 lanes side by side (a warp's load
+// of one vector is one contiguous 512 bytes): byte offset (((mt V + n / 4) 32 + lane) 4 + n % 4) 4 with V = b / 2.
+// A code c stands for level c - (2^b - 1) / 2.  Shifted into the mantissa of fp16 16 (4 bits: unit in the last place
+// 1/64, the code at bits 6..9) or 256 (8 bits: 1/4, bits 2..9) a code becomes the number 16 + c or 256 + c exactly, and
+// one half2 subtraction of 23.5 or 383.5 (both representable next to those bases, which 1024 + 7.5 would not be) gives
+// the level, the A operand; with B = (q 2^-k) * s split in two fp16 pieces the products are exact as in the 2-bit scan.
+template <int BITS>
+struct WideScan {
+    static constexpr int kTileBytes = kBlk * kD * BITS / 8;
+    static constexpr int kVec = BITS / 2;              // 16-byte vectors per lane and group of 16 tokens
+    __device__ static constexpr int word(int mt, int lane, int n) { return ((mt * kVec + n / 4) * 32 + lane) * 4 + n % 4; }
+};
+
+// q of head lane / 8, channels 32 j .. 32 j + 31, scaled by 2^-k only (the deeper scans need no per-k-step factor);
+// sq.unit turns accumulator units into logits for head lane % 4
+__device__ __forceinline__ void scan_setup_wide(ScanQuery& sq, const __nv_bfloat16* q_group, int G, int lane, float sm_scale) {
+    const int head = lane >> 3, j = lane & 3;
+    uint4 raw[4];   // channels 32 j .. 32 j + 31 of the head: the four lanes j of a column cover all 128
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        raw[x] = make_uint4(0u, 0u, 0u, 0u);
+        if (head < G) raw[x] = *reinterpret_cast<const uint4*>(q_group + head * kD + 32 * j + 8 * x);
+    }
+    const uint32_t* wds = reinterpret_cast<const uint32_t*>(raw);
+    // scale: the same power of two as the 2-bit scan (max over the head's channels)
+    float m = 0.f;
+#pragma unroll
+    for (int y = 0; y < 16; ++y)
+        m = fmaxf(m, fmaxf(fabsf(__uint_as_float(wds[y] << 16)), fabsf(__uint_as_float(wds[y] & 0xffff0000u))));
+    m = fmaxf(m, __shfl_xor_sync(kFull, m, 1));
+    m = fmaxf(m, __shfl_xor_sync(kFull, m, 2));
+    int e = 0;
+    (void)frexpf(m, &e);
+    const int k = min(max(e - 1, 0), 100);
+    const float inv = __uint_as_float((uint32_t)(127 - k) << 23);
+    sq.piece = (lane >> 2) & 1;
+    // B fragment of k-step i for column lane / 4 = (head, piece): registers 2 i and 2 i + 1 = channels 32 j + 4 i .. + 3
+#pragma unroll
+    for (int y = 0; y < 16; ++y) {
+        const __half2 h2 = __floats2half2_rn(__uint_as_float(wds[y] << 16) * inv, __uint_as_float(wds[y] & 0xffff0000u) * inv);
+        sq.qh[y] = *reinterpret_cast<const uint32_t*>(&h2);
+    }
+    const float inv_res = __shfl_sync(kFull, inv, 8 * (lane & 3));
+    sq.unit = sm_scale / inv_res;
+}
+
+// hint: bring a tile's codes and scales into L2 (one 128-byte line per lane and instruction)
+template <int BITS>
+__device__ __forceinline__ void wide_prefetch_l2(const unsigned char* codes_tile, const __half* scales_tile, int lane) {
+#pragma unroll
+    for (int o = 0; o < WideScan<BITS>::kTileBytes; o += 4096)
+        asm volatile("prefetch.global.L2 [%0];\n" ::"l"(codes_tile + o + lane * 128));
+    if (lane < 2) asm volatile("prefetch.global.L2 [%0];\n" ::"l"(reinterpret_cast<const unsigned char*>(scales_tile) + lane * 128));
+}
+
+// Block maximum of the approximate logits of head lane % 4 over the first `rows` tokens, codes and scales read straight
+// from global memory (the caller has prefetched the tile into L2), 32 tokens' worth of codes per round of loads.
+// PRECISE as in scan_mma.
+template <int BITS, bool PRECISE>
+__device__ __forceinline__ float scan_wide(const unsigned char* codes_tile, const __half* scales_tile, const ScanQuery& sq,
+                                           int lane, int rows, float& band) {
+    const int r = lane >> 2, j = lane & 3;
+    constexpr int kVec = WideScan<BITS>::kVec;
+    constexpr int kGroupsPerRound = 8 / kVec;            // 8 vectors per lane in flight: 4 groups (4 bits) or 2 (8 bits)
+    const uint4* src = reinterpret_cast<const uint4*>(codes_tile) + lane;
+    uint4 cv[8];
+#pragma unroll
+    for (int v = 0; v < 8; ++v) cv[v] = ldg_stream(src + v * 32);
+    // B operand: hi / lo piece of (q 2^-k) * s for this lane's column, k-step by k-step
+    uint32_t bfrag[16];
+    {
+        uint4 sv[4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) sv[x] = __ldg(reinterpret_cast<const uint4*>(scales_tile) + 4 * j + x);
+        const uint32_t* sc = reinterpret_cast<const uint32_t*>(sv);
+#pragma unroll
+        for (int y = 0; y < 16; ++y) {
+            const __half2 s2 = *reinterpret_cast<const __half2*>(&sc[y]);
+            const __half2 a = *reinterpret_cast<const __half2*>(&sq.qh[y]);
+            const __half2 hi = __hmul2(a, s2);
+            const __half2 lo = __hfma2(a, s2, __hneg2(hi));
+            const __half2 pick = sq.piece ? lo : hi;
+            bfrag[y] = *reinterpret_cast<const uint32_t*>(&pick);
+        }
+    }
+    float best = -INFINITY, amax = 0.f;
+    bool bad = false;
+#pragma unroll
+    for (int round = 0; round < 4 / kGroupsPerRound; ++round) {
+        if (round > 0) {
+#pragma unroll
+            for (int v = 0; v < 8; ++v) cv[v] = ldg_stream(src + (round * 8 + v) * 32);
+        }
+        const uint32_t* wr = reinterpret_cast<const uint32_t*>(cv);
+#pragma unroll
+        for (int gi = 0; gi < kGroupsPerRound; ++gi) {
+            const int mt = round * kGroupsPerRound + gi;
+            const uint32_t* w = wr + gi * kVec * 4;
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                uint32_t a[4];
+                if (BITS == 4) {
+                    const __half2 bias = __floats2half2_rn(23.5f, 23.5f);          // 16 + 7.5
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) {
+                        const uint32_t sh = 4 * x <= 6 ? w[i] << (6 - 4 * x) : w[i] >> (4 * x - 6);
+                        const uint32_t v = (sh & 0x03C003C0u) | 0x4C004C00u;     // 16 + c
+                        const __half2 lv = __hsub2(*reinterpret_cast<const __half2*>(&v), bias);
+                        a[x] = *reinterpret_cast<const uint32_t*>(&lv);
+                    }
+                } else {
+                    const __half2 bias = __floats2half2_rn(383.5f, 383.5f);        // 256 + 127.5
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) {
+                        const uint32_t word = w[2 * i + (x >> 1)];
+                        const uint32_t sh = (x & 1) ? word >> 6 : word << 2;
+                        const uint32_t v = (sh & 0x03FC03FCu) | 0x5C005C00u;     // 256 + c
+                        const __half2 lv = __hsub2(*reinterpret_cast<const __half2*>(&v), bias);
+                        a[x] = *reinterpret_cast<const uint32_t*>(&lv);
+                    }
+                }
+                if (PRECISE) {
+                    float part[4] = {0.f, 0.f, 0.f, 0.f};
+                    mma_f16(part, a[0], a[1], a[2], a[3], bfrag[2 * i], bfrag[2 * i + 1]);
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) acc[x] += part[x];
+                } else {
+                    mma_f16(acc, a[0], a[1], a[2], a[3], bfrag[2 * i], bfrag[2 * i + 1]);
+                }
+            }
+            const float t0 = acc[0] + acc[1], t1 = acc[2] + acc[3];    // hi + lo piece: token r, token r + 8
+            bad |= !(fabsf(t0) < INFINITY) || !(fabsf(t1) < INFINITY);
+            if (16 * mt + r < rows) { best = fmaxf(best, t0); amax = fmaxf(amax, fabsf(t0)); }
+            if (16 * mt + r + 8 < rows) { best = fmaxf(best, t1); amax = fmaxf(amax, fabsf(t1)); }
+        }
+    }
+    best = fmaxf(best, __shfl_xor_sync(kFull, best, 4));
+    best = fmaxf(best, __shfl_xor_sync(kFull, best, 8));
+    best = fmaxf(best, __shfl_xor_sync(kFull, best, 16));
+    amax = fmaxf(amax, __shfl_xor_sync(kFull, amax, 4));
+    amax = fmaxf(amax, __shfl_xor_sync(kFull, amax, 8));
+    amax = fmaxf(amax, __shfl_xor_sync(kFull, amax, 16));
+    // The level sums are centred (no offset term as in the 2-bit scan), so the accumulators are of the size of the
+    // scores themselves; the band follows the largest of them.
+    band = 4.f * kScanBandRel * amax * sq.unit;
+    if (__any_sync(kFull, bad)) return __int_as_float(0x7fc00000);
+    return best * sq.unit;
 }
 
 // The scan of one block in plain binary32 on the ordinary lanes, for blocks whose fp16 B operand overflowed (scales

@@ -30,7 +30,7 @@ class DeviceCache:
         self.v_cache = w.v_cache.to(device)
         self.block_table = None if w.block_table is None else torch.from_numpy(w.block_table).to(device)
         P, Hkv = w.num_pages, w.Hkv
-        self.k_quant = torch.zeros(P, Hkv, 2048, dtype=torch.uint8, device=device)
+        self.k_quant = torch.zeros(P, Hkv, 1024 * self.cfg.quant_bits, dtype=torch.uint8, device=device)
         self.k_scales = torch.zeros(P, Hkv, 128, dtype=torch.float16, device=device)
         self.workspace = new_workspace(self.cfg, w.B, w.max_blocks, device)
         odt = torch.float32 if self.cfg.out_dtype == 1 else torch.bfloat16

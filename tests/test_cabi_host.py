@@ -70,7 +70,7 @@ def test_documented_limits_of_the_static_entry_point_are_the_computed_ones():
 
 
 @pytest.mark.parametrize("field,value,status", [
-    ("head_dim", 64, 3), ("block_tokens", 32, 3), ("quant_bits", 4, 3), ("num_kv_heads", 5, 2),
+    ("head_dim", 64, 3), ("block_tokens", 32, 3), ("quant_bits", 3, 3), ("quant_bits", 16, 3), ("num_kv_heads", 5, 2),
     ("num_q_heads", 64, 3), ("n_local_blocks", -1, 2), ("out_dtype", 7, 3), ("sm_scale", -1.0, 2),
 ])
 def test_bad_config_is_rejected(field, value, status):
@@ -79,6 +79,15 @@ def test_bad_config_is_rejected(field, value, status):
     with pytest.raises(ffd.FfdError) as e:
         ffd.ffd_workspace_bytes(cfg, 1, 16)
     assert e.value.status == status
+
+
+def test_deeper_thumbnails_are_accepted_except_where_the_format_needs_two_bits():
+    for bits in (4, 8):
+        cfg = ffd.Config(32, 8, quant_bits=bits)
+        assert ffd.ffd_workspace_bytes(cfg, 1, 16) >= ffd.ffd_workspace_bytes(ffd.Config(32, 8), 1, 16) + 32 * 16 * 4
+        with pytest.raises(ffd.FfdError) as e:     # the 2 + 8 bit key format is defined on the 2-bit thumbnails
+            ffd.ffd_workspace_bytes_residual(cfg, 1, 16)
+        assert e.value.status == 3
 
 
 def test_null_and_range_arguments_are_rejected_before_any_launch(lib):

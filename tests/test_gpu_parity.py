@@ -51,7 +51,7 @@ def valid_row_mask(w):
 
 def check_quantize(ffd, oracle, w, dc):
     dc.quantize()
-    codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
+    codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks, bits=dc.cfg.quant_bits)
     g_codes = dc.canonical_codes().cpu().numpy()
     g_scales = dc.k_scales.cpu().view(torch.int16).numpy().view(np.uint16)
     vm, mapped = valid_row_mask(w)
@@ -97,7 +97,8 @@ def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None, k_res=Non
     kept = kept.cpu().numpy()
     bm = bm.cpu().numpy().astype(np.float64)
     r = oracle.decode(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), codes, scales, w.block_table, w.seq_lens,
-                      mb, delta, n_sink=dc.cfg.n_sink_blocks, n_local=dc.cfg.n_local_blocks, units=units, k_res=k_res)
+                      mb, delta, n_sink=dc.cfg.n_sink_blocks, n_local=dc.cfg.n_local_blocks, units=units, k_res=k_res,
+                      bits=dc.cfg.quant_bits)
     rows = units if units is not None else [(b, h) for b in range(B) for h in range(Hq)]
     mag = magnitude(r, w)
     differs = False
@@ -127,7 +128,7 @@ def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None, k_res=Non
     if differs:   # compare the output against the oracle's attention over the GPU's (equally valid) mask
         forced = np.where(kept == 255, 0, kept).astype(np.uint8)
         r = oracle.decode(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), codes, scales, w.block_table,
-                          w.seq_lens, mb, delta, forced_mask=forced, units=units, k_res=k_res)
+                          w.seq_lens, mb, delta, forced_mask=forced, units=units, k_res=k_res, bits=dc.cfg.quant_bits)
     idx = tuple(np.array(rows).T)
     err = np.abs(out[idx] - r.out[idx])
     assert err.max() < OUT_MAX * mag and err.mean() < OUT_MEAN * mag, (err.max(), err.mean(), mag)
@@ -193,6 +194,20 @@ def test_small_configs_residual_key_format(ffd, oracle, name, kw, _):
     dc.k_cache = None   # the residual decode must not need the 16-bit keys
     for delta in w.deltas:
         check_decode(ffd, oracle, w, dc, codes, scales, delta, k_res=k_res)
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+@pytest.mark.parametrize("name,kw,_", SMALL)
+def test_small_configs_deeper_thumbnails(ffd, oracle, name, kw, _, bits):
+    """App. "Bandwidth Proportionality of Quantization Depth": 4- and 8-bit thumbnails.  Codes and scales bit for bit,
+    masks and outputs against the oracle run at the same depth, at the bars of the 2-bit path."""
+    w = make_workload(name, **kw)
+    dc = DeviceCache(w, ffd.Config(w.Hq, w.Hkv, quant_bits=bits))
+    codes, scales = check_quantize(ffd, oracle, w, dc)
+    assert int(codes.max()) == (1 << bits) - 1
+    for delta in w.deltas:
+        check_decode(ffd, oracle, w, dc, codes, scales, delta)
+    check_decode(ffd, oracle, w, dc, codes, scales, 0.0)
 
 
 def test_bf16_output_is_rounding_of_fp32_output(ffd, oracle):
@@ -518,7 +533,7 @@ def test_append_writes_the_token_requantizes_its_block_and_bumps_the_length(ffd,
     sel = torch.from_numpy(np.broadcast_to(vm, tuple(k_all.shape)).copy()).cuda()
     assert torch.equal(dc.k_cache.view(torch.int16)[sel], k_all.view(torch.int16)[sel])
     assert torch.equal(dc.v_cache.view(torch.int16)[sel], v_all.view(torch.int16)[sel])
-    codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
+    codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks, bits=dc.cfg.quant_bits)
     g_codes = dc.canonical_codes().cpu().numpy()
     g_scales = dc.k_scales.cpu().view(torch.int16).numpy().view(np.uint16)
     assert np.array_equal(g_scales[mapped], scales[mapped])
@@ -775,6 +790,57 @@ def test_full_size_configs_every_row(ffd, oracle, name):
             check_decode(ffd, oracle, w, dc, codes, scales, w.deltas[0], k_res=k_res)
     finally:
         oracle.set_threads(min(8, oracle.max_threads()))
+
+
+@pytest.mark.parametrize("name,bits", [("C3", 4), ("C5", 4), ("C4", 8), ("C5", 8)])
+def test_full_size_configs_deeper_thumbnails(ffd, oracle, name, bits):
+    """4- and 8-bit thumbnails at the benchmark's sizes (the scan kernel of its own followed by the decode kernel):
+    every mapped tile and every (sequence, query head) row at the configuration's first delta."""
+    oracle.set_threads(oracle.max_threads())
+    try:
+        w = make_workload(name)
+        dc = DeviceCache(w, ffd.Config(w.Hq, w.Hkv, quant_bits=bits))
+        codes, scales = check_quantize(ffd, oracle, w, dc)
+        check_decode(ffd, oracle, w, dc, codes, scales, w.deltas[0])
+    finally:
+        oracle.set_threads(min(8, oracle.max_threads()))
+
+
+def test_deeper_thumbnails_edge_cases(ffd, oracle):
+    """Empty and one-token sequences, delta = inf (everything kept), a bad page index (reported, never kept, no fault)
+    and scales beyond the fp16 operand's range (reported, kept) on the two-kernel path of the deeper thumbnails."""
+    for bits in (4, 8):
+        w = make_workload("C5", B=24, lens=(1, 4000))
+        w.seq_lens[0] = 0
+        w.seq_lens[1] = 1
+        dc = DeviceCache(w, ffd.Config(w.Hq, w.Hkv, quant_bits=bits))
+        dc.seq_lens.copy_(torch.from_numpy(w.seq_lens))
+        codes, scales = check_quantize(ffd, oracle, w, dc)
+        live = [(b, h) for b in range(1, w.B) for h in range(w.Hq)]
+        check_decode(ffd, oracle, w, dc, codes, scales, 6.0, units=live)
+        check_decode(ffd, oracle, w, dc, codes, scales, INF, units=live)
+        assert torch.all(dc.out[0] == 0) and torch.all(torch.isinf(dc.lse[0]) & (dc.lse[0] < 0))   # the empty sequence
+        # a page index out of range in the middle of the longest sequence
+        b = int(np.argmax(w.seq_lens))
+        good = dc.block_table.clone()
+        dc.block_table[b, w.num_blocks(b) // 2] = w.num_pages + 5
+        kept = torch.full((w.B, w.Hq, w.max_blocks), 255, dtype=torch.uint8, device="cuda")
+        dc.decode(INF, kept_mask=kept)
+        torch.cuda.synchronize()
+        assert ffd.ffd_read_device_status(dc.workspace) & ffd.DEV_BAD_PAGE
+        assert int(kept[b, :, w.num_blocks(b) // 2].max()) == 0 and bool(torch.isfinite(dc.out).all())
+        dc.block_table.copy_(good)
+        ffd.ffd_workspace_init(dc.workspace)
+    # |q s| beyond fp16: keys of ~1e9 give scales at the fp16 maximum
+    w = make_workload("C5", B=24, lens=(1000, 3000), k_gain=3e8)
+    dc = DeviceCache(w, ffd.Config(w.Hq, w.Hkv, quant_bits=4))
+    dc.quantize()
+    kept = torch.full((w.B, w.Hq, w.max_blocks), 255, dtype=torch.uint8, device="cuda")
+    dc.decode(6.0, kept_mask=kept)
+    torch.cuda.synchronize()
+    assert ffd.ffd_read_device_status(dc.workspace) & ffd.DEV_RANGE
+    for b in range(w.B):
+        assert int(kept[b, :, : w.num_blocks(b)].min()) == 1
 
 
 LARGE = [
