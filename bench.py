@@ -227,10 +227,10 @@ def stats(xs):
 class Bench:
     """One workload resident on the device and the timing loops over it."""
 
-    def __init__(self, ffd, w, delta, shared=None):
+    def __init__(self, ffd, w, delta, shared=None, bits=2):
         from tests.device_cache import DeviceCache
         self.ffd, self.w, self.delta = ffd, w, delta
-        self.dc = DeviceCache(w, ffd.Config(w.Hq, w.Hkv, out_dtype=1))
+        self.dc = DeviceCache(w, ffd.Config(w.Hq, w.Hkv, out_dtype=1, quant_bits=bits))
         self.dc.quantize()
         self.first_token = torch.from_numpy(np.maximum(w.seq_lens - 1, 0)).to("cuda")
         if shared is None:
@@ -309,6 +309,36 @@ class Bench:
                 "fidelity": self.fidelity()}
 
 
+def depth_table(ffd, peak, steps):
+    """App. "Bandwidth Proportionality of Quantization Depth": the scan at 2, 4 and 8 bits on one scan-only workload
+    (sink needle in every head, delta 0: a handful of blocks kept), decode call alone (no tail re-quantize), cold L2.
+    kernel_us brackets the scan-select-attend kernel(s) of the call: the fused kernel at 2 bits, the scan kernel plus the
+    decode kernel at 4 and 8 bits."""
+    rows = []
+    w = make_workload("C2", N=131072, B=4)
+    tiles = sum(w.num_blocks(b) for b in range(w.B)) * w.Hkv
+    for bits in (2, 4, 8):
+        b = Bench(ffd, w, 0.0, bits=bits)
+        decode = lambda: b.dc.decode(0.0)
+        b.timed_loop(decode, 3)
+        step_us, _ = b.timed_loop(decode, steps)
+        _, kernel_us = b.timed_loop(decode, max(steps, 20), profile_kernel=True)
+        scan_bytes = tiles * (1024 * bits + 256)
+        t = statistics.mean(kernel_us)
+        rows.append({"bits": bits, "bytes_per_block_and_kv_head": 1024 * bits + 256, "scan_bytes": scan_bytes,
+                     "kept_tiles": b.kept_tiles, "total_tiles": tiles, "decode_us": statistics.mean(step_us),
+                     "kernel_us": stats(kernel_us), "scan_gbs": scan_bytes / (t * 1e-6) / 1e9,
+                     "frac": scan_bytes / (t * 1e-6) / 1e9 / peak})
+        del b
+        torch.cuda.empty_cache()
+    base = rows[0]
+    for r in rows:
+        r["bytes_ratio_vs_2bit"] = r["scan_bytes"] / base["scan_bytes"]
+        r["kernel_time_ratio_vs_2bit"] = r["kernel_us"]["mean"] / base["kernel_us"]["mean"]
+    return {"workload": "C2 recipe at batch 4, context 131072 (32 query / 8 KV heads), delta 0, decode call only",
+            "rows": rows}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -320,7 +350,8 @@ def main():
     ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--delta", type=float, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-extras", action="store_true", help="skip the secondary workloads (C4, C5) of the bench line")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the secondary workloads (C4, C5) and the quantization-depth table of the bench line")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -481,6 +512,7 @@ def main():
             del bx, wx
             torch.cuda.empty_cache()
         line["extra"] = extra
+        line["quantization_depth"] = depth_table(ffd, peak, min(args.steps, 30))
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(w, delta)
         one = cpu_baseline(w, delta, threads=1, rows_per_thread=8)

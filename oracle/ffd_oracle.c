@@ -258,6 +258,9 @@ typedef struct {
     double *out, *lse, *block_max, *mtilde;
     uint8_t* kept;
     const int8_t* k_res;        /* nullable: refine from Dequant(codes, k_res) instead of the 16-bit K */
+    int rule;                   /* selection rule, see ffd_oracle_decode */
+    int top_k;                  /* rule 3 only */
+    double* thr;                /* nullable [B,Hq,max_blocks]: the threshold every block's maximum was compared with */
 } decode_args;
 
 static void softmax_attention_over_mask(const decode_args* a, int b, int h, const uint8_t* keep, double* out,
@@ -336,11 +339,45 @@ static void decode_one(const decode_args* a, int b, int h) {
         if (blk < a->n_sink || blk >= nb - a->n_local)
             if (bm[blk] > mt) mt = bm[blk];
     a->mtilde[row] = mt;
-    /* top-delta test */
-    for (int blk = 0; blk < nb; ++blk) {
-        if (a->forced_mask) keep[blk] = a->forced_mask[row * a->max_blocks + blk];
-        else keep[blk] = isinf(a->delta) ? 1 : (bm[blk] >= mt - a->delta);
+    /* the threshold of every block under the selection rule */
+    double* thr = (double*)malloc(sizeof(double) * (size_t)(nb > 0 ? nb : 1));
+    if (a->rule == 0) {            /* Alg. 1 / Eq. 1: the pseudo-max of the sink and local blocks */
+        for (int blk = 0; blk < nb; ++blk) thr[blk] = mt - a->delta;
+    } else if (a->rule == 1) {     /* the comparison rule of Sec. 5.2: the maximum over all blocks (a first pass of its own) */
+        double m = -INFINITY;
+        for (int blk = 0; blk < nb; ++blk)
+            if (bm[blk] > m) m = bm[blk];
+        for (int blk = 0; blk < nb; ++blk) thr[blk] = m - a->delta;
+    } else if (a->rule == 2) {     /* a streaming scan's own reference: the pseudo-max raised by every block maximum
+                                      met so far, blocks taken in logical order, the block itself included */
+        double run = mt;
+        for (int blk = 0; blk < nb; ++blk) {
+            if (bm[blk] > run) run = bm[blk];
+            thr[blk] = run - a->delta;
+        }
+    } else {                       /* fixed budget (Fig. 1a): the top_k blocks by block maximum; blocks equal to the
+                                      k-th largest maximum are all kept; delta plays no part */
+        double tau = -INFINITY;
+        if (a->top_k < nb) {
+            /* the k-th largest by repeated extraction (k is small next to nb; clarity over speed) */
+            uint8_t* used = (uint8_t*)calloc((size_t)(nb > 0 ? nb : 1), 1);
+            for (int i = 0; i < a->top_k; ++i) {
+                int arg = -1;
+                for (int blk = 0; blk < nb; ++blk)
+                    if (!used[blk] && (arg < 0 || bm[blk] > bm[arg])) arg = blk;
+                used[arg] = 1;
+                tau = bm[arg];
+            }
+            free(used);
+        }
+        for (int blk = 0; blk < nb; ++blk) thr[blk] = tau;
     }
+    for (int blk = 0; blk < nb; ++blk) {
+        if (a->thr) a->thr[row * a->max_blocks + blk] = thr[blk];
+        if (a->forced_mask) keep[blk] = a->forced_mask[row * a->max_blocks + blk];
+        else keep[blk] = (a->rule != 3 && isinf(a->delta)) ? 1 : (bm[blk] >= thr[blk]);
+    }
+    free(thr);
     /* exact attention over the kept blocks */
     softmax_attention_over_mask(a, b, h, keep, a->out + row * D, a->lse + row);
 }
@@ -360,18 +397,24 @@ static int check_geometry(const decode_args* a) {
 
 /* Sparse decode step.  Rows of kept / block_max beyond a sequence's block count are left untouched.
  * k_res: NULL = refine from the 16-bit K; else from the 2-bit + 8-bit reconstruction (k_cache is then unused).
- * units: nullable list of n_units (b, h) pairs to compute; NULL = all B*Hq pairs. */
+ * units: nullable list of n_units (b, h) pairs to compute; NULL = all B*Hq pairs.
+ * rule: which reference the block maxima are compared with.  0 = the paper's method (Alg. 1, Eq. 1): m_tilde - delta.
+ * 1 = global approximate maximum - delta (Sec. 5.2's comparison).  2 = scan-order running maximum - delta: the pseudo-max
+ * raised by the block maxima met so far in logical block order (the whole sequence is one scan; the split geometry of an
+ * implementation plays no part).  3 = top-k by block maximum (Fig. 1a's fixed budget; the selection-overhead comparison
+ * of Sec. 4.4), ties with the k-th value kept, 1 <= top_k.  thr_out: nullable, the per-block thresholds. */
 int ffd_oracle_decode(const uint16_t* q, const uint16_t* k_cache, const uint16_t* v_cache, const uint8_t* codes,
                       const uint16_t* scales, const int32_t* block_table, const int32_t* seq_lens, int B, int Hq,
                       int Hkv, int D, int BLK, int max_blocks, int num_pages, int n_sink, int n_local,
                       double sm_scale, double delta, const uint8_t* forced_mask, const int32_t* units, int n_units,
                       double* out, double* lse, uint8_t* kept, double* block_max, double* mtilde, const int8_t* k_res,
-                      int bits) {
+                      int bits, int rule, int top_k, double* thr_out) {
     if (bits != 2 && bits != 4 && bits != 8) return 5;
+    if (rule < 0 || rule > 3 || (rule == 3 && top_k < 1)) return 6;
     if (k_res && bits != 2) return 5;             /* the residual format is defined on the 2-bit thumbnails */
     decode_args a = {q, k_cache, v_cache, scales, codes, block_table, seq_lens, B, Hq, Hkv, D, BLK, max_blocks,
                      num_pages, n_sink, n_local, sm_scale, delta, (double)((1 << bits) - 1) / 2.0, forced_mask, out, lse,
-                     block_max, mtilde, kept, k_res};
+                     block_max, mtilde, kept, k_res, rule, top_k, thr_out};
     int rc = check_geometry(&a);
     if (rc) return rc;
     if (isnan(delta) || delta < 0.0) return 4;
@@ -390,7 +433,7 @@ int ffd_oracle_dense(const uint16_t* q, const uint16_t* k_cache, const uint16_t*
                      const int32_t* seq_lens, int B, int Hq, int Hkv, int D, int BLK, int max_blocks, int num_pages,
                      double sm_scale, const int32_t* units, int n_units, double* out, double* lse) {
     decode_args a = {q, k_cache, v_cache, NULL, NULL, block_table, seq_lens, B, Hq, Hkv, D, BLK, max_blocks,
-                     num_pages, 0, 0, sm_scale, INFINITY, 1.5, NULL, out, lse, NULL, NULL, NULL, NULL};
+                     num_pages, 0, 0, sm_scale, INFINITY, 1.5, NULL, out, lse, NULL, NULL, NULL, NULL, 0, 0, NULL};
     int rc = check_geometry(&a);
     if (rc) return rc;
     int total = units ? n_units : B * Hq;

@@ -126,6 +126,10 @@ class DecodeResult:
     kept: np.ndarray       # uint8   [B, Hq, max_blocks]   (entries past a sequence's block count are 0)
     block_max: np.ndarray  # float64 [B, Hq, max_blocks]   (entries past the block count are -inf)
     mtilde: np.ndarray     # float64 [B, Hq]
+    thr: np.ndarray = None  # float64 [B, Hq, max_blocks]   the threshold each block maximum was compared with (nan past the block count)
+
+
+RULE_PSEUDO_MAX, RULE_GLOBAL_MAX, RULE_RUNNING_MAX, RULE_TOP_K = 0, 1, 2, 3
 
 
 def _units(units):
@@ -138,8 +142,14 @@ def _units(units):
 
 
 def decode(q, k_cache, v_cache, codes, scales, block_table, seq_lens, max_blocks, delta, *, n_sink=1, n_local=16,
-           sm_scale=None, forced_mask=None, units=None, k_res=None, bits: int = 2) -> DecodeResult:
+           sm_scale=None, forced_mask=None, units=None, k_res=None, bits: int = 2, rule: int = RULE_PSEUDO_MAX,
+           top_k: int = 0) -> DecodeResult:
     """Alg. 1: approximate scores -> pseudo-max -> top-delta -> exact attention over kept blocks.
+
+    ``rule``: the reference the block maxima are compared with.  RULE_PSEUDO_MAX is the paper's method; the others are
+    the comparison rules: RULE_GLOBAL_MAX (Sec. 5.2), RULE_RUNNING_MAX (the pseudo-max raised by the block maxima met so
+    far, blocks in logical order), RULE_TOP_K (fixed budget ``top_k`` blocks per head, ties with the k-th kept; ``delta``
+    unused).
 
     ``k_res`` (int8, from ``quantize_residual``): refine from Dequant(codes, k_res) instead of the 16-bit K.
 
@@ -162,6 +172,7 @@ def decode(q, k_cache, v_cache, codes, scales, block_table, seq_lens, max_blocks
     kept = np.zeros((B, Hq, max_blocks), dtype=np.uint8)
     bm = np.full((B, Hq, max_blocks), -np.inf, dtype=np.float64)
     mt = np.full((B, Hq), np.nan, dtype=np.float64)
+    thr = np.full((B, Hq, max_blocks), np.nan, dtype=np.float64)
     fm = None if forced_mask is None else np.ascontiguousarray(forced_mask, dtype=np.uint8)
     u, nu = _units(units)
     kr = None if k_res is None else np.ascontiguousarray(k_res, dtype=np.int8)
@@ -172,10 +183,11 @@ def decode(q, k_cache, v_cache, codes, scales, block_table, seq_lens, max_blocks
         _ptr(seq_lens, ctypes.c_int32), B, Hq, Hkv, D, BLK, int(max_blocks), P, int(n_sink), int(n_local),
         ctypes.c_double(sm_scale), ctypes.c_double(delta), _ptr(fm, ctypes.c_uint8), _ptr(u, ctypes.c_int32), nu,
         _ptr(out, ctypes.c_double), _ptr(lse, ctypes.c_double), _ptr(kept, ctypes.c_uint8),
-        _ptr(bm, ctypes.c_double), _ptr(mt, ctypes.c_double), _ptr(kr, ctypes.c_int8), int(bits))
+        _ptr(bm, ctypes.c_double), _ptr(mt, ctypes.c_double), _ptr(kr, ctypes.c_int8), int(bits), int(rule), int(top_k),
+        _ptr(thr, ctypes.c_double))
     if rc:
         raise ValueError(f"ffd_oracle_decode: error {rc}")
-    return DecodeResult(out, lse, kept, bm, mt)
+    return DecodeResult(out, lse, kept, bm, mt, thr)
 
 
 def dense(q, k_cache, v_cache, block_table, seq_lens, max_blocks, *, sm_scale=None, units=None):

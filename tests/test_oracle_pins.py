@@ -582,6 +582,64 @@ def test_mask_monotone_in_delta_nonempty_and_superset_of_global_max_rule(oracle,
     assert r2.kept[0, :, :nb].mean() > 0.9
 
 
+def test_selection_rule_variants_against_their_definitions(oracle):
+    """The comparison rules next to Alg. 1's pseudo-max (Fig. 1, Sec. 4.4 "Selection-Rule Overhead", Sec. 5.2).  The block
+    maxima are pinned elsewhere; here each rule's kept set is re-derived from them with numpy (sorting, accumulate) and the
+    rules are ordered as the mathematics says: global max  subset of  running max  subset of  pseudo-max."""
+    cases = [make_workload("C4", N=16384),                      # no sink needle: m_tilde below the global maximum
+             make_workload("C5", B=3, lens=(700, 3000)),        # paged, ragged
+             make_workload("C2", N=6000)]                       # sink needle: the three threshold rules coincide
+    strict = 0
+    for w in cases:
+        codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
+        for delta in (0.0, 3.0, 6.0):
+            base = _decode(oracle, w, codes, scales, delta)
+            glob = _decode(oracle, w, codes, scales, delta, rule=oracle.RULE_GLOBAL_MAX)
+            run = _decode(oracle, w, codes, scales, delta, rule=oracle.RULE_RUNNING_MAX)
+            assert np.array_equal(base.block_max, glob.block_max) and np.array_equal(base.block_max, run.block_max)
+            for b in range(w.B):
+                nb = w.num_blocks(b)
+                bm = base.block_max[b, :, :nb]
+                mt = base.mtilde[b][:, None]
+                assert np.array_equal(glob.kept[b, :, :nb], (bm >= bm.max(-1, keepdims=True) - delta).astype(np.uint8))
+                ref = np.maximum(np.maximum.accumulate(bm, axis=-1), mt)
+                assert np.array_equal(run.kept[b, :, :nb], (bm >= ref - delta).astype(np.uint8))
+                assert np.array_equal(run.thr[b, :, :nb], ref - delta)
+                g, r_, p_ = (x.kept[b, :, :nb].astype(bool) for x in (glob, run, base))
+                assert np.all(r_ | ~g) and np.all(p_ | ~r_)
+                strict += int((p_ & ~r_).sum() > 0) + int((r_ & ~g).sum() > 0)
+                # the block attaining the global maximum survives every rule
+                arg = bm.argmax(-1)
+                for x in (glob, run, base):
+                    assert np.all(x.kept[b, np.arange(w.Hq), arg] == 1)
+            # the outputs are the exact attention over each rule's own mask
+            forced = _decode(oracle, w, codes, scales, delta, forced_mask=run.kept)
+            assert np.array_equal(forced.out, run.out) and np.array_equal(forced.lse, run.lse)
+        # fixed budget: exactly k blocks when the k-th and (k+1)-th maxima differ, the k largest ones; k >= nb keeps all
+        for k in (1, 5, 40):
+            top = _decode(oracle, w, codes, scales, 6.0, rule=oracle.RULE_TOP_K, top_k=k)
+            for b in range(w.B):
+                nb = w.num_blocks(b)
+                bm = top.block_max[b, :, :nb]
+                order = np.sort(bm, axis=-1)[:, ::-1]
+                tau = order[:, min(k, nb) - 1] if k < nb else np.full(w.Hq, -np.inf)
+                want = bm >= tau[:, None]
+                assert np.array_equal(top.kept[b, :, :nb], want.astype(np.uint8))
+                distinct = (k >= nb) | (order[:, min(k, nb - 1)] < tau)
+                assert np.all(want.sum(-1)[distinct] == min(k, nb)) and np.all(want.sum(-1) >= min(k, nb))
+        everything = _decode(oracle, w, codes, scales, 0.0, rule=oracle.RULE_TOP_K, top_k=10 ** 6)
+        dense_o, dense_l = oracle.dense(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), w.block_table, w.seq_lens,
+                                        w.max_blocks)
+        assert np.abs(everything.out - dense_o).max() < 1e-12
+    assert strict >= 4, "the cases never separated the three threshold rules"
+    w = cases[2]
+    codes, scales = oracle.quantize(w.bits("k_cache"), w.block_table, w.seq_lens, w.max_blocks)
+    with pytest.raises(ValueError):
+        _decode(oracle, w, codes, scales, 6.0, rule=oracle.RULE_TOP_K, top_k=0)
+    with pytest.raises(ValueError):
+        _decode(oracle, w, codes, scales, 6.0, rule=7)
+
+
 def test_delta_zero_keeps_the_pseudo_max_block(oracle, small):
     w, codes, scales = small
     nb = w.num_blocks(0)
