@@ -214,6 +214,32 @@ ffd_status ffd_decode(const ffd_config* cfg, const void* q, const void* k_cache,
                       size_t workspace_bytes, void* stream);
 
 /*
+ * The decode step under one of the comparison selection rules (Fig. 1; Sec. 4.4 "Selection-Rule Overhead"; Sec. 5.2),
+ * for measuring what each rule costs and keeps next to the paper's own.  Same arguments, outputs, errors and workspace as
+ * ffd_decode, at every quantization depth; always runs as three kernels (scan of all blocks into the workspace, the rule,
+ * attention over the kept blocks), also where ffd_decode would fuse them.  rule:
+ *   FFD_RULE_PSEUDO_MAX   keep a block iff its maximum approximate score >= m_tilde - delta (Alg. 1, Eq. 1; what
+ *                         ffd_decode computes)
+ *   FFD_RULE_GLOBAL_MAX   ... >= (maximum over all blocks of the head) - delta: needs the whole scan before any decision
+ *   FFD_RULE_RUNNING_MAX  ... >= max(m_tilde, maxima of blocks 0 .. blk) - delta: the reference a streaming scan in logical
+ *                         block order has when it meets block blk; a function of the inputs only, whatever the split
+ *                         geometry of the kernels
+ *   FFD_RULE_TOP_K        the top_k blocks of each head by maximum approximate score (>= 1; blocks equal to the k-th value
+ *                         are all kept; top_k >= the head's block count keeps everything); delta is not used
+ * The kept sets are nested: global max within running max within pseudo-max.  `mtilde` in the workspace, kept_mask and
+ * block_max are written as by ffd_decode (block_max is NaN for a block whose page index is bad).
+ */
+#define FFD_RULE_PSEUDO_MAX 0
+#define FFD_RULE_GLOBAL_MAX 1
+#define FFD_RULE_RUNNING_MAX 2
+#define FFD_RULE_TOP_K 3
+ffd_status ffd_decode_select(const ffd_config* cfg, int32_t rule, int32_t top_k, const void* q, const void* k_cache,
+                             const void* v_cache, const void* k_quant, const void* k_scales, const int32_t* block_table,
+                             const int32_t* seq_lens, int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages,
+                             float delta, void* out, float* lse, uint8_t* kept_mask, float* block_max, void* workspace,
+                             size_t workspace_bytes, void* stream);
+
+/*
  * The same step on the 2 + 8 bit key format (Sec. 3.3, "Fine-grained refinement": a block that passes the filter
  * loads its 8-bit residual keys and its values; s_final = (q . k_quant + q . k_res) / sqrt(d), both dot products
  * accumulated without a full-precision key).  Selection is exactly ffd_decode's; the refined logit of a kept token is
@@ -286,7 +312,7 @@ ffd_status ffd_read_device_status(void* workspace, void* stream, uint32_t* statu
  * Limits and rules
  *   - Geometry: ffd_workspace_bytes(cfg, batch, max_blocks_per_seq) must not exceed FFD_STATIC_SCRATCH_BYTES,
  *     otherwise FFD_ERR_STATIC_LIMIT is returned and nothing is launched.  With 32 query / 8 KV heads on a 148-SM
- *     GPU the 8 MiB hold batch 1 up to about 117 K tokens of context, batch 4 up to about 28 K, batch 16 up to about
+ *     GPU the 8 MiB hold batch 1 up to about 113 K tokens of context, batch 4 up to about 27 K, batch 16 up to about
  *     6 K (ask ffd_workspace_bytes for the exact figure of a geometry).
  *   - First use on a device: the first call made while a given device is current looks up the device address of
  *     the array (cudaGetSymbolAddress) and remembers it.  Make that first call during start-up, outside of any

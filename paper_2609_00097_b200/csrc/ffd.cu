@@ -822,11 +822,14 @@ __device__ __noinline__ float scan_precise_from_global(const uint4* codes_tile, 
     return bm;
 }
 
-// ---- the scan on its own: 4- and 8-bit thumbnails on large geometries -------------------------------------------
-// One warp per block, many warps per SM: the thumbnails of a long cache stream through at memory speed, which the decode
-// kernel's seven fat warps per SM cannot do for codes this wide.  Writes the block maxima of the approximate logits
-// (precise accumulation, the arithmetic of m_tilde) for the decode kernel that follows: p.bmax[b][head][block]; NaN for a
-// block whose page index is bad (never kept, ignored by every maximum).
+// ---- scan, select and decode as three kernels -----------------------------------------------------------------
+// The path of the 4- and 8-bit thumbnails on large geometries and of the comparison selection rules (ffd_decode_select):
+//   scan_blocks_kernel   block maxima of the approximate logits of every block (Alg. 1 "Top-delta selection", the scores)
+//   select_kernel        the rule: which blocks each head keeps
+//   small_sparse_kernel<0>  exact attention over the kept blocks and the merge of the splits
+// Scan: one warp per block, many warps per SM; the codes of a long cache stream through, which the decode kernel's seven
+// fat warps per SM cannot do for codes this wide.  Writes p.bmax[b][head][block] (precise accumulation, the arithmetic
+// of m_tilde); NaN for a block whose page index is bad (never kept, ignored by every maximum).
 constexpr int kScanCtaBlocks = 64;   // blocks of one (sequence, KV head) per CTA: 8 per warp
 template <int BITS>
 __global__ void __launch_bounds__(256, 2) scan_blocks_kernel(DecodeParams p) {
@@ -851,6 +854,48 @@ __global__ void __launch_bounds__(256, 2) scan_blocks_kernel(DecodeParams p) {
             wide_prefetch_l2<BITS>(p.k_quant + tile * WideScan<BITS>::kTileBytes, p.k_scales + tile * kD, lane);
         }
     };
+    if constexpr (BITS == 2) {
+        // 2-bit thumbnails: the next block's codes and scales wait in registers while the current block is scored
+        ScanQuery sq;
+        scan_setup(sq, q_group, p.G, lane, p.sm_scale);
+        auto tile_of = [&](int blk) -> long long {
+            if (blk >= last) return -1;
+            const int page = page_of(p, b, blk);
+            return page < 0 ? -1 : (long long)page * p.Hkv + g;
+        };
+        auto load = [&](ScanRegs& sr, long long tile) {
+            if (tile >= 0)
+                scan_load(sr, reinterpret_cast<const uint4*>(p.k_quant + (size_t)tile * kCodeBytes),
+                          reinterpret_cast<const uint4*>(p.k_scales + (size_t)tile * kD), lane);
+        };
+        int blk = first + warp;
+        long long tile = tile_of(blk);
+        ScanRegs cur;
+        load(cur, tile);
+        for (; blk < last; blk += 8) {
+            const long long next_tile = tile_of(blk + 8);
+            ScanRegs nxt;
+            load(nxt, next_tile);
+            float bm = __int_as_float(0x7fc00000);
+            if (tile >= 0) {
+                const int rows = min(kBlk, n - blk * kBlk);
+                float band;
+                bm = scan_compute<true>(cur, sq, lane, rows, band);
+                if (bm != bm) {   // the fp16 operand overflowed: binary32 on the ordinary lanes
+                    bm = scan_block_wide(reinterpret_cast<const uint4*>(p.k_quant + (size_t)tile * kCodeBytes),
+                                         p.k_scales + (size_t)tile * kD, q_group, p.G, lane, rows, p.sm_scale, nullptr, 0);
+                    if (!(fabsf(bm) < INFINITY)) {
+                        if (j < p.G) atomicOr(p.status, kDevRange);
+                        bm = INFINITY;
+                    }
+                }
+            }
+            if (r == 0 && j < p.G) out[(size_t)j * p.max_blocks + blk] = bm;
+            tile = next_tile;
+            cur = nxt;
+        }
+        return;
+    }
     // the warp's first two tiles are on their way while it prepares its query fragments
     int blk = first + warp;
     int page = blk < last ? raw_page(blk) : -1;
@@ -878,6 +923,132 @@ __global__ void __launch_bounds__(256, 2) scan_blocks_kernel(DecodeParams p) {
         page = next_page;
         next_page = after;
         prefetch(after);
+    }
+}
+
+// ---- select: the rule that turns block maxima into decisions ----------------------------------------------------
+// One CTA per (sequence, KV head); the heads of the group one after the other.  Rules (ffd.h FFD_RULE_*):
+//   0 pseudo-max     keep = bm >= m_tilde - delta, m_tilde over the sink and local blocks (Alg. 1, Eq. 1)
+//   1 global max     keep = bm >= max over all blocks - delta (the comparison rule of Sec. 5.2: a reduction of its own)
+//   2 running max    keep = bm >= max(m_tilde, bm of blocks 0 .. blk) - delta: what a streaming scan in logical block
+//                    order knows when it meets the block
+//   3 top-k          keep = bm >= the k-th largest block maximum (Fig. 1a's fixed budget; ties kept): a radix select,
+//                    four passes over the head's maxima
+// Writes keep_bits (bit h of a block's byte = head h keeps it), m_tilde, and the kept_mask / block_max outputs.
+constexpr int kSelectThreads = 256;
+enum : int { kRulePseudoMax = 0, kRuleGlobalMax = 1, kRuleRunningMax = 2, kRuleTopK = 3 };
+
+__device__ __forceinline__ uint32_t select_key(float x) {   // order-preserving: larger float <-> larger key
+    const uint32_t u = __float_as_uint(x);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float select_unkey(uint32_t k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+__global__ void __launch_bounds__(kSelectThreads) select_kernel(DecodeParams p, int rule, int top_k) {
+    const int g = blockIdx.x, b = blockIdx.y;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    pdl_launch_dependents();
+    pdl_wait();
+    const int n = clamped_seq_len(p, b);
+    const int nb = (n + kBlk - 1) / kBlk;
+    const size_t head0 = (size_t)b * p.Hq + (size_t)g * p.G;
+    uint8_t* bits = p.keep_bits + ((size_t)b * p.Hkv + g) * p.max_blocks;
+    __shared__ float red_a[kSelectThreads / 32], red_b[kSelectThreads / 32];
+    __shared__ unsigned hist[256];
+    __shared__ unsigned sel_prefix, sel_remaining, sel_valid;
+    const int ns = min(p.n_sink, nb);
+    const int local_begin = max(nb - p.n_local, ns);
+    for (int h = 0; h < p.G; ++h) {
+        const float* v = p.bmax + (head0 + h) * p.max_blocks;
+        // m_tilde and the global maximum (NaN = bad page: fmaxf passes it over)
+        float mt = -INFINITY, gm = -INFINITY;
+        unsigned valid = 0;
+        for (int blk = tid; blk < nb; blk += kSelectThreads) {
+            const float x = v[blk];
+            gm = fmaxf(gm, x);
+            if (blk < ns || blk >= local_begin) mt = fmaxf(mt, x);
+            valid += x == x;
+        }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) {
+            mt = fmaxf(mt, __shfl_xor_sync(kFull, mt, o));
+            gm = fmaxf(gm, __shfl_xor_sync(kFull, gm, o));
+            valid += __shfl_xor_sync(kFull, valid, o);
+        }
+        __syncthreads();   // (the shared words of the previous head are no longer read)
+        if (lane == 0) { red_a[warp] = mt; red_b[warp] = gm; }
+        if (tid == 0) sel_valid = 0;
+        __syncthreads();
+        if (lane == 0) atomicAdd(&sel_valid, valid);
+#pragma unroll
+        for (int w = 0; w < kSelectThreads / 32; ++w) { mt = fmaxf(mt, red_a[w]); gm = fmaxf(gm, red_b[w]); }
+        if (tid == 0) p.mtilde[head0 + h] = mt;
+        float thr = (rule == kRuleGlobalMax ? gm : mt) - p.delta;   // delta = +inf: -inf, everything finite passes
+        if (rule == kRuleTopK) {
+            __syncthreads();
+            thr = -INFINITY;
+            if ((unsigned)top_k < sel_valid) {   // radix select of the k-th largest key, eight bits at a time
+                if (tid == 0) { sel_prefix = 0; sel_remaining = (unsigned)top_k; }
+                for (int shift = 24; shift >= 0; shift -= 8) {
+                    hist[tid] = 0;   // (kSelectThreads == 256 bins)
+                    __syncthreads();
+                    const unsigned prefix = sel_prefix;
+                    const unsigned high = shift == 24 ? 0u : 0xffffffffu << (shift + 8);
+                    for (int blk = tid; blk < nb; blk += kSelectThreads) {
+                        const float x = v[blk];
+                        if (x == x) {
+                            const uint32_t key = select_key(x);
+                            if ((key & high) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+                        }
+                    }
+                    __syncthreads();
+                    if (tid == 0) {
+                        unsigned left = sel_remaining;
+                        int bin = 255;
+                        for (; bin > 0 && hist[bin] < left; --bin) left -= hist[bin];
+                        sel_prefix = prefix | ((unsigned)bin << shift);
+                        sel_remaining = left;
+                    }
+                    __syncthreads();
+                }
+                thr = select_unkey(sel_prefix);
+            }
+        }
+        float carry = mt;   // rule 2: the reference before the current chunk
+        for (int base = 0; base < nb; base += kSelectThreads) {
+            const int blk = base + tid;
+            const float x = blk < nb ? v[blk] : __int_as_float(0x7fc00000);
+            float t = thr;
+            if (rule == kRuleRunningMax) {
+                float run = x == x ? x : -INFINITY;   // inclusive prefix maximum over the chunk
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const float y = __shfl_up_sync(kFull, run, o);
+                    if (lane >= o) run = fmaxf(run, y);
+                }
+                __syncthreads();
+                if (lane == 31) red_a[warp] = run;
+                __syncthreads();
+                float before = carry, total = carry;
+#pragma unroll
+                for (int w = 0; w < kSelectThreads / 32; ++w) {
+                    if (w < warp) before = fmaxf(before, red_a[w]);
+                    total = fmaxf(total, red_a[w]);
+                }
+                t = fmaxf(before, run) - p.delta;
+                carry = total;
+            }
+            if (blk < nb) {
+                const bool keep = x >= t;   // (NaN never passes)
+                const uint8_t old = h == 0 ? (uint8_t)0 : bits[blk];
+                bits[blk] = old | (uint8_t)((keep ? 1u : 0u) << h);
+                const size_t o = (head0 + h) * p.max_blocks + blk;
+                if (p.kept_mask) p.kept_mask[o] = keep ? 1 : 0;
+                if (p.block_max) p.block_max[o] = x;
+            }
+        }
     }
 }
 
@@ -935,8 +1106,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodePara
         if constexpr (BITS == 2) scan_setup(sq, q_group, p.G, lane, p.sm_scale);
         else if constexpr (BITS != 0) scan_setup_wide(sq, q_group, p.G, lane, p.sm_scale);
         constexpr size_t kCodeTile = BITS == 2 ? (size_t)kCodeBytes : (size_t)WideScan<BITS>::kTileBytes;
-        // BITS == 0: the block maxima come from the scan kernel that ran before this one (p.bmax)
-        const float* bmx = p.bmax + head0 * p.max_blocks;
+        // BITS == 0: the decisions come from the select kernel that ran before this one (p.keep_bits)
         // scan of one block, precise or fast.  2 bits: from the codes in registers, with the binary32 fallback when the
         // fp16 operand overflowed; deeper thumbnails: straight from global memory (an overflow there -- scales beyond
         // 30000 -- is reported and the block kept)
@@ -995,14 +1165,6 @@ __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodePara
                 return ref;
             };
             float best = -INFINITY;
-            if constexpr (BITS == 0) {   // every warp for itself: lane 4 r + j takes every eighth of the blocks for head j
-                if (j < p.G)
-                    for (int s = r; s < count; s += 8)
-                        best = fmaxf(best, bmx[(size_t)j * p.max_blocks + (s < ns ? s : local_begin + (s - ns))]);
-                best = fmaxf(best, __shfl_xor_sync(kFull, best, 4));
-                best = fmaxf(best, __shfl_xor_sync(kFull, best, 8));
-                best = fmaxf(best, __shfl_xor_sync(kFull, best, 16));
-            }
             BlockRef cur = ref_of(BITS == 0 ? count : warp);
             if constexpr (BITS != 2 && BITS != 0) {   // this warp's sink / local blocks on their way into L2 before the first is scanned
                 for (int s = warp; s < count; s += kWarps) {
@@ -1036,7 +1198,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodePara
 #pragma unroll
             for (int w = 0; w < kWarps; ++w) m = fmaxf(m, smax[w][j]);
             thr = m - p.delta;   // delta = +inf -> -inf: everything passes
-            if (split == 0 && warp == 0 && r == 0) p.mtilde[head0 + j] = m;
+            if (BITS != 0 && split == 0 && warp == 0 && r == 0) p.mtilde[head0 + j] = m;
         }
         attend_reset(st);
         attend_load_q(st.qa, q_group, p.G, lane);
@@ -1084,26 +1246,12 @@ __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodePara
             pending_keep = keep4;
         };
         if constexpr (BITS == 0) {
-            // Decisions from the stored maxima, 32 of the warp's blocks at a time (lane L looks at the L-th of them); only
-            // the kept ones cost a page lookup and a turn of the pipeline.
-            float thr_h[kMaxG];
-#pragma unroll
-            for (int h = 0; h < kMaxG; ++h) thr_h[h] = __shfl_sync(kFull, thr, h);
+            // The select kernel's decisions, 32 of the warp's blocks at a time (lane L looks at the L-th of them); only the
+            // kept ones cost a page lookup and a turn of the pipeline.
+            const uint8_t* bits = p.keep_bits + ((size_t)b * p.Hkv + g) * p.max_blocks;
             for (int base = blk_begin + warp; base < blk_end && ok; base += 32 * kWarps) {
                 const int mine = base + lane * kWarps;
-                unsigned k4 = 0;
-                if (mine < blk_end) {
-#pragma unroll
-                    for (int h = 0; h < kMaxG; ++h)
-                        if (h < p.G) {
-                            const float bm = bmx[(size_t)h * p.max_blocks + mine];
-                            const bool keep = bm >= thr_h[h];
-                            k4 |= (keep ? 1u : 0u) << h;
-                            const size_t o = (head0 + h) * p.max_blocks + mine;
-                            if (p.kept_mask) p.kept_mask[o] = keep ? 1 : 0;
-                            if (p.block_max) p.block_max[o] = bm;
-                        }
-                }
+                const unsigned k4 = mine < blk_end ? bits[mine] : 0u;
                 unsigned any = __ballot_sync(kFull, k4 != 0);
                 while (any && ok) {
                     const int src = __ffs(any) - 1;
@@ -1286,7 +1434,7 @@ struct Plan {
     int small_bps, small_splits;      // ... with these splits: at most one CTA per SM, never more splits than the dense path
     int wide_bps, wide_splits;        // the single-launch kernel on large geometries (deeper thumbnails): a few waves
     size_t off_arrive, off_mtilde, off_lens, off_units, off_qrec, off_ml, off_acc, off_fml, off_facc, total;
-    size_t off_bmax;
+    size_t off_bmax, off_keep;
     size_t off_scores, total_residual;   // 2 + 8 bit key format: the score tiles follow everything else
 };
 
@@ -1351,8 +1499,10 @@ static Plan make_plan(const ffd_config* cfg, int batch, int max_blocks, int sms)
     pl.off_fml = align_up(pl.off_acc + heads * pl.splits * kD * sizeof(float), 256);
     pl.off_facc = align_up(pl.off_fml + fslots * 2 * sizeof(float), 256);
     pl.total = align_up(pl.off_facc + fslots * kD * sizeof(float), 256);
-    pl.off_bmax = pl.total;   // deeper thumbnails only: the block maxima between the scan kernel and the decode kernel
-    if (cfg->quant_bits != 2) pl.total = align_up(pl.off_bmax + heads * (size_t)max_blocks * sizeof(float), 256);
+    // scan -> select -> decode: block maxima [B, Hq, max_blocks] and decision bytes [B, Hkv, max_blocks]
+    pl.off_bmax = pl.total;
+    pl.off_keep = align_up(pl.off_bmax + heads * (size_t)max_blocks * sizeof(float), 256);
+    pl.total = align_up(pl.off_keep + (size_t)units * max_blocks, 256);
     pl.off_scores = pl.total;
     pl.total_residual = pl.off_scores + (size_t)kResMaxCtas * kNB * kItemBlocksMax * kScoreTileFloats * sizeof(float);
     return pl;
@@ -1440,7 +1590,8 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
                              const int32_t* block_table, const int32_t* seq_lens, int batch, int max_blocks,
                              int num_pages, float delta, void* out, float* lse, uint8_t* kept_mask,
                              float* block_max, void* workspace, size_t workspace_bytes, void* stream,
-                             const AppendParams* append = nullptr, const void* k_res = nullptr) {
+                             const AppendParams* append = nullptr, const void* k_res = nullptr, int rule = -1,
+                             int top_k = 0) {   // rule >= 0: ffd_decode_select, always scan -> select -> decode
     const ffd_status st = check_decode_args(sparse, cfg, q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens,
                                             batch, max_blocks, num_pages, delta, out, lse, block_max, workspace, k_res);
     if (st) return st;
@@ -1486,6 +1637,7 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
     p.unit_list = reinterpret_cast<int2*>(ws + pl.off_units);
     p.res_scores = reinterpret_cast<float*>(ws + pl.off_scores);
     p.bmax = reinterpret_cast<float*>(ws + pl.off_bmax);
+    p.keep_bits = reinterpret_cast<uint8_t*>(ws + pl.off_keep);
     p.units = batch * cfg->num_kv_heads;
     const ItemGeom geom = item_geometry(p.units, max_blocks, sms);
     p.item_rows = geom.item_rows;
@@ -1509,14 +1661,13 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
         if (k_res && sms > kResMaxCtas) return FFD_ERR_UNSUPPORTED;
         // the work counters and class counts at ws + 64 are zero here: ffd_workspace_init zeroes them and the
         // combine kernel of every call leaves them zeroed for the next one (the kernels check the header's cookie)
-        // 4- / 8-bit thumbnails: the single-launch kernel on small geometries, a scan kernel followed by the same decode
-        // kernel on large ones
+        // 4- / 8-bit thumbnails: the single-launch kernel on small geometries, scan -> select -> decode on large ones;
+        // ffd_decode_select: scan -> select -> decode at every size and depth
         const bool deeper = cfg->quant_bits != 2;
-        if (deeper && (append || k_res)) return FFD_ERR_UNSUPPORTED;
-        if ((pl.small || deeper) && !append && !k_res) {   // little work: the whole step in one launch
-            // deeper thumbnails on a large geometry: the scan as a kernel of its own, then the same decode kernel taking
-            // its decisions from the stored block maxima
-            void (*kernel)(DecodeParams, uint32_t*) = !pl.small ? small_sparse_kernel<0>
+        if ((deeper || rule >= 0) && (append || k_res)) return FFD_ERR_UNSUPPORTED;
+        const bool three = rule >= 0 || (deeper && !pl.small);
+        if ((pl.small || three) && !append && !k_res) {   // little work: the whole step in one launch
+            void (*kernel)(DecodeParams, uint32_t*) = three ? small_sparse_kernel<0>
                                                       : cfg->quant_bits == 2 ? small_sparse_kernel<2>
                                                       : cfg->quant_bits == 4 ? small_sparse_kernel<4> : small_sparse_kernel<8>;
             if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem) != cudaSuccess)
@@ -1529,9 +1680,12 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
                 p.splits = pl.wide_splits;
             }
             if (prof) cudaEventRecord(g_prof_start, s);
-            if (!pl.small)
-                launch_pdl(cfg->quant_bits == 4 ? scan_blocks_kernel<4> : scan_blocks_kernel<8>,
-                           dim3((p.max_blocks + kScanCtaBlocks - 1) / kScanCtaBlocks, p.Hkv, batch), dim3(256), 0, s, p);
+            if (three) {
+                const dim3 scan_grid((p.max_blocks + kScanCtaBlocks - 1) / kScanCtaBlocks, p.Hkv, batch);
+                launch_pdl(cfg->quant_bits == 2 ? scan_blocks_kernel<2> : cfg->quant_bits == 4 ? scan_blocks_kernel<4> : scan_blocks_kernel<8>,
+                           scan_grid, dim3(256), 0, s, p);
+                launch_pdl(select_kernel, dim3(p.Hkv, batch), dim3(kSelectThreads), 0, s, p, rule < 0 ? (int)kRulePseudoMax : rule, top_k);
+            }
             launch_pdl(kernel, dim3(p.splits, p.Hkv, batch), dim3(kWarps * 32), kDecodeSmem, s, p,
                        reinterpret_cast<uint32_t*>(ws + pl.off_arrive));
             if (prof) cudaEventRecord(g_prof_stop, s);
@@ -1770,6 +1924,18 @@ ffd_status ffd_decode(const ffd_config* cfg, const void* q, const void* k_cache,
     return run_decode(true, cfg, q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, batch,
                       max_blocks_per_seq, num_pages, delta, out, lse, kept_mask, block_max, workspace,
                       workspace_bytes, stream);
+}
+
+ffd_status ffd_decode_select(const ffd_config* cfg, int32_t rule, int32_t top_k, const void* q, const void* k_cache,
+                             const void* v_cache, const void* k_quant, const void* k_scales, const int32_t* block_table,
+                             const int32_t* seq_lens, int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages,
+                             float delta, void* out, float* lse, uint8_t* kept_mask, float* block_max, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+    if (rule < FFD_RULE_PSEUDO_MAX || rule > FFD_RULE_TOP_K) return FFD_ERR_UNSUPPORTED;
+    if (rule == FFD_RULE_TOP_K && top_k < 1) return FFD_ERR_SHAPE;
+    return run_decode(true, cfg, q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens, batch,
+                      max_blocks_per_seq, num_pages, delta, out, lse, kept_mask, block_max, workspace,
+                      workspace_bytes, stream, nullptr, nullptr, rule, top_k);
 }
 
 ffd_status ffd_decode_residual(const ffd_config* cfg, const void* q, const void* k_res, const void* v_cache,

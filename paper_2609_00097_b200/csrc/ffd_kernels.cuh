@@ -86,7 +86,8 @@ struct DecodeParams {
     unsigned long long units_magic, hkv_magic;   // reciprocals for fast_div
     uint8_t* kept_mask;      // nullable [B, Hq, max_blocks]
     float* block_max;        // nullable [B, Hq, max_blocks]
-    float* bmax;             // deeper thumbnails on large geometries: [B, Hq, max_blocks] block maxima, scan kernel -> decode kernel (workspace)
+    float* bmax;             // scan kernel -> select kernel: [B, Hq, max_blocks] block maxima of the approximate logits (workspace)
+    uint8_t* keep_bits;      // select kernel -> decode kernel: [B, Hkv, max_blocks], bit h = head h of the group keeps the block (workspace)
     void* out;               // [B, Hq, 128] bf16 or fp32
     float* lse;              // nullable [B, Hq]
     int out_fp32;

@@ -29,7 +29,9 @@ DEV_BAD_WORKSPACE = 16
 EXPORTS = ["ffd_status_string", "ffd_workspace_bytes", "ffd_workspace_init", "ffd_quantize_keys", "ffd_decode",
            "ffd_decode_dense", "ffd_unpack_codes", "ffd_read_device_status", "ffd_profile_events", "ffd_decode_static",
            "ffd_append_kv", "ffd_append_decode", "ffd_quantize_residual", "ffd_decode_residual", "ffd_workspace_bytes_residual",
-           "ffd_quantize_keys_residual", "ffd_append_kv_residual"]
+           "ffd_quantize_keys_residual", "ffd_append_kv_residual", "ffd_decode_select"]
+
+RULE_PSEUDO_MAX, RULE_GLOBAL_MAX, RULE_RUNNING_MAX, RULE_TOP_K = 0, 1, 2, 3
 
 
 class FfdError(RuntimeError):
@@ -210,6 +212,17 @@ def ffd_decode(cfg: Config, q, k_cache, v_cache, k_quant, k_scales, block_table,
                                      _p(k_scales), _p(block_table), _p(seq_lens), q.shape[0], max_blocks_per_seq,
                                      k_cache.shape[0], ctypes.c_float(delta), _p(out), _p(lse), _p(kept_mask),
                                      _p(block_max), _p(workspace), workspace.numel(), _stream(stream)), "ffd_decode")
+
+
+def ffd_decode_select(cfg: Config, rule: int, top_k: int, q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens,
+                      delta: float, out, *, max_blocks_per_seq: int, workspace, lse=None, kept_mask=None, block_max=None,
+                      stream=None):
+    """ffd_decode under one of the comparison selection rules (RULE_*), as scan, select and decode kernels."""
+    _check(load_library().ffd_decode_select(ctypes.byref(cfg.c()), int(rule), int(top_k), _p(q), _p(k_cache), _p(v_cache),
+                                            _p(k_quant), _p(k_scales), _p(block_table), _p(seq_lens), q.shape[0],
+                                            max_blocks_per_seq, k_cache.shape[0], ctypes.c_float(delta), _p(out), _p(lse),
+                                            _p(kept_mask), _p(block_max), _p(workspace), workspace.numel(),
+                                            _stream(stream)), "ffd_decode_select")
 
 
 def ffd_append_decode(cfg: Config, k_new, v_new, q, k_cache, v_cache, k_quant, k_scales, block_table, seq_lens,

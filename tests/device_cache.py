@@ -8,7 +8,7 @@ from __future__ import annotations
 import torch
 
 from paper_2609_00097_b200.ffd import (Config, ffd_append_decode, ffd_append_kv, ffd_append_kv_residual, ffd_decode,
-                                        ffd_decode_dense, ffd_decode_residual, ffd_quantize_keys,
+                                        ffd_decode_dense, ffd_decode_residual, ffd_decode_select, ffd_quantize_keys,
                                         ffd_quantize_keys_residual, ffd_quantize_residual, ffd_unpack_codes,
                                         new_workspace)
 
@@ -81,6 +81,11 @@ class DeviceCache:
         ffd_decode(self.cfg, self.q, self.k_cache, self.v_cache, self.k_quant, self.k_scales, self.block_table,
                    self.seq_lens, delta, self.out, max_blocks_per_seq=self.w.max_blocks, workspace=self.workspace,
                    lse=self.lse, kept_mask=kept_mask, block_max=block_max)
+
+    def decode_select(self, rule, top_k, delta, kept_mask=None, block_max=None):
+        ffd_decode_select(self.cfg, rule, top_k, self.q, self.k_cache, self.v_cache, self.k_quant, self.k_scales,
+                          self.block_table, self.seq_lens, delta, self.out, max_blocks_per_seq=self.w.max_blocks,
+                          workspace=self.workspace, lse=self.lse, kept_mask=kept_mask, block_max=block_max)
 
     def dense(self):
         ffd_decode_dense(self.cfg, self.q, self.k_cache, self.v_cache, self.block_table, self.seq_lens, self.out,

@@ -76,10 +76,13 @@ def magnitude(r, w):
     return max(1.0, float(np.abs(finite).max()) / 64.0) if finite.size else 1.0
 
 
-def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None, k_res=None, expect_status=0):
-    """k_res (the oracle's residuals): check the 2 + 8 bit format's decode against the oracle's Dequant refinement."""
+def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None, k_res=None, expect_status=0, rule=None, top_k=0):
+    """k_res (the oracle's residuals): check the 2 + 8 bit format's decode against the oracle's Dequant refinement.
+    rule: check ffd_decode_select under that selection rule against the oracle run with the same rule."""
     B, Hq, mb = w.B, w.Hq, w.max_blocks
     gpu_decode = dc.decode if k_res is None else dc.decode_residual
+    if rule is not None:
+        gpu_decode = lambda delta, **kw: dc.decode_select(rule, top_k, delta, **kw)
     kept = torch.full((B, Hq, mb), 255, dtype=torch.uint8, device="cuda")
     bm = torch.full((B, Hq, mb), float("nan"), dtype=torch.float32, device="cuda")
     # without the block-max debug output the kernel may skip the tensor-core work of blocks whose scale-only upper
@@ -98,7 +101,7 @@ def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None, k_res=Non
     bm = bm.cpu().numpy().astype(np.float64)
     r = oracle.decode(w.bits("q"), w.bits("k_cache"), w.bits("v_cache"), codes, scales, w.block_table, w.seq_lens,
                       mb, delta, n_sink=dc.cfg.n_sink_blocks, n_local=dc.cfg.n_local_blocks, units=units, k_res=k_res,
-                      bits=dc.cfg.quant_bits)
+                      bits=dc.cfg.quant_bits, rule=rule or 0, top_k=top_k)
     rows = units if units is not None else [(b, h) for b in range(B) for h in range(Hq)]
     mag = magnitude(r, w)
     differs = False
@@ -123,7 +126,7 @@ def check_decode(ffd, oracle, w, dc, codes, scales, delta, units=None, k_res=Non
         diff = kept[b, hs, :nb] != r.kept[b, hs, :nb]
         if diff.any():
             differs = True
-            margin = np.abs(want_bm - (r.mtilde[b, hs, None] - delta))
+            margin = np.abs(want_bm - r.thr[b, hs, :nb])   # (m_tilde - delta under the paper's rule)
             assert np.all(margin[diff] < MASK_BAND * mag), (b, np.where(diff), margin[diff])
     if differs:   # compare the output against the oracle's attention over the GPU's (equally valid) mask
         forced = np.where(kept == 255, 0, kept).astype(np.uint8)
@@ -790,6 +793,62 @@ def test_full_size_configs_every_row(ffd, oracle, name):
             check_decode(ffd, oracle, w, dc, codes, scales, w.deltas[0], k_res=k_res)
     finally:
         oracle.set_threads(min(8, oracle.max_threads()))
+
+
+RULE_CASES = [
+    ("C1", dict()), ("C4", dict(N=16384)), ("C5", dict(B=4, lens=(1000, 5000))), ("C5", dict(B=20, lens=(300, 1500))),
+    ("C2", dict(N=6000, sink=False)), ("C3", dict(N=8192, B=8)),
+]
+
+
+@pytest.mark.parametrize("name,kw", RULE_CASES)
+def test_selection_rules_against_the_oracle(ffd, oracle, name, kw):
+    """ffd_decode_select (scan, select and decode as three kernels) under each rule against the oracle under the same
+    rule: masks (blocks within 1e-4 of their own threshold may differ), block maxima, outputs.  The pseudo-max rule through
+    this path must also reproduce ffd_decode's decisions."""
+    w = make_workload(name, **kw)
+    dc = DeviceCache(w)
+    codes, scales = check_quantize(ffd, oracle, w, dc)
+    delta = w.deltas[0]
+    for rule in (ffd.RULE_PSEUDO_MAX, ffd.RULE_GLOBAL_MAX, ffd.RULE_RUNNING_MAX):
+        check_decode(ffd, oracle, w, dc, codes, scales, delta, rule=rule)
+        check_decode(ffd, oracle, w, dc, codes, scales, 0.5, rule=rule)
+    check_decode(ffd, oracle, w, dc, codes, scales, INF, rule=ffd.RULE_RUNNING_MAX)
+    for k in (1, 7, 10 ** 6):
+        check_decode(ffd, oracle, w, dc, codes, scales, delta, rule=ffd.RULE_TOP_K, top_k=k)
+    a = torch.full((w.B, w.Hq, w.max_blocks), 255, dtype=torch.uint8, device="cuda")
+    b = a.clone()
+    dc.decode(delta, kept_mask=a)
+    out = dc.out.clone()
+    dc.decode_select(ffd.RULE_PSEUDO_MAX, 0, delta, kept_mask=b)
+    assert torch.equal(a, b) and (dc.out - out).abs().max().item() < 2e-5
+
+
+def test_selection_rules_full_size_and_deeper_thumbnails(ffd, oracle):
+    """The running-max and top-k rules at the benchmark's C4 size, and the rules on 4-bit thumbnails."""
+    oracle.set_threads(oracle.max_threads())
+    try:
+        w = make_workload("C4")
+        dc = DeviceCache(w)
+        codes, scales = check_quantize(ffd, oracle, w, dc)
+        check_decode(ffd, oracle, w, dc, codes, scales, 6.0, rule=ffd.RULE_RUNNING_MAX)
+        check_decode(ffd, oracle, w, dc, codes, scales, 6.0, rule=ffd.RULE_TOP_K, top_k=53)
+        w = make_workload("C5", B=8, lens=(3000, 9000))
+        dc = DeviceCache(w, ffd.Config(w.Hq, w.Hkv, quant_bits=4))
+        codes, scales = check_quantize(ffd, oracle, w, dc)
+        for rule, k in ((ffd.RULE_GLOBAL_MAX, 0), (ffd.RULE_RUNNING_MAX, 0), (ffd.RULE_TOP_K, 9)):
+            check_decode(ffd, oracle, w, dc, codes, scales, 6.0, rule=rule, top_k=k)
+    finally:
+        oracle.set_threads(min(8, oracle.max_threads()))
+
+
+def test_select_rejects_bad_rules(ffd, oracle):
+    w = make_workload("C1")
+    dc = DeviceCache(w)
+    dc.quantize()
+    for rule, k in ((4, 0), (-1, 0), (ffd.RULE_TOP_K, 0)):
+        with pytest.raises(ffd.FfdError):
+            dc.decode_select(rule, k, 6.0)
 
 
 @pytest.mark.parametrize("name,bits", [("C3", 4), ("C5", 4), ("C4", 8), ("C5", 8)])
