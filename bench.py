@@ -339,6 +339,44 @@ def depth_table(ffd, peak, steps):
             "rows": rows}
 
 
+def selection_table(ffd, w, delta, steps):
+    """Sec. 4.4 "Selection-Rule Overhead": the decode call under each selection rule at a matched keep ratio (top-k's k is
+    the mean number of blocks a head keeps under top-delta), all through ffd_decode_select's three kernels (scan, select,
+    decode), cold L2; the fused ffd_decode call beside them.  What differs between the rows is the select kernel (one
+    reduction more for the global max, a prefix scan for the running max, a four-pass radix select for top-k) and the
+    blocks each rule keeps."""
+    b = Bench(ffd, w, delta)
+    dc = b.dc
+    kept = torch.zeros(w.B, w.Hq, w.max_blocks, dtype=torch.uint8, device="cuda")
+    dc.decode(delta, kept_mask=kept)
+    k_match = max(1, round(b.kept_head_blocks / (w.B * w.Hq)))
+    rows = []
+
+    def measure(name, fn, mask_fn):
+        kept.zero_()
+        mask_fn(kept)
+        torch.cuda.synchronize()
+        frac = sum(int(kept[i, :, : w.num_blocks(i)].sum()) for i in range(w.B)) / b.head_blocks
+        loaded = union_kept_tiles(kept.cpu().numpy(), w) / b.total_tiles
+        b.timed_loop(fn, 3)
+        us, _ = b.timed_loop(fn, steps)
+        _, kus = b.timed_loop(fn, max(steps, 20), profile_kernel=True)
+        rows.append({"rule": name, "keep_ratio_per_head": frac, "loaded_fraction_of_kv_tiles": loaded,
+                     "decode_us": statistics.mean(us),
+                     "decode_us_median": statistics.median(us), "kernels_us": statistics.mean(kus)})
+
+    measure("top-delta, fused kernel (ffd_decode)", lambda: dc.decode(delta), lambda m: dc.decode(delta, kept_mask=m))
+    for name, rule, k in (("top-delta (pseudo-max)", ffd.RULE_PSEUDO_MAX, 0), ("global max", ffd.RULE_GLOBAL_MAX, 0),
+                          ("running max", ffd.RULE_RUNNING_MAX, 0), (f"top-k, k = {k_match}", ffd.RULE_TOP_K, k_match)):
+        measure(name, lambda r=rule, kk=k: dc.decode_select(r, kk, delta),
+                lambda m, r=rule, kk=k: dc.decode_select(r, kk, delta, kept_mask=m))
+    base = rows[1]["decode_us"]
+    for r in rows[1:]:
+        r["extra_us_vs_top_delta_same_path"] = r["decode_us"] - base
+        r["extra_us_per_head"] = (r["decode_us"] - base) / (w.B * w.Hq)
+    return {"workload": workload_config(w, delta, None)["workload"], "matched_k": k_match, "rows": rows}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -513,6 +551,7 @@ def main():
             torch.cuda.empty_cache()
         line["extra"] = extra
         line["quantization_depth"] = depth_table(ffd, peak, min(args.steps, 30))
+        line["selection_rules"] = selection_table(ffd, w, delta, min(args.steps, 30))
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(w, delta)
         one = cpu_baseline(w, delta, threads=1, rows_per_thread=8)

@@ -927,14 +927,15 @@ __global__ void __launch_bounds__(256, 2) scan_blocks_kernel(DecodeParams p) {
 }
 
 // ---- select: the rule that turns block maxima into decisions ----------------------------------------------------
-// One CTA per (sequence, KV head); the heads of the group one after the other.  Rules (ffd.h FFD_RULE_*):
+// One CTA per (sequence, query head).  Rules (ffd.h FFD_RULE_*):
 //   0 pseudo-max     keep = bm >= m_tilde - delta, m_tilde over the sink and local blocks (Alg. 1, Eq. 1)
 //   1 global max     keep = bm >= max over all blocks - delta (the comparison rule of Sec. 5.2: a reduction of its own)
 //   2 running max    keep = bm >= max(m_tilde, bm of blocks 0 .. blk) - delta: what a streaming scan in logical block
 //                    order knows when it meets the block
 //   3 top-k          keep = bm >= the k-th largest block maximum (Fig. 1a's fixed budget; ties kept): a radix select,
 //                    four passes over the head's maxima
-// Writes keep_bits (bit h of a block's byte = head h keeps it), m_tilde, and the kept_mask / block_max outputs.
+// Writes keep_bits (one byte per (block, head of the group), the bytes of a block side by side), m_tilde, and the
+// kept_mask / block_max outputs.
 constexpr int kSelectThreads = 256;
 enum : int { kRulePseudoMax = 0, kRuleGlobalMax = 1, kRuleRunningMax = 2, kRuleTopK = 3 };
 
@@ -947,24 +948,26 @@ __device__ __forceinline__ float select_unkey(uint32_t k) {
 }
 
 __global__ void __launch_bounds__(kSelectThreads) select_kernel(DecodeParams p, int rule, int top_k) {
-    const int g = blockIdx.x, b = blockIdx.y;
+    const int head = blockIdx.x, b = blockIdx.y;
+    const int g = head / p.G, h = head % p.G;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     pdl_launch_dependents();
     pdl_wait();
     const int n = clamped_seq_len(p, b);
     const int nb = (n + kBlk - 1) / kBlk;
     const size_t head0 = (size_t)b * p.Hq + (size_t)g * p.G;
-    uint8_t* bits = p.keep_bits + ((size_t)b * p.Hkv + g) * p.max_blocks;
+    uint8_t* bits = p.keep_bits + ((size_t)b * p.Hkv + g) * p.max_blocks * kMaxG + h;
     __shared__ float red_a[kSelectThreads / 32], red_b[kSelectThreads / 32];
     __shared__ unsigned hist[256];
     __shared__ unsigned sel_prefix, sel_remaining, sel_valid;
     const int ns = min(p.n_sink, nb);
     const int local_begin = max(nb - p.n_local, ns);
-    for (int h = 0; h < p.G; ++h) {
+    {
         const float* v = p.bmax + (head0 + h) * p.max_blocks;
         // m_tilde and the global maximum (NaN = bad page: fmaxf passes it over)
         float mt = -INFINITY, gm = -INFINITY;
         unsigned valid = 0;
+#pragma unroll 4
         for (int blk = tid; blk < nb; blk += kSelectThreads) {
             const float x = v[blk];
             gm = fmaxf(gm, x);
@@ -977,7 +980,6 @@ __global__ void __launch_bounds__(kSelectThreads) select_kernel(DecodeParams p, 
             gm = fmaxf(gm, __shfl_xor_sync(kFull, gm, o));
             valid += __shfl_xor_sync(kFull, valid, o);
         }
-        __syncthreads();   // (the shared words of the previous head are no longer read)
         if (lane == 0) { red_a[warp] = mt; red_b[warp] = gm; }
         if (tid == 0) sel_valid = 0;
         __syncthreads();
@@ -1042,8 +1044,7 @@ __global__ void __launch_bounds__(kSelectThreads) select_kernel(DecodeParams p, 
             }
             if (blk < nb) {
                 const bool keep = x >= t;   // (NaN never passes)
-                const uint8_t old = h == 0 ? (uint8_t)0 : bits[blk];
-                bits[blk] = old | (uint8_t)((keep ? 1u : 0u) << h);
+                bits[(size_t)blk * kMaxG] = keep ? 1 : 0;
                 const size_t o = (head0 + h) * p.max_blocks + blk;
                 if (p.kept_mask) p.kept_mask[o] = keep ? 1 : 0;
                 if (p.block_max) p.block_max[o] = x;
@@ -1248,10 +1249,13 @@ __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodePara
         if constexpr (BITS == 0) {
             // The select kernel's decisions, 32 of the warp's blocks at a time (lane L looks at the L-th of them); only the
             // kept ones cost a page lookup and a turn of the pipeline.
-            const uint8_t* bits = p.keep_bits + ((size_t)b * p.Hkv + g) * p.max_blocks;
+            static_assert(kMaxG == 4, "one 32-bit word of decision bytes per block");
+            const uint32_t* bits = reinterpret_cast<const uint32_t*>(p.keep_bits) + ((size_t)b * p.Hkv + g) * p.max_blocks;
+            const uint32_t group_mask = p.G >= 4 ? 0x01010101u : (1u << (8 * p.G)) - 1u & 0x01010101u;   // (bytes of absent heads are never written)
             for (int base = blk_begin + warp; base < blk_end && ok; base += 32 * kWarps) {
                 const int mine = base + lane * kWarps;
-                const unsigned k4 = mine < blk_end ? bits[mine] : 0u;
+                const uint32_t word = mine < blk_end ? bits[mine] & group_mask : 0u;
+                const unsigned k4 = (word & 1u) | ((word >> 7) & 2u) | ((word >> 14) & 4u) | ((word >> 21) & 8u);
                 unsigned any = __ballot_sync(kFull, k4 != 0);
                 while (any && ok) {
                     const int src = __ffs(any) - 1;
@@ -1499,10 +1503,10 @@ static Plan make_plan(const ffd_config* cfg, int batch, int max_blocks, int sms)
     pl.off_fml = align_up(pl.off_acc + heads * pl.splits * kD * sizeof(float), 256);
     pl.off_facc = align_up(pl.off_fml + fslots * 2 * sizeof(float), 256);
     pl.total = align_up(pl.off_facc + fslots * kD * sizeof(float), 256);
-    // scan -> select -> decode: block maxima [B, Hq, max_blocks] and decision bytes [B, Hkv, max_blocks]
+    // scan -> select -> decode: block maxima [B, Hq, max_blocks] and decision bytes [B, Hkv, max_blocks, 4]
     pl.off_bmax = pl.total;
     pl.off_keep = align_up(pl.off_bmax + heads * (size_t)max_blocks * sizeof(float), 256);
-    pl.total = align_up(pl.off_keep + (size_t)units * max_blocks, 256);
+    pl.total = align_up(pl.off_keep + (size_t)units * max_blocks * kMaxG, 256);
     pl.off_scores = pl.total;
     pl.total_residual = pl.off_scores + (size_t)kResMaxCtas * kNB * kItemBlocksMax * kScoreTileFloats * sizeof(float);
     return pl;
@@ -1684,7 +1688,7 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
                 const dim3 scan_grid((p.max_blocks + kScanCtaBlocks - 1) / kScanCtaBlocks, p.Hkv, batch);
                 launch_pdl(cfg->quant_bits == 2 ? scan_blocks_kernel<2> : cfg->quant_bits == 4 ? scan_blocks_kernel<4> : scan_blocks_kernel<8>,
                            scan_grid, dim3(256), 0, s, p);
-                launch_pdl(select_kernel, dim3(p.Hkv, batch), dim3(kSelectThreads), 0, s, p, rule < 0 ? (int)kRulePseudoMax : rule, top_k);
+                launch_pdl(select_kernel, dim3(p.Hq, batch), dim3(kSelectThreads), 0, s, p, rule < 0 ? (int)kRulePseudoMax : rule, top_k);
             }
             launch_pdl(kernel, dim3(p.splits, p.Hkv, batch), dim3(kWarps * 32), kDecodeSmem, s, p,
                        reinterpret_cast<uint32_t*>(ws + pl.off_arrive));

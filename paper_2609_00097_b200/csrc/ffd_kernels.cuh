@@ -87,7 +87,7 @@ struct DecodeParams {
     uint8_t* kept_mask;      // nullable [B, Hq, max_blocks]
     float* block_max;        // nullable [B, Hq, max_blocks]
     float* bmax;             // scan kernel -> select kernel: [B, Hq, max_blocks] block maxima of the approximate logits (workspace)
-    uint8_t* keep_bits;      // select kernel -> decode kernel: [B, Hkv, max_blocks], bit h = head h of the group keeps the block (workspace)
+    uint8_t* keep_bits;      // select kernel -> decode kernel: [B, Hkv, max_blocks, 4] bytes, byte h = head h of the group keeps the block (workspace)
     void* out;               // [B, Hq, 128] bf16 or fp32
     float* lse;              // nullable [B, Hq]
     int out_fp32;
