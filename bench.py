@@ -309,13 +309,13 @@ class Bench:
                 "fidelity": self.fidelity()}
 
 
-def depth_table(ffd, peak, steps):
+def depth_table(ffd, peak, steps, batch=4, context=131072):
     """App. "Bandwidth Proportionality of Quantization Depth": the scan at 2, 4 and 8 bits on one scan-only workload
     (sink needle in every head, delta 0: a handful of blocks kept), decode call alone (no tail re-quantize), cold L2.
     kernel_us brackets the scan-select-attend kernel(s) of the call: the fused kernel at 2 bits, the scan kernel plus the
     decode kernel at 4 and 8 bits."""
     rows = []
-    w = make_workload("C2", N=131072, B=4)
+    w = make_workload("C2", N=context, B=batch)
     tiles = sum(w.num_blocks(b) for b in range(w.B)) * w.Hkv
     for bits in (2, 4, 8):
         b = Bench(ffd, w, 0.0, bits=bits)
@@ -335,7 +335,7 @@ def depth_table(ffd, peak, steps):
     for r in rows:
         r["bytes_ratio_vs_2bit"] = r["scan_bytes"] / base["scan_bytes"]
         r["kernel_time_ratio_vs_2bit"] = r["kernel_us"]["mean"] / base["kernel_us"]["mean"]
-    return {"workload": "C2 recipe at batch 4, context 131072 (32 query / 8 KV heads), delta 0, decode call only",
+    return {"workload": f"C2 recipe at batch {batch}, context {context} (32 query / 8 KV heads), delta 0, decode call only",
             "rows": rows}
 
 
@@ -388,6 +388,10 @@ def main():
     ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--delta", type=float, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--table", default=None, choices=["depth", "selection"],
+                    help="print only the quantization-depth table (C2 recipe at --batch / --context, defaults 4 / 131072) or "
+                         "the selection-rule table (on --workload) as JSON and exit: small cases of them are what the ncu "
+                         "captures of the scan and select kernels run")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the secondary workloads (C4, C5) and the quantization-depth table of the bench line")
     args = ap.parse_args()
@@ -409,8 +413,14 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
+    if args.table == "depth":
+        print(json.dumps(depth_table(ffd, measured_peaks()[0], args.steps, args.batch or 4, args.context or 131072)), flush=True)
+        return
     w = make_workload(args.workload, **workload_overrides(args))
     delta = args.delta if args.delta is not None else w.deltas[0]
+    if args.table == "selection":
+        print(json.dumps(selection_table(ffd, w, delta, args.steps)), flush=True)
+        return
     bench = Bench(ffd, w, delta)
     dc, step, timed_loop = bench.dc, bench.step, bench.timed_loop
 

@@ -26,7 +26,12 @@
  *                                                            NULL = page b*max_blocks_per_seq + blk
  *       seq_lens int32 [batch]                               tokens in each sequence (0 allowed)
  *     Token t of sequence b lives in logical block t/64, row t%64.  Query head h uses KV head
- *     h / (num_q_heads / num_kv_heads).
+ *     h / (num_q_heads / num_kv_heads).  Group sizes G = num_q_heads / num_kv_heads: 1, 2, 3, 4, and also 6 and 8 in
+ *     ffd_workspace_bytes, ffd_workspace_init, ffd_quantize_keys, ffd_unpack_codes, ffd_decode, ffd_decode_dense and
+ *     ffd_decode_select.  A KV head with 6 or 8 query heads is served as two groups of 3 or 4 heads that read the same
+ *     tiles, so its codes and kept K/V tiles are read twice (same results as a kernel with wider fragments would give,
+ *     twice the traffic); the other entry points return FFD_ERR_UNSUPPORTED for G > 4, every entry point for G = 5, 7
+ *     and G > 8.
  *   - Physical order of k_quant: a (page, head) tile is 4 groups of 16 tokens, 512 bytes each.  Inside a
  *     group, 32 lanes own 16 bytes each: lane = 4*r + j holds 32-bit words W0..W3 for tokens r (W0, W2)
  *     and r+8 (W1, W3) of the group.  Bits [2i+1:2i] of the low / high half of W0 (W1) hold the codes of
@@ -63,7 +68,8 @@ typedef enum {
     FFD_ERR_NULL = 1,          /* a required pointer is NULL */
     FFD_ERR_SHAPE = 2,         /* batch / heads / block counts out of range */
     FFD_ERR_UNSUPPORTED = 3,   /* head_dim != 128, block_tokens != 64, quant_bits not 2, 4 or 8 (or not 2 where the entry
-                                  point needs the 2-bit thumbnails), group size not 1..4 ... */
+                                  point needs the 2-bit thumbnails), group size not 1..4 (6 and 8 where the
+                                  conventions above say so) ... */
     FFD_ERR_ALIGN = 4,         /* a device pointer is not 16-byte aligned */
     FFD_ERR_WORKSPACE = 5,     /* workspace smaller than ffd_workspace_bytes reports */
     FFD_ERR_DELTA = 6,         /* delta is NaN or negative */

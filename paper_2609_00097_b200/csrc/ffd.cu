@@ -538,7 +538,7 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
             tail_blk = pos / kBlk;
             if (tid < kD) {   // warps 0..3 append and re-quantize while the other warps already scan
                 const int row = pos % kBlk;
-                const size_t tile = (size_t)page * p.Hkv + g;
+                const size_t tile = tile_index(p, page, g);
                 const size_t unit = (size_t)b * p.Hkv + g;
                 const __nv_bfloat16 kn = ap.k_new[unit * kD + tid];
                 ap.v_cache[(tile * kBlk + row) * kD + tid] = ap.v_new[unit * kD + tid];
@@ -609,7 +609,7 @@ __global__ void __launch_bounds__(kPmWarps * 32) pseudomax_kernel(DecodeParams p
                                : (s < ns ? s : local_begin + (s - ns));
         const int page = page_of(p, b, blk);
         if (page < 0) continue;
-        const size_t tile = (size_t)page * p.Hkv + g;
+        const size_t tile = tile_index(p, page, g);
         const int rows = min(kBlk, n - blk * kBlk);
         float band;
         ScanRegs sr;
@@ -734,7 +734,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) dense_kernel(DecodeParams p) {
             if (page < 0) continue;
             ref.blk = blk;
             ref.rows = min(kBlk, n - blk * kBlk);
-            ref.tile = (size_t)page * p.Hkv + g;
+            ref.tile = tile_index(p, page, g);
             return ref;
         }
     };
@@ -850,7 +850,7 @@ __global__ void __launch_bounds__(256, 2) scan_blocks_kernel(DecodeParams p) {
     };
     auto prefetch = [&](int page) {
         if (page >= 0 && page < p.num_pages) {
-            const size_t tile = (size_t)page * p.Hkv + g;
+            const size_t tile = tile_index(p, page, g);
             wide_prefetch_l2<BITS>(p.k_quant + tile * WideScan<BITS>::kTileBytes, p.k_scales + tile * kD, lane);
         }
     };
@@ -861,7 +861,7 @@ __global__ void __launch_bounds__(256, 2) scan_blocks_kernel(DecodeParams p) {
         auto tile_of = [&](int blk) -> long long {
             if (blk >= last) return -1;
             const int page = page_of(p, b, blk);
-            return page < 0 ? -1 : (long long)page * p.Hkv + g;
+            return page < 0 ? -1 : (long long)tile_index(p, page, g);
         };
         auto load = [&](ScanRegs& sr, long long tile) {
             if (tile >= 0)
@@ -908,7 +908,7 @@ __global__ void __launch_bounds__(256, 2) scan_blocks_kernel(DecodeParams p) {
         const int after = blk + 16 < last ? raw_page(blk + 16) : -1;   // (read now, used for the hint one turn later)
         float bm = __int_as_float(0x7fc00000);
         if (page >= 0 && page < p.num_pages) {
-            const size_t tile = (size_t)page * p.Hkv + g;
+            const size_t tile = tile_index(p, page, g);
             float band;
             bm = scan_wide<BITS, true>(p.k_quant + tile * WideScan<BITS>::kTileBytes, p.k_scales + tile * kD, sq, lane,
                                        min(kBlk, n - blk * kBlk), band);
@@ -1006,12 +1006,25 @@ __global__ void __launch_bounds__(kSelectThreads) select_kernel(DecodeParams p, 
                         }
                     }
                     __syncthreads();
-                    if (tid == 0) {
-                        unsigned left = sel_remaining;
-                        int bin = 255;
-                        for (; bin > 0 && hist[bin] < left; --bin) left -= hist[bin];
-                        sel_prefix = prefix | ((unsigned)bin << shift);
-                        sel_remaining = left;
+                    if (warp == 0) {   // lane L owns bins 8 L .. 8 L + 7; the k-th largest is counted from the top bin down
+                        unsigned c[8], mine = 0;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) { c[i] = hist[8 * lane + i]; mine += c[i]; }
+                        unsigned incl = mine;   // keys in this lane's bins and in all higher ones
+#pragma unroll
+                        for (int o = 1; o < 32; o <<= 1) {
+                            const unsigned y = __shfl_down_sync(kFull, incl, o);
+                            if (lane + o < 32) incl += y;
+                        }
+                        const unsigned above = incl - mine, left = sel_remaining;
+                        __syncwarp();
+                        if (above < left && left <= incl) {   // exactly one lane
+                            unsigned l = left - above;
+                            int i = 7;
+                            for (; i > 0 && c[i] < l; --i) l -= c[i];
+                            sel_prefix = prefix | ((unsigned)(8 * lane + i) << shift);
+                            sel_remaining = l;
+                        }
                     }
                     __syncthreads();
                 }
@@ -1144,7 +1157,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodePara
         };
         auto prefetch_page = [&](int page) {
             if (page >= 0 && page < p.num_pages) {
-                const size_t tile = (size_t)page * p.Hkv + g;
+                const size_t tile = tile_index(p, page, g);
                 wide_prefetch_l2<BITS>(p.k_quant + tile * kCodeTile, p.k_scales + tile * kD, lane);
             }
         };
@@ -1161,7 +1174,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodePara
                 if (s < count) {
                     const int blk = s < ns ? s : local_begin + (s - ns);
                     const int page = page_of(p, b, blk);
-                    if (page >= 0) { ref.blk = blk; ref.rows = min(kBlk, n - blk * kBlk); ref.tile = (size_t)page * p.Hkv + g; }
+                    if (page >= 0) { ref.blk = blk; ref.rows = min(kBlk, n - blk * kBlk); ref.tile = tile_index(p, page, g); }
                 }
                 return ref;
             };
@@ -1220,7 +1233,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodePara
                 if (page < 0) continue;
                 ref.blk = blk;
                 ref.rows = min(kBlk, n - blk * kBlk);
-                ref.tile = (size_t)page * p.Hkv + g;
+                ref.tile = tile_index(p, page, g);
                 return ref;
             }
         };
@@ -1264,7 +1277,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodePara
                     const int blk = base + src * kWarps;
                     const int page = page_of(p, b, blk);
                     if (page < 0) continue;
-                    consume(BlockRef{blk, min(kBlk, n - blk * kBlk), (size_t)page * p.Hkv + g}, keep4);
+                    consume(BlockRef{blk, min(kBlk, n - blk * kBlk), tile_index(p, page, g)}, keep4);
                 }
             }
         }
@@ -1466,9 +1479,19 @@ static int device_sms() {
     return sms;
 }
 
+// Query heads per KV head: 1..4 directly; 6 and 8 as two groups of 3 or 4 heads that share the KV head's tiles (each
+// tile is then read once per group: correct, at twice the scan and K/V traffic of a kernel with wider fragments).
+static int group_shift(const ffd_config* cfg) {
+    const int G = cfg->num_q_heads / cfg->num_kv_heads;
+    return (G == 6 || G == 8) ? 1 : 0;
+}
+
 // Split geometry is a pure function of (batch, KV heads, max blocks, SM count) so that ffd_workspace_bytes and the
 // launch agree.  Aim for at least two CTAs per SM before making splits longer than 8 blocks.
-static Plan make_plan(const ffd_config* cfg, int batch, int max_blocks, int sms) {
+static Plan make_plan(const ffd_config* user_cfg, int batch, int max_blocks, int sms) {
+    ffd_config v = *user_cfg;   // the geometry is that of the groups the kernels work on (group_shift)
+    v.num_kv_heads <<= group_shift(user_cfg);
+    const ffd_config* cfg = &v;
     Plan pl;
     int bps = 32;
     const long units = (long)batch * cfg->num_kv_heads;
@@ -1512,13 +1535,14 @@ static Plan make_plan(const ffd_config* cfg, int batch, int max_blocks, int sms)
     return pl;
 }
 
-// two_bit_only: the entry point exists for the 2-bit thumbnails only (the 2 + 8 bit format, the device-side append)
-static ffd_status check_config(const ffd_config* cfg, bool two_bit_only = false) {
+// two_bit_only: the entry point exists for the 2-bit thumbnails only (the 2 + 8 bit format, the device-side append);
+// wide_groups: it also serves 6 and 8 query heads per KV head
+static ffd_status check_config(const ffd_config* cfg, bool two_bit_only = false, bool wide_groups = false) {
     if (!cfg) return FFD_ERR_NULL;
     if (cfg->head_dim != kD || cfg->block_tokens != kBlk) return FFD_ERR_UNSUPPORTED;
     if (cfg->quant_bits != 2 && (two_bit_only || (cfg->quant_bits != 4 && cfg->quant_bits != 8))) return FFD_ERR_UNSUPPORTED;
     if (cfg->num_q_heads <= 0 || cfg->num_kv_heads <= 0 || cfg->num_q_heads % cfg->num_kv_heads) return FFD_ERR_SHAPE;
-    if (cfg->num_q_heads / cfg->num_kv_heads > kMaxG) return FFD_ERR_UNSUPPORTED;
+    if (cfg->num_q_heads / cfg->num_kv_heads > kMaxG && !(wide_groups && group_shift(cfg))) return FFD_ERR_UNSUPPORTED;
     if (cfg->n_sink_blocks < 0 || cfg->n_local_blocks < 0 || cfg->n_sink_blocks + cfg->n_local_blocks < 1)
         return FFD_ERR_SHAPE;
     if (cfg->out_dtype != 0 && cfg->out_dtype != 1) return FFD_ERR_UNSUPPORTED;
@@ -1572,7 +1596,7 @@ static ffd_status check_decode_args(bool sparse, const ffd_config* cfg, const vo
                                     const int32_t* block_table, const int32_t* seq_lens, int batch, int max_blocks,
                                     int num_pages, float delta, const void* out, const float* lse,
                                     const float* block_max, const void* workspace, const void* k_res) {
-    ffd_status st = check_config(cfg);
+    ffd_status st = check_config(cfg, false, k_res == nullptr);
     if (st) return st;
     if (!q || (!k_cache && !k_res) || !v_cache || !seq_lens || !out || !workspace) return FFD_ERR_NULL;
     if (sparse && (!k_quant || !k_scales)) return FFD_ERR_NULL;
@@ -1580,7 +1604,7 @@ static ffd_status check_decode_args(bool sparse, const ffd_config* cfg, const vo
     if (st) return st;
     if (cfg->num_kv_heads > 65535 || cfg->num_q_heads > 65535) return FFD_ERR_SHAPE;
     if ((double)num_pages * cfg->num_kv_heads >= 2147483648.0) return FFD_ERR_SHAPE;
-    if ((long)batch * cfg->num_kv_heads >= 65536L) return FFD_ERR_SHAPE;   // fast_div: items * units < 2^48
+    if (((long)batch * cfg->num_kv_heads << group_shift(cfg)) >= 65536L) return FFD_ERR_SHAPE;   // fast_div: items * units < 2^48
     if (sparse && (isnan(delta) || delta < 0.f)) return FFD_ERR_DELTA;
     const void* ptrs[] = {q, k_cache, k_res, v_cache, k_quant, k_scales, block_table, seq_lens, out, lse, block_max,
                           workspace};
@@ -1615,7 +1639,10 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
     p.seq_lens = seq_lens;
     p.batch = batch;
     p.Hq = cfg->num_q_heads;
-    p.Hkv = cfg->num_kv_heads;
+    p.kv_shift = group_shift(cfg);
+    if (p.kv_shift && (append || k_res)) return FFD_ERR_UNSUPPORTED;
+    p.Hkv_phys = cfg->num_kv_heads;
+    p.Hkv = cfg->num_kv_heads << p.kv_shift;
     p.G = p.Hq / p.Hkv;
     p.max_blocks = max_blocks;
     p.num_pages = num_pages;
@@ -1642,13 +1669,13 @@ static ffd_status run_decode(bool sparse, const ffd_config* cfg, const void* q, 
     p.res_scores = reinterpret_cast<float*>(ws + pl.off_scores);
     p.bmax = reinterpret_cast<float*>(ws + pl.off_bmax);
     p.keep_bits = reinterpret_cast<uint8_t*>(ws + pl.off_keep);
-    p.units = batch * cfg->num_kv_heads;
+    p.units = batch * p.Hkv;
     const ItemGeom geom = item_geometry(p.units, max_blocks, sms);
     p.item_rows = geom.item_rows;
     p.rows_small = geom.rows_small;
     p.item_blocks = geom.item_blocks;
     p.units_magic = fast_div_magic((unsigned)p.units);
-    p.hkv_magic = fast_div_magic((unsigned)cfg->num_kv_heads);
+    p.hkv_magic = fast_div_magic((unsigned)p.Hkv);
     p.kept_mask = kept_mask;
     p.block_max = block_max;
     p.out = out;
@@ -1751,7 +1778,7 @@ const char* ffd_status_string(ffd_status status) {
 }
 
 ffd_status ffd_workspace_bytes(const ffd_config* cfg, int32_t batch, int32_t max_blocks_per_seq, size_t* bytes) {
-    ffd_status st = check_config(cfg);
+    ffd_status st = check_config(cfg, false, true);
     if (st) return st;
     if (!bytes) return FFD_ERR_NULL;
     st = check_geometry(batch, max_blocks_per_seq, 1);
@@ -1804,7 +1831,7 @@ ffd_status ffd_quantize_keys_residual(const ffd_config* cfg, const void* k_cache
 static ffd_status quantize_impl(const ffd_config* cfg, const void* k_cache, void* k_quant, void* k_scales, void* k_res,
                                 const int32_t* block_table, const int32_t* seq_lens, const int32_t* first_token,
                                 int32_t batch, int32_t max_blocks_per_seq, int32_t num_pages, void* stream) {
-    ffd_status st = check_config(cfg);
+    ffd_status st = check_config(cfg, false, k_res == nullptr);
     if (st) return st;
     if (!k_cache || !k_quant || !k_scales || !seq_lens) return FFD_ERR_NULL;
     st = check_geometry(batch, max_blocks_per_seq, num_pages);
@@ -1980,7 +2007,7 @@ ffd_status ffd_decode_dense(const ffd_config* cfg, const void* q, const void* k_
 
 ffd_status ffd_unpack_codes(const ffd_config* cfg, const void* k_quant, uint8_t* codes, int32_t num_pages,
                             void* stream) {
-    ffd_status st = check_config(cfg);
+    ffd_status st = check_config(cfg, false, true);
     if (st) return st;
     if (!k_quant || !codes) return FFD_ERR_NULL;
     if (num_pages <= 0) return FFD_ERR_SHAPE;

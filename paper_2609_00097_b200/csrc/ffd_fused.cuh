@@ -462,7 +462,7 @@ __device__ __forceinline__ bool cursor_next(const DecodeParams& p, ScanCursor& c
 __device__ __forceinline__ void ring_issue(const DecodeParams& p, const ScanCursor& c, uint32_t stage,
                                            volatile int* stage_tile, int lane) {
     const int page = __shfl_sync(kFull, c.pages, c.lb);   // -1: bad table entry (reported by the scheduler), skipped
-    const int tile = page >= 0 ? page * p.Hkv + c.it.g : -1;
+    const int tile = page >= 0 ? (int)tile_index(p, page, c.it.g) : -1;
     if (tile >= 0) {
         const uint4* codes = reinterpret_cast<const uint4*>(p.k_quant + (size_t)tile * kCodeBytes);
 #pragma unroll

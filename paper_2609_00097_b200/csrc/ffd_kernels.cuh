@@ -59,7 +59,9 @@ struct DecodeParams {
     const __half* k_scales;
     const int32_t* block_table;
     const int32_t* seq_lens;
-    int batch, Hq, Hkv, G, max_blocks, num_pages;
+    int batch, Hq, Hkv, G, max_blocks, num_pages;   // Hkv, G: the groups the kernels work on (see kv_shift)
+    int Hkv_phys, kv_shift;  // KV heads of the caches; a KV head with 6 or 8 query heads is served as 2^kv_shift = 2 groups of
+                             // 3 or 4 heads that read the same tiles: group g uses KV head g >> kv_shift
     int n_sink, n_local;
     int blocks_per_split, splits;
     float sm_scale;          // logit scale
@@ -233,6 +235,11 @@ __device__ __forceinline__ int page_of(const DecodeParams& p, int b, int blk) {
         return -1;
     }
     return page;
+}
+
+// (page, KV head) tile of group g
+__device__ __forceinline__ size_t tile_index(const DecodeParams& p, int page, int g) {
+    return (size_t)page * p.Hkv_phys + (g >> p.kv_shift);
 }
 
 __device__ __forceinline__ int clamped_seq_len(const DecodeParams& p, int b) {

@@ -82,7 +82,8 @@ class Workload:
 
 def make_workload(name: str, *, variant: int = 0, N: int | None = None, B: int | None = None,
                   lens: tuple | None = None, sink: bool | None = None, tail: int = 0, q_gain: float = 1.0,
-                  k_gain: float = 1.0, k_outliers: tuple | None = None, q_outliers: tuple | None = None) -> Workload:
+                  k_gain: float = 1.0, k_outliers: tuple | None = None, q_outliers: tuple | None = None,
+                  heads: tuple | None = None) -> Workload:
     """Build config ``name`` (C1..C5).  ``N`` / ``B`` / ``lens`` shrink or reshape it for tests; ``tail`` subtracts
     that many tokens from every sequence (ragged last block); ``variant`` k adds 10*k to the seed;
     ``sink=False`` gives the "no-sink" correctness variant; the gains and outlier channels are described in the
@@ -91,7 +92,7 @@ def make_workload(name: str, *, variant: int = 0, N: int | None = None, B: int |
     seed = cfg["seed"] + 10 * variant
     gen = torch.Generator().manual_seed(seed)
     Bn = B if B is not None else cfg["B"]
-    Hq, Hkv = cfg["Hq"], cfg["Hkv"]
+    Hq, Hkv = heads if heads is not None else (cfg["Hq"], cfg["Hkv"])   # heads = (query heads, KV heads) of a variant
     G = Hq // Hkv
     use_sink = cfg["sink"] if sink is None else sink
     lens = lens if lens is not None else cfg.get("lens")

@@ -71,7 +71,7 @@ def test_documented_limits_of_the_static_entry_point_are_the_computed_ones():
 
 @pytest.mark.parametrize("field,value,status", [
     ("head_dim", 64, 3), ("block_tokens", 32, 3), ("quant_bits", 3, 3), ("quant_bits", 16, 3), ("num_kv_heads", 5, 2),
-    ("num_q_heads", 64, 3), ("n_local_blocks", -1, 2), ("out_dtype", 7, 3), ("sm_scale", -1.0, 2),
+    ("num_q_heads", 40, 3), ("num_q_heads", 128, 3), ("n_local_blocks", -1, 2), ("out_dtype", 7, 3), ("sm_scale", -1.0, 2),
 ])
 def test_bad_config_is_rejected(field, value, status):
     cfg = ffd.Config(32, 8)
@@ -87,6 +87,16 @@ def test_deeper_thumbnails_are_accepted_except_where_the_format_needs_two_bits()
         assert ffd.ffd_workspace_bytes(cfg, 1, 16) == ffd.ffd_workspace_bytes(ffd.Config(32, 8), 1, 16)
         with pytest.raises(ffd.FfdError) as e:     # the 2 + 8 bit key format is defined on the 2-bit thumbnails
             ffd.ffd_workspace_bytes_residual(cfg, 1, 16)
+        assert e.value.status == 3
+
+
+def test_six_and_eight_query_heads_per_kv_head_are_accepted_where_documented():
+    for hq in (48, 64):
+        cfg = ffd.Config(hq, 8)
+        # two groups per KV head: the geometry of twice the KV heads
+        assert ffd.ffd_workspace_bytes(cfg, 2, 64) == ffd.ffd_workspace_bytes(ffd.Config(hq, 16), 2, 64)
+        with pytest.raises(ffd.FfdError) as e:
+            ffd.ffd_workspace_bytes_residual(cfg, 2, 64)
         assert e.value.status == 3
 
 

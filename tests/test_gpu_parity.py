@@ -795,6 +795,28 @@ def test_full_size_configs_every_row(ffd, oracle, name):
         oracle.set_threads(min(8, oracle.max_threads()))
 
 
+@pytest.mark.parametrize("heads", [(16, 2), (12, 2), (64, 8)])
+def test_six_and_eight_query_heads_per_kv_head(ffd, oracle, heads):
+    """GQA groups of 6 and 8 (served as two groups of 3 or 4 heads over the same KV tiles) on the single-launch path, the
+    persistent path, the dense path and the three-kernel path; refused by the entry points that are documented to."""
+    cases = [("C2", dict(N=8192, tail=5)), ("C5", dict(B=6, lens=(1000, 5000))), ("C5", dict(B=24, lens=(2000, 4200)))]
+    for name, kw in cases:
+        w = make_workload(name, heads=heads, **kw)
+        dc = DeviceCache(w)
+        codes, scales = check_quantize(ffd, oracle, w, dc)
+        check_decode(ffd, oracle, w, dc, codes, scales, 6.0)
+        check_decode(ffd, oracle, w, dc, codes, scales, 0.0)
+        check_dense(ffd, oracle, w, dc)
+        check_decode(ffd, oracle, w, dc, codes, scales, 6.0, rule=ffd.RULE_RUNNING_MAX)
+    with pytest.raises(ffd.FfdError) as e:
+        dc.quantize_residual()
+    assert e.value.status == 3
+    k_new = torch.zeros(w.B, w.Hkv, 128, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(ffd.FfdError) as e:
+        dc.append_decode(k_new, k_new, 6.0)
+    assert e.value.status == 3
+
+
 RULE_CASES = [
     ("C1", dict()), ("C4", dict(N=16384)), ("C5", dict(B=4, lens=(1000, 5000))), ("C5", dict(B=20, lens=(300, 1500))),
     ("C2", dict(N=6000, sink=False)), ("C3", dict(N=8192, B=8)),
