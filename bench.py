@@ -38,8 +38,8 @@ CODE_BYTES_PER_TILE = 2048 + 256          # packed 2-bit codes + fp16 scales of 
 KV_BYTES_PER_TILE = 2 * 64 * 128 * 2      # K tile + V tile of one kept (block, KV head)
 # dram__bytes_read + dram__bytes_write of one fused-kernel launch divided by the launch's algorithmic bytes, from
 # the ncu capture summarised in profiles/fused_sparse_kernel_C3_ctx32768.md (same kernel, same workload recipe at
-# context 32768; traffic grows in proportion to the blocks processed): (308.47 + 5.65) MB / 308.28 MB.
-NCU_TRAFFIC_RATIO = 1.018
+# context 32768; traffic grows in proportion to the blocks processed): (308.62 + 6.12) MB / 308.28 MB.
+NCU_TRAFFIC_RATIO = 1.021
 
 
 def measured_peaks():
