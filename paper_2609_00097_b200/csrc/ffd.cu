@@ -1093,6 +1093,11 @@ __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodePara
     const int r = lane >> 2, j = lane & 3;
     pdl_launch_dependents();
     pdl_wait();
+    // the query fragments first: their loads fly while the sequence length (which everything else hangs on) arrives
+    const __nv_bfloat16* q_group = p.q + ((size_t)b * p.Hq + (size_t)g * p.G) * kD;
+    ScanQuery sq;
+    if constexpr (BITS == 2) scan_setup(sq, q_group, p.G, lane, p.sm_scale);
+    else if constexpr (BITS != 0) scan_setup_wide(sq, q_group, p.G, lane, p.sm_scale);
     const int n = clamped_seq_len(p, b);
     const int nb = (n + kBlk - 1) / kBlk;
     const int blk_begin = split * p.blocks_per_split;
@@ -1110,15 +1115,11 @@ __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodePara
         mbar_init(vbar, 32);
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
-    const __nv_bfloat16* q_group = p.q + ((size_t)b * p.Hq + (size_t)g * p.G) * kD;
     const size_t head0 = (size_t)b * p.Hq + (size_t)g * p.G;
     AttendState st;
     bool ok = true;
     if (blk_begin >= nb) attend_reset(st);
     if (blk_begin < nb) {   // (uniform over the CTA; a split past the sequence's end only reports an empty partial)
-        ScanQuery sq;
-        if constexpr (BITS == 2) scan_setup(sq, q_group, p.G, lane, p.sm_scale);
-        else if constexpr (BITS != 0) scan_setup_wide(sq, q_group, p.G, lane, p.sm_scale);
         constexpr size_t kCodeTile = BITS == 2 ? (size_t)kCodeBytes : (size_t)WideScan<BITS>::kTileBytes;
         // BITS == 0: the decisions come from the select kernel that ran before this one (p.keep_bits)
         // scan of one block, precise or fast.  2 bits: from the codes in registers, with the binary32 fallback when the
@@ -1395,38 +1396,44 @@ __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodePara
         s_ml[x] = ml.y > 0.f ? ml : make_float2(-INFINITY, 0.f);
     }
     __syncthreads();
-    for (int item = threadIdx.x; item < p.G * (kD / 2); item += kWarps * 32) {
-        const int h = item / (kD / 2), c = (item % (kD / 2)) * 2;
+    // one work item = one head and four channels: G * 32 <= 128 items, a single pass of the CTA's 224 threads
+    for (int item = threadIdx.x; item < p.G * (kD / 4); item += kWarps * 32) {
+        const int h = item / (kD / 4), c = (item % (kD / 4)) * 4;
         const size_t base = (head0 + h) * p.splits;
         const float2* ml = s_ml + h * nsp;
         float M = -INFINITY;
         for (int sp = 0; sp < nsp; ++sp) M = fmaxf(M, ml[sp].x);
-        float L = 0.f, a0 = 0.f, a1 = 0.f;
+        float L = 0.f;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         if (M != -INFINITY) {
             for (int sp0 = 0; sp0 < nsp; sp0 += 8) {
-                float2 a[8];
+                float4 a[8];
                 float f[8];
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
                     const int sp = sp0 + u;
                     f[u] = sp < nsp ? exp2f(ml[sp].x - M) : 0.f;   // exp2(-inf) = 0 for empty splits
-                    a[u] = make_float2(0.f, 0.f);
-                    if (f[u] != 0.f) a[u] = __ldcg(reinterpret_cast<const float2*>(p.part_acc + (base + sp) * kD + c));
+                    a[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (f[u] != 0.f) a[u] = __ldcg(reinterpret_cast<const float4*>(p.part_acc + (base + sp) * kD + c));
                 }
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
                     if (sp0 + u < nsp) L += f[u] * ml[sp0 + u].y;
-                    a0 += f[u] * a[u].x;
-                    a1 += f[u] * a[u].y;
+                    acc.x += f[u] * a[u].x;
+                    acc.y += f[u] * a[u].y;
+                    acc.z += f[u] * a[u].z;
+                    acc.w += f[u] * a[u].w;
                 }
             }
         }
         const float inv = L > 0.f ? 1.f / L : 0.f;
         if (p.out_fp32) {
-            *reinterpret_cast<float2*>(static_cast<float*>(p.out) + (head0 + h) * kD + c) = make_float2(a0 * inv, a1 * inv);
+            *reinterpret_cast<float4*>(static_cast<float*>(p.out) + (head0 + h) * kD + c) =
+                make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
         } else {
-            *reinterpret_cast<__nv_bfloat162*>(static_cast<__nv_bfloat16*>(p.out) + (head0 + h) * kD + c) =
-                __floats2bfloat162_rn(a0 * inv, a1 * inv);
+            __nv_bfloat162* o = reinterpret_cast<__nv_bfloat162*>(static_cast<__nv_bfloat16*>(p.out) + (head0 + h) * kD + c);
+            o[0] = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+            o[1] = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
         }
         if (p.lse && c == 0) p.lse[head0 + h] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
     }
