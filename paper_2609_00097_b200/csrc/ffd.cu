@@ -1126,10 +1126,10 @@ __global__ void __launch_bounds__(kWarps * 32, 1) small_sparse_kernel(DecodePara
         // fp16 operand overflowed; deeper thumbnails: straight from global memory (an overflow there -- scales beyond
         // 30000 -- is reported and the block kept)
         auto judge = [&](bool precise, const ScanRegs& sr, size_t tile, int rows, float& band) {
-            float bm;
+            float bm = 0.f;
             if constexpr (BITS == 0) {
                 band = 0.f;
-                return 0.f;
+                return bm;
             } else if constexpr (BITS == 2) {
                 bm = precise ? scan_compute<true>(sr, sq, lane, rows, band) : scan_compute<false>(sr, sq, lane, rows, band);
             } else {
