@@ -808,6 +808,12 @@ def test_six_and_eight_query_heads_per_kv_head(ffd, oracle, heads):
         check_decode(ffd, oracle, w, dc, codes, scales, 0.0)
         check_dense(ffd, oracle, w, dc)
         check_decode(ffd, oracle, w, dc, codes, scales, 6.0, rule=ffd.RULE_RUNNING_MAX)
+    if heads == (16, 2):   # ... and on deeper thumbnails, single-launch and three-kernel path
+        for name, kw in cases[:1] + cases[2:]:
+            w4 = make_workload(name, heads=heads, **kw)
+            d4 = DeviceCache(w4, ffd.Config(w4.Hq, w4.Hkv, quant_bits=4))
+            c4, s4 = check_quantize(ffd, oracle, w4, d4)
+            check_decode(ffd, oracle, w4, d4, c4, s4, 6.0)
     with pytest.raises(ffd.FfdError) as e:
         dc.quantize_residual()
     assert e.value.status == 3
